@@ -1,0 +1,272 @@
+"""CPU fp64 oracle for K-cache-only ("slim") multi-head decode attention.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition that the
+CUDA library is checked against.  It is imported by the tests, by the smoke
+check and by the benchmark's CPU-baseline leg, never by the product path, and
+it imports nothing from the CUDA package.  Everything is numpy float64; the
+loops are over heads (and, in the ``*_loops`` functions, over scalars) exactly
+as the paper states the operations, with no tiling, fusion or reordering.
+
+Paper passages followed (arxiv 2503.05840):
+  Eq. 4, Eq. 5, Eq. 2   vanilla MHA: Q = X W_Q, K = X W_K, V = X W_V,
+                        head_i = softmax(Q_i K_i^T / sqrt(d_k)) V_i
+  Eq. 6                 W_KV = W_K^{-1} W_V,  V = K W_KV,  V_i = K W_KV,i
+  Eq. 7                 Option 1: softmax(.) [K W_KV,i]
+                        Option 2: [softmax(.) K] W_KV,i
+  Appendix "Support for RoPE"   encoding / decoding rotation formulas, and
+                        Option 1 of that appendix: raw keys are cached and
+                        rotated after they are read
+  Appendix "MHA complexity"     OP counts 2 n d_k (scores) and 2 n d
+                        (weighted sum of K) per head
+
+Readings where the paper is silent (the CUDA path takes the same ones):
+  * RoPE pairs element j with j + d_k/2 inside a head, frequency
+    theta_j = rope_theta ** (-2 j / d_k), angle = position * theta_j;
+    the rotation sign is the one printed in the appendix
+    (y1 = x1 cos + x2 sin, y2 = -x1 sin + x2 cos).  rope_theta == 0 means
+    "no positional rotation".
+  * The single decode query sits at position T-1 (the newest key is already
+    in the cache), key t sits at position t.  No causal mask is needed.
+  * d_v = d_k, head i owns columns i*d_k .. (i+1)*d_k-1 of every projection.
+  * A sequence of length 0 produces a zero output row.
+  * W_KV is obtained with a linear solve W_K W_KV = W_V rather than by
+    forming the inverse explicitly (same matrix up to rounding).
+
+Pins: tests/test_oracle_pins.py (closed forms, identities, brute force).
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------
+# RoPE (appendix "Support for RoPE")
+# --------------------------------------------------------------------------
+def rope_frequencies(d_k: int, rope_theta: float) -> np.ndarray:
+    """theta_j for j = 0 .. d_k/2 - 1 (float64)."""
+    if d_k % 2:
+        raise ValueError("d_k must be even for RoPE")
+    j = np.arange(d_k // 2, dtype=F64)
+    return np.power(F64(rope_theta), -2.0 * j / F64(d_k))
+
+
+def rope_encode(x: np.ndarray, positions, rope_theta: float) -> np.ndarray:
+    """Rotate head vectors x[..., d_k] sitting at `positions` (broadcast over
+    the leading axes of x).  Appendix formulas, pair (j, j + d_k/2):
+        y1 =  x1 cos(m theta) + x2 sin(m theta)
+        y2 = -x1 sin(m theta) + x2 cos(m theta)
+    """
+    x = np.asarray(x, dtype=F64)
+    if rope_theta == 0:
+        return x.copy()
+    d_k = x.shape[-1]
+    half = d_k // 2
+    ang = np.asarray(positions, dtype=F64)[..., None] * rope_frequencies(d_k, rope_theta)
+    c, s = np.cos(ang), np.sin(ang)
+    x1, x2 = x[..., :half], x[..., half:]
+    return np.concatenate([x1 * c + x2 * s, -x1 * s + x2 * c], axis=-1)
+
+
+def rope_decode(y: np.ndarray, positions, rope_theta: float) -> np.ndarray:
+    """Inverse rotation (appendix "RoPE decoding"), same cos/sin table:
+        x1 = y1 cos - y2 sin,   x2 = y1 sin + y2 cos
+    """
+    y = np.asarray(y, dtype=F64)
+    if rope_theta == 0:
+        return y.copy()
+    d_k = y.shape[-1]
+    half = d_k // 2
+    ang = np.asarray(positions, dtype=F64)[..., None] * rope_frequencies(d_k, rope_theta)
+    c, s = np.cos(ang), np.sin(ang)
+    y1, y2 = y[..., :half], y[..., half:]
+    return np.concatenate([y1 * c - y2 * s, y1 * s + y2 * c], axis=-1)
+
+
+# --------------------------------------------------------------------------
+# softmax (Eq. 2)
+# --------------------------------------------------------------------------
+def softmax(z: np.ndarray) -> np.ndarray:
+    """Softmax over the last axis: subtract the exact row maximum, exp, divide
+    by the sum.  float64 throughout."""
+    z = np.asarray(z, dtype=F64)
+    e = np.exp(z - np.max(z, axis=-1, keepdims=True))
+    return e / np.sum(e, axis=-1, keepdims=True)
+
+
+def attention_weights(q_i: np.ndarray, K_i: np.ndarray, rope_theta: float) -> np.ndarray:
+    """s = softmax(RoPE_{T-1}(q_i) . RoPE_t(K_i[t])^T / sqrt(d_k)) for one head.
+    q_i: [d_k], K_i: [T, d_k] (raw, un-rotated keys).  Returns [T]."""
+    T, d_k = K_i.shape
+    qr = rope_encode(q_i, T - 1, rope_theta)
+    Kr = rope_encode(K_i, np.arange(T), rope_theta)
+    return softmax(Kr @ qr / math.sqrt(d_k))
+
+
+# --------------------------------------------------------------------------
+# Eq. 6: W_KV
+# --------------------------------------------------------------------------
+def oracle_wkv(W_K: np.ndarray, W_V: np.ndarray) -> np.ndarray:
+    """W_KV = W_K^{-1} W_V in float64 (Eq. 6), by solving W_K W_KV = W_V."""
+    W_K = np.asarray(W_K, dtype=F64)
+    W_V = np.asarray(W_V, dtype=F64)
+    if W_K.ndim != 2 or W_K.shape[0] != W_K.shape[1]:
+        raise ValueError("W_K must be square (MHA with d = h d_k)")
+    return np.linalg.solve(W_K, W_V)
+
+
+# --------------------------------------------------------------------------
+# Eq. 4, 5, 2: vanilla MHA decode with an explicit V cache
+# --------------------------------------------------------------------------
+def oracle_vanilla(X: np.ndarray, W_Q: np.ndarray, W_K: np.ndarray, W_V: np.ndarray,
+                   H: int, rope_theta: float = 0.0, q: np.ndarray | None = None) -> np.ndarray:
+    """Output concat(head_1..head_h) (no W_O) for the LAST token of X attending
+    over all T = len(X) tokens.  X: [T, d].  If q is given it replaces
+    X[-1] W_Q (used where the query carries a bias)."""
+    X = np.asarray(X, dtype=F64)
+    T, d = X.shape
+    d_k = d // H
+    K = X @ np.asarray(W_K, dtype=F64)           # Eq. 4
+    V = X @ np.asarray(W_V, dtype=F64)           # Eq. 5
+    if q is None:
+        q = X[-1] @ np.asarray(W_Q, dtype=F64)   # Eq. 4, one query row
+    q = np.asarray(q, dtype=F64)
+    out = np.empty(d, dtype=F64)
+    for i in range(H):
+        sl = slice(i * d_k, (i + 1) * d_k)
+        s = attention_weights(q[sl], K[:, sl], rope_theta)
+        out[sl] = s @ V[:, sl]                   # Eq. 2
+    return out
+
+
+# --------------------------------------------------------------------------
+# Eq. 7: slim attention, one sequence
+# --------------------------------------------------------------------------
+def oracle_slim(q: np.ndarray, K: np.ndarray, W_KV: np.ndarray, H: int,
+                rope_theta: float = 0.0) -> np.ndarray:
+    """Eq. 7, Option 2: head_i = [softmax(.) K] W_KV,i with the FULL d-wide raw
+    keys in the weighted sum.  q: [d], K: [T, d] raw keys, W_KV: [d, d]."""
+    q = np.asarray(q, dtype=F64)
+    K = np.asarray(K, dtype=F64)
+    W_KV = np.asarray(W_KV, dtype=F64)
+    T, d = K.shape
+    d_k = d // H
+    out = np.empty(d, dtype=F64)
+    for i in range(H):
+        sl = slice(i * d_k, (i + 1) * d_k)
+        s = attention_weights(q[sl], K[:, sl], rope_theta)   # [T]
+        u = s @ K                                            # [d]   weighted sum of K
+        out[sl] = u @ W_KV[:, sl]                            # [d_k]
+    return out
+
+
+def oracle_slim_option1(q: np.ndarray, K: np.ndarray, W_KV: np.ndarray, H: int,
+                        rope_theta: float = 0.0) -> np.ndarray:
+    """Eq. 7, Option 1: V_i = K W_KV,i first, then softmax(.) V_i."""
+    q = np.asarray(q, dtype=F64)
+    K = np.asarray(K, dtype=F64)
+    W_KV = np.asarray(W_KV, dtype=F64)
+    T, d = K.shape
+    d_k = d // H
+    out = np.empty(d, dtype=F64)
+    for i in range(H):
+        sl = slice(i * d_k, (i + 1) * d_k)
+        s = attention_weights(q[sl], K[:, sl], rope_theta)
+        V_i = K @ W_KV[:, sl]                                # Eq. 6
+        out[sl] = s @ V_i
+    return out
+
+
+def oracle_slim_batch(q: np.ndarray, K: np.ndarray, lengths, W_KV: np.ndarray, H: int,
+                      rope_theta: float = 0.0) -> np.ndarray:
+    """Ragged batch: q [B, d], K [B, T_cap, d], lengths[b] rows valid.
+    Sequence b attends over K[b, :lengths[b]]; length 0 gives a zero row."""
+    q = np.asarray(q, dtype=F64)
+    B, d = q.shape
+    out = np.zeros((B, d), dtype=F64)
+    for b in range(B):
+        n = int(lengths[b])
+        if n > 0:
+            out[b] = oracle_slim(q[b], np.asarray(K[b][:n], dtype=F64), W_KV, H, rope_theta)
+    return out
+
+
+# --------------------------------------------------------------------------
+# Scalar-loop version with an operation counter (appendix "MHA complexity")
+# --------------------------------------------------------------------------
+def oracle_slim_loops(q, K, W_KV, H: int, rope_theta: float = 0.0):
+    """Same result as oracle_slim, written as scalar loops, for tiny inputs.
+    Returns (out, macs) where macs counts the multiply-accumulates of the two
+    attention products only (scores: T d_k per head; weighted sum of K: T d
+    per head), which the paper totals as 2 n d (h + 1) OPs = n d (h + 1) MACs."""
+    q = [float(v) for v in q]
+    K = [[float(v) for v in row] for row in K]
+    T, d = len(K), len(q)
+    d_k = d // H
+    half = d_k // 2
+    macs = 0
+    out = [0.0] * d
+    for i in range(H):
+        base = i * d_k
+        # rotate the query of this head to position T-1
+        qr = list(q[base:base + d_k])
+        if rope_theta != 0:
+            for j in range(half):
+                ang = (T - 1) * rope_theta ** (-2.0 * j / d_k)
+                c, s = math.cos(ang), math.sin(ang)
+                x1, x2 = q[base + j], q[base + j + half]
+                qr[j] = x1 * c + x2 * s
+                qr[j + half] = -x1 * s + x2 * c
+        z = []
+        for t in range(T):
+            kr = list(K[t][base:base + d_k])
+            if rope_theta != 0:
+                for j in range(half):
+                    ang = t * rope_theta ** (-2.0 * j / d_k)
+                    c, s = math.cos(ang), math.sin(ang)
+                    x1, x2 = K[t][base + j], K[t][base + j + half]
+                    kr[j] = x1 * c + x2 * s
+                    kr[j + half] = -x1 * s + x2 * c
+            acc = 0.0
+            for e in range(d_k):
+                acc += qr[e] * kr[e]
+                macs += 1
+            z.append(acc / math.sqrt(d_k))
+        zmax = max(z)
+        ez = [math.exp(v - zmax) for v in z]
+        tot = sum(ez)
+        s_w = [v / tot for v in ez]
+        u = [0.0] * d
+        for t in range(T):
+            for c_ in range(d):
+                u[c_] += s_w[t] * K[t][c_]
+                macs += 1
+        for c_ in range(d_k):
+            acc = 0.0
+            for r in range(d):
+                acc += u[r] * float(W_KV[r][base + c_])
+            out[base + c_] = acc
+    return np.array(out, dtype=F64), macs
+
+
+# --------------------------------------------------------------------------
+# Error norms used by the parity tests (stated in the benchmark spec's tolerances)
+# --------------------------------------------------------------------------
+def err_fp32_norm(got: np.ndarray, ref: np.ndarray) -> float:
+    """max_i |got_i - ref_i| / max(|ref_i|, RMS(ref)) over one output row."""
+    got = np.asarray(got, dtype=F64)
+    ref = np.asarray(ref, dtype=F64)
+    rms = math.sqrt(float(np.mean(ref * ref)))
+    den = np.maximum(np.abs(ref), rms if rms > 0 else 1.0)
+    return float(np.max(np.abs(got - ref) / den))
+
+
+def err_rms_norm(got: np.ndarray, ref: np.ndarray) -> float:
+    """max_i |got_i - ref_i| / RMS(ref) over one output row."""
+    got = np.asarray(got, dtype=F64)
+    ref = np.asarray(ref, dtype=F64)
+    rms = math.sqrt(float(np.mean(ref * ref)))
+    return float(np.max(np.abs(got - ref)) / (rms if rms > 0 else 1.0))

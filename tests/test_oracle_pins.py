@@ -1,0 +1,326 @@
+"""Pins for the CPU oracle: every check here is against something the paper or
+the mathematics fixes (closed forms, identities, brute force on tiny inputs,
+numbers printed in the paper), never against the oracle's own formula retyped.
+A few tests plant a plausible mistake in a copy of an oracle function and
+check that a pin catches it."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import slim_oracle as so
+from paper_2503_05840_b200 import synth
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rand_case(seed, T, d, H, well_conditioned=True):
+    g = np.random.default_rng(seed)
+    X = g.standard_normal((T, d))
+    W_Q = g.standard_normal((d, d)) / math.sqrt(d)
+    W_V = g.standard_normal((d, d)) / math.sqrt(d)
+    if well_conditioned:
+        Qo, _ = np.linalg.qr(g.standard_normal((d, d)))
+        W_K = Qo * g.uniform(0.5, 2.0, size=d)[None, :]
+    else:
+        W_K = g.standard_normal((d, d)) / math.sqrt(d)
+    return X, W_Q, W_K, W_V
+
+
+# ------------------------------------------------------------------ Eq. 6
+def test_wkv_closed_form_for_orthogonal_times_diagonal():
+    # W_K = Q diag(s)  =>  W_K^{-1} = diag(1/s) Q^T  exactly.
+    _, W_K, W_V, Qo, s = synth.make_weights(48, 123)
+    expect = (Qo.T @ W_V) / s[:, None]
+    got = so.oracle_wkv(W_K, W_V)
+    assert np.allclose(got, expect, rtol=1e-11, atol=1e-13)
+
+
+def test_wkv_hand_inverted_2x2_and_3x3():
+    W_K = np.array([[2.0, 1.0], [1.0, 1.0]])           # inverse [[1,-1],[-1,2]]
+    W_V = np.array([[3.0, 0.0], [1.0, 2.0]])
+    expect = np.array([[1.0, -1.0], [-1.0, 2.0]]) @ W_V
+    assert np.allclose(so.oracle_wkv(W_K, W_V), expect, atol=1e-14)
+    W_K3 = np.array([[1.0, 2.0, 0.0], [0.0, 1.0, 3.0], [0.0, 0.0, 1.0]])
+    inv3 = np.array([[1.0, -2.0, 6.0], [0.0, 1.0, -3.0], [0.0, 0.0, 1.0]])
+    W_V3 = np.arange(9.0).reshape(3, 3)
+    assert np.allclose(so.oracle_wkv(W_K3, W_V3), inv3 @ W_V3, atol=1e-13)
+
+
+def test_wkv_reconstructs_v_from_k():
+    # Eq. 6: K W_KV = V, and the appendix-A check W_K W_KV ~ W_V (numpy allclose defaults).
+    X, _, W_K, W_V = _rand_case(5, 9, 32, 4, well_conditioned=False)
+    W_KV = so.oracle_wkv(W_K, W_V)
+    assert np.allclose(W_K @ W_KV, W_V)
+    assert np.allclose((X @ W_K) @ W_KV, X @ W_V, rtol=1e-8, atol=1e-9)
+    assert np.allclose(np.linalg.inv(W_K) @ W_V, W_KV, rtol=1e-8, atol=1e-9)
+
+
+def test_wkv_rejects_non_square():
+    with pytest.raises(ValueError):
+        so.oracle_wkv(np.zeros((4, 6)), np.zeros((4, 6)))
+
+
+# ------------------------------------------------------------------ Eq. 7 == Eq. 2
+@pytest.mark.parametrize("T,d,H,theta", [(1, 8, 2, 0.0), (7, 16, 4, 0.0), (33, 32, 4, 1.0e4),
+                                         (64, 48, 6, 1.0e6), (130, 64, 2, 1.0e4)])
+def test_slim_equals_vanilla_and_option1_equals_option2(T, d, H, theta):
+    X, W_Q, W_K, W_V = _rand_case(100 + T, T, d, H)
+    ref = so.oracle_vanilla(X, W_Q, W_K, W_V, H, theta)
+    K = X @ W_K
+    q = X[-1] @ W_Q
+    W_KV = so.oracle_wkv(W_K, W_V)
+    o2 = so.oracle_slim(q, K, W_KV, H, theta)
+    o1 = so.oracle_slim_option1(q, K, W_KV, H, theta)
+    scale = np.max(np.abs(ref))
+    assert np.max(np.abs(o2 - ref)) <= 1e-11 * scale
+    assert np.max(np.abs(o1 - ref)) <= 1e-11 * scale
+    assert np.max(np.abs(o1 - o2)) <= 1e-11 * scale
+
+
+def test_config0_shape_slim_equals_vanilla():
+    cfg = synth.CONFIGS[0].scaled(context=300)
+    L = synth.make_layer(cfg, synth.layer_seed(0, 0))
+    X = L.X[0]
+    ref = so.oracle_vanilla(X, L.W_Q, L.W_K, L.W_V, cfg.H, cfg.rope_theta)
+    W_KV = so.oracle_wkv(L.W_K, L.W_V)
+    got = so.oracle_slim(X[-1] @ L.W_Q, X @ L.W_K, W_KV, cfg.H, cfg.rope_theta)
+    assert np.max(np.abs(got - ref)) <= 1e-11 * np.max(np.abs(ref))
+
+
+# ------------------------------------------------------------------ T = 1, T = 2
+@pytest.mark.parametrize("theta", [0.0, 1.0e4])
+def test_single_key_returns_its_value_row(theta):
+    X, W_Q, W_K, W_V = _rand_case(7, 1, 16, 4)
+    W_KV = so.oracle_wkv(W_K, W_V)
+    g = np.random.default_rng(0)
+    for _ in range(3):
+        q = g.standard_normal(16) * 5
+        out = so.oracle_slim(q, X @ W_K, W_KV, 4, theta)
+        assert np.allclose(out, (X @ W_V)[0], rtol=1e-10, atol=1e-12)
+
+
+def test_two_keys_is_a_logistic_blend_hand_computed():
+    # one head of width 2, no RoPE:  o = sig(a) v0 + (1 - sig(a)) v1,
+    # a = (q.k0 - q.k1)/sqrt(2), all numbers chosen by hand.
+    q = np.array([1.0, -2.0])
+    K = np.array([[0.5, 0.25], [-1.0, 0.75]])
+    W_KV = np.array([[2.0, 0.0], [1.0, -1.0]])
+    V = np.array([[0.5 * 2 + 0.25 * 1, -0.25], [-2.0 + 0.75, -0.75]])
+    s0 = (1.0 * 0.5 + -2.0 * 0.25) / math.sqrt(2.0)     # = 0
+    s1 = (1.0 * -1.0 + -2.0 * 0.75) / math.sqrt(2.0)    # = -2.5/sqrt2
+    w0 = 1.0 / (1.0 + math.exp(-(s0 - s1)))
+    expect = w0 * V[0] + (1.0 - w0) * V[1]
+    assert np.allclose(so.oracle_slim(q, K, W_KV, 1, 0.0), expect, rtol=1e-13)
+    assert np.allclose(so.oracle_slim_option1(q, K, W_KV, 1, 0.0), expect, rtol=1e-13)
+
+
+def test_two_keys_with_rope_hand_rotation_2d():
+    # d_k = 2: one frequency theta_0 = 1, so key t is rotated by angle t and the
+    # query (position 1) by angle 1, with the appendix's sign:
+    #   y1 = x1 cos + x2 sin ; y2 = -x1 sin + x2 cos
+    theta = 10000.0
+    q = np.array([0.3, -1.1])
+    K = np.array([[1.5, 0.2], [-0.4, 0.9]])
+    W_KV = np.array([[1.0, 2.0], [3.0, 4.0]])
+    c1, s1 = math.cos(1.0), math.sin(1.0)
+    qr = np.array([q[0] * c1 + q[1] * s1, -q[0] * s1 + q[1] * c1])
+    k0r = K[0]                                              # angle 0
+    k1r = np.array([K[1][0] * c1 + K[1][1] * s1, -K[1][0] * s1 + K[1][1] * c1])
+    z0 = float(qr @ k0r) / math.sqrt(2.0)
+    z1 = float(qr @ k1r) / math.sqrt(2.0)
+    w0 = math.exp(z0) / (math.exp(z0) + math.exp(z1))
+    V = K @ W_KV
+    expect = w0 * V[0] + (1 - w0) * V[1]
+    assert np.allclose(so.oracle_slim(q, K, W_KV, 1, theta), expect, rtol=1e-13)
+
+
+def test_rope_frequency_schedule_and_pairing_dk4():
+    # d_k = 4, theta = 10000: theta_0 = 1, theta_1 = 10000^(-1/2) = 0.01;
+    # element 0 pairs with 2, element 1 pairs with 3.
+    x = np.array([1.0, 2.0, 3.0, 4.0])
+    m = 3
+    y = so.rope_encode(x, m, 10000.0)
+    c0, s0 = math.cos(3.0), math.sin(3.0)
+    c1, s1 = math.cos(0.03), math.sin(0.03)
+    expect = np.array([1 * c0 + 3 * s0, 2 * c1 + 4 * s1, -1 * s0 + 3 * c0, -2 * s1 + 4 * c1])
+    assert np.allclose(y, expect, rtol=1e-14)
+    assert np.allclose(so.rope_frequencies(4, 10000.0), [1.0, 0.01], rtol=1e-14)
+
+
+# ------------------------------------------------------------------ uniform keys
+@pytest.mark.parametrize("theta", [0.0, 1.0e4])
+def test_identical_keys_return_their_value(theta):
+    g = np.random.default_rng(3)
+    d, H, T = 24, 3, 50
+    _, W_K, W_V, _, _ = synth.make_weights(d, 9)
+    k = g.standard_normal(d)
+    K = np.tile(k, (T, 1))
+    W_KV = so.oracle_wkv(W_K, W_V)
+    out = so.oracle_slim(g.standard_normal(d), K, W_KV, H, theta)
+    assert np.allclose(out, k @ W_KV, rtol=1e-10, atol=1e-12)
+
+
+# ------------------------------------------------------------------ softmax
+def test_softmax_rows_sum_to_one_and_shift_invariant():
+    g = np.random.default_rng(1)
+    z = g.standard_normal((5, 40)) * 30
+    p = so.softmax(z)
+    assert np.allclose(p.sum(axis=-1), 1.0, rtol=1e-14)
+    assert np.allclose(so.softmax(z + 123.456), p, rtol=1e-10)
+    assert np.allclose(so.softmax(np.array([0.0, math.log(3.0)])), [0.25, 0.75], rtol=1e-14)
+    assert np.all(np.isfinite(so.softmax(np.array([1e4, -1e4, 0.0]))))
+
+
+def test_attention_weights_sum_to_one():
+    g = np.random.default_rng(2)
+    w = so.attention_weights(g.standard_normal(8), g.standard_normal((19, 8)), 1.0e4)
+    assert abs(w.sum() - 1.0) < 1e-14 and np.all(w > 0)
+
+
+# ------------------------------------------------------------------ RoPE
+def test_rope_decode_inverts_encode_and_preserves_norm():
+    g = np.random.default_rng(4)
+    x = g.standard_normal((11, 3, 16))
+    pos = np.arange(11)[:, None] * 977
+    y = so.rope_encode(x, pos, 1.0e6)
+    assert np.allclose(so.rope_decode(y, pos, 1.0e6), x, rtol=1e-12, atol=1e-13)
+    assert np.allclose(np.linalg.norm(y, axis=-1), np.linalg.norm(x, axis=-1), rtol=1e-13)
+    assert not np.allclose(y[1:], x[1:])
+
+
+def test_rope_scores_depend_on_relative_position_only():
+    g = np.random.default_rng(5)
+    q, k = g.standard_normal(32), g.standard_normal(32)
+    a = so.rope_encode(q, 100, 1.0e4) @ so.rope_encode(k, 37, 1.0e4)
+    b = so.rope_encode(q, 100 + 555, 1.0e4) @ so.rope_encode(k, 37 + 555, 1.0e4)
+    c = so.rope_encode(q, 101, 1.0e4) @ so.rope_encode(k, 37, 1.0e4)
+    assert abs(a - b) < 1e-10
+    assert abs(a - c) > 1e-3
+
+
+def test_rope_theta_zero_is_identity_and_position_zero_is_identity():
+    x = np.arange(8.0)
+    assert np.array_equal(so.rope_encode(x, 5, 0.0), x)
+    assert np.allclose(so.rope_encode(x, 0, 1.0e4), x)
+
+
+def test_rotation_sign_is_a_real_convention():
+    # score = cos(D)(q1 k1 + q2 k2) + sin(D)(q1 k2 - q2 k1) with D the relative
+    # angle: turning both vectors the other way flips the sine term, so the
+    # printed sign has to be followed literally (it is not a free choice).
+    q, k = np.array([1.0, 0.0]), np.array([0.0, 1.0])
+    enc = so.rope_encode(q, 1, 10000.0) @ so.rope_encode(k, 0, 10000.0)
+    dec = so.rope_decode(q, 1, 10000.0) @ so.rope_decode(k, 0, 10000.0)
+    # query rotated by -1 rad (printed sign): (cos1, -sin1) . (0, 1) = -sin 1
+    assert abs(enc - (-math.sin(1.0))) < 1e-15
+    assert abs(dec - (+math.sin(1.0))) < 1e-15
+
+
+def test_key_bias_cancels_in_the_attention_weights_without_rope():
+    # appendix "Support for bias": a constant added to every key shifts all
+    # softmax arguments of one query by the same amount.
+    g = np.random.default_rng(6)
+    q, K, c = g.standard_normal(8), g.standard_normal((15, 8)), g.standard_normal(8)
+    assert np.allclose(so.attention_weights(q, K + c, 0.0), so.attention_weights(q, K, 0.0), rtol=1e-10)
+
+
+# ------------------------------------------------------------------ brute force + OP count
+@pytest.mark.parametrize("T,d,H,theta", [(5, 8, 2, 0.0), (6, 12, 3, 1.0e4), (9, 8, 1, 1.0e6)])
+def test_scalar_loops_match_vectorised_and_count_macs(T, d, H, theta):
+    X, W_Q, W_K, W_V = _rand_case(50 + T, T, d, H)
+    K, q = X @ W_K, X[-1] @ W_Q
+    W_KV = so.oracle_wkv(W_K, W_V)
+    out, macs = so.oracle_slim_loops(q, K, W_KV, H, theta)
+    assert np.allclose(out, so.oracle_slim(q, K, W_KV, H, theta), rtol=1e-11, atol=1e-13)
+    # appendix "MHA complexity": 2 n d (h+1) OPs = n d (h+1) multiply-accumulates
+    assert macs == T * d * (H + 1)
+
+
+# ------------------------------------------------------------------ ragged batch
+def test_batch_wrapper_masks_rows_beyond_length_and_zero_length():
+    g = np.random.default_rng(8)
+    d, H, B, Tc = 16, 2, 3, 12
+    _, W_K, W_V, _, _ = synth.make_weights(d, 1)
+    W_KV = so.oracle_wkv(W_K, W_V)
+    K = g.standard_normal((B, Tc, d))
+    q = g.standard_normal((B, d))
+    lengths = np.array([12, 0, 5])
+    K2 = K.copy()
+    K2[2, 5:] = np.nan
+    out = so.oracle_slim_batch(q, K2, lengths, W_KV, H, 1.0e4)
+    assert np.all(out[1] == 0)
+    assert np.allclose(out[0], so.oracle_slim(q[0], K[0], W_KV, H, 1.0e4))
+    assert np.allclose(out[2], so.oracle_slim(q[2], K[2, :5], W_KV, H, 1.0e4))
+
+
+# ------------------------------------------------------------------ planted mistakes
+def _slim_with(q, K, W_KV, H, theta, *, scale=None, transpose=False, q_pos_shift=0, full_d=True):
+    """oracle_slim with one deliberate defect, to show the pins notice it."""
+    T, d = K.shape
+    d_k = d // H
+    out = np.empty(d)
+    for i in range(H):
+        sl = slice(i * d_k, (i + 1) * d_k)
+        qr = so.rope_encode(q[sl], T - 1 + q_pos_shift, theta)
+        Kr = so.rope_encode(K[:, sl], np.arange(T), theta)
+        s = so.softmax(Kr @ qr / (math.sqrt(d_k) if scale is None else scale))
+        W = W_KV.T if transpose else W_KV
+        if full_d:
+            out[sl] = (s @ K) @ W[:, sl]
+        else:                       # wrongly uses only the head's own key slice
+            out[sl] = (s @ K[:, sl]) @ W[sl, sl]
+    return out
+
+
+def test_pins_catch_planted_mistakes():
+    T, d, H, theta = 40, 16, 2, 1.0e4
+    X, W_Q, W_K, W_V = _rand_case(77, T, d, H)
+    K, q = X @ W_K, X[-1] @ W_Q
+    W_KV = so.oracle_wkv(W_K, W_V)
+    ref = so.oracle_vanilla(X, W_Q, W_K, W_V, H, theta)
+    tol = 1e-9 * np.max(np.abs(ref))
+    assert np.max(np.abs(_slim_with(q, K, W_KV, H, theta) - ref)) < tol          # sane copy passes
+    assert np.max(np.abs(_slim_with(q, K, W_KV, H, theta, transpose=True) - ref)) > 1e3 * tol
+    assert np.max(np.abs(_slim_with(q, K, W_KV, H, theta, q_pos_shift=1) - ref)) > 1e3 * tol
+    assert np.max(np.abs(_slim_with(q, K, W_KV, H, theta, full_d=False) - ref)) > 1e3 * tol
+    # a dropped 1/sqrt(d_k) is caught by the hand-computed two-key blend:
+    q2 = np.array([1.0, -2.0]); K2 = np.array([[0.5, 0.25], [-1.0, 0.75]])
+    W2 = np.array([[2.0, 0.0], [1.0, -1.0]])
+    good = so.oracle_slim(q2, K2, W2, 1, 0.0)
+    bad = _slim_with(q2, K2, W2, 1, 0.0, scale=1.0)
+    assert np.max(np.abs(good - bad)) > 1e-3
+
+
+# ------------------------------------------------------------------ numbers printed in the paper
+def _rows(name):
+    with open(os.path.join(GOLD, name)) as f:
+        return [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+
+
+def test_kcache_accounting_matches_whisper_table():
+    for model, d, layers, cross, self_, base, opt1 in _rows("whisper_cache_sizes.txt"):
+        d, layers = int(d), int(layers)
+        cross_k = synth.kcache_values(d, layers, 1500)
+        self_k = synth.kcache_values(d, layers, 448)
+        assert abs(2 * cross_k / 1e6 - float(cross)) <= 0.051
+        assert abs(2 * self_k / 1e6 - float(self_)) <= 0.051
+        assert abs(2 * (cross_k + self_k) / 1e6 - float(base)) <= 0.051
+        assert abs((cross_k + self_k) / 1e6 - float(opt1)) <= 0.051   # K-cache only = half
+
+
+def test_kcache_accounting_matches_table1():
+    for model, d, layers, ctx, printed in _rows("table1_context_memory.txt"):
+        kv = 2 * synth.kcache_values(int(d), int(layers), int(ctx))
+        assert abs(kv - float(printed)) / float(printed) < 0.03
+
+
+# ------------------------------------------------------------------ error norms
+def test_error_norms():
+    ref = np.array([3.0, -4.0, 0.0, 0.0])            # RMS = 2.5
+    got = ref + np.array([0.0, 0.0, 0.25, 0.0])
+    assert abs(so.err_rms_norm(got, ref) - 0.1) < 1e-15
+    assert abs(so.err_fp32_norm(got, ref) - 0.1) < 1e-15
+    got2 = ref + np.array([0.3, 0.0, 0.0, 0.0])
+    assert abs(so.err_fp32_norm(got2, ref) - 0.1) < 1e-15   # relative to |ref_i| = 3
