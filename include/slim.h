@@ -1,0 +1,133 @@
+/*
+ * slim.h -- C ABI of the K-cache-only ("slim") multi-head decode-attention
+ * library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements one attention layer's generate-phase step of slim
+ * attention (arxiv 2503.05840): only keys are cached; values are recovered
+ * from keys through W_KV = W_K^{-1} W_V (Eq. 6) and the attention output is
+ * computed as   head_i = [ softmax(q_i K_i^T / sqrt(d_k)) K ] W_KV,i
+ * (Eq. 7, Option 2), with RoPE applied to the keys after they are read from
+ * the cache (appendix "Support for RoPE", Option 1).
+ *
+ * Conventions
+ *   - Row vectors, K = X W_K; every weight matrix is row-major [d_in][d_out];
+ *     head i owns columns i*d_k .. (i+1)*d_k-1.  Square MHA only: d = H*d_k.
+ *   - "device" pointers are CUDA device memory of the current device, "host"
+ *     pointers are ordinary host memory.  The caller owns every buffer it
+ *     passes; the library owns only what slim_create / slim_set_weights /
+ *     slim_cache_create allocate (W_KV, RoPE tables, tensor maps, a status word).
+ *   - Every call returns a slim_status; nothing throws across the ABI.
+ *   - Calls taking `stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) only enqueue work and return; device-side problems are reported
+ *     by slim_device_status.
+ *   - No call falls back to the CPU.  Without a usable CUDA device every
+ *     compute call returns SLIM_ERR_CUDA.
+ */
+#ifndef SLIM_H_
+#define SLIM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SLIM_OK = 0,
+  SLIM_ERR_INVALID_ARG = 1,  /* NULL pointer, non-positive size, bad enum          */
+  SLIM_ERR_UNSUPPORTED = 2,  /* d != H*d_k, odd d_k with RoPE, H > 64, ...          */
+  SLIM_ERR_SINGULAR = 3,     /* W_K has a (numerically) zero pivot                  */
+  SLIM_ERR_CAPACITY = 4,     /* append beyond t_cap / length beyond t_cap (device)  */
+  SLIM_ERR_OOM = 5,          /* a library-owned allocation failed                   */
+  SLIM_ERR_CUDA = 6,         /* CUDA runtime/driver error, or no device             */
+  SLIM_ERR_TIMEOUT = 7,      /* a bounded device-side wait ran out (device)         */
+  SLIM_ERR_NO_WEIGHTS = 8    /* slim_decode before slim_set_weights / slim_set_wkv  */
+} slim_status;
+
+typedef enum { SLIM_F32 = 0, SLIM_BF16 = 1 } slim_dtype;      /* cache / query dtype   */
+typedef enum { SLIM_HOST_F32 = 0, SLIM_HOST_F64 = 1 } slim_host_dtype;
+
+/* Kernel selection for slim_decode (slim_set_path). */
+typedef enum {
+  SLIM_PATH_AUTO = 0,     /* tensor-core path when the shape allows it, else generic */
+  SLIM_PATH_GENERIC = 1,  /* CUDA-core kernels (any supported shape, f32 or bf16)    */
+  SLIM_PATH_TC = 2        /* TMA + tcgen05 kernels (bf16; UNSUPPORTED if shape unfit) */
+} slim_path;
+
+/* Keys for slim_query. */
+typedef enum {
+  SLIM_Q_PATH_IN_USE = 0,        /* slim_path that slim_decode will take             */
+  SLIM_Q_LAUNCHES_PER_DECODE = 1,/* kernels one slim_decode enqueues                 */
+  SLIM_Q_MAX_UNITS = 2,          /* upper bound of (sequence, context-split) units   */
+  SLIM_Q_NUM_SMS = 3,
+  SLIM_Q_WORKERS = 4             /* context-split workers of the path in use         */
+} slim_query_key;
+
+typedef struct slim_ctx slim_ctx;     /* one attention layer: shape, W_KV, RoPE tables  */
+typedef struct slim_cache slim_cache; /* view of caller-owned key storage [B][t_cap][d] */
+
+/* One layer of shape (d, H, d_k); rope_theta = 0 disables RoPE; dtype is the
+ * type of the K-cache and of q.  Requires d == H*d_k (Eq. 6 needs a square
+ * W_K), H <= 64, d_k even.  Uses the current CUDA device.                      */
+slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta, int dtype);
+void        slim_destroy(slim_ctx* ctx);
+
+/* Eq. 6 with the appendix-A recipe: forms W_KV = W_K^{-1} W_V in float64 (LU
+ * with partial pivoting on the device, solving W_K W_KV = W_V) and stores it,
+ * rounded to the ctx dtype, as H column blocks [d][d_k].
+ *   W_K, W_V      host, row-major [d][d], host_dtype = SLIM_HOST_F32 | _F64
+ *   wkv_out       host [d][d] float64, receives the unrounded W_KV (may be NULL)
+ *   residual_out  receives max |W_K W_KV - W_V| (may be NULL)
+ * Synchronous.  SLIM_ERR_SINGULAR if a pivot is below 1e-13 * max|W_K| * d.   */
+slim_status slim_set_weights(slim_ctx* ctx, const void* W_K, const void* W_V, int host_dtype,
+                             double* wkv_out, double* residual_out);
+
+/* Load a precomputed W_KV (the paper stores it in the parameter file in place
+ * of W_V, Eq. 6).  W_KV: host, row-major [d][d].  Synchronous.                 */
+slim_status slim_set_wkv(slim_ctx* ctx, const void* W_KV, int host_dtype);
+
+/* Bytes of key storage for `batch` sequences of capacity t_cap, and of the
+ * scratch workspace slim_decode needs for such a cache (0 on bad arguments).  */
+size_t slim_cache_bytes(const slim_ctx* ctx, int batch, int t_cap);
+size_t slim_workspace_bytes(const slim_ctx* ctx, int batch, int t_cap);
+
+/* Wrap caller-owned device storage k_storage (layout [batch][t_cap][d], ctx
+ * dtype, 16-byte aligned; 1024-byte alignment recommended) as a K-cache of
+ * UN-ROTATED keys.  Builds the RoPE tables for positions < t_cap.  The storage
+ * must outlive the cache object; its contents are not touched.                */
+slim_status slim_cache_create(slim_ctx* ctx, slim_cache** out, void* k_storage, int batch, int t_cap);
+void        slim_cache_destroy(slim_cache* cache);
+
+/* Generate-phase cache update: for every sequence b write the n_new rows
+ * k_new[b][0..n_new) (device, [batch][n_new][d], ctx dtype, un-rotated keys
+ * k = x W_K) at rows positions[b] .. positions[b]+n_new-1 (device int32).
+ * A sequence whose rows would pass t_cap is left unwritten and the device
+ * status becomes SLIM_ERR_CAPACITY.                                            */
+slim_status slim_append_k(slim_ctx* ctx, slim_cache* cache, const void* k_new,
+                          const int32_t* positions, int n_new, void* stream);
+
+/* Eq. 7 Option 2 for one decode token per sequence.
+ *   q        device [batch][d], ctx dtype, un-rotated, bias (if any) included
+ *   lengths  device int32 [batch]; sequence b attends over cache rows
+ *            0 .. lengths[b]-1; the query sits at position lengths[b]-1;
+ *            lengths[b] == 0 gives a zero output row; lengths[b] > t_cap is
+ *            clamped and reported as SLIM_ERR_CAPACITY
+ *   o        device float32 [batch][d] = concat(head_1 .. head_H), no W_O
+ *   workspace device, >= slim_workspace_bytes(ctx, batch, t_cap), 256-byte
+ *            aligned; contents are scratch                                    */
+slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache,
+                        const int32_t* lengths, float* o, void* workspace, void* stream);
+
+/* Synchronises `stream`, returns the sticky device status (SLIM_OK,
+ * SLIM_ERR_CAPACITY or SLIM_ERR_TIMEOUT) and clears it.                        */
+slim_status slim_device_status(slim_ctx* ctx, void* stream);
+
+slim_status slim_set_path(slim_ctx* ctx, int path);
+long long   slim_query(const slim_ctx* ctx, int key);
+const char* slim_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLIM_H_ */

@@ -1,0 +1,165 @@
+"""ctypes binding of libslim.so: same names as the C ABI, argument marshalling
+only.  Every step of the decode path runs inside the library's CUDA kernels;
+torch is used by callers for device memory and streams.  If the shared library
+is missing or cannot be loaded this module raises -- there is no fallback."""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, byref, c_char_p, c_double, c_int, c_longlong, c_size_t, c_void_p
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libslim.so")
+
+SLIM_OK, SLIM_ERR_INVALID_ARG, SLIM_ERR_UNSUPPORTED, SLIM_ERR_SINGULAR, SLIM_ERR_CAPACITY, \
+    SLIM_ERR_OOM, SLIM_ERR_CUDA, SLIM_ERR_TIMEOUT, SLIM_ERR_NO_WEIGHTS = range(9)
+SLIM_F32, SLIM_BF16 = 0, 1
+SLIM_HOST_F32, SLIM_HOST_F64 = 0, 1
+SLIM_PATH_AUTO, SLIM_PATH_GENERIC, SLIM_PATH_TC = 0, 1, 2
+SLIM_Q_PATH_IN_USE, SLIM_Q_LAUNCHES_PER_DECODE, SLIM_Q_MAX_UNITS, SLIM_Q_NUM_SMS, SLIM_Q_WORKERS = range(5)
+
+# name -> (restype, argtypes); mirrors include/slim.h
+SIGNATURES = {
+    "slim_create": (c_int, [POINTER(c_void_p), c_int, c_int, c_int, c_double, c_int]),
+    "slim_destroy": (None, [c_void_p]),
+    "slim_set_weights": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_void_p, POINTER(c_double)]),
+    "slim_set_wkv": (c_int, [c_void_p, c_void_p, c_int]),
+    "slim_cache_bytes": (c_size_t, [c_void_p, c_int, c_int]),
+    "slim_workspace_bytes": (c_size_t, [c_void_p, c_int, c_int]),
+    "slim_cache_create": (c_int, [c_void_p, POINTER(c_void_p), c_void_p, c_int, c_int]),
+    "slim_cache_destroy": (None, [c_void_p]),
+    "slim_append_k": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]),
+    "slim_decode": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "slim_device_status": (c_int, [c_void_p, c_void_p]),
+    "slim_set_path": (c_int, [c_void_p, c_int]),
+    "slim_query": (c_longlong, [c_void_p, c_int]),
+    "slim_strerror": (c_char_p, [c_int]),
+}
+
+_lib = None
+
+
+class SlimError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {strerror(status)} (status {status})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load libslim.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2503_05840_b200.build` "
+                               "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def strerror(status: int) -> str:
+    return lib().slim_strerror(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != SLIM_OK:
+        raise SlimError(status, where)
+
+
+def _ptr(x) -> c_void_p:
+    """Raw address of a torch tensor / numpy array / int / None."""
+    if x is None:
+        return c_void_p(0)
+    if isinstance(x, int):
+        return c_void_p(x)
+    if isinstance(x, np.ndarray):
+        return c_void_p(x.ctypes.data)
+    return c_void_p(x.data_ptr())        # torch.Tensor
+
+
+def _host_mat(a):
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.float64:
+        return a, SLIM_HOST_F64
+    if a.dtype == np.float32:
+        return a, SLIM_HOST_F32
+    return np.ascontiguousarray(a, dtype=np.float64), SLIM_HOST_F64
+
+
+# ---- thin wrappers, same names as the C ABI ---------------------------------
+def slim_create(d: int, H: int, d_k: int, rope_theta: float, dtype: int) -> int:
+    h = c_void_p()
+    _check(lib().slim_create(byref(h), d, H, d_k, float(rope_theta), dtype), "slim_create")
+    return h.value
+
+
+def slim_destroy(ctx: int) -> None:
+    lib().slim_destroy(c_void_p(ctx))
+
+
+def slim_set_weights(ctx: int, W_K, W_V, want_wkv: bool = False):
+    """Returns (residual, W_KV float64 or None)."""
+    a, dt = _host_mat(W_K)
+    b, dt2 = _host_mat(W_V)
+    if dt != dt2:
+        a = np.ascontiguousarray(a, dtype=np.float64); b = np.ascontiguousarray(b, dtype=np.float64)
+        dt = SLIM_HOST_F64
+    out = np.empty(a.shape, dtype=np.float64) if want_wkv else None
+    res = c_double(0.0)
+    _check(lib().slim_set_weights(c_void_p(ctx), _ptr(a), _ptr(b), dt, _ptr(out), byref(res)), "slim_set_weights")
+    return res.value, out
+
+
+def slim_set_wkv(ctx: int, W_KV) -> None:
+    a, dt = _host_mat(W_KV)
+    _check(lib().slim_set_wkv(c_void_p(ctx), _ptr(a), dt), "slim_set_wkv")
+
+
+def slim_cache_bytes(ctx: int, batch: int, t_cap: int) -> int:
+    return lib().slim_cache_bytes(c_void_p(ctx), batch, t_cap)
+
+
+def slim_workspace_bytes(ctx: int, batch: int, t_cap: int) -> int:
+    return lib().slim_workspace_bytes(c_void_p(ctx), batch, t_cap)
+
+
+def slim_cache_create(ctx: int, k_storage, batch: int, t_cap: int) -> int:
+    h = c_void_p()
+    _check(lib().slim_cache_create(c_void_p(ctx), byref(h), _ptr(k_storage), batch, t_cap), "slim_cache_create")
+    return h.value
+
+
+def slim_cache_destroy(cache: int) -> None:
+    lib().slim_cache_destroy(c_void_p(cache))
+
+
+def slim_append_k(ctx: int, cache: int, k_new, positions, n_new: int, stream: int = 0) -> None:
+    _check(lib().slim_append_k(c_void_p(ctx), c_void_p(cache), _ptr(k_new), _ptr(positions), n_new,
+                               c_void_p(stream)), "slim_append_k")
+
+
+def slim_decode(ctx: int, q, cache: int, lengths, o, workspace, stream: int = 0) -> None:
+    _check(lib().slim_decode(c_void_p(ctx), _ptr(q), c_void_p(cache), _ptr(lengths), _ptr(o), _ptr(workspace),
+                             c_void_p(stream)), "slim_decode")
+
+
+def slim_device_status(ctx: int, stream: int = 0) -> int:
+    return lib().slim_device_status(c_void_p(ctx), c_void_p(stream))
+
+
+def slim_set_path(ctx: int, path: int) -> None:
+    _check(lib().slim_set_path(c_void_p(ctx), path), "slim_set_path")
+
+
+def slim_query(ctx: int, key: int) -> int:
+    return lib().slim_query(c_void_p(ctx), key)
+
+
+def slim_strerror(status: int) -> str:
+    return strerror(status)

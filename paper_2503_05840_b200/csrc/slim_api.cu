@@ -1,0 +1,325 @@
+// C-ABI entry points of libslim (argument checks, ownership, launch order).
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "slim_internal.h"
+
+size_t slim_tail_opart_floats(int d, int batch);
+
+namespace {
+
+inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+inline size_t esize(int dtype) { return dtype == SLIM_BF16 ? 2 : 4; }
+
+struct WsLayout {
+  size_t part_u, part_m, part_l, flags, o_part, total;
+  int units;
+};
+
+WsLayout ws_layout(const slim_ctx* ctx, int batch) {
+  WsLayout L;
+  L.units = ctx->num_sms + batch;
+  size_t off = 0;
+  L.part_u = off; off = align256(off + sizeof(float) * (size_t)L.units * ctx->H * ctx->d);
+  L.part_m = off; off = align256(off + sizeof(float) * (size_t)L.units * ctx->H);
+  L.part_l = off; off = align256(off + sizeof(float) * (size_t)L.units * ctx->H);
+  L.flags = off;  off = align256(off + sizeof(int) * (size_t)L.units);
+  L.o_part = off; off = align256(off + sizeof(float) * slim_tail_opart_floats(ctx->d, batch));
+  L.total = off;
+  return L;
+}
+
+int path_in_use(const slim_ctx* ctx) {
+  if (ctx->path_req == SLIM_PATH_GENERIC) return SLIM_PATH_GENERIC;
+  if (ctx->path_req == SLIM_PATH_TC) return ctx->tc_ok ? SLIM_PATH_TC : -1;
+  return ctx->tc_ok ? SLIM_PATH_TC : SLIM_PATH_GENERIC;
+}
+
+int min_tiles_for(const slim_ctx* ctx) {
+  int v = ctx->H / (2 * (int)esize(ctx->dtype));
+  return v < 2 ? 2 : v;
+}
+
+slim_status grow_rope_base(slim_ctx* ctx, int t_cap) {
+  if (ctx->rope_theta == 0.0) return SLIM_OK;
+  const int tiles = (t_cap + SLIM_TT - 1) / SLIM_TT + 1;
+  if (tiles <= ctx->rope_base_tiles) return SLIM_OK;
+  const int half = ctx->d_k / 2;
+  std::vector<float2> tab((size_t)tiles * half);
+  for (int j = 0; j < half; ++j) {
+    const double th = std::pow(ctx->rope_theta, -2.0 * j / ctx->d_k);
+    for (int t = 0; t < tiles; ++t) {
+      const double a = (double)t * SLIM_TT * th;
+      tab[(size_t)t * half + j] = make_float2((float)std::cos(a), (float)std::sin(a));
+    }
+  }
+  float2* dev = nullptr;
+  if (cudaMalloc(&dev, sizeof(float2) * tab.size()) != cudaSuccess) return SLIM_ERR_OOM;
+  if (cudaMemcpy(dev, tab.data(), sizeof(float2) * tab.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaFree(dev);
+    return SLIM_ERR_CUDA;
+  }
+  // the old table may still be referenced by enqueued work
+  cudaDeviceSynchronize();
+  cudaFree(ctx->rope_base);
+  ctx->rope_base = dev;
+  ctx->rope_base_tiles = tiles;
+  return SLIM_OK;
+}
+
+slim_status upload_f64(const void* src, int host_dtype, size_t n, double** dev_out) {
+  std::vector<double> tmp;
+  const double* h = nullptr;
+  if (host_dtype == SLIM_HOST_F64) {
+    h = static_cast<const double*>(src);
+  } else {
+    tmp.resize(n);
+    const float* f = static_cast<const float*>(src);
+    for (size_t i = 0; i < n; ++i) tmp[i] = (double)f[i];
+    h = tmp.data();
+  }
+  double* dev = nullptr;
+  if (cudaMalloc(&dev, sizeof(double) * n) != cudaSuccess) return SLIM_ERR_OOM;
+  if (cudaMemcpy(dev, h, sizeof(double) * n, cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaFree(dev);
+    return SLIM_ERR_CUDA;
+  }
+  *dev_out = dev;
+  return SLIM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* slim_strerror(int status) {
+  switch (status) {
+    case SLIM_OK: return "ok";
+    case SLIM_ERR_INVALID_ARG: return "invalid argument";
+    case SLIM_ERR_UNSUPPORTED: return "unsupported shape or option";
+    case SLIM_ERR_SINGULAR: return "W_K is singular to working precision";
+    case SLIM_ERR_CAPACITY: return "K-cache capacity exceeded";
+    case SLIM_ERR_OOM: return "out of device memory";
+    case SLIM_ERR_CUDA: return "CUDA error or no CUDA device";
+    case SLIM_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case SLIM_ERR_NO_WEIGHTS: return "W_KV has not been set";
+    default: return "unknown status";
+  }
+}
+
+slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta, int dtype) {
+  if (!out) return SLIM_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (d <= 0 || H <= 0 || d_k <= 0 || !(rope_theta >= 0.0) || (dtype != SLIM_F32 && dtype != SLIM_BF16))
+    return SLIM_ERR_INVALID_ARG;
+  if ((long long)H * d_k != d) return SLIM_ERR_UNSUPPORTED;       // Eq. 6 needs a square W_K
+  if (H > SLIM_MAX_H || d_k > 256 || (d_k & 1) || d > 16384 || (d % 8) != 0) return SLIM_ERR_UNSUPPORTED;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SLIM_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return SLIM_ERR_CUDA;
+  slim_ctx* c = new (std::nothrow) slim_ctx();
+  if (!c) return SLIM_ERR_OOM;
+  std::memset(c, 0, sizeof(*c));
+  c->d = d; c->H = H; c->d_k = d_k; c->dtype = dtype; c->rope_theta = rope_theta;
+  c->device = dev; c->num_sms = prop.multiProcessorCount;
+  c->path_req = SLIM_PATH_AUTO;
+  if (cudaMalloc(&c->status, sizeof(int)) != cudaSuccess) { delete c; return SLIM_ERR_OOM; }
+  cudaMemset(c->status, 0, sizeof(int));
+  if (cudaMalloc(&c->wkv, esize(dtype) * (size_t)d * d) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
+  if (rope_theta != 0.0) {
+    const int half = d_k / 2;
+    std::vector<float2> off((size_t)SLIM_TT * half);
+    for (int j = 0; j < half; ++j) {
+      const double th = std::pow(rope_theta, -2.0 * j / d_k);
+      for (int i = 0; i < SLIM_TT; ++i)
+        off[(size_t)i * half + j] = make_float2((float)std::cos(i * th), (float)std::sin(i * th));
+    }
+    if (cudaMalloc(&c->rope_off, sizeof(float2) * off.size()) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
+    if (cudaMemcpy(c->rope_off, off.data(), sizeof(float2) * off.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
+      slim_destroy(c);
+      return SLIM_ERR_CUDA;
+    }
+  }
+  c->tc_ok = prop.major == 10 ? slim_tc_shape_ok(d, H, d_k, dtype) : 0;
+  c->gen_workers = slim_generic_workers(c);
+  c->tc_workers = c->tc_ok ? slim_tc_workers(c) : 0;
+  if (c->tc_ok && c->tc_workers <= 0) c->tc_ok = 0;
+  *out = c;
+  return SLIM_OK;
+}
+
+void slim_destroy(slim_ctx* ctx) {
+  if (!ctx) return;
+  cudaFree(ctx->wkv);
+  cudaFree(ctx->rope_off);
+  cudaFree(ctx->rope_base);
+  cudaFree(ctx->status);
+  delete ctx;
+}
+
+slim_status slim_set_weights(slim_ctx* ctx, const void* W_K, const void* W_V, int host_dtype,
+                             double* wkv_out, double* residual_out) {
+  if (!ctx || !W_K || !W_V || (host_dtype != SLIM_HOST_F32 && host_dtype != SLIM_HOST_F64))
+    return SLIM_ERR_INVALID_ARG;
+  const int n = ctx->d;
+  const size_t nn = (size_t)n * n;
+  double *A = nullptr, *B = nullptr, *A0 = nullptr, *B0 = nullptr;
+  slim_status st = upload_f64(W_K, host_dtype, nn, &A);
+  if (st == SLIM_OK) st = upload_f64(W_V, host_dtype, nn, &B);
+  if (st == SLIM_OK && residual_out) {
+    if (cudaMalloc(&A0, sizeof(double) * nn) != cudaSuccess || cudaMalloc(&B0, sizeof(double) * nn) != cudaSuccess)
+      st = SLIM_ERR_OOM;
+    else if (cudaMemcpy(A0, A, sizeof(double) * nn, cudaMemcpyDeviceToDevice) != cudaSuccess ||
+             cudaMemcpy(B0, B, sizeof(double) * nn, cudaMemcpyDeviceToDevice) != cudaSuccess)
+      st = SLIM_ERR_CUDA;
+  }
+  int info = 0;
+  if (st == SLIM_OK) {
+    cudaError_t e = slim_wkv_solve(A, B, n, &info);
+    if (e == cudaErrorMemoryAllocation) st = SLIM_ERR_OOM;
+    else if (e != cudaSuccess) st = SLIM_ERR_CUDA;
+    else if (info != 0) st = SLIM_ERR_SINGULAR;
+  }
+  if (st == SLIM_OK && residual_out) {
+    if (slim_wkv_residual(A0, B, B0, n, residual_out) != cudaSuccess) st = SLIM_ERR_CUDA;
+  }
+  if (st == SLIM_OK && wkv_out) {
+    if (cudaMemcpy(wkv_out, B, sizeof(double) * nn, cudaMemcpyDeviceToHost) != cudaSuccess) st = SLIM_ERR_CUDA;
+  }
+  if (st == SLIM_OK) {
+    if (slim_wkv_store(B, ctx->d, ctx->H, ctx->d_k, ctx->dtype, ctx->wkv) != cudaSuccess ||
+        cudaDeviceSynchronize() != cudaSuccess)
+      st = SLIM_ERR_CUDA;
+    else
+      ctx->has_weights = 1;
+  }
+  cudaFree(A); cudaFree(B); cudaFree(A0); cudaFree(B0);
+  if (st != SLIM_OK) cudaGetLastError();
+  return st;
+}
+
+slim_status slim_set_wkv(slim_ctx* ctx, const void* W_KV, int host_dtype) {
+  if (!ctx || !W_KV || (host_dtype != SLIM_HOST_F32 && host_dtype != SLIM_HOST_F64)) return SLIM_ERR_INVALID_ARG;
+  double* X = nullptr;
+  slim_status st = upload_f64(W_KV, host_dtype, (size_t)ctx->d * ctx->d, &X);
+  if (st != SLIM_OK) return st;
+  if (slim_wkv_store(X, ctx->d, ctx->H, ctx->d_k, ctx->dtype, ctx->wkv) != cudaSuccess ||
+      cudaDeviceSynchronize() != cudaSuccess)
+    st = SLIM_ERR_CUDA;
+  else
+    ctx->has_weights = 1;
+  cudaFree(X);
+  return st;
+}
+
+size_t slim_cache_bytes(const slim_ctx* ctx, int batch, int t_cap) {
+  if (!ctx || batch <= 0 || t_cap <= 0) return 0;
+  return esize(ctx->dtype) * (size_t)batch * t_cap * ctx->d;
+}
+
+size_t slim_workspace_bytes(const slim_ctx* ctx, int batch, int t_cap) {
+  if (!ctx || batch <= 0 || t_cap <= 0 || batch > SLIM_MAX_BATCH) return 0;
+  return ws_layout(ctx, batch).total;
+}
+
+slim_status slim_cache_create(slim_ctx* ctx, slim_cache** out, void* k_storage, int batch, int t_cap) {
+  if (!out) return SLIM_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!ctx || !k_storage || batch <= 0 || t_cap <= 0) return SLIM_ERR_INVALID_ARG;
+  if (batch > SLIM_MAX_BATCH || ((uintptr_t)k_storage & 15)) return SLIM_ERR_UNSUPPORTED;
+  if ((long long)batch * t_cap > 0x7fffffffLL - 64) return SLIM_ERR_UNSUPPORTED;
+  slim_status st = grow_rope_base(ctx, t_cap);
+  if (st != SLIM_OK) return st;
+  slim_cache* c = new (std::nothrow) slim_cache();
+  if (!c) return SLIM_ERR_OOM;
+  c->ctx = ctx; c->k = k_storage; c->batch = batch; c->t_cap = t_cap; c->has_tmap = 0;
+  if (ctx->tc_ok) {
+    if (slim_tc_make_tmap(ctx, c) == cudaSuccess) c->has_tmap = 1;
+    else cudaGetLastError();
+  }
+  *out = c;
+  return SLIM_OK;
+}
+
+void slim_cache_destroy(slim_cache* cache) { delete cache; }
+
+slim_status slim_append_k(slim_ctx* ctx, slim_cache* cache, const void* k_new, const int32_t* positions,
+                          int n_new, void* stream) {
+  if (!ctx || !cache || !k_new || !positions || cache->ctx != ctx) return SLIM_ERR_INVALID_ARG;
+  if (n_new <= 0 || n_new > 65535) return SLIM_ERR_INVALID_ARG;
+  if (n_new > cache->t_cap) return SLIM_ERR_CAPACITY;
+  if (slim_launch_append(ctx, cache, k_new, positions, n_new, (cudaStream_t)stream) != cudaSuccess)
+    return SLIM_ERR_CUDA;
+  return SLIM_OK;
+}
+
+slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,
+                        float* o, void* workspace, void* stream) {
+  if (!ctx || !q || !cache || !lengths || !o || !workspace || cache->ctx != ctx) return SLIM_ERR_INVALID_ARG;
+  if (((uintptr_t)workspace & 255) || ((uintptr_t)q & 15) || ((uintptr_t)o & 15)) return SLIM_ERR_INVALID_ARG;
+  if (!ctx->has_weights) return SLIM_ERR_NO_WEIGHTS;
+  int path = path_in_use(ctx);
+  if (path < 0) return SLIM_ERR_UNSUPPORTED;
+  if (path == SLIM_PATH_TC && !cache->has_tmap) {
+    if (ctx->path_req == SLIM_PATH_TC) return SLIM_ERR_UNSUPPORTED;
+    path = SLIM_PATH_GENERIC;
+  }
+  const WsLayout L = ws_layout(ctx, cache->batch);
+  char* ws = static_cast<char*>(workspace);
+  SlimDecodeParams p;
+  p.d = ctx->d; p.H = ctx->H; p.d_k = ctx->d_k; p.half = ctx->d_k / 2;
+  p.batch = cache->batch; p.t_cap = cache->t_cap;
+  p.rope = ctx->rope_theta != 0.0; p.dtype = ctx->dtype;
+  p.workers = path == SLIM_PATH_TC ? ctx->tc_workers : ctx->gen_workers;
+  p.min_tiles = min_tiles_for(ctx);
+  p.qscale = (float)(1.4426950408889634 / std::sqrt((double)ctx->d_k));
+  p.q = q; p.k = cache->k; p.lengths = lengths;
+  p.rope_base = ctx->rope_base; p.rope_off = ctx->rope_off; p.wkv = ctx->wkv;
+  p.part_u = reinterpret_cast<float*>(ws + L.part_u);
+  p.part_m = reinterpret_cast<float*>(ws + L.part_m);
+  p.part_l = reinterpret_cast<float*>(ws + L.part_l);
+  p.unit_flags = reinterpret_cast<int*>(ws + L.flags);
+  p.u = reinterpret_cast<float*>(ws + L.o_part);
+  p.o = o; p.status = ctx->status;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = path == SLIM_PATH_TC ? slim_launch_tc(ctx, cache, p, st) : slim_launch_generic(ctx, p, st);
+  if (e == cudaSuccess) e = slim_launch_tail(ctx, p, st);
+  if (e != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
+  return SLIM_OK;
+}
+
+slim_status slim_device_status(slim_ctx* ctx, void* stream) {
+  if (!ctx) return SLIM_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
+  int v = 0;
+  if (cudaMemcpy(&v, ctx->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return SLIM_ERR_CUDA;
+  if (v != 0) cudaMemset(ctx->status, 0, sizeof(int));
+  return (slim_status)v;
+}
+
+slim_status slim_set_path(slim_ctx* ctx, int path) {
+  if (!ctx || path < SLIM_PATH_AUTO || path > SLIM_PATH_TC) return SLIM_ERR_INVALID_ARG;
+  if (path == SLIM_PATH_TC && !ctx->tc_ok) return SLIM_ERR_UNSUPPORTED;
+  ctx->path_req = path;
+  return SLIM_OK;
+}
+
+long long slim_query(const slim_ctx* ctx, int key) {
+  if (!ctx) return -1;
+  const int path = path_in_use(ctx);
+  switch (key) {
+    case SLIM_Q_PATH_IN_USE: return path;
+    case SLIM_Q_LAUNCHES_PER_DECODE: return path == SLIM_PATH_TC ? 4 : 3;
+    case SLIM_Q_MAX_UNITS: return ctx->num_sms;   // + batch, known only per cache
+    case SLIM_Q_NUM_SMS: return ctx->num_sms;
+    case SLIM_Q_WORKERS: return path == SLIM_PATH_TC ? ctx->tc_workers : ctx->gen_workers;
+    default: return -1;
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,224 @@
+// Generic CUDA-core decode kernel (any supported shape, f32 or bf16 cache).
+//
+// One CTA = (worker, d-slice).  For every context tile of its worker the CTA
+//   A. computes the softmax arguments of ALL heads for the tile rows
+//      (Eq. 2 with keys rotated after the read, RoPE appendix Option 1),
+//   B. updates the running max / sum per head (online softmax),
+//   C. accumulates U[h][col] += p[h][t] * K[t][col] for the columns it owns
+//      (Eq. 7 Option 2: weighted sum of the full-width raw keys),
+// and at the end of a unit writes the partial (m, l, U) for the combine.
+// CTAs of the same worker recompute step A redundantly (the key rows come
+// from L2 after the first touch); the tensor-core path removes that.
+#include "slim_internal.h"
+#include "slim_sched.cuh"
+
+namespace {
+
+__device__ __forceinline__ float ld_k(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float ld_k(const __nv_bfloat16* p) {
+  return __bfloat162float(__ldg(reinterpret_cast<const __nv_bfloat16*>(p)));
+}
+
+constexpr int GEN_THREADS = 256;
+
+template <typename KT, int HP, int COLS>
+__global__ void __launch_bounds__(GEN_THREADS)
+slim_generic_kernel(SlimDecodeParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* s_q = reinterpret_cast<float*>(smem_raw);                 // [d]
+  float* s_S = s_q + p.d;                                           // [HP][TT]
+  float* s_P = s_S + HP * SLIM_TT;                                  // [HP][TT]
+  float* s_alpha = s_P + HP * SLIM_TT;                              // [HP]
+  float* s_m = s_alpha + HP;                                        // [HP]
+  float* s_l = s_m + HP;                                            // [HP]
+  int* s_prefix = reinterpret_cast<int*>(s_l + HP);                 // [batch+1]
+
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int w = blockIdx.y;
+  const int col0 = blockIdx.x * (GEN_THREADS * COLS);
+  const KT* __restrict__ Kc = reinterpret_cast<const KT*>(p.k);
+  const KT* __restrict__ Q = reinterpret_cast<const KT*>(p.q);
+  const int d = p.d, H = p.H, dk = p.d_k, half = p.half;
+
+  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles,
+                                        s_prefix, p.status);
+  if (sc.total_tiles == 0 || w >= sc.workers_eff) return;
+  const int g_begin = slim_worker_start(sc, w), g_end = slim_worker_start(sc, w + 1);
+
+  float acc[HP][COLS];
+
+  int g = g_begin;
+  while (g < g_end) {
+    const int b = slim_seq_of_tile(s_prefix, p.batch, g);
+    const int seg_end = min(g_end, s_prefix[b + 1]);
+    const int tile0 = g - s_prefix[b], tile1 = seg_end - s_prefix[b];
+    const int unit = w + b;
+    int len = p.lengths[b];
+    len = min(max(len, 0), p.t_cap);
+
+    // ---- a2: rotate and scale the query of this sequence --------------------
+    __syncthreads();
+    {
+      const int m = len - 1, mt = m / SLIM_TT, mi = m % SLIM_TT;
+      for (int e = tid; e < d; e += GEN_THREADS) {
+        const int h = e / dk, jj = e - h * dk;
+        float v;
+        if (p.rope) {
+          const int j = jj < half ? jj : jj - half;
+          const float2 cb = p.rope_base[(size_t)mt * half + j], co = p.rope_off[mi * half + j];
+          const float c = cb.x * co.x - cb.y * co.y, s = cb.y * co.x + cb.x * co.y;
+          const float q1 = ld_k(Q + (size_t)b * d + h * dk + j);
+          const float q2 = ld_k(Q + (size_t)b * d + h * dk + j + half);
+          v = jj < half ? (q1 * c + q2 * s) : (-q1 * s + q2 * c);
+        } else {
+          v = ld_k(Q + (size_t)b * d + e);
+        }
+        s_q[e] = v * p.qscale;
+      }
+      if (tid < HP) { s_m[tid] = -INFINITY; s_l[tid] = 0.f; }
+#pragma unroll
+      for (int h = 0; h < HP; ++h)
+#pragma unroll
+        for (int c = 0; c < COLS; ++c) acc[h][c] = 0.f;
+    }
+    __syncthreads();
+
+    for (int tile = tile0; tile < tile1; ++tile) {
+      const int t0 = tile * SLIM_TT;
+      const KT* __restrict__ Kt = Kc + ((size_t)b * p.t_cap + t0) * d;
+
+      // ---- A: softmax arguments for all heads, rows of this tile ------------
+      for (int pi = wid; pi < H * SLIM_TT; pi += GEN_THREADS / 32) {
+        const int h = pi / SLIM_TT, t = pi - h * SLIM_TT;
+        float a = 0.f;
+        if (t0 + t < len) {
+          const KT* kr = Kt + (size_t)t * d + h * dk;
+          const float* qh = s_q + h * dk;
+          for (int j = lane; j < half; j += 32) {
+            const float k1 = ld_k(kr + j), k2 = ld_k(kr + j + half);
+            const float q1 = qh[j], q2 = qh[j + half];
+            if (p.rope) {
+              const float2 cb = p.rope_base[(size_t)tile * half + j], co = p.rope_off[t * half + j];
+              const float c = cb.x * co.x - cb.y * co.y, s = cb.y * co.x + cb.x * co.y;
+              a += c * (q1 * k1 + q2 * k2) + s * (q1 * k2 - q2 * k1);
+            } else {
+              a += q1 * k1 + q2 * k2;
+            }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        } else {
+          a = -INFINITY;
+        }
+        if (lane == 0) s_S[h * SLIM_TT + t] = a;
+      }
+      __syncthreads();
+
+      // ---- B: online softmax per head ---------------------------------------
+      for (int h = wid; h < H; h += GEN_THREADS / 32) {
+        const float s = lane < SLIM_TT ? s_S[h * SLIM_TT + lane] : -INFINITY;
+        float mx = s;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        const float m_old = s_m[h];
+        const float m_new = fmaxf(m_old, mx);
+        const float pr = (s == -INFINITY) ? 0.f : exp2f(s - m_new);
+        float ps = pr;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
+        const float alpha = exp2f(m_old - m_new);      // 0 on the first tile
+        if (lane < SLIM_TT) s_P[h * SLIM_TT + lane] = pr;
+        if (lane == 0) { s_alpha[h] = alpha; s_m[h] = m_new; s_l[h] = s_l[h] * alpha + ps; }
+      }
+      __syncthreads();
+
+      // ---- C: U[h][col] = alpha U[h][col] + sum_t p[h][t] K[t][col] ----------
+      float kv[COLS][SLIM_TT];
+#pragma unroll
+      for (int c = 0; c < COLS; ++c) {
+        const int col = col0 + tid + c * GEN_THREADS;
+#pragma unroll
+        for (int t = 0; t < SLIM_TT; ++t)
+          kv[c][t] = (col < d && t0 + t < len) ? ld_k(Kt + (size_t)t * d + col) : 0.f;
+      }
+#pragma unroll
+      for (int h = 0; h < HP; ++h) {
+        if (h < H) {
+          const float al = s_alpha[h];
+          const float4* P4 = reinterpret_cast<const float4*>(s_P + h * SLIM_TT);
+          float pv[SLIM_TT];
+#pragma unroll
+          for (int i = 0; i < SLIM_TT / 4; ++i) {
+            const float4 v = P4[i];
+            pv[4 * i] = v.x; pv[4 * i + 1] = v.y; pv[4 * i + 2] = v.z; pv[4 * i + 3] = v.w;
+          }
+#pragma unroll
+          for (int c = 0; c < COLS; ++c) {
+            float a = acc[h][c] * al;
+#pragma unroll
+            for (int t = 0; t < SLIM_TT; ++t) a = fmaf(pv[t], kv[c][t], a);
+            acc[h][c] = a;
+          }
+        }
+      }
+      __syncthreads();
+    }
+
+    // ---- partial of this unit -------------------------------------------------
+#pragma unroll
+    for (int h = 0; h < HP; ++h) {
+      if (h < H) {
+#pragma unroll
+        for (int c = 0; c < COLS; ++c) {
+          const int col = col0 + tid + c * GEN_THREADS;
+          if (col < d) p.part_u[((size_t)unit * H + h) * d + col] = acc[h][c];
+        }
+      }
+    }
+    if (blockIdx.x == 0 && tid < H) {
+      p.part_m[(size_t)unit * H + tid] = s_m[tid];
+      p.part_l[(size_t)unit * H + tid] = s_l[tid];
+    }
+    g = seg_end;
+  }
+}
+
+template <typename KT, int HP, int COLS>
+cudaError_t launch_one(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st) {
+  const int dsplit = (p.d + GEN_THREADS * COLS - 1) / (GEN_THREADS * COLS);
+  const size_t smem = sizeof(float) * (p.d + 2 * HP * SLIM_TT + 3 * HP) + sizeof(int) * (p.batch + 1);
+  auto kern = slim_generic_kernel<KT, HP, COLS>;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  dim3 grid(dsplit, p.workers);
+  kern<<<grid, GEN_THREADS, smem, st>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+// Columns per thread: 2 for H <= 32 (64 accumulators), 1 above.
+int slim_generic_dsplit(const slim_ctx* ctx) {
+  const int cols = ctx->H <= 32 ? 2 : 1;
+  return (ctx->d + GEN_THREADS * cols - 1) / (GEN_THREADS * cols);
+}
+
+int slim_generic_workers(const slim_ctx* ctx) {
+  // about two CTAs per SM in flight, shared between the d-slices of a worker
+  int w = (2 * ctx->num_sms) / slim_generic_dsplit(ctx);
+  if (w < 1) w = 1;
+  if (w > ctx->num_sms) w = ctx->num_sms;
+  return w;
+}
+
+cudaError_t slim_launch_generic(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st) {
+  const bool bf = p.dtype == SLIM_BF16;
+  if (p.H <= 8) {
+    return bf ? launch_one<__nv_bfloat16, 8, 2>(ctx, p, st) : launch_one<float, 8, 2>(ctx, p, st);
+  } else if (p.H <= 32) {
+    return bf ? launch_one<__nv_bfloat16, 32, 2>(ctx, p, st) : launch_one<float, 32, 2>(ctx, p, st);
+  }
+  return bf ? launch_one<__nv_bfloat16, 64, 1>(ctx, p, st) : launch_one<float, 64, 1>(ctx, p, st);
+}

@@ -1,0 +1,84 @@
+// Internal declarations shared by the translation units of libslim.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/slim.h"
+
+// Context tile: every kernel walks the context in tiles of SLIM_TT rows that
+// start at absolute positions that are multiples of SLIM_TT.  The RoPE base
+// table has one entry per tile and the offset table one per row of a tile.
+#define SLIM_TT 16
+#define SLIM_MAX_H 64
+#define SLIM_MAX_BATCH 4096
+
+// Parameters every decode kernel receives (passed by value).
+struct SlimDecodeParams {
+  int d, H, d_k, half;           // half = d_k / 2
+  int batch, t_cap;
+  int rope;                      // 0 / 1
+  int dtype;                     // slim_dtype
+  int workers;                   // context-split workers (W)
+  int min_tiles;                 // a worker gets at least this many tiles if it gets any
+  float qscale;                  // log2(e) / sqrt(d_k)
+  const void* q;                 // [batch][d]
+  const void* k;                 // [batch][t_cap][d]
+  const int32_t* lengths;        // [batch]
+  const float2* rope_base;       // [ceil(t_cap/TT)+1][half]  (cos, sin) of TT*tile*theta_j
+  const float2* rope_off;        // [TT][half]                (cos, sin) of i*theta_j
+  const void* wkv;               // [H][d][d_k] ctx dtype
+  float* part_u;                 // [units][H][d]
+  float* part_m;                 // [units][H]   reference exponent (log2 domain)
+  float* part_l;                 // [units][H]   sum of 2^(s - m)
+  int* unit_flags;               // [units]      1 = unit must be redone exactly
+  float* u;                      // [batch][H][d] combined
+  float* o;                      // [batch][d]
+  int* status;                   // sticky device status word
+};
+
+struct slim_ctx {
+  int d, H, d_k, dtype;
+  double rope_theta;
+  int device;
+  int num_sms;
+  int path_req;                  // slim_path requested
+  int has_weights;
+  void* wkv;                     // device [H][d][d_k] ctx dtype
+  float2* rope_off;              // device [TT][half]
+  float2* rope_base;             // device table, grown by slim_cache_create
+  int rope_base_tiles;
+  int* status;                   // device status word
+  int tc_ok;                     // shape fits the tensor-core path
+  int tc_workers;                // clusters the tensor-core kernel runs
+  int gen_workers;
+};
+
+struct slim_cache {
+  slim_ctx* ctx;
+  void* k;
+  int batch, t_cap;
+  alignas(64) unsigned char tmap[128];   // CUtensorMap for the tensor-core path
+  int has_tmap;
+};
+
+// ---- launchers implemented in the kernel translation units -----------------
+int  slim_generic_workers(const slim_ctx* ctx);
+int  slim_generic_dsplit(const slim_ctx* ctx);
+cudaError_t slim_launch_generic(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st);
+cudaError_t slim_launch_tail(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st);
+cudaError_t slim_launch_append(const slim_ctx* ctx, const slim_cache* c, const void* k_new,
+                               const int32_t* positions, int n_new, cudaStream_t st);
+// fp64 solve W_K X = W_V on the device; A and B are device row-major [n][n]
+// float64, both overwritten; X is returned in B.  info: 0 ok, 1 singular.
+cudaError_t slim_wkv_solve(double* A, double* B, int n, int* info_host);
+cudaError_t slim_wkv_residual(const double* Wk, const double* X, const double* Wv, int n, double* res_host);
+cudaError_t slim_wkv_store(const double* X, int d, int H, int d_k, int dtype, void* dst);
+
+// tensor-core path (slim_tc.cu)
+int  slim_tc_shape_ok(int d, int H, int d_k, int dtype);
+int  slim_tc_workers(const slim_ctx* ctx);
+cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c);
+cudaError_t slim_launch_tc(const slim_ctx* ctx, const slim_cache* c, const SlimDecodeParams& p, cudaStream_t st);

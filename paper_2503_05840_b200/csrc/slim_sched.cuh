@@ -1,0 +1,78 @@
+// Device-side work schedule shared by all decode kernels.
+//
+// The context of sequence b is cut into tiles of SLIM_TT rows.  All tiles of
+// the batch are laid end to end (sequence 0 first) and cut into W_eff equal
+// contiguous ranges, one per worker ("stream-K" over the ragged batch).  The
+// part of a worker's range that falls into one sequence is a *unit*: it
+// produces one partial (m, l, U[H][d]) for the log-sum-exp combine.  Because
+// (worker, sequence) pairs are monotone along the tile line, unit id =
+// worker + sequence is unique and < workers + batch.  The schedule is a pure
+// function of `lengths`, so every CTA (and the combine kernel) recomputes it
+// and the result is deterministic.
+#pragma once
+#include "slim_internal.h"
+
+struct SlimSched {
+  int total_tiles;   // NT
+  int workers_eff;   // W_eff <= workers
+};
+
+// Exclusive prefix of per-sequence tile counts into s_prefix[0..batch]
+// (shared memory, batch+1 ints).  Must be called by all threads of the CTA
+// (uses __syncthreads).  Lengths are clamped to [0, t_cap]; a length above
+// t_cap also raises SLIM_ERR_CAPACITY in *status.
+__device__ __forceinline__ SlimSched slim_sched_build(const int32_t* __restrict__ lengths, int batch,
+                                                      int t_cap, int workers, int min_tiles,
+                                                      int* s_prefix, int* status) {
+  const int tid = threadIdx.x + threadIdx.y * blockDim.x;
+  const int nthr = blockDim.x * blockDim.y;
+  for (int b = tid; b < batch; b += nthr) {
+    int len = lengths[b];
+    if (len > t_cap) { len = t_cap; atomicMax(status, (int)SLIM_ERR_CAPACITY); }
+    if (len < 0) len = 0;
+    s_prefix[b + 1] = (len + SLIM_TT - 1) / SLIM_TT;
+  }
+  if (tid == 0) s_prefix[0] = 0;
+  __syncthreads();
+  if (tid < 32) {
+    // warp 0: each lane scans a contiguous chunk, then the chunk sums are scanned.
+    const int chunk = (batch + 31) / 32;
+    const int lo = tid * chunk, hi = min(batch, lo + chunk);
+    int sum = 0;
+    for (int b = lo; b < hi; ++b) sum += s_prefix[b + 1];
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (tid >= o) incl += v;
+    }
+    int run = incl - sum;
+    for (int b = lo; b < hi; ++b) { run += s_prefix[b + 1]; s_prefix[b + 1] = run; }
+  }
+  __syncthreads();
+  SlimSched s;
+  s.total_tiles = s_prefix[batch];
+  int we = s.total_tiles / (min_tiles > 0 ? min_tiles : 1);
+  if (we < 1) we = 1;
+  s.workers_eff = we < workers ? we : workers;
+  return s;
+}
+
+__device__ __forceinline__ int slim_worker_start(const SlimSched& s, int w) {
+  return (int)(((long long)w * s.total_tiles) / s.workers_eff);
+}
+
+// Worker that owns global tile g (0 <= g < total_tiles).
+__device__ __forceinline__ int slim_worker_of_tile(const SlimSched& s, int g) {
+  return (int)((((long long)g + 1) * s.workers_eff - 1) / s.total_tiles);
+}
+
+// Sequence that owns global tile g: prefix[b] <= g < prefix[b+1].
+__device__ __forceinline__ int slim_seq_of_tile(const int* s_prefix, int batch, int g) {
+  int lo = 0, hi = batch;            // invariant: prefix[lo] <= g < prefix[hi]
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (s_prefix[mid] <= g) lo = mid; else hi = mid;
+  }
+  return lo;
+}

@@ -1,0 +1,189 @@
+// Tail of the decode step: log-sum-exp combine of the context-split partials
+// fused with the per-head projection o_h = u_h W_KV,h (Eq. 7 Option 2), and the
+// K-cache append.
+//
+//   tail1: CTA (head h, j-slice js).  For a tile of sequences it rebuilds
+//          u[b][h][j] = sum_s w_s U_s[h][j] / sum_s w_s l_s over the units of b
+//          (w_s = 2^(m_s - M)), keeps it in shared memory, and multiplies by
+//          W_KV[h][j][0..d_k): a partial sum over its j-slice, written to
+//          o_part[js][b][h*d_k + c].
+//   tail2: o[b][:] = sum_js o_part[js][b][:]   (fixed order => deterministic)
+#include "slim_internal.h"
+#include "slim_sched.cuh"
+
+namespace {
+
+constexpr int JR = 256;        // rows of W_KV,h (= columns of u) per tail1 CTA
+constexpr int BT_MAX = 32;     // sequences per pass
+constexpr int BPT = 8;         // sequences per thread
+
+__device__ __forceinline__ float ld_w(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float ld_w(const __nv_bfloat16* p) { return __bfloat162float(__ldg(p)); }
+
+template <typename WT>
+__global__ void __launch_bounds__(256) slim_tail1_kernel(SlimDecodeParams p, int bg_count, float* o_part) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* s_u = reinterpret_cast<float*>(smem_raw);              // [BT][JR]
+  float* s_wgt = s_u + BT_MAX * JR;                             // [BT][workers]
+  int* s_wlo = reinterpret_cast<int*>(s_wgt + BT_MAX * p.workers);   // [BT]
+  int* s_wn = s_wlo + BT_MAX;                                   // [BT]
+  int* s_prefix = s_wn + BT_MAX;                                // [batch+1]
+
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nwarp = blockDim.x >> 5;
+  const int h = blockIdx.x, js = blockIdx.y;
+  const int d = p.d, H = p.H, dk = p.d_k;
+  const int j0 = js * JR, jn = min(JR, d - j0);
+  const int BT = bg_count * BPT;
+  const WT* __restrict__ W = reinterpret_cast<const WT*>(p.wkv) + ((size_t)h * d + j0) * dk;
+
+  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles,
+                                        s_prefix, p.status);
+  const int c = tid % dk, bg = tid / dk;          // blockDim.x == dk * bg_count
+
+  for (int b0 = 0; b0 < p.batch; b0 += BT) {
+    const int nb = min(BT, p.batch - b0);
+    __syncthreads();
+    // ---- combine weights per sequence (one warp per sequence) ----------------
+    for (int bi = wid; bi < nb; bi += nwarp) {
+      const int b = b0 + bi;
+      const int g_lo = s_prefix[b], g_hi = s_prefix[b + 1];
+      int wlo = 0, wn = 0;
+      if (g_hi > g_lo) {
+        wlo = slim_worker_of_tile(sc, g_lo);
+        wn = slim_worker_of_tile(sc, g_hi - 1) - wlo + 1;
+        float M = -INFINITY;
+        for (int i = lane; i < wn; i += 32) {
+          const size_t ui = (size_t)(wlo + i + b) * H + h;
+          M = fmaxf(M, p.part_m[ui] + log2f(p.part_l[ui]));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        float L = 0.f;
+        for (int i = lane; i < wn; i += 32) {
+          const size_t ui = (size_t)(wlo + i + b) * H + h;
+          const float wg = exp2f(p.part_m[ui] - M);
+          s_wgt[bi * p.workers + i] = wg;
+          L += wg * p.part_l[ui];
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+        const float inv = 1.f / L;
+        __syncwarp();
+        for (int i = lane; i < wn; i += 32) s_wgt[bi * p.workers + i] *= inv;
+      }
+      if (lane == 0) { s_wlo[bi] = wlo; s_wn[bi] = wn; }
+    }
+    __syncthreads();
+    // ---- a7: u tile = weighted sum of the partials --------------------------
+    for (int e = tid; e < nb * JR; e += blockDim.x) {
+      const int bi = e / JR, j = e - bi * JR;
+      float v = 0.f;
+      if (j < jn) {
+        const int b = b0 + bi, wlo = s_wlo[bi], wn = s_wn[bi];
+        const float* wg = s_wgt + bi * p.workers;
+        for (int i = 0; i < wn; ++i)
+          v = fmaf(wg[i], __ldg(p.part_u + ((size_t)(wlo + i + b) * H + h) * d + j0 + j), v);
+      }
+      s_u[bi * JR + j] = v;
+    }
+    __syncthreads();
+    // ---- a8: partial projection over this j-slice ------------------------------
+    if (bg < bg_count) {
+      float acc[BPT];
+#pragma unroll
+      for (int i = 0; i < BPT; ++i) acc[i] = 0.f;
+      const float* ub = s_u + (bg * BPT) * JR;
+      int j = 0;
+      for (; j + 4 <= jn; j += 4) {
+        const float w0 = ld_w(W + (size_t)(j + 0) * dk + c), w1 = ld_w(W + (size_t)(j + 1) * dk + c);
+        const float w2 = ld_w(W + (size_t)(j + 2) * dk + c), w3 = ld_w(W + (size_t)(j + 3) * dk + c);
+#pragma unroll
+        for (int i = 0; i < BPT; ++i) {
+          const float4 uv = *reinterpret_cast<const float4*>(ub + i * JR + j);
+          acc[i] = fmaf(uv.x, w0, acc[i]); acc[i] = fmaf(uv.y, w1, acc[i]);
+          acc[i] = fmaf(uv.z, w2, acc[i]); acc[i] = fmaf(uv.w, w3, acc[i]);
+        }
+      }
+      for (; j < jn; ++j) {
+        const float w0 = ld_w(W + (size_t)j * dk + c);
+#pragma unroll
+        for (int i = 0; i < BPT; ++i) acc[i] = fmaf(ub[i * JR + j], w0, acc[i]);
+      }
+#pragma unroll
+      for (int i = 0; i < BPT; ++i) {
+        const int bi = bg * BPT + i;
+        if (bi < nb) o_part[((size_t)js * p.batch + b0 + bi) * d + h * dk + c] = acc[i];
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) slim_tail2_kernel(const float* __restrict__ o_part, float* __restrict__ o,
+                                                         int n, int nsplit) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  float a = 0.f;
+  for (int s = 0; s < nsplit; ++s) a += o_part[(size_t)s * n + i];
+  o[i] = a;
+}
+
+template <typename KT>
+__global__ void slim_append_kernel(KT* __restrict__ cache, const KT* __restrict__ k_new,
+                                   const int32_t* __restrict__ positions, int d, int t_cap, int n_new,
+                                   int* status) {
+  const int b = blockIdx.x, r = blockIdx.y;
+  const int pos = positions[b];
+  if (pos < 0 || pos + n_new > t_cap) {
+    if (threadIdx.x == 0) atomicMax(status, (int)SLIM_ERR_CAPACITY);
+    return;
+  }
+  const KT* src = k_new + ((size_t)b * n_new + r) * d;
+  KT* dst = cache + ((size_t)b * t_cap + pos + r) * d;
+  for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = src[e];
+}
+
+}  // namespace
+
+size_t slim_tail_opart_floats(int d, int batch) { return (size_t)((d + JR - 1) / JR) * batch * d; }
+
+cudaError_t slim_launch_tail(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st) {
+  const int nsplit = (p.d + JR - 1) / JR;
+  int bg_count = 256 / p.d_k;
+  if (bg_count < 1) bg_count = 1;
+  if (bg_count > BT_MAX / BPT) bg_count = BT_MAX / BPT;
+  const int threads = ((p.d_k * bg_count + 31) / 32) * 32;
+  // o_part lives behind u in the workspace
+  float* o_part = p.u;
+  const size_t smem = sizeof(float) * ((size_t)BT_MAX * JR + (size_t)BT_MAX * p.workers) +
+                      sizeof(int) * (2 * BT_MAX + p.batch + 1);
+  cudaError_t e;
+  dim3 grid(p.H, nsplit);
+  if (p.dtype == SLIM_BF16) {
+    auto kern = slim_tail1_kernel<__nv_bfloat16>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, threads, smem, st>>>(p, bg_count, o_part);
+  } else {
+    auto kern = slim_tail1_kernel<float>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, threads, smem, st>>>(p, bg_count, o_part);
+  }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const int n = p.batch * p.d;
+  slim_tail2_kernel<<<(n + 255) / 256, 256, 0, st>>>(o_part, p.o, n, nsplit);
+  return cudaGetLastError();
+}
+
+cudaError_t slim_launch_append(const slim_ctx* ctx, const slim_cache* c, const void* k_new,
+                               const int32_t* positions, int n_new, cudaStream_t st) {
+  dim3 grid(c->batch, n_new);
+  if (ctx->dtype == SLIM_BF16)
+    slim_append_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((__nv_bfloat16*)c->k, (const __nv_bfloat16*)k_new,
+                                                            positions, ctx->d, c->t_cap, n_new, ctx->status);
+  else
+    slim_append_kernel<float><<<grid, 256, 0, st>>>((float*)c->k, (const float*)k_new, positions, ctx->d,
+                                                    c->t_cap, n_new, ctx->status);
+  return cudaGetLastError();
+}

@@ -1,0 +1,314 @@
+// Eq. 6 on the device in float64:  solve W_K X = W_V  (X = W_KV) by blocked LU
+// with partial pivoting on the augmented matrix M = [W_K | W_V] (n x 2n),
+// followed by a blocked back substitution.  Offline set-up work; written for
+// clarity and a few seconds at n = 4096, not for peak FP64 rate.
+#include "slim_internal.h"
+
+namespace {
+
+constexpr int NB = 32;          // panel width
+
+// --- panel factorisation: columns [k0, k0+kb) of rows [k0, n) ---------------
+// One CTA.  Row swaps are applied to the panel columns only; piv[k0+j] records
+// the row exchanged with row k0+j.  info[0] = 1 if a pivot is too small.
+__global__ void __launch_bounds__(1024) lu_panel_kernel(double* __restrict__ M, int ld, int n, int k0, int kb,
+                                                        int* __restrict__ piv, int* info, double tiny) {
+  __shared__ double s_val[32];
+  __shared__ int s_idx[32];
+  __shared__ double s_row[NB];
+  __shared__ int s_p;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
+  for (int j = 0; j < kb; ++j) {
+    const int col = k0 + j;
+    // arg max |M[i][col]| over i >= col
+    double best = -1.0; int bi = col;
+    for (int i = col + tid; i < n; i += blockDim.x) {
+      const double v = fabs(M[(size_t)i * ld + col]);
+      if (v > best) { best = v; bi = i; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const double ov = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+    }
+    if (lane == 0) { s_val[wid] = best; s_idx[wid] = bi; }
+    __syncthreads();
+    if (wid == 0) {
+      best = lane < nw ? s_val[lane] : -1.0; bi = lane < nw ? s_idx[lane] : 0x7fffffff;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const double ov = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+      }
+      if (lane == 0) {
+        s_p = bi; piv[col] = bi;
+        if (!(best > tiny)) info[0] = 1;
+      }
+    }
+    __syncthreads();
+    const int prow = s_p;
+    // swap rows col <-> prow inside the panel, keep the pivot row in smem
+    if (tid < kb) {
+      const double a = M[(size_t)col * ld + k0 + tid], b = M[(size_t)prow * ld + k0 + tid];
+      M[(size_t)col * ld + k0 + tid] = b;
+      M[(size_t)prow * ld + k0 + tid] = a;
+      s_row[tid] = b;
+    }
+    __syncthreads();
+    const double pv = s_row[j];
+    const double rinv = (pv != 0.0) ? 1.0 / pv : 0.0;
+    for (int i = col + 1 + tid; i < n; i += blockDim.x) {
+      double* r = M + (size_t)i * ld + k0;
+      const double l = r[j] * rinv;
+      r[j] = l;
+      for (int jj = j + 1; jj < kb; ++jj) r[jj] -= l * s_row[jj];
+    }
+    __syncthreads();
+  }
+}
+
+// --- apply the panel's row exchanges to every column outside the panel --------
+__global__ void lu_swap_kernel(double* __restrict__ M, int ld, int ncols, int k0, int kb,
+                               const int* __restrict__ piv) {
+  int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= ncols - kb) return;
+  if (c >= k0) c += kb;                       // skip the panel columns
+  for (int j = 0; j < kb; ++j) {
+    const int r0 = k0 + j, r1 = piv[r0];
+    if (r1 != r0) {
+      const double a = M[(size_t)r0 * ld + c], b = M[(size_t)r1 * ld + c];
+      M[(size_t)r0 * ld + c] = b; M[(size_t)r1 * ld + c] = a;
+    }
+  }
+}
+
+// --- U12 = L11^{-1} A12 (unit lower), one thread per column -----------------
+__global__ void lu_trsm_lower_kernel(double* __restrict__ M, int ld, int ncols, int k0, int kb) {
+  __shared__ double s_L[NB][NB + 1];
+  for (int e = threadIdx.x; e < kb * kb; e += blockDim.x)
+    s_L[e / kb][e % kb] = M[(size_t)(k0 + e / kb) * ld + k0 + e % kb];
+  __syncthreads();
+  const int c = k0 + kb + blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= ncols) return;
+  double x[NB];
+#pragma unroll
+  for (int r = 0; r < NB; ++r) {
+    if (r < kb) {
+      double v = M[(size_t)(k0 + r) * ld + c];
+#pragma unroll
+      for (int s = 0; s < NB; ++s) if (s < r) v -= s_L[r][s] * x[s];
+      x[r] = v;
+      M[(size_t)(k0 + r) * ld + c] = v;
+    }
+  }
+}
+
+// --- C[r0:r1, c0:c1] -= A[r0:r1, k0:k0+kb] * B[k0:k0+kb, c0:c1]   (all inside M)
+// 64x64 tile per CTA, 16x16 threads, 4x4 outputs per thread.
+__global__ void __launch_bounds__(256) lu_gemm_kernel(double* __restrict__ M, int ld, int r0, int r1, int c0, int c1,
+                                                      int k0, int kb) {
+  __shared__ double s_A[64][NB + 1];
+  __shared__ double s_B[NB][64 + 1];
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int rb = r0 + blockIdx.y * 64, cb = c0 + blockIdx.x * 64;
+  for (int e = threadIdx.x; e < 64 * NB; e += 256) {
+    const int r = e / NB, k = e % NB;
+    s_A[r][k] = (rb + r < r1 && k < kb) ? M[(size_t)(rb + r) * ld + k0 + k] : 0.0;
+  }
+  for (int e = threadIdx.x; e < NB * 64; e += 256) {
+    const int k = e / 64, c = e % 64;
+    s_B[k][c] = (cb + c < c1 && k < kb) ? M[(size_t)(k0 + k) * ld + cb + c] : 0.0;
+  }
+  __syncthreads();
+  double acc[4][4] = {};
+#pragma unroll 8
+  for (int k = 0; k < NB; ++k) {
+    double a[4], b[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { a[i] = s_A[ty + 16 * i][k]; b[i] = s_B[k][tx + 16 * i]; }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int r = rb + ty + 16 * i, c = cb + tx + 16 * j;
+      if (r < r1 && c < c1) M[(size_t)r * ld + c] -= acc[i][j];
+    }
+}
+
+// --- X[k0:k0+kb, :] = U11^{-1} Y[k0:k0+kb, :] (upper, non-unit), thread per column of the right half
+__global__ void lu_trsm_upper_kernel(double* __restrict__ M, int ld, int n, int k0, int kb) {
+  __shared__ double s_U[NB][NB + 1];
+  for (int e = threadIdx.x; e < kb * kb; e += blockDim.x)
+    s_U[e / kb][e % kb] = M[(size_t)(k0 + e / kb) * ld + k0 + e % kb];
+  __syncthreads();
+  const int c = n + blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= 2 * n) return;
+  double x[NB];
+#pragma unroll
+  for (int rr = 0; rr < NB; ++rr) {
+    const int r = NB - 1 - rr;
+    if (r < kb) {
+      double v = M[(size_t)(k0 + r) * ld + c];
+#pragma unroll
+      for (int s = 0; s < NB; ++s) if (s > r && s < kb) v -= s_U[r][s] * x[s];
+      v /= s_U[r][r];
+      x[r] = v;
+      M[(size_t)(k0 + r) * ld + c] = v;
+    }
+  }
+}
+
+__global__ void pack_aug_kernel(const double* __restrict__ A, const double* __restrict__ B, double* __restrict__ M, int n) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (size_t)n * n) return;
+  const size_t r = i / n, c = i % n;
+  M[r * 2 * n + c] = A[i];
+  M[r * 2 * n + n + c] = B[i];
+}
+
+__global__ void unpack_x_kernel(const double* __restrict__ M, double* __restrict__ X, int n) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (size_t)n * n) return;
+  const size_t r = i / n, c = i % n;
+  X[i] = M[r * 2 * n + n + c];
+}
+
+__global__ void absmax_kernel(const double* __restrict__ A, size_t n, double* out) {
+  double m = 0.0;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    m = fmax(m, fabs(A[i]));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0)   // non-negative doubles order like their bit patterns
+    atomicMax(reinterpret_cast<unsigned long long*>(out), (unsigned long long)__double_as_longlong(m));
+}
+
+// residual: max | Wk X - Wv |, 64x64 tiles
+__global__ void __launch_bounds__(256) residual_kernel(const double* __restrict__ Wk, const double* __restrict__ X,
+                                                       const double* __restrict__ Wv, int n, double* out) {
+  __shared__ double s_A[64][NB + 1];
+  __shared__ double s_B[NB][64 + 1];
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int rb = blockIdx.y * 64, cb = blockIdx.x * 64;
+  double acc[4][4] = {};
+  for (int k0 = 0; k0 < n; k0 += NB) {
+    for (int e = threadIdx.x; e < 64 * NB; e += 256) {
+      const int r = e / NB, k = e % NB;
+      s_A[r][k] = (rb + r < n && k0 + k < n) ? Wk[(size_t)(rb + r) * n + k0 + k] : 0.0;
+    }
+    for (int e = threadIdx.x; e < NB * 64; e += 256) {
+      const int k = e / 64, c = e % 64;
+      s_B[k][c] = (cb + c < n && k0 + k < n) ? X[(size_t)(k0 + k) * n + cb + c] : 0.0;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int k = 0; k < NB; ++k) {
+      double a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { a[i] = s_A[ty + 16 * i][k]; b[i] = s_B[k][tx + 16 * i]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  double m = 0.0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int r = rb + ty + 16 * i, c = cb + tx + 16 * j;
+      if (r < n && c < n) m = fmax(m, fabs(acc[i][j] - Wv[(size_t)r * n + c]));
+    }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0)
+    atomicMax(reinterpret_cast<unsigned long long*>(out), (unsigned long long)__double_as_longlong(m));
+}
+
+template <typename WT>
+__global__ void store_wkv_kernel(const double* __restrict__ X, WT* __restrict__ dst, int d, int H, int dk) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (size_t)d * d) return;
+  const int c = (int)(i % dk);
+  const size_t rest = i / dk;
+  const int j = (int)(rest % d), h = (int)(rest / d);
+  const double v = X[(size_t)j * d + h * dk + c];
+  if constexpr (sizeof(WT) == 2) dst[i] = __double2bfloat16(v); else dst[i] = (float)v;
+}
+
+#define CK(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) { cudaFree(M); cudaFree(piv); cudaFree(scal); return e_; } } while (0)
+
+}  // namespace
+
+cudaError_t slim_wkv_solve(double* A, double* B, int n, int* info_host) {
+  double* M = nullptr; int* piv = nullptr; double* scal = nullptr;   // scal: [0] = max|A| bits, [1] = info
+  const int ld = 2 * n;
+  CK(cudaMalloc(&M, sizeof(double) * (size_t)n * ld));
+  CK(cudaMalloc(&piv, sizeof(int) * n));
+  CK(cudaMalloc(&scal, 16));
+  CK(cudaMemset(scal, 0, 16));
+  const size_t nn = (size_t)n * n;
+  pack_aug_kernel<<<(unsigned)((nn + 255) / 256), 256>>>(A, B, M, n);
+  absmax_kernel<<<256, 256>>>(A, nn, scal);
+  double amax = 0.0;
+  CK(cudaMemcpy(&amax, scal, sizeof(double), cudaMemcpyDeviceToHost));
+  const double tiny = 1e-13 * amax * n;
+  int* info = reinterpret_cast<int*>(scal + 1);
+  for (int k0 = 0; k0 < n; k0 += NB) {
+    const int kb = (n - k0 < NB) ? n - k0 : NB;
+    lu_panel_kernel<<<1, 1024>>>(M, ld, n, k0, kb, piv, info, tiny);
+    lu_swap_kernel<<<(ld - kb + 255) / 256, 256>>>(M, ld, ld, k0, kb, piv);
+    const int rest_c = ld - (k0 + kb);
+    lu_trsm_lower_kernel<<<(rest_c + 127) / 128, 128>>>(M, ld, ld, k0, kb);
+    const int rest_r = n - (k0 + kb);
+    if (rest_r > 0) {
+      dim3 g((rest_c + 63) / 64, (rest_r + 63) / 64);
+      lu_gemm_kernel<<<g, 256>>>(M, ld, k0 + kb, n, k0 + kb, ld, k0, kb);
+    }
+  }
+  // back substitution on the right half: U X = Y
+  const int nblk = (n + NB - 1) / NB;
+  for (int blk = nblk - 1; blk >= 0; --blk) {
+    const int k0 = blk * NB, kb = (n - k0 < NB) ? n - k0 : NB;
+    lu_trsm_upper_kernel<<<(n + 127) / 128, 128>>>(M, ld, n, k0, kb);
+    if (k0 > 0) {
+      dim3 g((n + 63) / 64, (k0 + 63) / 64);
+      lu_gemm_kernel<<<g, 256>>>(M, ld, 0, k0, n, ld, k0, kb);
+    }
+  }
+  unpack_x_kernel<<<(unsigned)((nn + 255) / 256), 256>>>(M, B, n);
+  CK(cudaGetLastError());
+  CK(cudaMemcpy(info_host, info, sizeof(int), cudaMemcpyDeviceToHost));
+  cudaFree(M); cudaFree(piv); cudaFree(scal);
+  return cudaSuccess;
+}
+
+cudaError_t slim_wkv_residual(const double* Wk, const double* X, const double* Wv, int n, double* res_host) {
+  double* out = nullptr;
+  cudaError_t e = cudaMalloc(&out, sizeof(double));
+  if (e != cudaSuccess) return e;
+  cudaMemset(out, 0, sizeof(double));
+  dim3 g((n + 63) / 64, (n + 63) / 64);
+  residual_kernel<<<g, 256>>>(Wk, X, Wv, n, out);
+  e = cudaMemcpy(res_host, out, sizeof(double), cudaMemcpyDeviceToHost);
+  cudaFree(out);
+  return e;
+}
+
+cudaError_t slim_wkv_store(const double* X, int d, int H, int d_k, int dtype, void* dst) {
+  const size_t nn = (size_t)d * d;
+  if (dtype == SLIM_BF16)
+    store_wkv_kernel<__nv_bfloat16><<<(unsigned)((nn + 255) / 256), 256>>>(X, (__nv_bfloat16*)dst, d, H, d_k);
+  else
+    store_wkv_kernel<float><<<(unsigned)((nn + 255) / 256), 256>>>(X, (float*)dst, d, H, d_k);
+  return cudaGetLastError();
+}

@@ -164,3 +164,40 @@ def kcache_bytes_per_step(cfg: SlimConfig, lengths: np.ndarray) -> int:
     sizeof(dtype)  (the 'n d reads' of Table 2, per layer and sequence)."""
     size = 2 if cfg.dtype == "bf16" else 4
     return int(cfg.layers) * int(np.sum(lengths, dtype=np.int64)) * cfg.d * size
+
+
+# ---------------------------------------------------------------- device-side drawing (full-size configs)
+def make_weights_torch(d: int, seed: int, device):
+    """Same recipe as make_weights, drawn and factorised on `device` in float64
+    (used where the host QR of a 4096 x 4096 matrix per layer would dominate
+    set-up).  Returns (W_Q, W_K, W_V, Qorth, s) as float64 tensors."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    G = torch.randn((d, d), generator=g, dtype=torch.float64, device=device)
+    Qo, R = torch.linalg.qr(G)
+    Qo = Qo * torch.sign(torch.diagonal(R))[None, :]
+    s = torch.rand(d, generator=g, dtype=torch.float64, device=device) * 1.5 + 0.5
+    W_K = Qo * s[None, :]
+    W_V = torch.randn((d, d), generator=g, dtype=torch.float64, device=device) / d ** 0.5
+    W_Q = torch.randn((d, d), generator=g, dtype=torch.float64, device=device) / d ** 0.5
+    return W_Q, W_K, W_V, Qo, s
+
+
+def fill_layer_torch(cfg: SlimConfig, seed: int, W_Q, W_K, lengths, k_out, q_out) -> None:
+    """Draw X per sequence on the device, write K = X W_K (rounded to the cache
+    dtype) into k_out[b, :len_b] and q = x_n W_Q into q_out[b].  Rows beyond
+    len_b are left as they are."""
+    import torch
+    g = torch.Generator(device=k_out.device)
+    g.manual_seed(seed + 7)
+    for b in range(cfg.batch):
+        n = int(lengths[b])
+        if n == 0:
+            continue
+        X = torch.randn((n, cfg.d), generator=g, dtype=torch.float64, device=k_out.device)
+        if cfg.rmsnorm_x:
+            X = X / torch.sqrt(torch.mean(X * X, dim=1, keepdim=True))
+        k_out[b, :n] = (X @ W_K).to(k_out.dtype)
+        q_out[b] = (X[-1] @ W_Q).to(q_out.dtype)
+        del X

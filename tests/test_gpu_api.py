@@ -1,0 +1,247 @@
+"""GPU tests of the boundary: set_weights against the oracle, append, error
+statuses, and properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import slim_oracle as so
+from paper_2503_05840_b200 import binding as B
+from paper_2503_05840_b200 import synth
+from paper_2503_05840_b200.layer import SlimLayer, to_device_keys
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.mark.parametrize("d,H", [(32, 2), (96, 3), (384, 6), (1000, 10), (1280, 20)])
+def test_set_weights_matches_oracle_and_closed_form(d, H):
+    W_Q, W_K, W_V, Qo, s = synth.make_weights(d, 77 + d)
+    layer = SlimLayer(d, H, d // H, 0.0, "f32", 1, 16, DEV)
+    try:
+        res, wkv = layer.set_weights(W_K, W_V, want_wkv=True)
+        ref = so.oracle_wkv(W_K, W_V)
+        closed = (Qo.T @ W_V) / s[:, None]
+        assert np.allclose(wkv, ref, rtol=1e-9, atol=1e-11)
+        assert np.allclose(wkv, closed, rtol=1e-9, atol=1e-11)
+        assert res <= 1e-12 * d
+        assert np.allclose(W_K @ wkv, W_V)          # the appendix-A check
+        # float32 host weights are accepted too
+        res32, wkv32 = layer.set_weights(W_K.astype(np.float32), W_V.astype(np.float32), want_wkv=True)
+        ref32 = so.oracle_wkv(W_K.astype(np.float32).astype(np.float64), W_V.astype(np.float32).astype(np.float64))
+        assert np.allclose(wkv32, ref32, rtol=1e-8, atol=1e-10)
+    finally:
+        layer.close()
+
+
+def test_set_weights_general_matrix_with_pivoting():
+    g = np.random.default_rng(5)
+    d = 200
+    W_K = g.standard_normal((d, d))
+    W_K[0, 0] = 0.0                       # forces a row exchange at the first step
+    W_V = g.standard_normal((d, d))
+    layer = SlimLayer(d, 4, d // 4, 0.0, "f32", 1, 16, DEV)
+    try:
+        res, wkv = layer.set_weights(W_K, W_V, want_wkv=True)
+        ref = so.oracle_wkv(W_K, W_V)
+        assert np.max(np.abs(wkv - ref)) <= 1e-8 * np.max(np.abs(ref))
+    finally:
+        layer.close()
+
+
+def test_singular_w_k_is_reported():
+    d = 64
+    W_K = np.ones((d, d))
+    layer = SlimLayer(d, 2, 32, 0.0, "f32", 1, 16, DEV)
+    try:
+        with pytest.raises(B.SlimError) as ei:
+            layer.set_weights(W_K, np.eye(d))
+        assert ei.value.status == B.SLIM_ERR_SINGULAR
+        q = torch.zeros((1, d), device=DEV)
+        with pytest.raises(B.SlimError) as ei:
+            layer.decode(q, torch.ones(1, dtype=torch.int32, device=DEV))
+        assert ei.value.status == B.SLIM_ERR_NO_WEIGHTS
+    finally:
+        layer.close()
+
+
+def test_set_wkv_equals_set_weights():
+    cfg = synth.SlimConfig("x", 256, 4, 64, 2, 64, 1, 1.0e4, "bf16")
+    L = synth.make_layer(cfg, 31)
+    outs = []
+    for mode in ("solve", "direct"):
+        layer = SlimLayer(cfg.d, cfg.H, cfg.d_k, cfg.rope_theta, cfg.dtype, cfg.batch, cfg.context, DEV)
+        try:
+            layer.k.copy_(to_device_keys(L.K, cfg.dtype, DEV))
+            if mode == "solve":
+                layer.set_weights(L.W_K, L.W_V)
+            else:
+                layer.set_wkv(so.oracle_wkv(L.W_K, L.W_V))
+            q = to_device_keys(L.q, cfg.dtype, DEV)
+            outs.append(layer.decode(q, torch.from_numpy(L.lengths).to(DEV)).cpu().numpy())
+        finally:
+            layer.close()
+    assert np.allclose(outs[0], outs[1], rtol=1e-5, atol=1e-6)
+
+
+@pytest.mark.parametrize("dtype,theta", [("f32", 0.0), ("bf16", 1.0e4)])
+def test_append_then_decode_equals_prefilled_cache(dtype, theta):
+    cfg = synth.SlimConfig("app", 256, 4, 64, 3, 80, 1, theta, dtype)
+    lengths = np.array([80, 37, 5], dtype=np.int32)
+    L = synth.make_layer(cfg, 555, lengths=lengths)
+    W_KV = so.oracle_wkv(L.W_K, L.W_V)
+    a = SlimLayer(cfg.d, cfg.H, cfg.d_k, theta, dtype, cfg.batch, cfg.context, DEV)
+    b = SlimLayer(cfg.d, cfg.H, cfg.d_k, theta, dtype, cfg.batch, cfg.context, DEV)
+    try:
+        Kd = to_device_keys(L.K, dtype, DEV)
+        a.k.copy_(Kd)
+        a.set_wkv(W_KV); b.set_wkv(W_KV)
+        # b: feed the keys through slim_append_k, first a bulk of len-3 rows, then three single rows
+        pos = torch.zeros(3, dtype=torch.int32, device=DEV)
+        bulk = int(lengths.min()) - 3
+        b.append_k(Kd[:, :bulk].contiguous(), pos)
+        cur = np.full(3, bulk, dtype=np.int32)
+        while np.any(cur < lengths):
+            step = torch.zeros((3, 1, cfg.d), dtype=Kd.dtype, device=DEV)
+            posd = torch.from_numpy(np.minimum(cur, lengths - 1).astype(np.int32)).to(DEV)
+            for i in range(3):
+                step[i, 0] = Kd[i, min(cur[i], lengths[i] - 1)]
+            b.append_k(step, posd)
+            cur = np.minimum(cur + 1, lengths)
+        assert b.device_status() == B.SLIM_OK
+        for i in range(3):
+            assert torch.equal(b.k[i, :lengths[i]], a.k[i, :lengths[i]])
+        q = to_device_keys(L.q, dtype, DEV)
+        ld = torch.from_numpy(lengths).to(DEV)
+        oa = a.decode(q, ld).clone()
+        ob = b.decode(q, ld).clone()
+        assert torch.equal(oa, ob)
+    finally:
+        a.close(); b.close()
+
+
+def test_append_beyond_capacity_sets_status_and_writes_nothing():
+    layer = SlimLayer(64, 2, 32, 0.0, "f32", 2, 8, DEV)
+    try:
+        layer.k.fill_(7.0)
+        k_new = torch.ones((2, 2, 64), device=DEV)
+        layer.append_k(k_new, torch.tensor([7, 0], dtype=torch.int32, device=DEV))   # seq 0: rows 7,8 -> overflow
+        assert layer.device_status() == B.SLIM_ERR_CAPACITY
+        assert layer.device_status() == B.SLIM_OK            # status is cleared by the read
+        assert torch.all(layer.k[0] == 7.0)
+        assert torch.all(layer.k[1, :2] == 1.0) and torch.all(layer.k[1, 2:] == 7.0)
+    finally:
+        layer.close()
+
+
+def test_length_beyond_capacity_is_clamped_and_reported():
+    cfg = synth.SlimConfig("cap", 128, 2, 64, 1, 40, 1, 0.0, "f32")
+    L = synth.make_layer(cfg, 3)
+    layer = SlimLayer(cfg.d, cfg.H, cfg.d_k, 0.0, "f32", 1, 40, DEV)
+    try:
+        layer.k.copy_(to_device_keys(L.K, "f32", DEV))
+        layer.set_weights(L.W_K, L.W_V)
+        q = to_device_keys(L.q, "f32", DEV)
+        good = layer.decode(q, torch.tensor([40], dtype=torch.int32, device=DEV)).clone()
+        assert layer.device_status() == B.SLIM_OK
+        got = layer.decode(q, torch.tensor([41], dtype=torch.int32, device=DEV)).clone()
+        assert layer.device_status() == B.SLIM_ERR_CAPACITY
+        assert torch.equal(got, good)
+    finally:
+        layer.close()
+
+
+def _paths(layer):
+    paths = [B.SLIM_PATH_GENERIC]
+    try:
+        layer.set_path(B.SLIM_PATH_TC); paths.append(B.SLIM_PATH_TC)
+    except B.SlimError:
+        pass
+    layer.set_path(B.SLIM_PATH_AUTO)
+    return paths
+
+
+def test_poisoned_rows_beyond_length_do_not_leak_and_runs_are_bitwise_repeatable():
+    cfg = synth.SlimConfig("poison", 1024, 8, 128, 4, 700, 1, 1.0e6, "bf16")
+    lengths = np.array([700, 333, 17, 640], dtype=np.int32)
+    L = synth.make_layer(cfg, 42, lengths=lengths)
+    layer = SlimLayer(cfg.d, cfg.H, cfg.d_k, cfg.rope_theta, "bf16", cfg.batch, cfg.context, DEV)
+    try:
+        Kd = to_device_keys(L.K, "bf16", DEV)
+        layer.set_weights(L.W_K, L.W_V)
+        q = to_device_keys(L.q, "bf16", DEV)
+        ld = torch.from_numpy(lengths).to(DEV)
+        for path in _paths(layer):
+            layer.set_path(path)
+            layer.k.copy_(Kd)
+            clean = layer.decode(q, ld).clone()
+            for b in range(4):
+                layer.k[b, lengths[b]:] = float("nan")
+            nan_run = layer.decode(q, ld).clone()
+            for b in range(4):
+                layer.k[b, lengths[b]:] = float("inf")
+            inf_run = layer.decode(q, ld).clone()
+            assert torch.equal(clean, nan_run), f"path {path}"
+            assert torch.equal(clean, inf_run), f"path {path}"
+            again = layer.decode(q, ld).clone()
+            assert torch.equal(inf_run, again)
+    finally:
+        layer.close()
+
+
+def test_row_permutation_invariance_without_rope_and_identical_keys():
+    cfg = synth.SlimConfig("perm", 1280, 20, 64, 2, 1500, 1, 0.0, "bf16")
+    L = synth.make_layer(cfg, 8)
+    layer = SlimLayer(cfg.d, cfg.H, cfg.d_k, 0.0, "bf16", cfg.batch, cfg.context, DEV)
+    try:
+        Kd = to_device_keys(L.K, "bf16", DEV)
+        W_KV = so.oracle_wkv(L.W_K, L.W_V)
+        layer.set_wkv(W_KV)
+        q = to_device_keys(L.q, "bf16", DEV)
+        ld = torch.from_numpy(L.lengths).to(DEV)
+        g = torch.Generator(device="cpu"); g.manual_seed(0)
+        perm = torch.randperm(1500, generator=g).to(DEV)
+        for path in _paths(layer):
+            layer.set_path(path)
+            layer.k.copy_(Kd)
+            base = layer.decode(q, ld).clone()
+            layer.k.copy_(Kd[:, perm])
+            shuffled = layer.decode(q, ld).clone()
+            rms = base.pow(2).mean().sqrt()
+            assert (base - shuffled).abs().max() <= 2e-3 * rms
+            # all keys identical: the output is that key's value row, whatever q is
+            layer.k.copy_(Kd[:, :1].expand(-1, 1500, -1))
+            same = layer.decode(q, ld).cpu().numpy().astype(np.float64)
+            for b in range(2):
+                v = L.K[b, 0].astype(np.float64) @ W_KV
+                assert so.err_rms_norm(same[b], v) <= 2e-2
+    finally:
+        layer.close()
+
+
+def test_scores_far_above_the_first_tile_are_handled():
+    # later keys score much higher than the first tile's: exercises the
+    # reference-exponent handling of every path (and its exact redo, if any).
+    cfg = synth.SlimConfig("ramp", 512, 4, 128, 2, 400, 1, 0.0, "bf16")
+    L = synth.make_layer(cfg, 77)
+    K = L.K.copy()
+    q = L.q.copy()
+    for b in range(2):
+        qn = q[b] / np.linalg.norm(q[b])
+        ramp = np.linspace(0.0, 60.0 if b == 0 else 400.0, 400)[:, None]
+        K[b] = synth.round_to_bf16(K[b] + ramp * qn[None, :] * 8.0)
+    layer = SlimLayer(cfg.d, cfg.H, cfg.d_k, 0.0, "bf16", cfg.batch, cfg.context, DEV)
+    try:
+        W_KV = so.oracle_wkv(L.W_K, L.W_V)
+        layer.set_wkv(W_KV)
+        layer.k.copy_(to_device_keys(K, "bf16", DEV))
+        qd = to_device_keys(q, "bf16", DEV)
+        ld = torch.from_numpy(L.lengths).to(DEV)
+        ref = so.oracle_slim_batch(q, K, L.lengths, W_KV, cfg.H, 0.0)
+        for path in _paths(layer):
+            layer.set_path(path)
+            got = layer.decode(qd, ld).cpu().numpy().astype(np.float64)
+            assert layer.device_status() == B.SLIM_OK
+            for b in range(2):
+                assert so.err_rms_norm(got[b], ref[b]) <= 2e-2, f"path {path} seq {b}"
+    finally:
+        layer.close()

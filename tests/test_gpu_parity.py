@@ -1,0 +1,156 @@
+"""GPU parity: the CUDA library (through the C ABI) against the CPU fp64 oracle
+on the same seeded inputs.  Tolerances (from the benchmark spec):
+  f32 cache : max_i |err_i| / max(|ref_i|, RMS(ref)) <= 1e-4 per sequence
+  bf16 cache: max_i |err_i| / RMS(ref) <= 2e-2 per sequence, oracle run on the
+              same bf16-rounded K and q, with unrounded float64 W_KV."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import slim_oracle as so
+from paper_2503_05840_b200 import binding as B
+from paper_2503_05840_b200 import synth
+from paper_2503_05840_b200.layer import SlimLayer, to_device_keys
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}
+DEV = "cuda:0"
+
+
+def _err(got, ref, dtype):
+    return so.err_fp32_norm(got, ref) if dtype == "f32" else so.err_rms_norm(got, ref)
+
+
+def _paths(layer):
+    """Kernel paths available for this shape on this device."""
+    paths = [B.SLIM_PATH_GENERIC]
+    try:
+        layer.set_path(B.SLIM_PATH_TC)
+        paths.append(B.SLIM_PATH_TC)
+    except B.SlimError:
+        pass
+    layer.set_path(B.SLIM_PATH_AUTO)
+    return paths
+
+
+def _run_host_case(cfg, L, check_paths=True):
+    layer = SlimLayer(cfg.d, cfg.H, cfg.d_k, cfg.rope_theta, cfg.dtype, cfg.batch, cfg.context, DEV)
+    try:
+        layer.k.copy_(to_device_keys(L.K, cfg.dtype, DEV))
+        res, _ = layer.set_weights(L.W_K, L.W_V)
+        assert res < 1e-9
+        q = to_device_keys(L.q, cfg.dtype, DEV)
+        lengths = torch.from_numpy(L.lengths).to(DEV)
+        W_KV = so.oracle_wkv(L.W_K, L.W_V)
+        ref = so.oracle_slim_batch(L.q, L.K, L.lengths, W_KV, cfg.H, cfg.rope_theta)
+        worst = {}
+        for path in (_paths(layer) if check_paths else [B.SLIM_PATH_AUTO]):
+            layer.set_path(path)
+            layer.o.fill_(float("nan"))
+            got = layer.decode(q, lengths).cpu().numpy().astype(np.float64)
+            assert layer.device_status() == B.SLIM_OK
+            assert np.all(np.isfinite(got)), f"path {path}: non-finite output"
+            e = 0.0
+            for b in range(cfg.batch):
+                if L.lengths[b] == 0:
+                    assert np.all(got[b] == 0)
+                else:
+                    e = max(e, _err(got[b], ref[b], cfg.dtype))
+            worst[path] = e
+            assert e <= TOL[cfg.dtype], f"path {path}: error {e:.3e} > {TOL[cfg.dtype]}"
+        return worst
+    finally:
+        layer.close()
+
+
+SMALL_SHAPES = [
+    # d, H, d_k, theta, dtype
+    (64, 2, 32, 0.0, "f32"),
+    (64, 2, 32, 1.0e4, "f32"),
+    (384, 6, 64, 0.0, "f32"),
+    (256, 4, 64, 1.0e4, "bf16"),
+    (192, 2, 96, 1.0e4, "bf16"),
+    (512, 32, 16, 1.0e6, "bf16"),
+    (1024, 64, 16, 1.0e4, "f32"),
+    (1280, 20, 64, 0.0, "bf16"),
+    (768, 8, 96, 1.0e4, "bf16"),
+    (1024, 8, 128, 1.0e6, "bf16"),
+]
+
+
+@pytest.mark.parametrize("d,H,d_k,theta,dtype", SMALL_SHAPES)
+def test_small_ragged_batch_matches_oracle(d, H, d_k, theta, dtype):
+    lengths = np.array([1, 2, 15, 16, 17, 33, 100, 0, 257, 300], dtype=np.int32)
+    cfg = synth.SlimConfig("small", d, H, d_k, len(lengths), 300, 1, theta, dtype)
+    L = synth.make_layer(cfg, 1234 + d + H, lengths=lengths)
+    _run_host_case(cfg, L)
+
+
+@pytest.mark.parametrize("T", [1, 16, 31, 32, 33, 1000, 2049])
+def test_single_sequence_lengths(T):
+    cfg = synth.SlimConfig("single", 512, 4, 128, 1, max(T, 16), 1, 1.0e4, "bf16")
+    L = synth.make_layer(cfg, 99 + T, lengths=np.array([T], dtype=np.int32))
+    _run_host_case(cfg, L)
+
+
+def test_config0_whisper_tiny_shape_full():
+    cfg = synth.CONFIGS[0]
+    _run_host_case(cfg, synth.make_layer(cfg, synth.layer_seed(0, 0)))
+
+
+def test_config1_phi3_mini_shape_full():
+    cfg = synth.CONFIGS[1]
+    _run_host_case(cfg, synth.make_layer(cfg, synth.layer_seed(1, 0)))
+
+
+def test_config3_whisper_large_cross_shape_one_layer():
+    cfg = synth.CONFIGS[3].scaled(layers=1)
+    _run_host_case(cfg, synth.make_layer(cfg, synth.layer_seed(3, 0)))
+
+
+def _run_device_case(cfg, config_index, sample):
+    """Full-size configs: inputs drawn on the GPU; the stored K bits of the
+    sampled sequences are copied back for the oracle."""
+    seed = synth.layer_seed(config_index, 0)
+    lengths = synth.make_lengths(cfg, seed)
+    layer = SlimLayer(cfg.d, cfg.H, cfg.d_k, cfg.rope_theta, cfg.dtype, cfg.batch, cfg.context, DEV)
+    try:
+        W_Q, W_K, W_V, _, _ = synth.make_weights_torch(cfg.d, seed, DEV)
+        q = torch.zeros((cfg.batch, cfg.d), dtype=layer.tdtype, device=DEV)
+        layer.k.fill_(float("nan"))            # rows beyond each length are poison
+        synth.fill_layer_torch(cfg, seed, W_Q, W_K, lengths, layer.k, q)
+        W_K_h, W_V_h = W_K.cpu().numpy(), W_V.cpu().numpy()
+        res, wkv = layer.set_weights(W_K_h, W_V_h, want_wkv=True)
+        assert res < 1e-9
+        W_KV = so.oracle_wkv(W_K_h, W_V_h)
+        assert np.allclose(wkv, W_KV, rtol=1e-8, atol=1e-10)
+        lens_dev = torch.from_numpy(lengths).to(DEV)
+        outs = {}
+        for path in _paths(layer):
+            layer.set_path(path)
+            layer.o.fill_(float("nan"))
+            outs[path] = layer.decode(q, lens_dev).cpu().numpy().astype(np.float64)
+            assert layer.device_status() == B.SLIM_OK
+            assert np.all(np.isfinite(outs[path]))
+        for b in sample:
+            n = int(lengths[b])
+            Kb = layer.k[b, :n].float().cpu().numpy()
+            qb = q[b].float().cpu().numpy()
+            ref = so.oracle_slim(qb, Kb, W_KV, cfg.H, cfg.rope_theta)
+            for path, got in outs.items():
+                e = _err(got[b], ref, cfg.dtype)
+                assert e <= TOL[cfg.dtype], f"path {path} seq {b}: error {e:.3e}"
+    finally:
+        layer.close()
+
+
+def test_config2_codellama_shape_one_layer_sampled_sequences():
+    cfg = synth.CONFIGS[2].scaled(layers=1)
+    lengths = synth.make_lengths(cfg, synth.layer_seed(2, 0))
+    sample = sorted({0, int(np.argmin(lengths)), int(np.argmax(lengths))})
+    _run_device_case(cfg, 2, sample)
+
+
+def test_config4_long_context_full():
+    _run_device_case(synth.CONFIGS[4], 4, [0])
