@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Benchmark of the slim-attention decode path (one process per GPU).
+
+A *step* is one decode token for every sequence of the batch through all
+layers of the workload: per layer slim_append_k (the new key row) followed by
+slim_decode.  The default workload is the CodeLlama-7B-shaped configuration
+(32 layers, d=4096, H=32, d_k=128, batch 16, ragged contexts U[8192,16384],
+bf16 K-cache, RoPE theta 1e6) with seeded synthetic data.
+
+  value      decode tokens/s with all inputs resident in HBM (CUDA events)
+  e2e        the same through host buffers: per step the queries and new keys
+             are copied from pinned host memory and the outputs copied back
+  roofline   K-cache bytes per main-kernel launch / its CUDA-event duration,
+             against the measured HBM copy rate
+  cpu_baseline  the fp64 oracle timed on the host cores on a bounded sample
+
+`--impl reference` times the oracle alone (there is no reference code to run).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="index into the five workload shapes")
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (0 = the config's)")
+    ap.add_argument("--path", default="auto", choices=["auto", "generic", "tc"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thr = threading.Thread(target=self._read, daemon=True)
+            self.thr.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], None, set()
+        for ts, line in self.rows:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            inside = t0 <= ts <= t1 + 0.1
+            try:
+                if inside:
+                    sm.append(float(parts[1]))
+                mx = float(parts[2])
+            except ValueError:
+                continue
+            if inside:
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        if not sm:      # timed region shorter than the sampling period: use every sample
+            for ts, line in self.rows:
+                parts = [x.strip() for x in line.split(",")]
+                try:
+                    sm.append(float(parts[1]))
+                except (ValueError, IndexError):
+                    pass
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_sample_seconds(cfg, lengths, get_seq, W_KV):
+    """Time the oracle, as it stands, on one (layer, sequence) of the workload."""
+    from oracle import slim_oracle as so
+    b = int(np.argmin(np.abs(lengths - np.mean(lengths))))
+    q, K = get_seq(b)
+    t0 = time.perf_counter()
+    so.oracle_slim(q, K, W_KV, cfg.H, cfg.rope_theta)
+    dt = time.perf_counter() - t0
+    return b, dt
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    """The CPU oracle as the reference arm: one step = one (layer, sequence)
+    sample of the workload; throughput is scaled to whole decode tokens."""
+    from oracle import slim_oracle as so
+    from paper_2503_05840_b200 import synth
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = synth.CONFIGS[args.config]
+    layers = args.layers or cfg.layers
+    seed = synth.layer_seed(args.config, 0)
+    lengths = synth.make_lengths(cfg, seed)
+    # bounded sample: one sequence of one layer, context capped so a step stays in seconds
+    n = int(min(int(np.mean(lengths)), 4096))
+    g = np.random.Generator(np.random.Philox(seed))
+    s = g.uniform(0.5, 2.0, size=cfg.d)
+    K = synth.round_to_dtype(g.standard_normal((n, cfg.d)) * s[None, :], cfg.dtype).astype(np.float64)
+    q = synth.round_to_dtype(g.standard_normal(cfg.d), cfg.dtype).astype(np.float64)
+    W_KV = g.standard_normal((cfg.d, cfg.d)) / np.sqrt(cfg.d)
+    for _ in range(max(1, min(args.warmup, 1))):
+        so.oracle_slim(q, K, W_KV, cfg.H, cfg.rope_theta)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        so.oracle_slim(q, K, W_KV, cfg.H, cfg.rope_theta)
+    dt = (time.perf_counter() - t0) / args.steps
+    # seconds per (layer, sequence) at the mean context, then per decode token (all layers)
+    per_token = dt * (float(np.mean(lengths)) / n) * layers
+    value = 1.0 / per_token
+    cores = host_threads()
+    sample = f"oracle_slim on 1 layer x 1 sequence x {n} context rows per step, scaled to {layers} layers and mean context {int(np.mean(lengths))}"
+    line = {"impl": "reference", "metric": "decode_attention_tokens_per_s", "value": value, "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"config{args.config}:{cfg.name}", "layers": layers, "batch": cfg.batch,
+                       "context": cfg.context, "d": cfg.d, "H": cfg.H, "d_k": cfg.d_k},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_2503_05840_b200 import binding as B
+    from paper_2503_05840_b200 import build as _build
+    from paper_2503_05840_b200 import synth
+    from paper_2503_05840_b200.layer import SlimLayer
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    if rank == 0:
+        _build.build()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+        dist.barrier()
+    dev = f"cuda:{local}"
+    torch.cuda.set_device(local)
+
+    cfg = synth.CONFIGS[args.config]
+    layers_n = args.layers or cfg.layers
+    cfg = cfg.scaled(layers=layers_n)
+    path = {"auto": B.SLIM_PATH_AUTO, "generic": B.SLIM_PATH_GENERIC, "tc": B.SLIM_PATH_TC}[args.path]
+
+    # ---- set-up (untimed): per-layer weights, W_KV solve, K-cache fill -----------
+    seed0 = synth.layer_seed(args.config, 0) + 100000 * rank
+    lengths = synth.make_lengths(cfg, synth.layer_seed(args.config, 0))      # same ragged mix on every rank
+    lens_dev = torch.from_numpy(lengths).to(dev)
+    pos_dev = (lens_dev - 1).clamp(min=0).to(torch.int32)
+    layers = []
+    ws = None
+    q_all = torch.zeros((layers_n, cfg.batch, cfg.d), dtype=torch.bfloat16 if cfg.dtype == "bf16" else torch.float32,
+                        device=dev)
+    knew_all = torch.zeros_like(q_all)
+    o_all = torch.zeros((layers_n, cfg.batch, cfg.d), dtype=torch.float32, device=dev)
+    wkv_last = None
+    t_setup = time.time()
+    for li in range(layers_n):
+        lay = SlimLayer(cfg.d, cfg.H, cfg.d_k, cfg.rope_theta, cfg.dtype, cfg.batch, cfg.context, dev, workspace=ws)
+        ws = lay.workspace
+        lay.set_path(path)
+        W_Q, W_K, W_V, _, _ = synth.make_weights_torch(cfg.d, seed0 + li, dev)
+        synth.fill_layer_torch(cfg, seed0 + li, W_Q, W_K, lengths, lay.k, q_all[li])
+        want = (li == layers_n - 1)
+        res, wkv = lay.set_weights(W_K.cpu().numpy(), W_V.cpu().numpy(), want_wkv=want)
+        if want:
+            wkv_last = wkv
+        assert res < 1e-8, f"W_KV residual {res}"
+        for b in range(cfg.batch):          # the step re-appends the newest key row
+            if lengths[b] > 0:
+                knew_all[li, b] = lay.k[b, int(lengths[b]) - 1]
+        del W_Q, W_K, W_V
+        layers.append(lay)
+    torch.cuda.synchronize()
+    t_setup = time.time() - t_setup
+    stream = torch.cuda.current_stream()
+
+    def step():
+        for li, lay in enumerate(layers):
+            lay.append_k(knew_all[li].unsqueeze(1), pos_dev)
+            lay.decode(q_all[li], lens_dev, o_all[li])
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        barrier()
+        return ms
+
+    # ---- device-resident timing ------------------------------------------------
+    for _ in range(max(args.warmup, 3)):
+        step()
+    for lay in layers[:1]:
+        assert lay.device_status() == B.SLIM_OK
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    t0 = time.time()
+    ms_total = timed(step, args.steps)
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1) if rank == 0 else None
+    ms_step = ms_total / args.steps
+    tokens = cfg.batch * world
+    value = tokens / (ms_step * 1e-3)
+
+    # ---- attribution pass: CUDA events around the main kernel of every decode ----
+    for lay in layers:
+        lay.profile(True)
+    main_ms, tail_ms, n_launch = 0.0, 0.0, 0
+    for _ in range(min(args.steps, 5)):
+        step()
+        for lay in layers:
+            a, b = lay.profile_read()
+            main_ms += a; tail_ms += b; n_launch += 1
+    for lay in layers:
+        lay.profile(False)
+    main_ms /= n_launch; tail_ms /= n_launch
+    k_bytes_layer = synth.kcache_bytes_per_step(cfg.scaled(layers=1), lengths)
+    peak, peak_kind = measured_peaks()
+    achieved = k_bytes_layer / (main_ms * 1e-3) / 1e9
+    step_gbs = k_bytes_layer * layers_n / (ms_step * 1e-3) / 1e9
+
+    # ---- end to end through host buffers -----------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        q_host = q_all.cpu().pin_memory()
+        k_host = knew_all.cpu().pin_memory()
+        o_host = torch.empty(o_all.shape, dtype=torch.float32).pin_memory()
+
+        def step_e2e():
+            q_all.copy_(q_host, non_blocking=True)
+            knew_all.copy_(k_host, non_blocking=True)
+            step()
+            o_host.copy_(o_all, non_blocking=True)
+
+        for _ in range(3):
+            step_e2e()
+        ms_e2e = timed(step_e2e, args.steps) / args.steps
+        e2e = {"value": tokens / (ms_e2e * 1e-3), "unit": "tokens/s",
+               "h2d_bytes_per_step": int(q_host.numel() * q_host.element_size() * 2),
+               "d2h_bytes_per_step": int(o_host.numel() * 4), "ms_per_step": ms_e2e}
+
+    # ---- CPU oracle baseline on a bounded sample (rank 0, N=1 only) ----------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import slim_oracle as so
+        lay = layers[-1]
+        W_KV = wkv_last
+        b = int(np.argmin(np.abs(lengths - np.mean(lengths))))
+        n_full = int(lengths[b])
+        n = min(n_full, 4096)                       # bounded: ~10-30 s of host work
+        Kb = lay.k[b, :n].float().cpu().numpy().astype(np.float64)
+        qb = q_all[-1, b].float().cpu().numpy().astype(np.float64)
+        tt = time.perf_counter()
+        ref = so.oracle_slim(qb, Kb, W_KV, cfg.H, cfg.rope_theta)
+        dt = time.perf_counter() - tt
+        per_token = dt * (float(np.mean(lengths)) / n) * layers_n
+        cpu = {"value": 1.0 / per_token, "unit": "tokens/s", "cores": host_threads(), "kind": "oracle",
+               "sample": f"oracle_slim on layer {layers_n - 1}, sequence {b}, first {n} of {n_full} context rows "
+                         f"({dt:.2f} s), scaled to mean context {int(np.mean(lengths))} x {layers_n} layers"}
+        # the same sample doubles as a live parity check of what was timed
+        lens_chk = lens_dev.clone(); lens_chk[b] = n
+        got = lay.decode(q_all[-1], lens_chk).cpu().numpy().astype(np.float64)[b]
+        err = so.err_rms_norm(got, ref) if cfg.dtype == "bf16" else so.err_fp32_norm(got, ref)
+        cpu["parity_err_on_sample"] = err
+
+    status = layers[0].device_status()
+    if rank == 0:
+        launches = sum(1 + lay.query(B.SLIM_Q_LAUNCHES_PER_DECODE) for lay in layers)
+        line = {
+            "metric": "decode_attention_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
+            "data": "synthetic",
+            "config": {"workload": f"config{args.config}:{cfg.name}", "layers": layers_n, "batch_per_gpu": cfg.batch,
+                       "global_batch": tokens, "context": cfg.context, "sum_lengths": int(lengths.sum()),
+                       "d": cfg.d, "H": cfg.H, "d_k": cfg.d_k, "rope_theta": cfg.rope_theta,
+                       "parallelism": f"replicas x{world} (batch-sharded, no collective)",
+                       "l2": "inputs larger than L2 (K-cache per step >> 126 MB)" if k_bytes_layer * layers_n > 2.6e8
+                             else "K-cache per step fits L2: warm-cache number",
+                       "path": {1: "generic", 2: "tc"}[layers[0].query(B.SLIM_Q_PATH_IN_USE)]},
+            "kcache_gbs": step_gbs, "kcache_frac_of_8000": step_gbs / 8000.0, "kcache_frac_of_measured": step_gbs / peak,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "peak_kind": peak_kind, "kernel": "main decode kernel (per layer launch)",
+                         "main_ms": main_ms, "tail_ms": tail_ms, "bytes_per_launch": k_bytes_layer},
+            "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": launches, "clocks": clocks,
+            "device_status": int(status), "setup_s": t_setup,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -36,7 +36,7 @@ extern "C" {
 typedef enum {
   SLIM_OK = 0,
   SLIM_ERR_INVALID_ARG = 1,  /* NULL pointer, non-positive size, bad enum          */
-  SLIM_ERR_UNSUPPORTED = 2,  /* d != H*d_k, odd d_k with RoPE, H > 64, ...          */
+  SLIM_ERR_UNSUPPORTED = 2,  /* d != H*d_k, d_k not a multiple of 16, H > 64, ...   */
   SLIM_ERR_SINGULAR = 3,     /* W_K has a (numerically) zero pivot                  */
   SLIM_ERR_CAPACITY = 4,     /* append beyond t_cap / length beyond t_cap (device)  */
   SLIM_ERR_OOM = 5,          /* a library-owned allocation failed                   */
@@ -69,7 +69,7 @@ typedef struct slim_cache slim_cache; /* view of caller-owned key storage [B][t_
 
 /* One layer of shape (d, H, d_k); rope_theta = 0 disables RoPE; dtype is the
  * type of the K-cache and of q.  Requires d == H*d_k (Eq. 6 needs a square
- * W_K), H <= 64, d_k even.  Uses the current CUDA device.                      */
+ * W_K), H <= 64, d_k a multiple of 16 and <= 256.  Uses the current CUDA device. */
 slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta, int dtype);
 void        slim_destroy(slim_ctx* ctx);
 
@@ -122,6 +122,13 @@ slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache,
 /* Synchronises `stream`, returns the sticky device status (SLIM_OK,
  * SLIM_ERR_CAPACITY or SLIM_ERR_TIMEOUT) and clears it.                        */
 slim_status slim_device_status(slim_ctx* ctx, void* stream);
+
+/* Kernel timing for roofline reports.  While enabled, slim_decode records CUDA
+ * events on its stream before the main (K-reading) kernel, after it, and after
+ * the combine/projection tail.  slim_profile_read waits for the last decode of
+ * this ctx to finish and returns the two durations in milliseconds.           */
+slim_status slim_profile_enable(slim_ctx* ctx, int enable);
+slim_status slim_profile_read(slim_ctx* ctx, float* main_ms, float* tail_ms);
 
 slim_status slim_set_path(slim_ctx* ctx, int path);
 long long   slim_query(const slim_ctx* ctx, int key);

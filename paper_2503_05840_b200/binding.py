@@ -33,6 +33,8 @@ SIGNATURES = {
     "slim_append_k": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]),
     "slim_decode": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "slim_device_status": (c_int, [c_void_p, c_void_p]),
+    "slim_profile_enable": (c_int, [c_void_p, c_int]),
+    "slim_profile_read": (c_int, [c_void_p, POINTER(ctypes.c_float), POINTER(ctypes.c_float)]),
     "slim_set_path": (c_int, [c_void_p, c_int]),
     "slim_query": (c_longlong, [c_void_p, c_int]),
     "slim_strerror": (c_char_p, [c_int]),
@@ -151,6 +153,17 @@ def slim_decode(ctx: int, q, cache: int, lengths, o, workspace, stream: int = 0)
 
 def slim_device_status(ctx: int, stream: int = 0) -> int:
     return lib().slim_device_status(c_void_p(ctx), c_void_p(stream))
+
+
+def slim_profile_enable(ctx: int, enable: bool) -> None:
+    _check(lib().slim_profile_enable(c_void_p(ctx), 1 if enable else 0), "slim_profile_enable")
+
+
+def slim_profile_read(ctx: int):
+    """(main_ms, tail_ms) of the last slim_decode of this ctx."""
+    a, b = ctypes.c_float(0), ctypes.c_float(0)
+    _check(lib().slim_profile_read(c_void_p(ctx), byref(a), byref(b)), "slim_profile_read")
+    return a.value, b.value
 
 
 def slim_set_path(ctx: int, path: int) -> None:

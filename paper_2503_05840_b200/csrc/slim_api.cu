@@ -16,11 +16,11 @@ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 inline size_t esize(int dtype) { return dtype == SLIM_BF16 ? 2 : 4; }
 
 struct WsLayout {
-  size_t part_u, part_m, part_l, flags, o_part, total;
+  size_t part_u, part_m, part_l, flags, o_part, scores, total;
   int units;
 };
 
-WsLayout ws_layout(const slim_ctx* ctx, int batch) {
+WsLayout ws_layout(const slim_ctx* ctx, int batch, int t_cap) {
   WsLayout L;
   L.units = ctx->num_sms + batch;
   size_t off = 0;
@@ -29,6 +29,7 @@ WsLayout ws_layout(const slim_ctx* ctx, int batch) {
   L.part_l = off; off = align256(off + sizeof(float) * (size_t)L.units * ctx->H);
   L.flags = off;  off = align256(off + sizeof(int) * (size_t)L.units);
   L.o_part = off; off = align256(off + sizeof(float) * slim_tail_opart_floats(ctx->d, batch));
+  L.scores = off; off = align256(off + sizeof(float) * (size_t)batch * ctx->H * t_cap);   // generic path only
   L.total = off;
   return L;
 }
@@ -117,7 +118,7 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
   if (d <= 0 || H <= 0 || d_k <= 0 || !(rope_theta >= 0.0) || (dtype != SLIM_F32 && dtype != SLIM_BF16))
     return SLIM_ERR_INVALID_ARG;
   if ((long long)H * d_k != d) return SLIM_ERR_UNSUPPORTED;       // Eq. 6 needs a square W_K
-  if (H > SLIM_MAX_H || d_k > 256 || (d_k & 1) || d > 16384 || (d % 8) != 0) return SLIM_ERR_UNSUPPORTED;
+  if (H > SLIM_MAX_H || d_k > 256 || (d_k % 16) != 0 || d > 16384) return SLIM_ERR_UNSUPPORTED;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return SLIM_ERR_CUDA;
   cudaDeviceProp prop;
@@ -159,6 +160,8 @@ void slim_destroy(slim_ctx* ctx) {
   cudaFree(ctx->rope_off);
   cudaFree(ctx->rope_base);
   cudaFree(ctx->status);
+  for (int i = 0; i < 3; ++i)
+    if (ctx->prof_ev[i]) cudaEventDestroy(ctx->prof_ev[i]);
   delete ctx;
 }
 
@@ -224,7 +227,7 @@ size_t slim_cache_bytes(const slim_ctx* ctx, int batch, int t_cap) {
 
 size_t slim_workspace_bytes(const slim_ctx* ctx, int batch, int t_cap) {
   if (!ctx || batch <= 0 || t_cap <= 0 || batch > SLIM_MAX_BATCH) return 0;
-  return ws_layout(ctx, batch).total;
+  return ws_layout(ctx, batch, t_cap).total;
 }
 
 slim_status slim_cache_create(slim_ctx* ctx, slim_cache** out, void* k_storage, int batch, int t_cap) {
@@ -269,7 +272,7 @@ slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, c
     if (ctx->path_req == SLIM_PATH_TC) return SLIM_ERR_UNSUPPORTED;
     path = SLIM_PATH_GENERIC;
   }
-  const WsLayout L = ws_layout(ctx, cache->batch);
+  const WsLayout L = ws_layout(ctx, cache->batch, cache->t_cap);
   char* ws = static_cast<char*>(workspace);
   SlimDecodeParams p;
   p.d = ctx->d; p.H = ctx->H; p.d_k = ctx->d_k; p.half = ctx->d_k / 2;
@@ -287,8 +290,17 @@ slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   p.u = reinterpret_cast<float*>(ws + L.o_part);
   p.o = o; p.status = ctx->status;
   cudaStream_t st = (cudaStream_t)stream;
-  cudaError_t e = path == SLIM_PATH_TC ? slim_launch_tc(ctx, cache, p, st) : slim_launch_generic(ctx, p, st);
+  if (ctx->prof_on) cudaEventRecord(ctx->prof_ev[0], st);
+  cudaError_t e;
+  if (path == SLIM_PATH_TC) {
+    e = slim_launch_tc(ctx, cache, p, st);
+    if (e == cudaSuccess) e = slim_launch_exact_flagged(ctx, p, st);
+  } else {
+    e = slim_launch_generic(ctx, p, reinterpret_cast<float*>(ws + L.scores), st);
+  }
+  if (ctx->prof_on) cudaEventRecord(ctx->prof_ev[1], st);
   if (e == cudaSuccess) e = slim_launch_tail(ctx, p, st);
+  if (ctx->prof_on) { cudaEventRecord(ctx->prof_ev[2], st); ctx->prof_valid = 1; }
   if (e != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
   return SLIM_OK;
 }
@@ -300,6 +312,27 @@ slim_status slim_device_status(slim_ctx* ctx, void* stream) {
   if (cudaMemcpy(&v, ctx->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return SLIM_ERR_CUDA;
   if (v != 0) cudaMemset(ctx->status, 0, sizeof(int));
   return (slim_status)v;
+}
+
+slim_status slim_profile_enable(slim_ctx* ctx, int enable) {
+  if (!ctx) return SLIM_ERR_INVALID_ARG;
+  if (enable && !ctx->prof_ev[0]) {
+    for (int i = 0; i < 3; ++i)
+      if (cudaEventCreate(&ctx->prof_ev[i]) != cudaSuccess) return SLIM_ERR_CUDA;
+  }
+  ctx->prof_on = enable ? 1 : 0;
+  ctx->prof_valid = 0;
+  return SLIM_OK;
+}
+
+slim_status slim_profile_read(slim_ctx* ctx, float* main_ms, float* tail_ms) {
+  if (!ctx || !main_ms || !tail_ms) return SLIM_ERR_INVALID_ARG;
+  if (!ctx->prof_on || !ctx->prof_valid) return SLIM_ERR_INVALID_ARG;
+  if (cudaEventSynchronize(ctx->prof_ev[2]) != cudaSuccess) return SLIM_ERR_CUDA;
+  if (cudaEventElapsedTime(main_ms, ctx->prof_ev[0], ctx->prof_ev[1]) != cudaSuccess ||
+      cudaEventElapsedTime(tail_ms, ctx->prof_ev[1], ctx->prof_ev[2]) != cudaSuccess)
+    return SLIM_ERR_CUDA;
+  return SLIM_OK;
 }
 
 slim_status slim_set_path(slim_ctx* ctx, int path) {
@@ -314,7 +347,7 @@ long long slim_query(const slim_ctx* ctx, int key) {
   const int path = path_in_use(ctx);
   switch (key) {
     case SLIM_Q_PATH_IN_USE: return path;
-    case SLIM_Q_LAUNCHES_PER_DECODE: return path == SLIM_PATH_TC ? 4 : 3;
+    case SLIM_Q_LAUNCHES_PER_DECODE: return 4;   // tc: main, exact redo, tail1, tail2; generic: scores, accum, tail1, tail2
     case SLIM_Q_MAX_UNITS: return ctx->num_sms;   // + batch, known only per cache
     case SLIM_Q_NUM_SMS: return ctx->num_sms;
     case SLIM_Q_WORKERS: return path == SLIM_PATH_TC ? ctx->tc_workers : ctx->gen_workers;

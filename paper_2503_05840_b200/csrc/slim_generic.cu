@@ -1,14 +1,20 @@
-// Generic CUDA-core decode kernel (any supported shape, f32 or bf16 cache).
+// Generic CUDA-core decode kernels (any supported shape, f32 or bf16 cache).
 //
-// One CTA = (worker, d-slice).  For every context tile of its worker the CTA
-//   A. computes the softmax arguments of ALL heads for the tile rows
-//      (Eq. 2 with keys rotated after the read, RoPE appendix Option 1),
-//   B. updates the running max / sum per head (online softmax),
-//   C. accumulates U[h][col] += p[h][t] * K[t][col] for the columns it owns
-//      (Eq. 7 Option 2: weighted sum of the full-width raw keys),
-// and at the end of a unit writes the partial (m, l, U) for the combine.
-// CTAs of the same worker recompute step A redundantly (the key rows come
-// from L2 after the first touch); the tensor-core path removes that.
+// Two passes over the keys:
+//   slim_scores_kernel  softmax arguments s[b][h][t] (log2 domain) of every
+//                       head for every cached row (Eq. 2, keys rotated after
+//                       the read, RoPE appendix Option 1), 16-byte coalesced
+//                       row reads, written to a scratch array;
+//   slim_accum_kernel   CTA = (worker, d-slice): online softmax per head over
+//                       its context tiles and U[h][col] += p[h][t] K[t][col]
+//                       for the columns it owns (Eq. 7 Option 2: weighted sum
+//                       of the full-width raw keys); writes the partial
+//                       (m, l, U) of each unit for the combine.
+// The keys are read twice here; the tensor-core path reads them once.
+//
+// slim_exact_kernel is the single-pass variant (scores recomputed per
+// d-slice).  It is only used to redo, exactly, the rare units the tensor-core
+// kernel flags because a softmax argument ran away from its reference.
 #include "slim_internal.h"
 #include "slim_sched.cuh"
 
@@ -23,7 +29,7 @@ constexpr int GEN_THREADS = 256;
 
 template <typename KT, int HP, int COLS>
 __global__ void __launch_bounds__(GEN_THREADS)
-slim_generic_kernel(SlimDecodeParams p) {
+slim_exact_kernel(SlimDecodeParams p, int only_flagged) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* s_q = reinterpret_cast<float*>(smem_raw);                 // [d]
   float* s_S = s_q + p.d;                                           // [HP][TT]
@@ -53,6 +59,7 @@ slim_generic_kernel(SlimDecodeParams p) {
     const int seg_end = min(g_end, s_prefix[b + 1]);
     const int tile0 = g - s_prefix[b], tile1 = seg_end - s_prefix[b];
     const int unit = w + b;
+    if (only_flagged && p.unit_flags[unit] == 0) { g = seg_end; continue; }
     int len = p.lengths[b];
     len = min(max(len, 0), p.t_cap);
 
@@ -183,42 +190,263 @@ slim_generic_kernel(SlimDecodeParams p) {
   }
 }
 
+// ---------------------------------------------------------------------------
+// pass 1: softmax arguments
+// ---------------------------------------------------------------------------
+template <typename KT> struct Vec;
+template <> struct Vec<float> {
+  static constexpr int N = 4;
+  __device__ static void load(const float* p, float (&v)[4]) {
+    const float4 x = __ldg(reinterpret_cast<const float4*>(p));
+    v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+  }
+};
+template <> struct Vec<__nv_bfloat16> {
+  static constexpr int N = 8;
+  __device__ static void load(const __nv_bfloat16* p, float (&v)[8]) {
+    const uint4 x = __ldg(reinterpret_cast<const uint4*>(p));
+    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+};
+
+// One CTA walks tiles g = blockIdx.x, blockIdx.x + gridDim.x, ...  A warp owns
+// rows of the tile; a lane owns "pair vectors": VEC consecutive elements j of
+// the first half of a head together with their partners j + d_k/2.
+template <typename KT>
+__global__ void __launch_bounds__(GEN_THREADS)
+slim_scores_kernel(SlimDecodeParams p, float* __restrict__ scores) {
+  constexpr int VEC = Vec<KT>::N;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* s_q = reinterpret_cast<float*>(smem_raw);                         // [d] rotated, scaled query
+  float* s_part = s_q + p.d;                                                // [TT][d / (2 VEC)]
+  int* s_prefix = reinterpret_cast<int*>(s_part + SLIM_TT * (p.d / (2 * VEC)));
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int d = p.d, H = p.H, dk = p.d_k, half = p.half;
+  const int npv = d / (2 * VEC), pv_per_head = half / VEC;
+  const KT* __restrict__ Kc = reinterpret_cast<const KT*>(p.k);
+  const KT* __restrict__ Q = reinterpret_cast<const KT*>(p.q);
+
+  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status);
+  int cur_b = -1;
+  for (int g = blockIdx.x; g < sc.total_tiles; g += gridDim.x) {
+    const int b = slim_seq_of_tile(s_prefix, p.batch, g);
+    const int tile = g - s_prefix[b], t0 = tile * SLIM_TT;
+    const int len = min(max(p.lengths[b], 0), p.t_cap);
+    __syncthreads();
+    if (b != cur_b) {                       // a2: rotate + scale the query of sequence b
+      cur_b = b;
+      const int m = len - 1, mt = m / SLIM_TT, mi = m % SLIM_TT;
+      for (int e = tid; e < d; e += GEN_THREADS) {
+        const int h = e / dk, jj = e - h * dk;
+        float v;
+        if (p.rope) {
+          const int j = jj < half ? jj : jj - half;
+          const float2 cb = p.rope_base[(size_t)mt * half + j], co = p.rope_off[mi * half + j];
+          const float c = cb.x * co.x - cb.y * co.y, s = cb.y * co.x + cb.x * co.y;
+          const float q1 = ld_k(Q + (size_t)b * d + h * dk + j), q2 = ld_k(Q + (size_t)b * d + h * dk + j + half);
+          v = jj < half ? (q1 * c + q2 * s) : (-q1 * s + q2 * c);
+        } else {
+          v = ld_k(Q + (size_t)b * d + e);
+        }
+        s_q[e] = v * p.qscale;
+      }
+      __syncthreads();
+    }
+    for (int t = wid; t < SLIM_TT; t += GEN_THREADS / 32) {
+      if (t0 + t >= len) continue;
+      const KT* kr = Kc + ((size_t)b * p.t_cap + t0 + t) * d;
+      for (int pv = lane; pv < npv; pv += 32) {
+        const int h = pv / pv_per_head, j0 = (pv - h * pv_per_head) * VEC;
+        float k1[VEC], k2[VEC];
+        Vec<KT>::load(kr + h * dk + j0, k1);
+        Vec<KT>::load(kr + h * dk + half + j0, k2);
+        const float* q1 = s_q + h * dk + j0;
+        const float* q2 = q1 + half;
+        float a = 0.f;
+        if (p.rope) {
+          const float2* cbp = p.rope_base + (size_t)tile * half + j0;
+          const float2* cop = p.rope_off + t * half + j0;
+#pragma unroll
+          for (int x = 0; x < VEC; ++x) {
+            const float2 cb = __ldg(cbp + x), co = __ldg(cop + x);
+            const float c = cb.x * co.x - cb.y * co.y, s = cb.y * co.x + cb.x * co.y;
+            a += c * (q1[x] * k1[x] + q2[x] * k2[x]) + s * (q1[x] * k2[x] - q2[x] * k1[x]);
+          }
+        } else {
+#pragma unroll
+          for (int x = 0; x < VEC; ++x) a += q1[x] * k1[x] + q2[x] * k2[x];
+        }
+        s_part[t * npv + pv] = a;
+      }
+    }
+    __syncthreads();
+    for (int e = tid; e < H * SLIM_TT; e += GEN_THREADS) {
+      const int h = e / SLIM_TT, t = e - h * SLIM_TT;
+      if (t0 + t < len) {
+        float a = 0.f;
+        for (int x = 0; x < pv_per_head; ++x) a += s_part[t * npv + h * pv_per_head + x];
+        scores[((size_t)b * H + h) * p.t_cap + t0 + t] = a;
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// pass 2: online softmax + weighted sum of the raw keys
+// ---------------------------------------------------------------------------
+template <typename KT, int HP>
+__global__ void __launch_bounds__(GEN_THREADS, 2)
+slim_accum_kernel(SlimDecodeParams p, const float* __restrict__ scores) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* s_P = reinterpret_cast<float*>(smem_raw);                  // [HP][TT]
+  float* s_alpha = s_P + HP * SLIM_TT;                              // [HP]
+  float* s_m = s_alpha + HP;                                        // [HP]
+  float* s_l = s_m + HP;                                            // [HP]
+  int* s_prefix = reinterpret_cast<int*>(s_l + HP);                 // [batch+1]
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int w = blockIdx.y;
+  const int col = blockIdx.x * GEN_THREADS + tid;
+  const KT* __restrict__ Kc = reinterpret_cast<const KT*>(p.k);
+  const int d = p.d, H = p.H;
+
+  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status);
+  if (sc.total_tiles == 0 || w >= sc.workers_eff) return;
+  const int g_begin = slim_worker_start(sc, w), g_end = slim_worker_start(sc, w + 1);
+  float acc[HP];
+  int g = g_begin;
+  while (g < g_end) {
+    const int b = slim_seq_of_tile(s_prefix, p.batch, g);
+    const int seg_end = min(g_end, s_prefix[b + 1]);
+    const int tile0 = g - s_prefix[b], tile1 = seg_end - s_prefix[b];
+    const int unit = w + b;
+    const int len = min(max(p.lengths[b], 0), p.t_cap);
+    __syncthreads();
+    if (tid < HP) { s_m[tid] = -INFINITY; s_l[tid] = 0.f; }
+#pragma unroll
+    for (int h = 0; h < HP; ++h) acc[h] = 0.f;
+    __syncthreads();
+    for (int tile = tile0; tile < tile1; ++tile) {
+      const int t0 = tile * SLIM_TT;
+      const KT* __restrict__ Kt = Kc + ((size_t)b * p.t_cap + t0) * d;
+      float kv[SLIM_TT];
+#pragma unroll
+      for (int t = 0; t < SLIM_TT; ++t) kv[t] = (col < d && t0 + t < len) ? ld_k(Kt + (size_t)t * d + col) : 0.f;
+      // ---- a5: online softmax, one warp per head ----
+      for (int h = wid; h < H; h += GEN_THREADS / 32) {
+        const float s = (lane < SLIM_TT && t0 + lane < len)
+                            ? __ldg(scores + ((size_t)b * H + h) * p.t_cap + t0 + lane) : -INFINITY;
+        float mx = s;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        const float m_old = s_m[h], m_new = fmaxf(m_old, mx);
+        const float pr = (s == -INFINITY) ? 0.f : exp2f(s - m_new);
+        float ps = pr;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
+        const float alpha = exp2f(m_old - m_new);
+        if (lane < SLIM_TT) s_P[h * SLIM_TT + lane] = pr;
+        if (lane == 0) { s_alpha[h] = alpha; s_m[h] = m_new; s_l[h] = s_l[h] * alpha + ps; }
+      }
+      __syncthreads();
+      // ---- a6: U[h][col] = alpha U[h][col] + sum_t p[h][t] K[t][col] ----
+#pragma unroll
+      for (int h = 0; h < HP; ++h) {
+        if (h < H) {
+          const float4* P4 = reinterpret_cast<const float4*>(s_P + h * SLIM_TT);
+          float a = acc[h] * s_alpha[h];
+#pragma unroll
+          for (int i = 0; i < SLIM_TT / 4; ++i) {
+            const float4 v = P4[i];
+            a = fmaf(v.x, kv[4 * i], a); a = fmaf(v.y, kv[4 * i + 1], a);
+            a = fmaf(v.z, kv[4 * i + 2], a); a = fmaf(v.w, kv[4 * i + 3], a);
+          }
+          acc[h] = a;
+        }
+      }
+      __syncthreads();
+    }
+    if (col < d) {
+#pragma unroll
+      for (int h = 0; h < HP; ++h)
+        if (h < H) p.part_u[((size_t)unit * H + h) * d + col] = acc[h];
+    }
+    if (blockIdx.x == 0 && tid < H) {
+      p.part_m[(size_t)unit * H + tid] = s_m[tid];
+      p.part_l[(size_t)unit * H + tid] = s_l[tid];
+    }
+    g = seg_end;
+  }
+}
+
 template <typename KT, int HP, int COLS>
-cudaError_t launch_one(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st) {
+cudaError_t launch_exact(const SlimDecodeParams& p, int only_flagged, cudaStream_t st) {
   const int dsplit = (p.d + GEN_THREADS * COLS - 1) / (GEN_THREADS * COLS);
   const size_t smem = sizeof(float) * (p.d + 2 * HP * SLIM_TT + 3 * HP) + sizeof(int) * (p.batch + 1);
-  auto kern = slim_generic_kernel<KT, HP, COLS>;
+  auto kern = slim_exact_kernel<KT, HP, COLS>;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
   dim3 grid(dsplit, p.workers);
-  kern<<<grid, GEN_THREADS, smem, st>>>(p);
+  kern<<<grid, GEN_THREADS, smem, st>>>(p, only_flagged);
+  return cudaGetLastError();
+}
+
+template <typename KT>
+cudaError_t launch_two_pass(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, cudaStream_t st) {
+  constexpr int VEC = Vec<KT>::N;
+  {
+    const size_t smem = sizeof(float) * (p.d + SLIM_TT * (p.d / (2 * VEC))) + sizeof(int) * (p.batch + 1);
+    auto kern = slim_scores_kernel<KT>;
+    if (smem > 48 * 1024) {
+      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+    }
+    kern<<<4 * ctx->num_sms, GEN_THREADS, smem, st>>>(p, scores);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  const int dsplit = (p.d + GEN_THREADS - 1) / GEN_THREADS;
+  dim3 grid(dsplit, p.workers);
+  if (p.H <= 8) {
+    const size_t smem = sizeof(float) * (8 * SLIM_TT + 3 * 8) + sizeof(int) * (p.batch + 1);
+    slim_accum_kernel<KT, 8><<<grid, GEN_THREADS, smem, st>>>(p, scores);
+  } else if (p.H <= 32) {
+    const size_t smem = sizeof(float) * (32 * SLIM_TT + 3 * 32) + sizeof(int) * (p.batch + 1);
+    slim_accum_kernel<KT, 32><<<grid, GEN_THREADS, smem, st>>>(p, scores);
+  } else {
+    const size_t smem = sizeof(float) * (64 * SLIM_TT + 3 * 64) + sizeof(int) * (p.batch + 1);
+    slim_accum_kernel<KT, 64><<<grid, GEN_THREADS, smem, st>>>(p, scores);
+  }
   return cudaGetLastError();
 }
 
 }  // namespace
 
-// Columns per thread: 2 for H <= 32 (64 accumulators), 1 above.
-int slim_generic_dsplit(const slim_ctx* ctx) {
-  const int cols = ctx->H <= 32 ? 2 : 1;
-  return (ctx->d + GEN_THREADS * cols - 1) / (GEN_THREADS * cols);
-}
+int slim_generic_dsplit(const slim_ctx* ctx) { return (ctx->d + GEN_THREADS - 1) / GEN_THREADS; }
 
 int slim_generic_workers(const slim_ctx* ctx) {
-  // about two CTAs per SM in flight, shared between the d-slices of a worker
-  int w = (2 * ctx->num_sms) / slim_generic_dsplit(ctx);
+  // about three CTAs per SM in flight, shared between the d-slices of a worker
+  int w = (3 * ctx->num_sms) / slim_generic_dsplit(ctx);
   if (w < 1) w = 1;
   if (w > ctx->num_sms) w = ctx->num_sms;
   return w;
 }
 
-cudaError_t slim_launch_generic(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st) {
+cudaError_t slim_launch_generic(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, cudaStream_t st) {
+  return p.dtype == SLIM_BF16 ? launch_two_pass<__nv_bfloat16>(ctx, p, scores, st)
+                              : launch_two_pass<float>(ctx, p, scores, st);
+}
+
+// Redo exactly the units whose flag is set (schedule taken from p.workers / p.min_tiles).
+cudaError_t slim_launch_exact_flagged(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st) {
   const bool bf = p.dtype == SLIM_BF16;
-  if (p.H <= 8) {
-    return bf ? launch_one<__nv_bfloat16, 8, 2>(ctx, p, st) : launch_one<float, 8, 2>(ctx, p, st);
-  } else if (p.H <= 32) {
-    return bf ? launch_one<__nv_bfloat16, 32, 2>(ctx, p, st) : launch_one<float, 32, 2>(ctx, p, st);
-  }
-  return bf ? launch_one<__nv_bfloat16, 64, 1>(ctx, p, st) : launch_one<float, 64, 1>(ctx, p, st);
+  if (p.H <= 8) return bf ? launch_exact<__nv_bfloat16, 8, 2>(p, 1, st) : launch_exact<float, 8, 2>(p, 1, st);
+  if (p.H <= 32) return bf ? launch_exact<__nv_bfloat16, 32, 2>(p, 1, st) : launch_exact<float, 32, 2>(p, 1, st);
+  return bf ? launch_exact<__nv_bfloat16, 64, 1>(p, 1, st) : launch_exact<float, 64, 1>(p, 1, st);
 }

@@ -13,7 +13,7 @@
 // table has one entry per tile and the offset table one per row of a tile.
 #define SLIM_TT 16
 #define SLIM_MAX_H 64
-#define SLIM_MAX_BATCH 4096
+#define SLIM_MAX_BATCH 2048
 
 // Parameters every decode kernel receives (passed by value).
 struct SlimDecodeParams {
@@ -54,6 +54,8 @@ struct slim_ctx {
   int tc_ok;                     // shape fits the tensor-core path
   int tc_workers;                // clusters the tensor-core kernel runs
   int gen_workers;
+  int prof_on, prof_valid;
+  cudaEvent_t prof_ev[3];
 };
 
 struct slim_cache {
@@ -67,7 +69,8 @@ struct slim_cache {
 // ---- launchers implemented in the kernel translation units -----------------
 int  slim_generic_workers(const slim_ctx* ctx);
 int  slim_generic_dsplit(const slim_ctx* ctx);
-cudaError_t slim_launch_generic(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st);
+cudaError_t slim_launch_generic(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, cudaStream_t st);
+cudaError_t slim_launch_exact_flagged(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st);
 cudaError_t slim_launch_tail(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st);
 cudaError_t slim_launch_append(const slim_ctx* ctx, const slim_cache* c, const void* k_new,
                                const int32_t* positions, int n_new, cudaStream_t st);

@@ -1,9 +1,661 @@
-// Tensor-core (TMA + tcgen05) decode path -- placeholder until the kernel lands.
-#include "slim_internal.h"
+// Tensor-core decode path for sm_100a: TMA-staged K tiles, CUDA-core scores
+// with RoPE in registers, tcgen05 (UMMA) weighted sum of the raw keys with the
+// accumulator in tensor memory.
+//
+// Work split.  A *worker* is a cluster of two CTAs; CTA r of the pair owns the
+// key columns [r d/2, (r+1) d/2) and therefore the heads that live in those
+// columns.  Both CTAs walk the same context tiles (16 rows) of the worker's
+// units.  Per tile and CTA:
+//   producer warp   one TMA load brings the [16 x d/2] slice of the tile into a
+//                   128-byte-swizzled shared-memory stage (each key byte is
+//                   staged exactly once in the whole GPU);
+//   score warps     (two heads each) read the stage, rotate the keys in
+//                   registers (RoPE appendix, Option 1), form the softmax
+//                   arguments of their heads (Eq. 2), turn them into
+//                   p = 2^(s - m_ref) and write the bf16 probabilities of their
+//                   heads into the P tile of BOTH CTAs (distributed shared
+//                   memory), because every head weights the full key row;
+//   MMA warp        U^T[128 cols x 32 heads] += K_tile^T[128 x 16] P^T[16 x 32]
+//                   for every 128-column chunk of the slice: one tcgen05.mma
+//                   per chunk, A = the staged keys (MN-major, straight from
+//                   the TMA layout), B = the P tile, D in tensor memory
+//                   (Eq. 7 Option 2: the weighted sum of the full-width keys).
+// At the end of a unit warps 0-3 read U from tensor memory and write the
+// partial (m_ref, l, U) for the log-sum-exp combine.
+//
+// Softmax reference.  m_ref of a (unit, head) is the maximum argument of the
+// unit's first tile and is never changed, so the accumulator is never rescaled.
+// 2^(s - m_ref) is exact in relative terms for any exponent below 2^127; a later
+// argument more than 96 (log2 units) above m_ref sets the unit's flag and the
+// unit is redone by the exact CUDA-core kernel afterwards.  l is accumulated
+// from the bf16-rounded p, so U / l stays an exact weighted mean of key rows.
+//
+// Every wait on an mbarrier is bounded in time; a wait that runs out sets the
+// device status to SLIM_ERR_TIMEOUT, all roles leave their loops, and the CTA
+// frees its tensor memory and exits.
+#include <cuda.h>
+#include <cstring>
 
-int slim_tc_shape_ok(int, int, int, int) { return 0; }
-int slim_tc_workers(const slim_ctx*) { return 0; }
-cudaError_t slim_tc_make_tmap(const slim_ctx*, slim_cache*) { return cudaErrorNotSupported; }
-cudaError_t slim_launch_tc(const slim_ctx*, const slim_cache*, const SlimDecodeParams&, cudaStream_t) {
-  return cudaErrorNotSupported;
+#include "slim_internal.h"
+#include "slim_sched.cuh"
+
+namespace {
+
+constexpr int TC_NP = 4;                 // P-tile stages
+constexpr int TC_P_BYTES = 1024;         // [32 heads][16 rows] bf16
+constexpr int TC_MAX_NS = 8;             // K stages
+constexpr float TC_XMAX = 96.f;          // largest exponent accepted above m_ref
+constexpr unsigned long long TC_WAIT_NS = 2000000000ull;
+
+struct TcGeom {
+  int dsl;          // key columns per CTA (d / 2)
+  int nch;          // 128-column chunks per CTA
+  int nc64;         // 64-column TMA chunks per CTA
+  int hl;           // heads per CTA
+  int nsw;          // score warps (two heads each)
+  int nswl;         // launched score/epilogue warps = max(4, nsw)
+  int ns;           // K stages
+  int stage_bytes;  // 16 * dsl * 2
+  int tmem_cols;    // power of two >= 32 * nch
+};
+
+// ------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ unsigned long long globaltimer() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank) {
+  uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank)); return r;
+}
+__device__ __forceinline__ void st_cluster_u16(uint32_t cluster_addr, unsigned short v) {
+  asm volatile("st.shared::cluster.u16 [%0], %1;" ::"r"(cluster_addr), "h"(v) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the wait ran out or another thread of the CTA gave up.
+template <bool CLUSTER>
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer();
+  unsigned spins = 0;
+  while (true) {
+    if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (globaltimer() - t0 > TC_WAIT_NS) {
+        *abort_flag = 1;
+        atomicMax(status, (int)SLIM_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {   // arrives on the barrier at this offset in both CTAs
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptors (sm_100 format: version 1 at bit 46).
+// A: K_tile^T chunk, M = 128 key columns x K = 16 rows, MN-major, 128-byte
+//    swizzle: two 64-column atoms 2048 B apart (leading offset), 8-row groups
+//    1024 B apart (stride offset).
+__device__ __forceinline__ uint64_t desc_a(uint32_t addr) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(2048 >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// B: P tile, N = 32 heads x K = 16 rows, K-major, no swizzle: 8x8 core matrices
+//    of 128 B; the two K halves 128 B apart (leading), 8-head groups 256 B apart (stride).
+__device__ __forceinline__ uint64_t desc_b(uint32_t addr) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(128 >> 4) << 16) | ((uint64_t)(256 >> 4) << 32) |
+         (1ull << 46);
+}
+// bf16 x bf16 -> f32, A MN-major, B K-major, M = 128, N = 32.
+constexpr uint32_t TC_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
+
+__device__ __forceinline__ uint32_t p_offset(int n, int k) {
+  return (uint32_t)((n & 7) * 16 + (n >> 3) * 256 + (k >> 3) * 128 + (k & 7) * 2);
+}
+
+__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts128_zero(uint32_t addr) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
+}
+
+// ------------------------------------------------------------------ the kernel
+template <int DK, bool ROPE>
+__global__ void __launch_bounds__(320, 1)
+slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams p, const TcGeom g) {
+  constexpr int PAIRS = DK / 2;                   // rotation pairs (j, j + DK/2) per head
+  constexpr int OCT = PAIRS / 8;                  // 8-pair groups per head
+  constexpr int JL = OCT <= 2 ? 2 : (OCT <= 4 ? 4 : (OCT <= 8 ? 8 : 16));   // lanes along j
+  constexpr int TG = 32 / JL;                     // row groups per warp
+  constexpr int RT = SLIM_TT / TG;                // rows per thread  (2 RT == JL)
+  static_assert(2 * RT == JL, "lane mapping");
+
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw_u32 = smem_u32(smem_raw);
+  const uint32_t base = (raw_u32 + 1023u) & ~1023u;
+  unsigned char* sm = smem_raw + (base - raw_u32);
+  const uint32_t k_stage0 = base;
+  const uint32_t p_stage0 = base + (uint32_t)g.ns * g.stage_bytes;
+  const uint32_t bars = p_stage0 + TC_NP * TC_P_BYTES;
+  const uint32_t bar_k_full = bars, bar_k_empty = bars + 8 * TC_MAX_NS;
+  const uint32_t bar_p_full = bars + 16 * TC_MAX_NS, bar_p_empty = bar_p_full + 8 * TC_NP;
+  const uint32_t bar_u_full = bar_p_empty + 8 * TC_NP, bar_u_empty = bar_u_full + 8;
+  unsigned char* misc = sm + (bar_u_empty + 8 - base);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 4);
+  int* s_prefix = reinterpret_cast<int*>(misc + 8);
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t rank = cluster_ctarank();
+  const int w = blockIdx.x >> 1;                  // worker = cluster index
+  const int producer_warp = g.nswl, mma_warp = g.nswl + 1;
+
+  // ---- set-up -------------------------------------------------------------------
+  if (tid == 0) {
+    for (int i = 0; i < g.ns; ++i) { mbar_init(bar_k_full + 8 * i, 1); mbar_init(bar_k_empty + 8 * i, g.nsw + 1); }
+    for (int i = 0; i < TC_NP; ++i) { mbar_init(bar_p_full + 8 * i, 2 * g.nsw * 32); mbar_init(bar_p_empty + 8 * i, 2); }
+    mbar_init(bar_u_full, 1);
+    mbar_init(bar_u_empty, 4);
+    *s_abort = 0;
+    fence_mbar_init();
+  }
+  for (int i = tid; i < TC_NP * TC_P_BYTES / 16; i += blockDim.x) sts128_zero(p_stage0 + 16 * i);
+  fence_proxy_async();
+  if (warp == mma_warp) tmem_alloc(smem_u32(s_tmem), (uint32_t)g.tmem_cols);
+  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status);
+  const bool have_work = sc.total_tiles > 0 && w < sc.workers_eff;
+  const int g_begin = have_work ? slim_worker_start(sc, w) : 0;
+  const int g_end = have_work ? slim_worker_start(sc, w + 1) : 0;
+  if (rank == 0 && have_work) {                   // clear the redo flags of this worker's units
+    const int b_lo = slim_seq_of_tile(s_prefix, p.batch, g_begin), b_hi = slim_seq_of_tile(s_prefix, p.batch, g_end - 1);
+    for (int b = b_lo + tid; b <= b_hi; b += blockDim.x) p.unit_flags[w + b] = 0;
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+
+  if (have_work) {
+    if (warp < g.nswl) {
+      // =========================== score / epilogue warps ===========================
+      const bool scorer = warp < g.nsw;
+      const int jl = lane % JL, tg = lane / JL;
+      const bool active = scorer && jl < OCT;
+      const int hl0 = 2 * warp;
+      const int nh = scorer ? min(2, g.hl - hl0) : 0;
+      const int my_hh = jl / RT, my_r = jl % RT, my_row = tg * RT + my_r;
+      const bool my_head_valid = my_hh < nh;
+      const int my_n = (int)rank * g.hl + hl0 + my_hh;           // global head of the value this lane owns
+      const uint32_t my_poff = p_offset(my_n & 31, my_row);
+      // shuffle masks that keep the head bit (value RT) fixed
+      float2 off_first[8], stepv[8];
+      if (ROPE && active) {
+#pragma unroll
+        for (int x = 0; x < 8; ++x) {
+          off_first[x] = p.rope_off[(tg * RT) * PAIRS + 8 * jl + x];
+          stepv[x] = p.rope_off[1 * PAIRS + 8 * jl + x];
+        }
+      }
+      // byte offsets of this thread's 16-byte key units inside a stage, per head and half
+      uint32_t koff[2][2], kunit[2][2];
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          const int col = (hl0 + hh) * DK + hf * PAIRS + 8 * jl;
+          koff[hh][hf] = (uint32_t)(col >> 6) * 2048u;
+          kunit[hh][hf] = (uint32_t)((col & 63) >> 3);
+        }
+
+      int it = 0, uc = 0;
+      bool ok = true;
+      for (int gg = g_begin; gg < g_end && ok; ++uc) {
+        const int b = slim_seq_of_tile(s_prefix, p.batch, gg);
+        const int seg_end = min(g_end, s_prefix[b + 1]);
+        const int tile0 = gg - s_prefix[b], ntile = seg_end - gg;
+        const int unit = w + b;
+        const int len = min(max(p.lengths[b], 0), p.t_cap);
+        // ---- a2: this thread's slice of the rotated, scaled query ----
+        float q1[2][8], q2[2][8];
+        if (active) {
+          const __nv_bfloat16* Q = reinterpret_cast<const __nv_bfloat16*>(p.q) + (size_t)b * p.d;
+          float cm[8], sn[8];
+          if (ROPE) {
+            const int m = len - 1, mt = m / SLIM_TT, mi = m % SLIM_TT;
+#pragma unroll
+            for (int x = 0; x < 8; ++x) {
+              const float2 cb = p.rope_base[(size_t)mt * PAIRS + 8 * jl + x], co = p.rope_off[mi * PAIRS + 8 * jl + x];
+              cm[x] = cb.x * co.x - cb.y * co.y; sn[x] = cb.y * co.x + cb.x * co.y;
+            }
+          }
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            if (hh < nh) {
+              const int n = (int)rank * g.hl + hl0 + hh;
+              float a[8], c[8];
+              unpack8(__ldg(reinterpret_cast<const uint4*>(Q + n * DK + 8 * jl)), a);
+              unpack8(__ldg(reinterpret_cast<const uint4*>(Q + n * DK + PAIRS + 8 * jl)), c);
+#pragma unroll
+              for (int x = 0; x < 8; ++x) {
+                if (ROPE) {
+                  q1[hh][x] = (a[x] * cm[x] + c[x] * sn[x]) * p.qscale;
+                  q2[hh][x] = (-a[x] * sn[x] + c[x] * cm[x]) * p.qscale;
+                } else {
+                  q1[hh][x] = a[x] * p.qscale; q2[hh][x] = c[x] * p.qscale;
+                }
+              }
+            } else {
+#pragma unroll
+              for (int x = 0; x < 8; ++x) { q1[hh][x] = 0.f; q2[hh][x] = 0.f; }
+            }
+          }
+        }
+        float mref = 0.f, lsum = 0.f;
+
+        for (int kt = 0; kt < ntile && ok; ++kt, ++it) {
+          const int tile = tile0 + kt, t0 = tile * SLIM_TT;
+          const int st = it % g.ns, ps = it % TC_NP;
+          const uint32_t kbase = k_stage0 + (uint32_t)st * g.stage_bytes;
+          float sv = 0.f;
+          if (scorer) {
+            ok = mbar_wait<false>(bar_k_full + 8 * st, (it / g.ns) & 1, s_abort, p.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            // rows at or beyond the sequence end must not reach the tensor core (0 x NaN)
+            if (t0 + SLIM_TT > len) {
+              const int nz = len - t0;
+              for (int c64 = warp; c64 < g.nc64; c64 += g.nsw)
+                for (int e = lane; e < (SLIM_TT - nz) * 8; e += 32)
+                  sts128_zero(kbase + (uint32_t)c64 * 2048u + (uint32_t)(nz + (e >> 3)) * 128u + (uint32_t)(e & 7) * 16u);
+            }
+            // ---- a4: softmax arguments of this warp's heads ----
+            float acc[2][RT];
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+              for (int r = 0; r < RT; ++r) acc[hh][r] = 0.f;
+            if (active) {
+              float2 cur[8];
+              if (ROPE) {
+                const float4* bp = reinterpret_cast<const float4*>(p.rope_base + (size_t)tile * PAIRS + 8 * jl);
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                  const float4 v = __ldg(bp + x);
+                  const float2 o0 = off_first[2 * x], o1 = off_first[2 * x + 1];
+                  cur[2 * x] = make_float2(v.x * o0.x - v.y * o0.y, v.y * o0.x + v.x * o0.y);
+                  cur[2 * x + 1] = make_float2(v.z * o1.x - v.w * o1.y, v.w * o1.x + v.z * o1.y);
+                }
+              }
+#pragma unroll
+              for (int r = 0; r < RT; ++r) {
+                const int row = tg * RT + r;
+                const uint32_t rbase = kbase + (uint32_t)row * 128u;
+                const uint32_t sw = (uint32_t)(row & 7);
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                  if (hh < nh) {
+                    float k1[8], k2[8];
+                    unpack8(lds128(rbase + koff[hh][0] + ((kunit[hh][0] ^ sw) << 4)), k1);
+                    unpack8(lds128(rbase + koff[hh][1] + ((kunit[hh][1] ^ sw) << 4)), k2);
+                    float a = acc[hh][r];
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) {
+                      if (ROPE) {
+                        const float A = fmaf(q1[hh][x], k1[x], q2[hh][x] * k2[x]);
+                        const float Bv = fmaf(q1[hh][x], k2[x], -(q2[hh][x] * k1[x]));
+                        a = fmaf(cur[x].x, A, a);
+                        a = fmaf(cur[x].y, Bv, a);
+                      } else {
+                        a = fmaf(q1[hh][x], k1[x], a);
+                        a = fmaf(q2[hh][x], k2[x], a);
+                      }
+                    }
+                    acc[hh][r] = a;
+                  }
+                }
+                if (ROPE && r + 1 < RT) {
+#pragma unroll
+                  for (int x = 0; x < 8; ++x) {
+                    const float2 c = cur[x], s = stepv[x];
+                    cur[x] = make_float2(c.x * s.x - c.y * s.y, c.y * s.x + c.x * s.y);
+                  }
+                }
+              }
+            }
+            // sum over the lanes that share (head, row), then pick this lane's value
+#pragma unroll
+            for (int o = 1; o < JL; o <<= 1)
+#pragma unroll
+              for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+                for (int r = 0; r < RT; ++r) acc[hh][r] += __shfl_xor_sync(0xffffffffu, acc[hh][r], o);
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+              for (int r = 0; r < RT; ++r)
+                if (hh == my_hh && r == my_r) sv = acc[hh][r];
+            const bool valid = my_head_valid && (t0 + my_row < len);
+            // ---- a5: probabilities against the fixed reference of this unit ----
+            if (kt == 0) {
+              float mx = valid ? sv : -INFINITY;
+#pragma unroll
+              for (int o = 1; o < 32; o <<= 1)
+                if (o != RT) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+              mref = mx;
+              lsum = 0.f;
+            }
+            float x = sv - mref;
+            if (valid && x > TC_XMAX) { p.unit_flags[unit] = 1; x = TC_XMAX; }
+            const float pf = valid ? exp2f(x) : 0.f;
+            const __nv_bfloat16 pb = __float2bfloat16_rn(pf);
+            lsum += __bfloat162float(pb);
+            // the P stage is free once the MMAs of tile it - TC_NP are done in both CTAs
+            ok = mbar_wait<false>(bar_p_empty + 8 * ps, ((it / TC_NP) & 1) ^ 1, s_abort, p.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const uint32_t paddr = p_stage0 + (uint32_t)ps * TC_P_BYTES + my_poff;
+            if (my_head_valid) {
+              st_cluster_u16(mapa(paddr, 0), __bfloat16_as_ushort(pb));
+              st_cluster_u16(mapa(paddr, 1), __bfloat16_as_ushort(pb));
+            }
+            fence_proxy_async();
+            mbar_arrive_cluster(mapa(bar_p_full + 8 * ps, 0));
+            mbar_arrive_cluster(mapa(bar_p_full + 8 * ps, 1));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_k_empty + 8 * st);
+          }
+        }
+        if (!ok) break;
+        // ---- partial of this unit: (m_ref, l) per head, then U from tensor memory ----
+        if (scorer) {
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1)
+            if (o != RT) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
+          if (my_head_valid && tg == 0 && my_r == 0) {
+            p.part_m[(size_t)unit * p.H + my_n] = mref;
+            p.part_l[(size_t)unit * p.H + my_n] = lsum;
+          }
+        }
+        if (warp < 4) {
+          ok = mbar_wait<false>(bar_u_full, uc & 1, s_abort, p.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          float* dst = p.part_u + (size_t)unit * p.H * p.d + (size_t)rank * g.dsl + warp * 32 + lane;
+          for (int c = 0; c < g.nch; ++c) {
+            uint32_t r[32];
+            tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), r);
+#pragma unroll
+            for (int n = 0; n < 32; ++n)
+              if (n < p.H) dst[(size_t)n * p.d + c * 128] = __uint_as_float(r[n]);
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_u_empty);
+        }
+        gg = seg_end;
+      }
+    } else if (warp == producer_warp) {
+      // =========================== TMA producer ===========================
+      if (lane == 0) {
+        int it = 0;
+        bool ok = true;
+        for (int gg = g_begin; gg < g_end && ok;) {
+          const int b = slim_seq_of_tile(s_prefix, p.batch, gg);
+          const int seg_end = min(g_end, s_prefix[b + 1]);
+          const int tile0 = gg - s_prefix[b], ntile = seg_end - gg;
+          for (int kt = 0; kt < ntile; ++kt, ++it) {
+            const int st = it % g.ns;
+            ok = mbar_wait<false>(bar_k_empty + 8 * st, ((it / g.ns) & 1) ^ 1, s_abort, p.status);
+            if (!ok) break;
+            mbar_arrive_expect_tx(bar_k_full + 8 * st, (uint32_t)g.stage_bytes);
+            tma_load_3d(k_stage0 + (uint32_t)st * g.stage_bytes, &tmap, bar_k_full + 8 * st, 0,
+                        b * p.t_cap + (tile0 + kt) * SLIM_TT, (int)rank * g.nc64);
+          }
+          gg = seg_end;
+        }
+        if (!ok) {
+          // gave up: let the loads that were issued land before the CTA goes away
+          const int issued = it < g.ns ? it : g.ns;
+          for (int k = 0; k < issued; ++k) {
+            const int j = it - 1 - k, st = j % g.ns;
+            const unsigned long long t0 = globaltimer();
+            while (!mbar_try_wait(bar_k_full + 8 * st, (j / g.ns) & 1) && globaltimer() - t0 < TC_WAIT_NS) {}
+          }
+        }
+      }
+    } else if (warp == mma_warp) {
+      // =========================== MMA issuer ===========================
+      if (lane == 0) {
+        int it = 0, uc = 0;
+        bool ok = true;
+        for (int gg = g_begin; gg < g_end && ok; ++uc) {
+          const int b = slim_seq_of_tile(s_prefix, p.batch, gg);
+          const int seg_end = min(g_end, s_prefix[b + 1]);
+          const int ntile = seg_end - gg;
+          for (int kt = 0; kt < ntile; ++kt, ++it) {
+            const int st = it % g.ns, ps = it % TC_NP;
+            ok = mbar_wait<false>(bar_k_full + 8 * st, (it / g.ns) & 1, s_abort, p.status);
+            if (ok) ok = mbar_wait<true>(bar_p_full + 8 * ps, (it / TC_NP) & 1, s_abort, p.status);
+            if (ok && kt == 0 && uc > 0) ok = mbar_wait<false>(bar_u_empty, (uc - 1) & 1, s_abort, p.status);
+            if (!ok) break;
+            fence_proxy_async();
+            tc_fence_after();
+            const uint64_t bd = desc_b(p_stage0 + (uint32_t)ps * TC_P_BYTES);
+            const uint32_t kbase = k_stage0 + (uint32_t)st * g.stage_bytes;
+            for (int c = 0; c < g.nch; ++c)
+              umma_bf16(tmem_base + (uint32_t)(c * 32), desc_a(kbase + (uint32_t)c * 4096u), bd, TC_IDESC, kt > 0 ? 1u : 0u);
+            umma_commit(bar_k_empty + 8 * st);
+            umma_commit_pair(bar_p_empty + 8 * ps);
+            if (kt == ntile - 1) umma_commit(bar_u_full);
+          }
+          gg = seg_end;
+        }
+      }
+    }
+  }
+
+  // ---- teardown: nobody may still write into a CTA that has left ------------------
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == mma_warp) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, (uint32_t)g.tmem_cols);
+  }
+}
+
+// ------------------------------------------------------------------ host side
+TcGeom make_geom(int d, int H, int d_k, int smem_limit) {
+  TcGeom g;
+  g.dsl = d / 2;
+  g.nch = g.dsl / 128;
+  g.nc64 = g.dsl / 64;
+  g.hl = H / 2;
+  g.nsw = (g.hl + 1) / 2;
+  g.nswl = g.nsw < 4 ? 4 : g.nsw;
+  g.stage_bytes = SLIM_TT * g.dsl * 2;
+  int ns = (smem_limit - 16 * 1024) / g.stage_bytes;
+  g.ns = ns > TC_MAX_NS ? TC_MAX_NS : ns;
+  int cols = 32;
+  while (cols < 32 * g.nch) cols <<= 1;
+  g.tmem_cols = cols;
+  return g;
+}
+
+size_t tc_smem_bytes(const TcGeom& g, int batch) {
+  size_t need = 1024 + (size_t)g.ns * g.stage_bytes + TC_NP * TC_P_BYTES + 16 * TC_MAX_NS + 16 * TC_NP + 16 + 8 +
+                sizeof(int) * (batch + 1) + 64;
+  const size_t floor_bytes = 120 * 1024;         // one CTA per SM: tensor memory is not shared
+  return need < floor_bytes ? floor_bytes : need;
+}
+
+typedef void (*tc_kernel_t)(const CUtensorMap, const SlimDecodeParams, const TcGeom);
+
+tc_kernel_t pick_kernel(int d_k, bool rope) {
+  switch (d_k) {
+    case 64: return rope ? slim_tc_kernel<64, true> : slim_tc_kernel<64, false>;
+    case 96: return rope ? slim_tc_kernel<96, true> : slim_tc_kernel<96, false>;
+    case 128: return rope ? slim_tc_kernel<128, true> : slim_tc_kernel<128, false>;
+    default: return nullptr;
+  }
+}
+
+constexpr int TC_SMEM_LIMIT = 227 * 1024;
+
+}  // namespace
+
+int slim_tc_shape_ok(int d, int H, int d_k, int dtype) {
+  if (dtype != SLIM_BF16) return 0;
+  if (d_k != 64 && d_k != 96 && d_k != 128) return 0;
+  if ((H & 1) || H > 32 || H < 2) return 0;
+  if (d % 256 != 0 || d > 4096) return 0;          // d/2 in 128-column chunks, <= 512 TMEM columns
+  return 1;
+}
+
+int slim_tc_workers(const slim_ctx* ctx) {
+  tc_kernel_t kern = pick_kernel(ctx->d_k, ctx->rope_theta != 0.0);
+  if (!kern) return 0;
+  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, TC_SMEM_LIMIT);
+  if (g.ns < 2) return 0;
+  const size_t smem = tc_smem_bytes(g, SLIM_MAX_BATCH);
+  if (smem > (size_t)TC_SMEM_LIMIT) return 0;
+  if (cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_LIMIT) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * (ctx->num_sms / 2));
+  cfg.blockDim = dim3((g.nswl + 2) * 32);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  int nclusters = 0;
+  if (cudaOccupancyMaxActiveClusters(&nclusters, (const void*)kern, &cfg) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  const int cap = ctx->num_sms / 2;
+  return nclusters < cap ? nclusters : cap;
+}
+
+cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c) {
+  typedef CUresult (*encode_t)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static encode_t encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return e;
+    if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+    encode = (encode_t)fn;
+  }
+  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, TC_SMEM_LIMIT);
+  // dim0: 64 contiguous elements; dim1: cache rows (stride d elements); dim2: 64-column chunks
+  const cuuint64_t dims[3] = {64, (cuuint64_t)c->batch * (cuuint64_t)c->t_cap, (cuuint64_t)(ctx->d / 64)};
+  const cuuint64_t strides[2] = {(cuuint64_t)ctx->d * 2, 128};
+  const cuuint32_t box[3] = {64, SLIM_TT, (cuuint32_t)g.nc64};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = encode(reinterpret_cast<CUtensorMap*>(c->tmap), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, c->k, dims,
+                      strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+cudaError_t slim_launch_tc(const slim_ctx* ctx, const slim_cache* c, const SlimDecodeParams& p, cudaStream_t st) {
+  tc_kernel_t kern = pick_kernel(ctx->d_k, ctx->rope_theta != 0.0);
+  if (!kern || !c->has_tmap) return cudaErrorNotSupported;
+  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, TC_SMEM_LIMIT);
+  const size_t smem = tc_smem_bytes(g, p.batch);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * p.workers);
+  cfg.blockDim = dim3((g.nswl + 2) * 32);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  CUtensorMap map;
+  memcpy(&map, c->tmap, sizeof(map));
+  return cudaLaunchKernelEx(&cfg, kern, map, p, g);
 }

@@ -11,7 +11,7 @@ from . import binding as B
 
 class SlimLayer:
     def __init__(self, d: int, H: int, d_k: int, rope_theta: float, dtype: str, batch: int, t_cap: int,
-                 device: str = "cuda:0"):
+                 device: str = "cuda:0", workspace: "torch.Tensor | None" = None):
         if not torch.cuda.is_available():
             raise RuntimeError("SlimLayer needs a CUDA device (there is no CPU fallback)")
         self.device = torch.device(device)
@@ -22,8 +22,11 @@ class SlimLayer:
             self.ctx = B.slim_create(d, H, d_k, rope_theta, B.SLIM_BF16 if dtype == "bf16" else B.SLIM_F32)
             self.k = torch.zeros((batch, t_cap, d), dtype=self.tdtype, device=self.device)
             self.cache = B.slim_cache_create(self.ctx, self.k, batch, t_cap)
-            self.workspace = torch.empty(B.slim_workspace_bytes(self.ctx, batch, t_cap), dtype=torch.uint8,
-                                         device=self.device)
+            need = B.slim_workspace_bytes(self.ctx, batch, t_cap)
+            if workspace is None:      # layers that run one after another on a stream may share one
+                workspace = torch.empty(need, dtype=torch.uint8, device=self.device)
+            assert workspace.numel() >= need and workspace.data_ptr() % 256 == 0
+            self.workspace = workspace
             self.o = torch.empty((batch, d), dtype=torch.float32, device=self.device)
 
     # ---- set-up -------------------------------------------------------------
@@ -52,6 +55,12 @@ class SlimLayer:
         B.slim_decode(self.ctx, q, self.cache, lengths, o, self.workspace,
                       torch.cuda.current_stream(self.device).cuda_stream)
         return o
+
+    def profile(self, enable: bool) -> None:
+        B.slim_profile_enable(self.ctx, enable)
+
+    def profile_read(self):
+        return B.slim_profile_read(self.ctx)
 
     def device_status(self) -> int:
         return B.slim_device_status(self.ctx, torch.cuda.current_stream(self.device).cuda_stream)
