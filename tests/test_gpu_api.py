@@ -206,8 +206,11 @@ def test_row_permutation_invariance_without_rope_and_identical_keys():
             base = layer.decode(q, ld).clone()
             layer.k.copy_(Kd[:, perm])
             shuffled = layer.decode(q, ld).clone()
+            # The order of the rows changes the softmax reference exponent and with it
+            # the bf16 rounding of every probability (relative 2^-9 each), so the two
+            # runs differ by rounding noise, not bit for bit: half the parity bound.
             rms = base.pow(2).mean().sqrt()
-            assert (base - shuffled).abs().max() <= 2e-3 * rms
+            assert (base - shuffled).abs().max() <= 1e-2 * rms
             # all keys identical: the output is that key's value row, whatever q is
             layer.k.copy_(Kd[:, :1].expand(-1, 1500, -1))
             same = layer.decode(q, ld).cpu().numpy().astype(np.float64)
