@@ -9,12 +9,18 @@
 //   producer warp   one TMA load brings the [16 x d/2] slice of the tile into a
 //                   128-byte-swizzled shared-memory stage (each key byte is
 //                   staged exactly once in the whole GPU);
-//   score warps     (two heads each) read the stage, rotate the keys in
-//                   registers (RoPE appendix, Option 1), form the softmax
-//                   arguments of their heads (Eq. 2), turn them into
-//                   p = 2^(s - m_ref) and write the bf16 probabilities of their
-//                   heads into the P tile of BOTH CTAs (distributed shared
-//                   memory), because every head weights the full key row;
+//   score warps     (two heads each) read the stage and form the softmax
+//                   arguments of their heads (Eq. 2).  A thread owns one head,
+//                   eight rotation pairs and every RP-th row of the tile.  The
+//                   rotation of the RoPE appendix (Option 1: keys are rotated
+//                   after the read) is moved onto the query: with q^ the query
+//                   at its own position, q^ . RoPE_t(k) = Q(t) . k where
+//                   Q(t) = q^ e^{i t theta} per pair, and Q is stepped from row
+//                   to row by one packed complex multiplication in registers
+//                   (re-seeded from the tables every TC_RESEED tiles).  The
+//                   arguments become p = 2^(s - m_ref); the bf16 probabilities
+//                   are written into the P tile of BOTH CTAs (distributed
+//                   shared memory), because every head weights the full key row;
 //   MMA warp        U^T[128 cols x 32 heads] += K_tile^T[128 x 16] P^T[16 x 32]
 //                   for every 128-column chunk of the slice: one tcgen05.mma
 //                   per chunk, A = the staged keys (MN-major, straight from
@@ -45,6 +51,7 @@ constexpr int TC_NP = 4;                 // P-tile stages
 constexpr int TC_P_BYTES = 1024;         // [32 heads][16 rows] bf16
 constexpr int TC_MAX_NS = 8;             // K stages
 constexpr float TC_XMAX = 96.f;          // largest exponent accepted above m_ref
+constexpr int TC_RESEED = 32;            // tiles between exact re-seeds of the stepped query rotation
 constexpr unsigned long long TC_WAIT_NS = 2000000000ull;
 
 struct TcGeom {
@@ -192,16 +199,47 @@ __device__ __forceinline__ void sts128_zero(uint32_t addr) {
   asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
 }
 
+// ------------------------------------------------------------------ packed fp32 helpers
+// Two fp32 values in one 64-bit register; sm_100 executes add/mul/fma on both halves
+// with one instruction.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 d; asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi)); return d;
+}
+__device__ __forceinline__ float sum2(f32x2 v) {
+  float lo, hi; asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); return lo + hi;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+  f32x2 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d;
+}
+// the two bf16 of a 32-bit word as (low element, high element) in fp32
+__device__ __forceinline__ f32x2 unpack2(uint32_t w) {
+  f32x2 d;
+  asm("{\n\t.reg .b32 lo, hi;\n\tshl.b32 lo, %1, 16;\n\tand.b32 hi, %1, 0xffff0000;\n\tmov.b64 %0, {lo, hi};\n\t}" : "=l"(d) : "r"(w));
+  return d;
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y;
+}
+
 // ------------------------------------------------------------------ the kernel
 template <int DK, bool ROPE>
 __global__ void __launch_bounds__(320, 1)
 slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams p, const TcGeom g) {
   constexpr int PAIRS = DK / 2;                   // rotation pairs (j, j + DK/2) per head
   constexpr int OCT = PAIRS / 8;                  // 8-pair groups per head
-  constexpr int JL = OCT <= 2 ? 2 : (OCT <= 4 ? 4 : (OCT <= 8 ? 8 : 16));   // lanes along j
-  constexpr int TG = 32 / JL;                     // row groups per warp
-  constexpr int RT = SLIM_TT / TG;                // rows per thread  (2 RT == JL)
-  static_assert(2 * RT == JL, "lane mapping");
+  constexpr int JL = OCT <= 4 ? 4 : 8;            // lanes along j (lanes >= OCT idle)
+  constexpr int RT = JL;                          // rows per thread and tile
+  constexpr int RP = SLIM_TT / RT;                // a thread owns rows rp, rp + RP, ...
+  constexpr int HL = JL * RP;                     // lanes per head
+  constexpr int HW = 32 / HL;                     // heads per warp
+  static_assert(HW == 2, "TcGeom assumes two heads per score warp");
 
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_u32 = smem_u32(smem_raw);
@@ -226,7 +264,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   // ---- set-up -------------------------------------------------------------------
   if (tid == 0) {
     for (int i = 0; i < g.ns; ++i) { mbar_init(bar_k_full + 8 * i, 1); mbar_init(bar_k_empty + 8 * i, g.nsw + 1); }
-    for (int i = 0; i < TC_NP; ++i) { mbar_init(bar_p_full + 8 * i, 2 * g.nsw * 32); mbar_init(bar_p_empty + 8 * i, 2); }
+    for (int i = 0; i < TC_NP; ++i) { mbar_init(bar_p_full + 8 * i, 2 * g.nsw); mbar_init(bar_p_empty + 8 * i, 2); }
     mbar_init(bar_u_full, 1);
     mbar_init(bar_u_empty, 4);
     *s_abort = 0;
@@ -253,33 +291,30 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
     if (warp < g.nswl) {
       // =========================== score / epilogue warps ===========================
       const bool scorer = warp < g.nsw;
-      const int jl = lane % JL, tg = lane / JL;
-      const bool active = scorer && jl < OCT;
-      const int hl0 = 2 * warp;
-      const int nh = scorer ? min(2, g.hl - hl0) : 0;
-      const int my_hh = jl / RT, my_r = jl % RT, my_row = tg * RT + my_r;
-      const bool my_head_valid = my_hh < nh;
-      const int my_n = (int)rank * g.hl + hl0 + my_hh;           // global head of the value this lane owns
+      const int jl = lane % JL, rp = (lane / JL) % RP, hw = lane / HL;
+      const int hl = HW * warp + hw;                             // head within this CTA
+      const bool head_valid = scorer && hl < g.hl;
+      const bool active = head_valid && jl < OCT;
+      const int my_n = (int)rank * g.hl + hl;                    // global head
+      const int my_row = rp + RP * jl;                           // row whose argument this lane ends up with
       const uint32_t my_poff = p_offset(my_n & 31, my_row);
-      // shuffle masks that keep the head bit (value RT) fixed
-      float2 off_first[8], stepv[8];
+      // byte offsets of this thread's two 16-byte key units (first / second half of the head)
+      uint32_t koff[2], kunit[2];
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        const int col = hl * DK + hf * PAIRS + 8 * jl;
+        koff[hf] = (uint32_t)(col >> 6) * 2048u;
+        kunit[hf] = (uint32_t)((col & 63) >> 3);
+      }
+      // e^{i RP theta}: one step of this thread's rows
+      f32x2 stc[4], sts[4], stn[4];
       if (ROPE && active) {
 #pragma unroll
-        for (int x = 0; x < 8; ++x) {
-          off_first[x] = p.rope_off[(tg * RT) * PAIRS + 8 * jl + x];
-          stepv[x] = p.rope_off[1 * PAIRS + 8 * jl + x];
+        for (int x = 0; x < 4; ++x) {
+          const float2 a = p.rope_off[RP * PAIRS + 8 * jl + 2 * x], b = p.rope_off[RP * PAIRS + 8 * jl + 2 * x + 1];
+          stc[x] = pack2(a.x, b.x); sts[x] = pack2(a.y, b.y); stn[x] = pack2(-a.y, -b.y);
         }
       }
-      // byte offsets of this thread's 16-byte key units inside a stage, per head and half
-      uint32_t koff[2][2], kunit[2][2];
-#pragma unroll
-      for (int hh = 0; hh < 2; ++hh)
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          const int col = (hl0 + hh) * DK + hf * PAIRS + 8 * jl;
-          koff[hh][hf] = (uint32_t)(col >> 6) * 2048u;
-          kunit[hh][hf] = (uint32_t)((col & 63) >> 3);
-        }
 
       int it = 0, uc = 0;
       bool ok = true;
@@ -289,41 +324,33 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
         const int tile0 = gg - s_prefix[b], ntile = seg_end - gg;
         const int unit = w + b;
         const int len = min(max(p.lengths[b], 0), p.t_cap);
-        // ---- a2: this thread's slice of the rotated, scaled query ----
-        float q1[2][8], q2[2][8];
+        // ---- a2: this thread's slice of the query at its own position, scaled ----
+        float qh1[8], qh2[8];
+#pragma unroll
+        for (int x = 0; x < 8; ++x) { qh1[x] = 0.f; qh2[x] = 0.f; }
         if (active) {
-          const __nv_bfloat16* Q = reinterpret_cast<const __nv_bfloat16*>(p.q) + (size_t)b * p.d;
-          float cm[8], sn[8];
+          const __nv_bfloat16* Q = reinterpret_cast<const __nv_bfloat16*>(p.q) + (size_t)b * p.d + my_n * DK + 8 * jl;
+          float a[8], c[8];
+          unpack8(__ldg(reinterpret_cast<const uint4*>(Q)), a);
+          unpack8(__ldg(reinterpret_cast<const uint4*>(Q + PAIRS)), c);
           if (ROPE) {
             const int m = len - 1, mt = m / SLIM_TT, mi = m % SLIM_TT;
 #pragma unroll
             for (int x = 0; x < 8; ++x) {
               const float2 cb = p.rope_base[(size_t)mt * PAIRS + 8 * jl + x], co = p.rope_off[mi * PAIRS + 8 * jl + x];
-              cm[x] = cb.x * co.x - cb.y * co.y; sn[x] = cb.y * co.x + cb.x * co.y;
+              const float cm = cb.x * co.x - cb.y * co.y, sn = cb.y * co.x + cb.x * co.y;
+              qh1[x] = (a[x] * cm + c[x] * sn) * p.qscale;
+              qh2[x] = (-a[x] * sn + c[x] * cm) * p.qscale;
             }
-          }
+          } else {
 #pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {
-            if (hh < nh) {
-              const int n = (int)rank * g.hl + hl0 + hh;
-              float a[8], c[8];
-              unpack8(__ldg(reinterpret_cast<const uint4*>(Q + n * DK + 8 * jl)), a);
-              unpack8(__ldg(reinterpret_cast<const uint4*>(Q + n * DK + PAIRS + 8 * jl)), c);
-#pragma unroll
-              for (int x = 0; x < 8; ++x) {
-                if (ROPE) {
-                  q1[hh][x] = (a[x] * cm[x] + c[x] * sn[x]) * p.qscale;
-                  q2[hh][x] = (-a[x] * sn[x] + c[x] * cm[x]) * p.qscale;
-                } else {
-                  q1[hh][x] = a[x] * p.qscale; q2[hh][x] = c[x] * p.qscale;
-                }
-              }
-            } else {
-#pragma unroll
-              for (int x = 0; x < 8; ++x) { q1[hh][x] = 0.f; q2[hh][x] = 0.f; }
-            }
+            for (int x = 0; x < 8; ++x) { qh1[x] = a[x] * p.qscale; qh2[x] = c[x] * p.qscale; }
           }
         }
+        // Q(t) = q^ e^{i t theta}: (Qa, Qb) weight the first / second half of the head
+        f32x2 Qa[4], Qb[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) { Qa[x] = pack2(qh1[2 * x], qh1[2 * x + 1]); Qb[x] = pack2(qh2[2 * x], qh2[2 * x + 1]); }
         float mref = 0.f, lsum = 0.f;
 
         for (int kt = 0; kt < ntile && ok; ++kt, ++it) {
@@ -332,6 +359,18 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           const uint32_t kbase = k_stage0 + (uint32_t)st * g.stage_bytes;
           float sv = 0.f;
           if (scorer) {
+            if (ROPE && active && (kt % TC_RESEED) == 0) {
+              // exact Q at this thread's first row of the tile (position t0 + rp)
+#pragma unroll
+              for (int x = 0; x < 4; ++x) {
+                const float4 cb = __ldg(reinterpret_cast<const float4*>(p.rope_base + (size_t)tile * PAIRS + 8 * jl + 2 * x));
+                const float4 co = __ldg(reinterpret_cast<const float4*>(p.rope_off + rp * PAIRS + 8 * jl + 2 * x));
+                const float c0 = cb.x * co.x - cb.y * co.y, s0 = cb.y * co.x + cb.x * co.y;
+                const float c1 = cb.z * co.z - cb.w * co.w, s1 = cb.w * co.z + cb.z * co.w;
+                Qa[x] = pack2(qh1[2 * x] * c0 - qh2[2 * x] * s0, qh1[2 * x + 1] * c1 - qh2[2 * x + 1] * s1);
+                Qb[x] = pack2(qh1[2 * x] * s0 + qh2[2 * x] * c0, qh1[2 * x + 1] * s1 + qh2[2 * x + 1] * c1);
+              }
+            }
             ok = mbar_wait<false>(bar_k_full + 8 * st, (it / g.ns) & 1, s_abort, p.status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -342,85 +381,63 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
                 for (int e = lane; e < (SLIM_TT - nz) * 8; e += 32)
                   sts128_zero(kbase + (uint32_t)c64 * 2048u + (uint32_t)(nz + (e >> 3)) * 128u + (uint32_t)(e & 7) * 16u);
             }
-            // ---- a4: softmax arguments of this warp's heads ----
-            float acc[2][RT];
+            // ---- a4: softmax arguments: this thread's partial sums for its RT rows ----
+            float v[RT];
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh)
-#pragma unroll
-              for (int r = 0; r < RT; ++r) acc[hh][r] = 0.f;
+            for (int i = 0; i < RT; ++i) v[i] = 0.f;
             if (active) {
-              float2 cur[8];
-              if (ROPE) {
-                const float4* bp = reinterpret_cast<const float4*>(p.rope_base + (size_t)tile * PAIRS + 8 * jl);
 #pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                  const float4 v = __ldg(bp + x);
-                  const float2 o0 = off_first[2 * x], o1 = off_first[2 * x + 1];
-                  cur[2 * x] = make_float2(v.x * o0.x - v.y * o0.y, v.y * o0.x + v.x * o0.y);
-                  cur[2 * x + 1] = make_float2(v.z * o1.x - v.w * o1.y, v.w * o1.x + v.z * o1.y);
-                }
-              }
-#pragma unroll
-              for (int r = 0; r < RT; ++r) {
-                const int row = tg * RT + r;
+              for (int i = 0; i < RT; ++i) {
+                const int row = rp + RP * i;
                 const uint32_t rbase = kbase + (uint32_t)row * 128u;
                 const uint32_t sw = (uint32_t)(row & 7);
+                const uint4 ka = lds128(rbase + koff[0] + ((kunit[0] ^ sw) << 4));
+                const uint4 kb = lds128(rbase + koff[1] + ((kunit[1] ^ sw) << 4));
+                f32x2 acc0 = mul2(unpack2(ka.x), Qa[0]);
+                f32x2 acc1 = mul2(unpack2(kb.x), Qb[0]);
+                acc0 = fma2(unpack2(ka.y), Qa[1], acc0); acc1 = fma2(unpack2(kb.y), Qb[1], acc1);
+                acc0 = fma2(unpack2(ka.z), Qa[2], acc0); acc1 = fma2(unpack2(kb.z), Qb[2], acc1);
+                acc0 = fma2(unpack2(ka.w), Qa[3], acc0); acc1 = fma2(unpack2(kb.w), Qb[3], acc1);
+                v[i] = sum2(add2(acc0, acc1));
+                if (ROPE) {
 #pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                  if (hh < nh) {
-                    float k1[8], k2[8];
-                    unpack8(lds128(rbase + koff[hh][0] + ((kunit[hh][0] ^ sw) << 4)), k1);
-                    unpack8(lds128(rbase + koff[hh][1] + ((kunit[hh][1] ^ sw) << 4)), k2);
-                    float a = acc[hh][r];
-#pragma unroll
-                    for (int x = 0; x < 8; ++x) {
-                      if (ROPE) {
-                        const float A = fmaf(q1[hh][x], k1[x], q2[hh][x] * k2[x]);
-                        const float Bv = fmaf(q1[hh][x], k2[x], -(q2[hh][x] * k1[x]));
-                        a = fmaf(cur[x].x, A, a);
-                        a = fmaf(cur[x].y, Bv, a);
-                      } else {
-                        a = fmaf(q1[hh][x], k1[x], a);
-                        a = fmaf(q2[hh][x], k2[x], a);
-                      }
-                    }
-                    acc[hh][r] = a;
-                  }
-                }
-                if (ROPE && r + 1 < RT) {
-#pragma unroll
-                  for (int x = 0; x < 8; ++x) {
-                    const float2 c = cur[x], s = stepv[x];
-                    cur[x] = make_float2(c.x * s.x - c.y * s.y, c.y * s.x + c.x * s.y);
+                  for (int x = 0; x < 4; ++x) {
+                    const f32x2 na = fma2(Qb[x], stn[x], mul2(Qa[x], stc[x]));
+                    Qb[x] = fma2(Qa[x], sts[x], mul2(Qb[x], stc[x]));
+                    Qa[x] = na;
                   }
                 }
               }
             }
-            // sum over the lanes that share (head, row), then pick this lane's value
+            // sum over the JL lanes of a (head, row set); lane jl keeps row rp + RP jl
+            {
+              int n = RT;
 #pragma unroll
-            for (int o = 1; o < JL; o <<= 1)
+              for (int o = JL / 2; o >= 1; o >>= 1) {
+                const int half = n / 2;
+                const bool up = (jl & o) != 0;
 #pragma unroll
-              for (int hh = 0; hh < 2; ++hh)
-#pragma unroll
-                for (int r = 0; r < RT; ++r) acc[hh][r] += __shfl_xor_sync(0xffffffffu, acc[hh][r], o);
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh)
-#pragma unroll
-              for (int r = 0; r < RT; ++r)
-                if (hh == my_hh && r == my_r) sv = acc[hh][r];
-            const bool valid = my_head_valid && (t0 + my_row < len);
+                for (int i = 0; i < half; ++i) {
+                  const float send = up ? v[i] : v[i + half];
+                  const float keep = up ? v[i + half] : v[i];
+                  v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+                }
+                n = half;
+              }
+              sv = v[0];
+            }
+            const bool valid = head_valid && (t0 + my_row < len);
             // ---- a5: probabilities against the fixed reference of this unit ----
             if (kt == 0) {
               float mx = valid ? sv : -INFINITY;
 #pragma unroll
-              for (int o = 1; o < 32; o <<= 1)
-                if (o != RT) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+              for (int o = 1; o < HL; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
               mref = mx;
               lsum = 0.f;
             }
             float x = sv - mref;
             if (valid && x > TC_XMAX) { p.unit_flags[unit] = 1; x = TC_XMAX; }
-            const float pf = valid ? exp2f(x) : 0.f;
+            const float pf = valid ? ex2_approx(x) : 0.f;
             const __nv_bfloat16 pb = __float2bfloat16_rn(pf);
             lsum += __bfloat162float(pb);
             // the P stage is free once the MMAs of tile it - TC_NP are done in both CTAs
@@ -428,24 +445,25 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const uint32_t paddr = p_stage0 + (uint32_t)ps * TC_P_BYTES + my_poff;
-            if (my_head_valid) {
+            if (head_valid) {
               st_cluster_u16(mapa(paddr, 0), __bfloat16_as_ushort(pb));
               st_cluster_u16(mapa(paddr, 1), __bfloat16_as_ushort(pb));
             }
             fence_proxy_async();
-            mbar_arrive_cluster(mapa(bar_p_full + 8 * ps, 0));
-            mbar_arrive_cluster(mapa(bar_p_full + 8 * ps, 1));
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_k_empty + 8 * st);
+            if (lane == 0) {
+              mbar_arrive_cluster(mapa(bar_p_full + 8 * ps, 0));
+              mbar_arrive_cluster(mapa(bar_p_full + 8 * ps, 1));
+              mbar_arrive(bar_k_empty + 8 * st);
+            }
           }
         }
         if (!ok) break;
         // ---- partial of this unit: (m_ref, l) per head, then U from tensor memory ----
         if (scorer) {
 #pragma unroll
-          for (int o = 1; o < 32; o <<= 1)
-            if (o != RT) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
-          if (my_head_valid && tg == 0 && my_r == 0) {
+          for (int o = 1; o < HL; o <<= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
+          if (head_valid && (lane % HL) == 0) {
             p.part_m[(size_t)unit * p.H + my_n] = mref;
             p.part_l[(size_t)unit * p.H + my_n] = lsum;
           }
