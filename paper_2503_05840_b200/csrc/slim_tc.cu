@@ -19,8 +19,10 @@
 //                   to row by one packed complex multiplication in registers
 //                   (re-seeded from the tables every TC_RESEED tiles).  The
 //                   arguments become p = 2^(s - m_ref); the bf16 probabilities
-//                   are written into the P tile of BOTH CTAs (distributed
-//                   shared memory), because every head weights the full key row;
+//                   are shipped into the P tile of BOTH CTAs with st.async
+//                   (distributed shared memory; the bytes complete on the
+//                   receiver's p_full barrier, so no thread waits on a remote
+//                   fence), because every head weights the full key row;
 //   MMA warp        U^T[128 cols x 32 heads] += K_tile^T[128 x 16] P^T[16 x 32]
 //                   for every 128-column chunk of the slice: one tcgen05.mma
 //                   per chunk, A = the staged keys (MN-major, straight from
@@ -40,6 +42,7 @@
 // device status to SLIM_ERR_TIMEOUT, all roles leave their loops, and the CTA
 // frees its tensor memory and exits.
 #include <cuda.h>
+#include <cstdlib>
 #include <cstring>
 
 #include "slim_internal.h"
@@ -50,6 +53,7 @@ namespace {
 constexpr int TC_NP = 4;                 // P-tile stages
 constexpr int TC_P_BYTES = 1024;         // [32 heads][16 rows] bf16
 constexpr int TC_MAX_NS = 8;             // K stages
+constexpr int TC_MAX_SW = 16;            // score warps
 constexpr float TC_XMAX = 96.f;          // largest exponent accepted above m_ref
 constexpr int TC_RESEED = 32;            // tiles between exact re-seeds of the stepped query rotation
 constexpr unsigned long long TC_WAIT_NS = 2000000000ull;
@@ -59,7 +63,7 @@ struct TcGeom {
   int nch;          // 128-column chunks per CTA
   int nc64;         // 64-column TMA chunks per CTA
   int hl;           // heads per CTA
-  int nsw;          // score warps (two heads each)
+  int nsw;          // score warps (tc_heads_per_warp heads each)
   int nswl;         // launched score/epilogue warps = max(4, nsw)
   int ns;           // K stages
   int stage_bytes;  // 16 * dsl * 2
@@ -81,15 +85,19 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
 __device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank) {
   uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank)); return r;
 }
-__device__ __forceinline__ void st_cluster_u16(uint32_t cluster_addr, unsigned short v) {
-  asm volatile("st.shared::cluster.u16 [%0], %1;" ::"r"(cluster_addr), "h"(v) : "memory");
+// 16 bytes into (possibly another CTA's) shared memory; the same 16 bytes are
+// counted as completed on the mbarrier at cluster_bar, which lives in the target CTA.
+__device__ __forceinline__ void st_async_v4(uint32_t cluster_addr, const uint4& v, uint32_t cluster_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+               ::"r"(cluster_addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(cluster_bar) : "memory");
 }
+__device__ __forceinline__ void sts_u16(uint32_t addr, unsigned short v) {
+  asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
@@ -228,18 +236,27 @@ __device__ __forceinline__ float ex2_approx(float x) {
   float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y;
 }
 
+// Lane mapping of the score warps: JL lanes share a (head, row set); a thread
+// owns RT rows of the tile; 16 / RT row sets and JL lanes make one head.
+__host__ __device__ constexpr int tc_jl(int dk) { return dk / 16 <= 4 ? 4 : 8; }
+__host__ __device__ constexpr int tc_heads_per_warp(int dk, int rt) { return 32 / (tc_jl(dk) * (SLIM_TT / rt)); }
+__host__ __device__ constexpr int tc_threads(int dk, int rt) {
+  // up to 16 heads per CTA, at least four score/epilogue warps, plus the producer and MMA warps
+  return 32 * ((16 / tc_heads_per_warp(dk, rt) < 4 ? 4 : 16 / tc_heads_per_warp(dk, rt)) + 2);
+}
+
 // ------------------------------------------------------------------ the kernel
-template <int DK, bool ROPE>
-__global__ void __launch_bounds__(320, 1)
+template <int DK, bool ROPE, int RT>
+__global__ void __launch_bounds__(tc_threads(DK, RT), 1)
 slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams p, const TcGeom g) {
   constexpr int PAIRS = DK / 2;                   // rotation pairs (j, j + DK/2) per head
   constexpr int OCT = PAIRS / 8;                  // 8-pair groups per head
-  constexpr int JL = OCT <= 4 ? 4 : 8;            // lanes along j (lanes >= OCT idle)
-  constexpr int RT = JL;                          // rows per thread and tile
-  constexpr int RP = SLIM_TT / RT;                // a thread owns rows rp, rp + RP, ...
+  constexpr int JL = tc_jl(DK);                   // lanes along j (lanes >= OCT idle)
+  constexpr int RP = SLIM_TT / RT;                // a thread owns the RT rows rp, rp + RP, ...
+  constexpr int DUP = JL / RT;                    // lanes that end up with the same row's sum
   constexpr int HL = JL * RP;                     // lanes per head
   constexpr int HW = 32 / HL;                     // heads per warp
-  static_assert(HW == 2, "TcGeom assumes two heads per score warp");
+  static_assert(RT <= JL && HL <= 32 && HW == tc_heads_per_warp(DK, RT), "lane mapping");
 
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_u32 = smem_u32(smem_raw);
@@ -247,7 +264,8 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   unsigned char* sm = smem_raw + (base - raw_u32);
   const uint32_t k_stage0 = base;
   const uint32_t p_stage0 = base + (uint32_t)g.ns * g.stage_bytes;
-  const uint32_t bars = p_stage0 + TC_NP * TC_P_BYTES;
+  const uint32_t stg0 = p_stage0 + TC_NP * TC_P_BYTES;            // per-warp P staging: 2 x 64 B
+  const uint32_t bars = stg0 + TC_MAX_SW * 128;
   const uint32_t bar_k_full = bars, bar_k_empty = bars + 8 * TC_MAX_NS;
   const uint32_t bar_p_full = bars + 16 * TC_MAX_NS, bar_p_empty = bar_p_full + 8 * TC_NP;
   const uint32_t bar_u_full = bar_p_empty + 8 * TC_NP, bar_u_empty = bar_u_full + 8;
@@ -264,7 +282,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   // ---- set-up -------------------------------------------------------------------
   if (tid == 0) {
     for (int i = 0; i < g.ns; ++i) { mbar_init(bar_k_full + 8 * i, 1); mbar_init(bar_k_empty + 8 * i, g.nsw + 1); }
-    for (int i = 0; i < TC_NP; ++i) { mbar_init(bar_p_full + 8 * i, 2 * g.nsw); mbar_init(bar_p_empty + 8 * i, 2); }
+    for (int i = 0; i < TC_NP; ++i) { mbar_init(bar_p_full + 8 * i, 1 + g.nsw); mbar_init(bar_p_empty + 8 * i, 2); }
     mbar_init(bar_u_full, 1);
     mbar_init(bar_u_empty, 4);
     *s_abort = 0;
@@ -296,8 +314,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
       const bool head_valid = scorer && hl < g.hl;
       const bool active = head_valid && jl < OCT;
       const int my_n = (int)rank * g.hl + hl;                    // global head
-      const int my_row = rp + RP * jl;                           // row whose argument this lane ends up with
-      const uint32_t my_poff = p_offset(my_n & 31, my_row);
+      const int my_row = rp + RP * (jl / DUP);                   // row whose argument this lane ends up with
       // byte offsets of this thread's two 16-byte key units (first / second half of the head)
       uint32_t koff[2], kunit[2];
 #pragma unroll
@@ -409,20 +426,24 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
                 }
               }
             }
-            // sum over the JL lanes of a (head, row set); lane jl keeps row rp + RP jl
+            // sum over the JL lanes of a (head, row set); lane jl keeps row rp + RP (jl / DUP)
             {
               int n = RT;
 #pragma unroll
               for (int o = JL / 2; o >= 1; o >>= 1) {
-                const int half = n / 2;
-                const bool up = (jl & o) != 0;
+                if (n > 1) {
+                  const int half = n / 2;
+                  const bool up = (jl & o) != 0;
 #pragma unroll
-                for (int i = 0; i < half; ++i) {
-                  const float send = up ? v[i] : v[i + half];
-                  const float keep = up ? v[i + half] : v[i];
-                  v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+                  for (int i = 0; i < half; ++i) {
+                    const float send = up ? v[i] : v[i + half];
+                    const float keep = up ? v[i + half] : v[i];
+                    v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+                  }
+                  n = half;
+                } else {
+                  v[0] += __shfl_xor_sync(0xffffffffu, v[0], o);
                 }
-                n = half;
               }
               sv = v[0];
             }
@@ -439,21 +460,33 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             if (valid && x > TC_XMAX) { p.unit_flags[unit] = 1; x = TC_XMAX; }
             const float pf = valid ? ex2_approx(x) : 0.f;
             const __nv_bfloat16 pb = __float2bfloat16_rn(pf);
-            lsum += __bfloat162float(pb);
+            if ((jl % DUP) == 0) lsum += __bfloat162float(pb);
             // the P stage is free once the MMAs of tile it - TC_NP are done in both CTAs
             ok = mbar_wait<false>(bar_p_empty + 8 * ps, ((it / TC_NP) & 1) ^ 1, s_abort, p.status);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            const uint32_t paddr = p_stage0 + (uint32_t)ps * TC_P_BYTES + my_poff;
-            if (head_valid) {
-              st_cluster_u16(mapa(paddr, 0), __bfloat16_as_ushort(pb));
-              st_cluster_u16(mapa(paddr, 1), __bfloat16_as_ushort(pb));
+            {
+              // stage this warp's probabilities in the K-major order of the P tile, then ship
+              // them in 16-byte pieces (8 rows of one head) to both CTAs
+              const uint32_t stg = stg0 + (uint32_t)warp * 128u + (uint32_t)(it & 1) * 64u;
+              if ((jl % DUP) == 0) sts_u16(stg + (uint32_t)(hw * 16 + my_row) * 2u, __bfloat16_as_ushort(pb));
+              __syncwarp();
+              if (lane < 4 * HW) {
+                const int hsel = lane >> 2, half = (lane >> 1) & 1, dest = lane & 1;
+                const int hl_s = HW * warp + hsel;
+                if (hl_s < g.hl) {
+                  const uint4 pv = lds128(stg + (uint32_t)(hsel * 16 + half * 8) * 2u);
+                  const int n_s = (int)rank * g.hl + hl_s;
+                  const uint32_t dst = p_stage0 + (uint32_t)ps * TC_P_BYTES + p_offset(n_s & 31, half * 8);
+                  st_async_v4(mapa(dst, dest), pv, mapa(bar_p_full + 8 * ps, dest));
+                }
+              }
             }
-            fence_proxy_async();
+            // The local arrival releases this warp's zero-fill of the K stage (if any) to the
+            // MMA thread, whose proxy fence orders it before the tensor-core reads.
             __syncwarp();
             if (lane == 0) {
-              mbar_arrive_cluster(mapa(bar_p_full + 8 * ps, 0));
-              mbar_arrive_cluster(mapa(bar_p_full + 8 * ps, 1));
+              mbar_arrive(bar_p_full + 8 * ps);
               mbar_arrive(bar_k_empty + 8 * st);
             }
           }
@@ -521,6 +554,11 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
       if (lane == 0) {
         int it = 0, uc = 0;
         bool ok = true;
+        // p_full of a tile completes on: this thread's arming arrival + the local score
+        // warps' arrivals + 32 bytes per head shipped by the score warps of both CTAs
+        const int total_it = g_end - g_begin;
+        const uint32_t p_bytes = (uint32_t)p.H * 32u;
+        for (int i = 0; i < TC_NP && i < total_it; ++i) mbar_arrive_expect_tx(bar_p_full + 8 * i, p_bytes);
         for (int gg = g_begin; gg < g_end && ok; ++uc) {
           const int b = slim_seq_of_tile(s_prefix, p.batch, gg);
           const int seg_end = min(g_end, s_prefix[b + 1]);
@@ -531,7 +569,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             if (ok) ok = mbar_wait<true>(bar_p_full + 8 * ps, (it / TC_NP) & 1, s_abort, p.status);
             if (ok && kt == 0 && uc > 0) ok = mbar_wait<false>(bar_u_empty, (uc - 1) & 1, s_abort, p.status);
             if (!ok) break;
-            fence_proxy_async();
+            fence_proxy_async_smem();        // P pieces and zero-filled key rows -> tensor-core reads
             tc_fence_after();
             const uint64_t bd = desc_b(p_stage0 + (uint32_t)ps * TC_P_BYTES);
             const uint32_t kbase = k_stage0 + (uint32_t)st * g.stage_bytes;
@@ -539,6 +577,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
               umma_bf16(tmem_base + (uint32_t)(c * 32), desc_a(kbase + (uint32_t)c * 4096u), bd, TC_IDESC, kt > 0 ? 1u : 0u);
             umma_commit(bar_k_empty + 8 * st);
             umma_commit_pair(bar_p_empty + 8 * ps);
+            if (it + TC_NP < total_it) mbar_arrive_expect_tx(bar_p_full + 8 * ps, p_bytes);
             if (kt == ntile - 1) umma_commit(bar_u_full);
           }
           gg = seg_end;
@@ -559,13 +598,14 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
 }
 
 // ------------------------------------------------------------------ host side
-TcGeom make_geom(int d, int H, int d_k, int smem_limit) {
+TcGeom make_geom(int d, int H, int d_k, int rt, int smem_limit) {
   TcGeom g;
   g.dsl = d / 2;
   g.nch = g.dsl / 128;
   g.nc64 = g.dsl / 64;
   g.hl = H / 2;
-  g.nsw = (g.hl + 1) / 2;
+  const int hw = tc_heads_per_warp(d_k, rt);
+  g.nsw = (g.hl + hw - 1) / hw;
   g.nswl = g.nsw < 4 ? 4 : g.nsw;
   g.stage_bytes = SLIM_TT * g.dsl * 2;
   int ns = (smem_limit - 16 * 1024) / g.stage_bytes;
@@ -577,7 +617,7 @@ TcGeom make_geom(int d, int H, int d_k, int smem_limit) {
 }
 
 size_t tc_smem_bytes(const TcGeom& g, int batch) {
-  size_t need = 1024 + (size_t)g.ns * g.stage_bytes + TC_NP * TC_P_BYTES + 16 * TC_MAX_NS + 16 * TC_NP + 16 + 8 +
+  size_t need = 1024 + (size_t)g.ns * g.stage_bytes + TC_NP * TC_P_BYTES + TC_MAX_SW * 128 + 16 * TC_MAX_NS + 16 * TC_NP + 16 + 8 +
                 sizeof(int) * (batch + 1) + 64;
   const size_t floor_bytes = 120 * 1024;         // one CTA per SM: tensor memory is not shared
   return need < floor_bytes ? floor_bytes : need;
@@ -585,11 +625,25 @@ size_t tc_smem_bytes(const TcGeom& g, int batch) {
 
 typedef void (*tc_kernel_t)(const CUtensorMap, const SlimDecodeParams, const TcGeom);
 
-tc_kernel_t pick_kernel(int d_k, bool rope) {
-  switch (d_k) {
-    case 64: return rope ? slim_tc_kernel<64, true> : slim_tc_kernel<64, false>;
-    case 96: return rope ? slim_tc_kernel<96, true> : slim_tc_kernel<96, false>;
-    case 128: return rope ? slim_tc_kernel<128, true> : slim_tc_kernel<128, false>;
+// Rows per thread and tile.  Measured on the d = 4096 / 32-head shape: 8 rows per
+// thread (8 score warps) beats 4 rows (16 warps); the stepped query rotation is
+// re-used over more rows and fewer warps contend for the issue slots.
+// SLIM_TC_RT overrides the choice for sweeps.
+int tc_rows_per_thread(int d_k) {
+  const char* e = getenv("SLIM_TC_RT");
+  const int want = e ? atoi(e) : 0;
+  if (d_k == 64) return want == 2 ? 2 : 4;
+  return want == 4 ? 4 : 8;
+}
+
+tc_kernel_t pick_kernel(int d_k, bool rope, int rt) {
+  switch (d_k * 16 + rt) {
+    case 64 * 16 + 2: return rope ? slim_tc_kernel<64, true, 2> : slim_tc_kernel<64, false, 2>;
+    case 64 * 16 + 4: return rope ? slim_tc_kernel<64, true, 4> : slim_tc_kernel<64, false, 4>;
+    case 96 * 16 + 4: return rope ? slim_tc_kernel<96, true, 4> : slim_tc_kernel<96, false, 4>;
+    case 96 * 16 + 8: return rope ? slim_tc_kernel<96, true, 8> : slim_tc_kernel<96, false, 8>;
+    case 128 * 16 + 4: return rope ? slim_tc_kernel<128, true, 4> : slim_tc_kernel<128, false, 4>;
+    case 128 * 16 + 8: return rope ? slim_tc_kernel<128, true, 8> : slim_tc_kernel<128, false, 8>;
     default: return nullptr;
   }
 }
@@ -607,9 +661,10 @@ int slim_tc_shape_ok(int d, int H, int d_k, int dtype) {
 }
 
 int slim_tc_workers(const slim_ctx* ctx) {
-  tc_kernel_t kern = pick_kernel(ctx->d_k, ctx->rope_theta != 0.0);
+  const int rt = tc_rows_per_thread(ctx->d_k);
+  tc_kernel_t kern = pick_kernel(ctx->d_k, ctx->rope_theta != 0.0, rt);
   if (!kern) return 0;
-  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, TC_SMEM_LIMIT);
+  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, rt, TC_SMEM_LIMIT);
   if (g.ns < 2) return 0;
   const size_t smem = tc_smem_bytes(g, SLIM_MAX_BATCH);
   if (smem > (size_t)TC_SMEM_LIMIT) return 0;
@@ -647,7 +702,7 @@ cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c) {
     if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
     encode = (encode_t)fn;
   }
-  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, TC_SMEM_LIMIT);
+  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, tc_rows_per_thread(ctx->d_k), TC_SMEM_LIMIT);
   // dim0: 64 contiguous elements; dim1: cache rows (stride d elements); dim2: 64-column chunks
   const cuuint64_t dims[3] = {64, (cuuint64_t)c->batch * (cuuint64_t)c->t_cap, (cuuint64_t)(ctx->d / 64)};
   const cuuint64_t strides[2] = {(cuuint64_t)ctx->d * 2, 128};
@@ -660,9 +715,10 @@ cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c) {
 }
 
 cudaError_t slim_launch_tc(const slim_ctx* ctx, const slim_cache* c, const SlimDecodeParams& p, cudaStream_t st) {
-  tc_kernel_t kern = pick_kernel(ctx->d_k, ctx->rope_theta != 0.0);
+  const int rt = tc_rows_per_thread(ctx->d_k);
+  tc_kernel_t kern = pick_kernel(ctx->d_k, ctx->rope_theta != 0.0, rt);
   if (!kern || !c->has_tmap) return cudaErrorNotSupported;
-  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, TC_SMEM_LIMIT);
+  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, rt, TC_SMEM_LIMIT);
   const size_t smem = tc_smem_bytes(g, p.batch);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * p.workers);
