@@ -1,0 +1,63 @@
+"""World-size-2 check (gloo, CPU) of the replica logic bench.py uses for N > 1:
+distinct per-rank seeds, identical length mix, max-over-ranks timing, whole-job
+throughput.  No GPU and no CUDA library is touched."""
+import os
+import socket
+import sys
+
+import numpy as np
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    p = s.getsockname()[1]
+    s.close()
+    return p
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    import torch.distributed as dist
+    from paper_2503_05840_b200 import replicas, synth
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    r, w, _ = replicas.rank_info()
+    cfg = synth.CONFIGS[2].scaled(batch=4, context=256, ragged_min=128, d=64, H=2, d_k=32)
+    base = synth.layer_seed(2, 0)
+    lengths = synth.make_lengths(cfg, base)                       # same on every rank
+    L = synth.make_layer(cfg, replicas.replica_seed(base, r), lengths=lengths)
+    ms = replicas.max_over_ranks(10.0 + 5.0 * r, dist)            # rank 1 is the slow one
+    dist.barrier()
+    out.put((r, w, lengths.tolist(), float(L.K[0, 0, 0]), ms, replicas.job_throughput(cfg.batch, w, ms)))
+    dist.destroy_process_group()
+
+
+def test_two_replicas_share_only_timing():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(60)
+        assert p.exitcode == 0
+    (r0, w0, len0, k0, ms0, v0), (r1, w1, len1, k1, ms1, v1) = res
+    assert (r0, r1) == (0, 1) and w0 == w1 == 2
+    assert len0 == len1                                  # equal work per rank
+    assert k0 != k1                                      # different data per rank
+    assert ms0 == ms1 == 15.0                            # slowest rank's time on both
+    assert np.isclose(v0, 4 * 2 / 15e-3) and v0 == v1    # units of all ranks / that time
+
+
+def test_single_process_needs_no_group():
+    sys.path.insert(0, ROOT)
+    from paper_2503_05840_b200 import replicas
+    assert replicas.max_over_ranks(3.5) == 3.5
+    assert replicas.replica_seed(7, 0) == 7 and replicas.replica_seed(7, 3) != replicas.replica_seed(7, 2)
