@@ -42,7 +42,8 @@ typedef enum {
   SLIM_ERR_OOM = 5,          /* a library-owned allocation failed                   */
   SLIM_ERR_CUDA = 6,         /* CUDA runtime/driver error, or no device             */
   SLIM_ERR_TIMEOUT = 7,      /* a bounded device-side wait ran out (device)         */
-  SLIM_ERR_NO_WEIGHTS = 8    /* slim_decode before slim_set_weights / slim_set_wkv  */
+  SLIM_ERR_NO_WEIGHTS = 8,   /* slim_decode before slim_set_weights / slim_set_wkv  */
+  SLIM_ERR_STATIC_WS = 9     /* slim_decode_static_ws: scratch need above the built-in maximum */
 } slim_status;
 
 typedef enum { SLIM_F32 = 0, SLIM_BF16 = 1 } slim_dtype;      /* cache / query dtype   */
@@ -118,6 +119,30 @@ slim_status slim_append_k(slim_ctx* ctx, slim_cache* cache, const void* k_new,
  *            aligned; contents are scratch                                    */
 slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache,
                         const int32_t* lengths, float* o, void* workspace, void* stream);
+
+/* slim_decode for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; this is a convenience of the library.)  Some hosts of this code must
+ * not call cudaMalloc or any allocator while they run: a serving loop whose memory
+ * pool is frozen after start-up, a plug-in that is handed a device it does not own,
+ * code running where an allocation would synchronise the whole device.  For them the
+ * scratch that slim_decode takes as `workspace` lives in a fixed array inside the
+ * library: slim_static_workspace_max() bytes (16 MiB) of device memory that every
+ * GPU which loads the library keeps until the process exits.  Same arguments and
+ * result as slim_decode, minus `workspace`; no device or host memory is allocated or
+ * freed by the call.
+ *   - If slim_workspace_bytes(ctx, batch, t_cap) of the cache exceeds the maximum,
+ *     nothing is launched and SLIM_ERR_STATIC_WS is returned (use slim_decode with
+ *     your own workspace for such sizes; the need grows with batch, H*d and the SM count).
+ *   - The ctx's device must be the current device.  The first call on a device looks
+ *     up the array's device address (once per device); make that first call before
+ *     starting any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the previous
+ *     call left.  The kernels write every word before they read it, so nothing needs
+ *     clearing, but two calls whose kernels overlap on the GPU (different streams,
+ *     different ctx objects) race on it: run them one after another.              */
+size_t      slim_static_workspace_max(void);
+slim_status slim_decode_static_ws(slim_ctx* ctx, const void* q, const slim_cache* cache,
+                                  const int32_t* lengths, float* o, void* stream);
 
 /* Synchronises `stream`, returns the sticky device status (SLIM_OK,
  * SLIM_ERR_CAPACITY or SLIM_ERR_TIMEOUT) and clears it.                        */

@@ -14,7 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libslim.so")
 
 SLIM_OK, SLIM_ERR_INVALID_ARG, SLIM_ERR_UNSUPPORTED, SLIM_ERR_SINGULAR, SLIM_ERR_CAPACITY, \
-    SLIM_ERR_OOM, SLIM_ERR_CUDA, SLIM_ERR_TIMEOUT, SLIM_ERR_NO_WEIGHTS = range(9)
+    SLIM_ERR_OOM, SLIM_ERR_CUDA, SLIM_ERR_TIMEOUT, SLIM_ERR_NO_WEIGHTS, SLIM_ERR_STATIC_WS = range(10)
 SLIM_F32, SLIM_BF16 = 0, 1
 SLIM_HOST_F32, SLIM_HOST_F64 = 0, 1
 SLIM_PATH_AUTO, SLIM_PATH_GENERIC, SLIM_PATH_TC = 0, 1, 2
@@ -32,6 +32,8 @@ SIGNATURES = {
     "slim_cache_destroy": (None, [c_void_p]),
     "slim_append_k": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]),
     "slim_decode": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "slim_static_workspace_max": (c_size_t, []),
+    "slim_decode_static_ws": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "slim_device_status": (c_int, [c_void_p, c_void_p]),
     "slim_profile_enable": (c_int, [c_void_p, c_int]),
     "slim_profile_read": (c_int, [c_void_p, POINTER(ctypes.c_float), POINTER(ctypes.c_float)]),
@@ -149,6 +151,16 @@ def slim_append_k(ctx: int, cache: int, k_new, positions, n_new: int, stream: in
 def slim_decode(ctx: int, q, cache: int, lengths, o, workspace, stream: int = 0) -> None:
     _check(lib().slim_decode(c_void_p(ctx), _ptr(q), c_void_p(cache), _ptr(lengths), _ptr(o), _ptr(workspace),
                              c_void_p(stream)), "slim_decode")
+
+
+def slim_static_workspace_max() -> int:
+    return lib().slim_static_workspace_max()
+
+
+def slim_decode_static_ws(ctx: int, q, cache: int, lengths, o, stream: int = 0) -> None:
+    """slim_decode with the library's built-in scratch: for callers that must not allocate."""
+    _check(lib().slim_decode_static_ws(c_void_p(ctx), _ptr(q), c_void_p(cache), _ptr(lengths), _ptr(o),
+                                       c_void_p(stream)), "slim_decode_static_ws")
 
 
 def slim_device_status(ctx: int, stream: int = 0) -> int:

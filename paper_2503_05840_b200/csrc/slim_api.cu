@@ -3,12 +3,20 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
 #include "slim_internal.h"
 
 size_t slim_tail_opart_floats(int d, int batch);
+
+// Built-in scratch for slim_decode_static_ws: device memory that exists from the moment
+// the library is loaded on a GPU until the process exits, so that entry point never has
+// to ask an allocator for anything.  In host code this name is only a handle for
+// cudaGetSymbolAddress; the real device address is looked up once per device below.
+#define SLIM_STATIC_WS_BYTES (16u << 20)
+static __device__ __align__(256) unsigned char slim_static_ws[SLIM_STATIC_WS_BYTES];
 
 namespace {
 
@@ -93,6 +101,27 @@ slim_status upload_f64(const void* src, int host_dtype, size_t n, double** dev_o
   return SLIM_OK;
 }
 
+// Device address of slim_static_ws on `device` (which must be the current device).
+// Looked up on the first call per device and remembered.
+constexpr int kMaxDevices = 64;
+void* g_static_ws_ptr[kMaxDevices] = {};
+std::mutex g_static_ws_mutex;
+
+slim_status static_ws_address(int device, void** out) {
+  if (device < 0 || device >= kMaxDevices) return SLIM_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_ws_mutex);
+  if (!g_static_ws_ptr[device]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, slim_static_ws) != cudaSuccess || !ptr) {
+      cudaGetLastError();
+      return SLIM_ERR_CUDA;
+    }
+    g_static_ws_ptr[device] = ptr;
+  }
+  *out = g_static_ws_ptr[device];
+  return SLIM_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -108,6 +137,7 @@ const char* slim_strerror(int status) {
     case SLIM_ERR_CUDA: return "CUDA error or no CUDA device";
     case SLIM_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     case SLIM_ERR_NO_WEIGHTS: return "W_KV has not been set";
+    case SLIM_ERR_STATIC_WS: return "this batch / capacity needs more scratch than the built-in static workspace holds";
     default: return "unknown status";
   }
 }
@@ -303,6 +333,24 @@ slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   if (ctx->prof_on) { cudaEventRecord(ctx->prof_ev[2], st); ctx->prof_valid = 1; }
   if (e != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
   return SLIM_OK;
+}
+
+size_t slim_static_workspace_max(void) { return SLIM_STATIC_WS_BYTES; }
+
+slim_status slim_decode_static_ws(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,
+                                  float* o, void* stream) {
+  if (!ctx || !q || !cache || !lengths || !o || cache->ctx != ctx) return SLIM_ERR_INVALID_ARG;
+  const size_t need = ws_layout(ctx, cache->batch, cache->t_cap).total;
+  if (need > (size_t)SLIM_STATIC_WS_BYTES) return SLIM_ERR_STATIC_WS;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
+  if (dev != ctx->device) return SLIM_ERR_INVALID_ARG;          // the ctx's device must be current
+  void* ws = nullptr;
+  const slim_status st = static_ws_address(dev, &ws);
+  if (st != SLIM_OK) return st;
+  // Nothing in the scratch has to start at zero: every word the kernels read was written
+  // earlier in the same call (partials, redo flags, projection slices).
+  return slim_decode(ctx, q, cache, lengths, o, ws, stream);
 }
 
 slim_status slim_device_status(slim_ctx* ctx, void* stream) {
