@@ -24,7 +24,7 @@ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 inline size_t esize(int dtype) { return dtype == SLIM_BF16 ? 2 : 4; }
 
 struct WsLayout {
-  size_t part_u, part_m, part_l, flags, o_part, scores, total;
+  size_t part_u, part_m, part_l, flags, o_part, scores, u_tiled, total;
   int units;
 };
 
@@ -38,6 +38,7 @@ WsLayout ws_layout(const slim_ctx* ctx, int batch, int t_cap) {
   L.flags = off;  off = align256(off + sizeof(int) * (size_t)L.units);
   L.o_part = off; off = align256(off + sizeof(float) * slim_tail_opart_floats(ctx->d, batch));
   L.scores = off; off = align256(off + sizeof(float) * (size_t)batch * ctx->H * t_cap);   // generic path only
+  L.u_tiled = off; off = align256(off + (ctx->proj_ok ? slim_proj_u_bytes(ctx->d, ctx->H, batch) : 0));   // tensor-core tail only
   L.total = off;
   return L;
 }
@@ -175,6 +176,12 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
       slim_destroy(c);
       return SLIM_ERR_CUDA;
     }
+  }
+  c->proj_ok = prop.major == 10 ? slim_proj_shape_ok(d, H, d_k, dtype) : 0;
+  if (c->proj_ok && slim_proj_make_wmap(c) != cudaSuccess) { cudaGetLastError(); c->proj_ok = 0; }
+  {
+    const char* e = getenv("SLIM_TAIL");                 // "cuda" forces the CUDA-core tail (sweeps, tests)
+    if (e && !strcmp(e, "cuda")) c->proj_ok = 0;
   }
   c->tc_ok = prop.major == 10 ? slim_tc_shape_ok(d, H, d_k, dtype) : 0;
   c->gen_workers = slim_generic_workers(c);
@@ -329,7 +336,15 @@ slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, c
     e = slim_launch_generic(ctx, p, reinterpret_cast<float*>(ws + L.scores), st);
   }
   if (ctx->prof_on) cudaEventRecord(ctx->prof_ev[1], st);
-  if (e == cudaSuccess) e = slim_launch_tail(ctx, p, st);
+  if (e == cudaSuccess) {
+    if (ctx->proj_ok) {
+      float* o_part = reinterpret_cast<float*>(ws + L.o_part);
+      e = slim_launch_proj(ctx, p, reinterpret_cast<unsigned char*>(ws + L.u_tiled), o_part, st);
+      if (e == cudaSuccess) e = slim_launch_sum_slices(o_part, o, p.batch * p.d, slim_proj_jsplit(ctx->d), st);
+    } else {
+      e = slim_launch_tail(ctx, p, st);
+    }
+  }
   if (ctx->prof_on) { cudaEventRecord(ctx->prof_ev[2], st); ctx->prof_valid = 1; }
   if (e != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
   return SLIM_OK;
@@ -395,7 +410,8 @@ long long slim_query(const slim_ctx* ctx, int key) {
   const int path = path_in_use(ctx);
   switch (key) {
     case SLIM_Q_PATH_IN_USE: return path;
-    case SLIM_Q_LAUNCHES_PER_DECODE: return 4;   // tc: main, exact redo, tail1, tail2; generic: scores, accum, tail1, tail2
+    case SLIM_Q_LAUNCHES_PER_DECODE:              // main (tc: + exact redo; generic: scores + accum), then the tail
+      return 2 + (ctx->proj_ok ? 3 : 2);          // combine, projection, slice sum  |  combine+projection, slice sum
     case SLIM_Q_MAX_UNITS: return ctx->num_sms;   // + batch, known only per cache
     case SLIM_Q_NUM_SMS: return ctx->num_sms;
     case SLIM_Q_WORKERS: return path == SLIM_PATH_TC ? ctx->tc_workers : ctx->gen_workers;

@@ -56,6 +56,8 @@ struct slim_ctx {
   int gen_workers;
   int prof_on, prof_valid;
   cudaEvent_t prof_ev[3];
+  int proj_ok;                   // tensor-core combine + projection usable for this shape
+  alignas(64) unsigned char wmap[128];   // CUtensorMap over W_KV for the projection kernel
 };
 
 struct slim_cache {
@@ -85,3 +87,16 @@ int  slim_tc_shape_ok(int d, int H, int d_k, int dtype);
 int  slim_tc_workers(const slim_ctx* ctx);
 cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c);
 cudaError_t slim_launch_tc(const slim_ctx* ctx, const slim_cache* c, const SlimDecodeParams& p, cudaStream_t st);
+
+// 3-D tiled tensor map with 128-byte swizzle over bf16 data (driver entry point looked up once)
+cudaError_t slim_tmap_encode_3d(void* out_map, void* base, const unsigned long long dims[3],
+                                const unsigned long long strides[2], const unsigned int box[3]);
+
+// tensor-core combine + projection (slim_proj.cu)
+int    slim_proj_shape_ok(int d, int H, int d_k, int dtype);
+int    slim_proj_jsplit(int d);
+size_t slim_proj_u_bytes(int d, int H, int batch);
+cudaError_t slim_proj_make_wmap(slim_ctx* ctx);
+cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, unsigned char* u_tiled, float* o_part,
+                             cudaStream_t st);
+cudaError_t slim_launch_sum_slices(const float* o_part, float* o, int n, int nsplit, cudaStream_t st);

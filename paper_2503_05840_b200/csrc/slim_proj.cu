@@ -1,0 +1,289 @@
+// Tail of the decode step on the tensor cores (bf16 caches, d_k = 64 or 128):
+//
+//   slim_combine_kernel   log-sum-exp combine of the context-split partials:
+//                         u[b][h][:] = sum_s w_s U_s[h][:] / sum_s w_s l_s over the
+//                         units s of sequence b.  u is written as a bf16 pair
+//                         (hi = bf16(u), lo = bf16(u - hi)) directly in the
+//                         shared-memory operand layout of the projection MMA, so
+//                         the projection kernel fetches it with plain bulk copies.
+//   slim_proj_tc_kernel   the per-head projection o_h = u_h W_KV,h of Eq. 7
+//                         (Option 2) for 16 sequences at a time:
+//                         O^T[128 x N] += W_tile^T[128 x 16] u^T[16 x N] with one
+//                         tcgen05.mma per 16 rows of W_KV,h; A = the TMA-staged
+//                         weights used MN-major, B = the u tiles, D in tensor
+//                         memory.  N = 32 per head (16 sequences x {hi, lo}); for
+//                         d_k = 64 two heads share an instruction (M = 2 x 64,
+//                         N = 2 x 32) and the off-diagonal quadrants are ignored.
+//                         A CTA owns (head group, slice of the d rows of W_KV,h,
+//                         16-sequence group) and writes a projection slice that
+//                         slim_tail2_kernel sums in a fixed order.
+//
+// Every mbarrier wait is bounded in time; a wait that runs out sets the device
+// status to SLIM_ERR_TIMEOUT and the CTA drains and exits.
+#include <cstring>
+
+#include "slim_internal.h"
+#include "slim_sched.cuh"
+#include "slim_ptx.cuh"
+
+namespace {
+using namespace slim_ptx;
+
+constexpr int PJ_ROWS = 64;                    // rows of W_KV,h per stage (4 MMA k-steps)
+constexpr int PJ_W_BYTES = PJ_ROWS * 128 * 2;  // two 64-column atoms x 64 rows x 128 B
+constexpr int PJ_NS = 4;                       // stages
+constexpr int PJ_BG = 16;                      // sequences per MMA (N = 32 per head: hi and lo)
+
+struct ProjGeom {
+  int hp;        // heads per MMA: 1 (d_k = 128) or 2 (d_k = 64)
+  int hg;        // head groups = H / hp
+  int jsplit;    // slices of the d rows of W_KV,h
+  int nst;       // stages per CTA = d / 64 / jsplit
+  int nbg;       // 16-sequence groups
+  int u_bytes;   // bytes of u per stage = 4 k-steps x hp x 1 KB
+};
+
+__device__ __forceinline__ uint32_t u_offset(int n, int k) {      // K-major 8x8 core matrices, N = 32
+  return (uint32_t)((n & 7) * 16 + (n >> 3) * 256 + (k >> 3) * 128 + (k & 7) * 2);
+}
+
+__global__ void __launch_bounds__(256)
+slim_combine_kernel(const SlimDecodeParams p, unsigned char* __restrict__ u_tiled, const int hp) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* s_w = reinterpret_cast<float*>(smem_raw);                 // [workers]
+  int* s_info = reinterpret_cast<int*>(s_w + p.workers);           // wlo, wn
+  int* s_prefix = s_info + 2;                                      // [batch+1]
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int h = blockIdx.x, b = blockIdx.y, bg = b / PJ_BG, n = b % PJ_BG;
+  const int d = p.d, H = p.H;
+
+  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status);
+  if (tid < 32) {
+    int wlo = 0, wn = 0;
+    if (b < p.batch && s_prefix[b + 1] > s_prefix[b]) {
+      wlo = slim_worker_of_tile(sc, s_prefix[b]);
+      wn = slim_worker_of_tile(sc, s_prefix[b + 1] - 1) - wlo + 1;
+      float M = -INFINITY;
+      for (int i = lane; i < wn; i += 32) {
+        const size_t ui = (size_t)(wlo + i + b) * H + h;
+        M = fmaxf(M, p.part_m[ui] + log2f(p.part_l[ui]));
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+      float L = 0.f;
+      for (int i = lane; i < wn; i += 32) {
+        const size_t ui = (size_t)(wlo + i + b) * H + h;
+        const float wg = exp2f(p.part_m[ui] - M);
+        s_w[i] = wg;
+        L += wg * p.part_l[ui];
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+      const float inv = 1.f / L;
+      __syncwarp();
+      for (int i = lane; i < wn; i += 32) s_w[i] *= inv;
+    }
+    if (lane == 0) { s_info[0] = wlo; s_info[1] = wn; }
+  }
+  __syncthreads();
+  const int wlo = s_info[0], wn = s_info[1];
+  const size_t tile_bytes = (size_t)1024 * hp;
+  unsigned char* dst_h = u_tiled + ((size_t)(bg * (H / hp) + h / hp) * (d / 16)) * tile_bytes + (size_t)(h % hp) * 1024;
+  for (int jg = tid; jg < d / 8; jg += blockDim.x) {
+    const int j0 = jg * 8;
+    float acc[8];
+#pragma unroll
+    for (int x = 0; x < 8; ++x) acc[x] = 0.f;
+    for (int i = 0; i < wn; ++i) {
+      const float wg = s_w[i];
+      const float4* U = reinterpret_cast<const float4*>(p.part_u + ((size_t)(wlo + i + b) * H + h) * d + j0);
+      const float4 a = __ldg(U), c = __ldg(U + 1);
+      acc[0] = fmaf(wg, a.x, acc[0]); acc[1] = fmaf(wg, a.y, acc[1]); acc[2] = fmaf(wg, a.z, acc[2]); acc[3] = fmaf(wg, a.w, acc[3]);
+      acc[4] = fmaf(wg, c.x, acc[4]); acc[5] = fmaf(wg, c.y, acc[5]); acc[6] = fmaf(wg, c.z, acc[6]); acc[7] = fmaf(wg, c.w, acc[7]);
+    }
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const __nv_bfloat16 h0 = __float2bfloat16_rn(acc[2 * x]), h1 = __float2bfloat16_rn(acc[2 * x + 1]);
+      const __nv_bfloat16 l0 = __float2bfloat16_rn(acc[2 * x] - __bfloat162float(h0));
+      const __nv_bfloat16 l1 = __float2bfloat16_rn(acc[2 * x + 1] - __bfloat162float(h1));
+      hi[x] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+      lo[x] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+    }
+    unsigned char* t = dst_h + (size_t)(j0 / 16) * tile_bytes;
+    *reinterpret_cast<uint4*>(t + u_offset(n, j0 & 15)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    *reinterpret_cast<uint4*>(t + u_offset(PJ_BG + n, j0 & 15)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+  }
+}
+
+__global__ void __launch_bounds__(128)
+slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned char* __restrict__ u_tiled,
+                    float* __restrict__ o_part, const ProjGeom g, const int d, const int d_k, const int batch,
+                    int* status) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw_u32 = smem_u32(smem_raw);
+  const uint32_t base = (raw_u32 + 1023u) & ~1023u;
+  unsigned char* sm = smem_raw + (base - raw_u32);
+  const uint32_t stage_bytes = (uint32_t)(PJ_W_BYTES + g.u_bytes);
+  const uint32_t bars = base + PJ_NS * stage_bytes;
+  const uint32_t bar_full = bars, bar_empty = bars + 8 * PJ_NS, bar_done = bars + 16 * PJ_NS;
+  unsigned char* misc = sm + (bar_done + 8 - base);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 4);
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int hg = blockIdx.x, js = blockIdx.y, bg = blockIdx.z;
+  const uint32_t tmem_cols = (uint32_t)(32 * g.hp);
+
+  if (tid == 0) {
+    for (int i = 0; i < PJ_NS; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
+    mbar_init(bar_done, 1);
+    *s_abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(s_tmem), tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  const int row0 = js * g.nst * PJ_ROWS;                      // first row of W_KV,h of this CTA
+
+  if (warp == 0 && lane == 0) {
+    // =========================== producer ===========================
+    const unsigned char* usrc = u_tiled + ((size_t)(bg * g.hg + hg) * (d / 16) + row0 / 16) * ((size_t)1024 * g.hp);
+    int s = 0;
+    bool ok = true;
+    for (; s < g.nst; ++s) {
+      const int st = s % PJ_NS;
+      ok = mbar_wait<false>(bar_empty + 8 * st, ((s / PJ_NS) & 1) ^ 1, s_abort, status);
+      if (!ok) break;
+      const uint32_t dst = base + (uint32_t)st * stage_bytes;
+      mbar_arrive_expect_tx(bar_full + 8 * st, stage_bytes);
+      if (g.hp == 1) tma_load_3d(dst, &wmap, bar_full + 8 * st, 0, hg * d + row0 + s * PJ_ROWS, 0);
+      else           tma_load_3d(dst, &wmap, bar_full + 8 * st, 0, row0 + s * PJ_ROWS, 2 * hg);
+      bulk_load(dst + PJ_W_BYTES, usrc + (size_t)s * g.u_bytes, (uint32_t)g.u_bytes, bar_full + 8 * st);
+    }
+    if (!ok) {
+      // gave up: let the copies that were issued land before the CTA goes away
+      const int issued = s < PJ_NS ? s : PJ_NS;
+      for (int k = 0; k < issued; ++k) {
+        const int j = s - 1 - k, st = j % PJ_NS;
+        const unsigned long long t0 = globaltimer();
+        while (!mbar_try_wait(bar_full + 8 * st, (j / PJ_NS) & 1) && globaltimer() - t0 < SLIM_WAIT_NS) {}
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // =========================== MMA issuer ===========================
+    const uint32_t idesc = umma_idesc((uint32_t)(32 * g.hp));
+    bool ok = true;
+    for (int s = 0; s < g.nst && ok; ++s) {
+      const int st = s % PJ_NS;
+      ok = mbar_wait<false>(bar_full + 8 * st, (s / PJ_NS) & 1, s_abort, status);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t wbase = base + (uint32_t)st * stage_bytes, ubase = wbase + PJ_W_BYTES;
+#pragma unroll
+      for (int kk = 0; kk < PJ_ROWS / 16; ++kk)
+        umma_bf16(tmem_base, desc_a(wbase + (uint32_t)kk * 2048u, PJ_ROWS * 128), desc_b(ubase + (uint32_t)(kk * 1024 * g.hp)),
+                  idesc, (s | kk) ? 1u : 0u);
+      umma_commit(bar_empty + 8 * st);
+      if (s == g.nst - 1) umma_commit(bar_done);
+    }
+  }
+  __syncwarp();
+  // =========================== epilogue: all four warps ===========================
+  {
+    bool ok = mbar_wait<false>(bar_done, 0, s_abort, status);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after();
+      const int m = warp * 32 + lane;                           // accumulator row = TMEM lane
+      const int upper = g.hp == 2 ? (warp >> 1) : 0;            // d_k = 64: lanes 64..127 hold the second head
+      const int head = hg * g.hp + upper;
+      const int c = g.hp == 2 ? (m & 63) : m;
+      uint32_t r[32];
+      tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(32 * upper), r);
+      if (c < d_k) {
+#pragma unroll
+        for (int n = 0; n < PJ_BG; ++n) {
+          const int b = bg * PJ_BG + n;
+          if (b < batch)
+            o_part[((size_t)js * batch + b) * d + head * d_k + c] = __uint_as_float(r[n]) + __uint_as_float(r[PJ_BG + n]);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, tmem_cols);
+  }
+}
+
+ProjGeom make_proj_geom(int d, int H, int d_k, int batch) {
+  ProjGeom g;
+  g.hp = 128 / d_k;
+  g.hg = H / g.hp;
+  const int stages = d / PJ_ROWS;
+  int js = 1;
+  for (int c = 1; c <= 8; ++c)
+    if (stages % c == 0) js = c;
+  g.jsplit = js;
+  g.nst = stages / js;
+  g.nbg = (batch + PJ_BG - 1) / PJ_BG;
+  g.u_bytes = (PJ_ROWS / 16) * 1024 * g.hp;
+  return g;
+}
+
+size_t proj_smem_bytes(const ProjGeom& g) { return 1024 + (size_t)PJ_NS * (PJ_W_BYTES + g.u_bytes) + 16 * PJ_NS + 8 + 16 + 64; }
+
+}  // namespace
+
+int slim_proj_shape_ok(int d, int H, int d_k, int dtype) {
+  if (dtype != SLIM_BF16) return 0;
+  if (d_k != 64 && d_k != 128) return 0;
+  if (d % PJ_ROWS != 0 || H % (128 / d_k) != 0) return 0;
+  return 1;
+}
+
+int slim_proj_jsplit(int d) { return make_proj_geom(d, 2, 64, 1).jsplit; }
+
+size_t slim_proj_u_bytes(int d, int H, int batch) {
+  return (size_t)((batch + PJ_BG - 1) / PJ_BG) * PJ_BG * H * d * sizeof(float);
+}
+
+cudaError_t slim_proj_make_wmap(slim_ctx* ctx) {
+  const int d = ctx->d, d_k = ctx->d_k, H = ctx->H;
+  unsigned long long dims[3], strides[2];
+  unsigned int box[3] = {64, PJ_ROWS, 2};
+  if (d_k == 128) {          // (64 columns, H*d rows, 2 column halves)
+    dims[0] = 64; dims[1] = (unsigned long long)H * d; dims[2] = 2;
+    strides[0] = 256; strides[1] = 128;
+  } else {                   // d_k = 64: (64 columns, d rows, H heads)
+    dims[0] = 64; dims[1] = d; dims[2] = H;
+    strides[0] = 128; strides[1] = (unsigned long long)d * 128;
+  }
+  cudaError_t e = slim_tmap_encode_3d(ctx->wmap, ctx->wkv, dims, strides, box);
+  if (e != cudaSuccess) return e;
+  const ProjGeom g = make_proj_geom(d, H, d_k, 1);
+  return cudaFuncSetAttribute((const void*)slim_proj_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)proj_smem_bytes(g));
+}
+
+cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, unsigned char* u_tiled, float* o_part,
+                             cudaStream_t st) {
+  const ProjGeom g = make_proj_geom(p.d, p.H, p.d_k, p.batch);
+  {
+    dim3 grid(p.H, g.nbg * PJ_BG);
+    const size_t smem = sizeof(float) * p.workers + sizeof(int) * (2 + p.batch + 1) + 16;
+    slim_combine_kernel<<<grid, 256, smem, st>>>(p, u_tiled, g.hp);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  CUtensorMap map;
+  memcpy(&map, ctx->wmap, sizeof(map));
+  dim3 grid(g.hg, g.jsplit, g.nbg);
+  slim_proj_tc_kernel<<<grid, 128, proj_smem_bytes(g), st>>>(map, u_tiled, o_part, g, p.d, p.d_k, p.batch, p.status);
+  return cudaGetLastError();
+}

@@ -144,7 +144,15 @@ __global__ void slim_append_kernel(KT* __restrict__ cache, const KT* __restrict_
 
 }  // namespace
 
-size_t slim_tail_opart_floats(int d, int batch) { return (size_t)((d + JR - 1) / JR) * batch * d; }
+size_t slim_tail_opart_floats(int d, int batch) {
+  const int slices = (d + JR - 1) / JR;
+  return (size_t)(slices > 8 ? slices : 8) * batch * d;      // the tensor-core projection writes up to 8 slices
+}
+
+cudaError_t slim_launch_sum_slices(const float* o_part, float* o, int n, int nsplit, cudaStream_t st) {
+  slim_tail2_kernel<<<(n + 255) / 256, 256, 0, st>>>(o_part, o, n, nsplit);
+  return cudaGetLastError();
+}
 
 cudaError_t slim_launch_tail(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st) {
   const int nsplit = (p.d + JR - 1) / JR;
