@@ -162,6 +162,8 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
   c->path_req = SLIM_PATH_AUTO;
   if (cudaMalloc(&c->status, sizeof(int)) != cudaSuccess) { delete c; return SLIM_ERR_OOM; }
   cudaMemset(c->status, 0, sizeof(int));
+  if (cudaMalloc(&c->any_flag, sizeof(int)) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
+  cudaMemset(c->any_flag, 0, sizeof(int));
   if (cudaMalloc(&c->wkv, esize(dtype) * (size_t)d * d) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
   if (rope_theta != 0.0) {
     const int half = d_k / 2;
@@ -197,6 +199,7 @@ void slim_destroy(slim_ctx* ctx) {
   cudaFree(ctx->rope_off);
   cudaFree(ctx->rope_base);
   cudaFree(ctx->status);
+  cudaFree(ctx->any_flag);
   for (int i = 0; i < 3; ++i)
     if (ctx->prof_ev[i]) cudaEventDestroy(ctx->prof_ev[i]);
   delete ctx;
@@ -325,7 +328,7 @@ slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   p.part_l = reinterpret_cast<float*>(ws + L.part_l);
   p.unit_flags = reinterpret_cast<int*>(ws + L.flags);
   p.u = reinterpret_cast<float*>(ws + L.o_part);
-  p.o = o; p.status = ctx->status;
+  p.o = o; p.status = ctx->status; p.any_flag = ctx->any_flag;
   cudaStream_t st = (cudaStream_t)stream;
   if (ctx->prof_on) cudaEventRecord(ctx->prof_ev[0], st);
   cudaError_t e;

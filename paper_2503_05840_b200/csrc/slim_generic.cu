@@ -41,6 +41,7 @@ slim_exact_kernel(SlimDecodeParams p, int only_flagged) {
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int w = blockIdx.y;
+  if (only_flagged && *p.any_flag == 0) return;         // nothing was flagged in this decode
   const int col0 = blockIdx.x * (GEN_THREADS * COLS);
   const KT* __restrict__ Kc = reinterpret_cast<const KT*>(p.k);
   const KT* __restrict__ Q = reinterpret_cast<const KT*>(p.q);

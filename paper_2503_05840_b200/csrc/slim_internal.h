@@ -37,6 +37,7 @@ struct SlimDecodeParams {
   float* u;                      // [batch][H][d] combined
   float* o;                      // [batch][d]
   int* status;                   // sticky device status word
+  int* any_flag;                 // set to 1 by a kernel that flags a unit
 };
 
 struct slim_ctx {
@@ -57,6 +58,7 @@ struct slim_ctx {
   int prof_on, prof_valid;
   cudaEvent_t prof_ev[3];
   int proj_ok;                   // tensor-core combine + projection usable for this shape
+  int* any_flag;                 // device: 1 while some unit of the current decode is flagged for the exact redo
   alignas(64) unsigned char wmap[128];   // CUtensorMap over W_KV for the projection kernel
 };
 

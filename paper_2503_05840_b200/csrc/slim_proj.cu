@@ -56,6 +56,7 @@ slim_combine_kernel(const SlimDecodeParams p, unsigned char* __restrict__ u_tile
   const int tid = threadIdx.x, lane = tid & 31;
   const int h = blockIdx.x, b = blockIdx.y, bg = b / PJ_BG, n = b % PJ_BG;
   const int d = p.d, H = p.H;
+  if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) *p.any_flag = 0;   // the redo kernel has consumed it
 
   const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status);
   if (tid < 32) {

@@ -292,7 +292,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
               lsum = 0.f;
             }
             float x = sv - mref;
-            if (valid && x > TC_XMAX) { p.unit_flags[unit] = 1; x = TC_XMAX; }
+            if (valid && x > TC_XMAX) { p.unit_flags[unit] = 1; *p.any_flag = 1; x = TC_XMAX; }
             const float pf = valid ? ex2_approx(x) : 0.f;
             const __nv_bfloat16 pb = __float2bfloat16_rn(pf);
             if ((jl % DUP) == 0) lsum += __bfloat162float(pb);
