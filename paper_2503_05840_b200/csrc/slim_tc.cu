@@ -115,11 +115,13 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   const int producer_warp = g.nswl, mma_warp = g.nswl + 1;
 
   // ---- set-up -------------------------------------------------------------------
+  const int nepi = (g.nswl / 4) * 4;              // warps that drain the accumulator at a unit's end
   if (tid == 0) {
+    prefetch_tensormap(&tmap);
     for (int i = 0; i < g.ns; ++i) { mbar_init(bar_k_full + 8 * i, 1); mbar_init(bar_k_empty + 8 * i, g.nsw + 1); }
     for (int i = 0; i < TC_NP; ++i) { mbar_init(bar_p_full + 8 * i, 1 + g.nsw); mbar_init(bar_p_empty + 8 * i, 2); }
     mbar_init(bar_u_full, 1);
-    mbar_init(bar_u_empty, 4);
+    mbar_init(bar_u_empty, nepi);
     *s_abort = 0;
     fence_mbar_init();
   }
@@ -133,6 +135,17 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   if (rank == 0 && have_work) {                   // clear the redo flags of this worker's units
     const int b_lo = slim_seq_of_tile(s_prefix, p.batch, g_begin), b_hi = slim_seq_of_tile(s_prefix, p.batch, g_end - 1);
     for (int b = b_lo + tid; b <= b_hi; b += blockDim.x) p.unit_flags[w + b] = 0;
+  }
+  // The first loads need only this CTA's barriers (ready since the __syncthreads inside
+  // slim_sched_build): start them before the cluster-wide set-up finishes.
+  const int pre_issued = have_work ? min(g.ns, g_end - g_begin) : 0;
+  if (warp == producer_warp && lane == 0) {
+    for (int it = 0; it < pre_issued; ++it) {
+      const int gg = g_begin + it, b = slim_seq_of_tile(s_prefix, p.batch, gg);
+      mbar_arrive_expect_tx(bar_k_full + 8 * it, (uint32_t)g.stage_bytes);
+      tma_load_3d(k_stage0 + (uint32_t)it * g.stage_bytes, &tmap, bar_k_full + 8 * it, 0,
+                  b * p.t_cap + (gg - s_prefix[b]) * SLIM_TT, (int)rank * g.nc64);
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -336,18 +349,34 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             p.part_l[(size_t)unit * p.H + my_n] = lsum;
           }
         }
-        if (warp < 4) {
+        if (warp < nepi) {
+          // Warp w drains TMEM lanes 32 (w & 3) .. +31 (the only ones it can reach) for the
+          // chunks w >> 2, w >> 2 + nepi / 4, ...; the next chunk is fetched while this one
+          // is stored.
           ok = mbar_wait<false>(bar_u_full, uc & 1, s_abort, p.status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
-          float* dst = p.part_u + (size_t)unit * p.H * p.d + (size_t)rank * g.dsl + warp * 32 + lane;
-          for (int c = 0; c < g.nch; ++c) {
-            uint32_t r[32];
-            tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), r);
+          const int q = warp & 3, cstep = nepi >> 2;
+          const uint32_t tlane = tmem_base + ((uint32_t)(q * 32) << 16);
+          float* dst = p.part_u + (size_t)unit * p.H * p.d + (size_t)rank * g.dsl + q * 32 + lane;
+          uint32_t ra[32], rb[32];
+          int c = warp >> 2;
+          if (c < g.nch) tmem_ld32_issue(tlane + (uint32_t)(c * 32), ra);
+          while (c < g.nch) {
+            tmem_ld_wait();
+            if (c + cstep < g.nch) tmem_ld32_issue(tlane + (uint32_t)((c + cstep) * 32), rb);
 #pragma unroll
             for (int n = 0; n < 32; ++n)
-              if (n < p.H) dst[(size_t)n * p.d + c * 128] = __uint_as_float(r[n]);
+              if (n < p.H) dst[(size_t)n * p.d + c * 128] = __uint_as_float(ra[n]);
+            c += cstep;
+            if (c >= g.nch) break;
+            tmem_ld_wait();
+            if (c + cstep < g.nch) tmem_ld32_issue(tlane + (uint32_t)((c + cstep) * 32), ra);
+#pragma unroll
+            for (int n = 0; n < 32; ++n)
+              if (n < p.H) dst[(size_t)n * p.d + c * 128] = __uint_as_float(rb[n]);
+            c += cstep;
           }
           tc_fence_before();
           __syncwarp();
@@ -365,6 +394,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           const int seg_end = min(g_end, s_prefix[b + 1]);
           const int tile0 = gg - s_prefix[b], ntile = seg_end - gg;
           for (int kt = 0; kt < ntile; ++kt, ++it) {
+            if (it < pre_issued) continue;          // issued during set-up
             const int st = it % g.ns;
             ok = mbar_wait<false>(bar_k_empty + 8 * st, ((it / g.ns) & 1) ^ 1, s_abort, p.status);
             if (!ok) break;
