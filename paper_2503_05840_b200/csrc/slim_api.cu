@@ -35,7 +35,7 @@ WsLayout ws_layout(const slim_ctx* ctx, int batch, int t_cap) {
   L.part_u = off; off = align256(off + sizeof(float) * (size_t)L.units * ctx->H * ctx->d);
   L.part_m = off; off = align256(off + sizeof(float) * (size_t)L.units * ctx->H);
   L.part_l = off; off = align256(off + sizeof(float) * (size_t)L.units * ctx->H);
-  L.flags = off;  off = align256(off + sizeof(int) * (size_t)L.units);
+  L.flags = off;  off = align256(off + sizeof(int) * 2 * (size_t)L.units);
   L.o_part = off; off = align256(off + sizeof(float) * slim_tail_opart_floats(ctx->d, batch));
   L.scores = off; off = align256(off + sizeof(float) * (size_t)batch * ctx->H * t_cap);   // generic path only
   L.u_tiled = off; off = align256(off + (ctx->proj_ok ? slim_proj_u_bytes(ctx->d, ctx->H, batch) : 0));   // tensor-core tail only
@@ -320,6 +320,7 @@ slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   p.rope = ctx->rope_theta != 0.0; p.dtype = ctx->dtype;
   p.workers = path == SLIM_PATH_TC ? ctx->tc_workers : ctx->gen_workers;
   p.min_tiles = min_tiles_for(ctx);
+  p.unit_cost = path == SLIM_PATH_TC ? (ctx->H + 3) / 4 : 0;   // measured: a drain costs about H/4 tiles
   p.qscale = (float)(1.4426950408889634 / std::sqrt((double)ctx->d_k));
   p.q = q; p.k = cache->k; p.lengths = lengths;
   p.rope_base = ctx->rope_base; p.rope_off = ctx->rope_off; p.wkv = ctx->wkv;

@@ -47,8 +47,7 @@ slim_exact_kernel(SlimDecodeParams p, int only_flagged) {
   const KT* __restrict__ Q = reinterpret_cast<const KT*>(p.q);
   const int d = p.d, H = p.H, dk = p.d_k, half = p.half;
 
-  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles,
-                                        s_prefix, p.status);
+  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
   if (sc.total_tiles == 0 || w >= sc.workers_eff) return;
   const int g_begin = slim_worker_start(sc, w), g_end = slim_worker_start(sc, w + 1);
 
@@ -60,7 +59,7 @@ slim_exact_kernel(SlimDecodeParams p, int only_flagged) {
     const int seg_end = min(g_end, s_prefix[b + 1]);
     const int tile0 = g - s_prefix[b], tile1 = seg_end - s_prefix[b];
     const int unit = w + b;
-    if (only_flagged && p.unit_flags[unit] == 0) { g = seg_end; continue; }
+    if (only_flagged && (p.unit_flags[2 * unit] | p.unit_flags[2 * unit + 1]) == 0) { g = seg_end; continue; }
     int len = p.lengths[b];
     len = min(max(len, 0), p.t_cap);
 
@@ -232,7 +231,7 @@ slim_scores_kernel(SlimDecodeParams p, float* __restrict__ scores) {
   const KT* __restrict__ Kc = reinterpret_cast<const KT*>(p.k);
   const KT* __restrict__ Q = reinterpret_cast<const KT*>(p.q);
 
-  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status);
+  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
   int cur_b = -1;
   for (int g = blockIdx.x; g < sc.total_tiles; g += gridDim.x) {
     const int b = slim_seq_of_tile(s_prefix, p.batch, g);
@@ -315,7 +314,7 @@ slim_accum_kernel(SlimDecodeParams p, const float* __restrict__ scores) {
   const KT* __restrict__ Kc = reinterpret_cast<const KT*>(p.k);
   const int d = p.d, H = p.H;
 
-  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status);
+  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
   if (sc.total_tiles == 0 || w >= sc.workers_eff) return;
   const int g_begin = slim_worker_start(sc, w), g_end = slim_worker_start(sc, w + 1);
   float acc[HP];

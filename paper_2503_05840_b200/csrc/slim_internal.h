@@ -23,6 +23,7 @@ struct SlimDecodeParams {
   int dtype;                     // slim_dtype
   int workers;                   // context-split workers (W)
   int min_tiles;                 // a worker gets at least this many tiles if it gets any
+  int unit_cost;                 // tiles of time that closing a unit costs a worker (schedule)
   float qscale;                  // log2(e) / sqrt(d_k)
   const void* q;                 // [batch][d]
   const void* k;                 // [batch][t_cap][d]
@@ -33,7 +34,7 @@ struct SlimDecodeParams {
   float* part_u;                 // [units][H][d]
   float* part_m;                 // [units][H]   reference exponent (log2 domain)
   float* part_l;                 // [units][H]   sum of 2^(s - m)
-  int* unit_flags;               // [units]      1 = unit must be redone exactly
+  int* unit_flags;               // [units][2]   1 = unit must be redone exactly (one word per CTA of the pair)
   float* u;                      // [batch][H][d] combined
   float* o;                      // [batch][d]
   int* status;                   // sticky device status word

@@ -58,7 +58,7 @@ slim_combine_kernel(const SlimDecodeParams p, unsigned char* __restrict__ u_tile
   const int d = p.d, H = p.H;
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) *p.any_flag = 0;   // the redo kernel has consumed it
 
-  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status);
+  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
   if (tid < 32) {
     int wlo = 0, wn = 0;
     if (b < p.batch && s_prefix[b + 1] > s_prefix[b]) {

@@ -9,12 +9,21 @@
 // worker + sequence is unique and < workers + batch.  The schedule is a pure
 // function of `lengths`, so every CTA (and the combine kernel) recomputes it
 // and the result is deterministic.
+//
+// Closing a unit costs a worker about `unit_cost` tiles of time (draining the
+// accumulator, restarting the pipeline), so the cut is made on a *virtual*
+// line in which every boundary between two sequences is unit_cost slots wide:
+// a worker whose range crosses a boundary gets that many tiles fewer.
 #pragma once
 #include "slim_internal.h"
 
 struct SlimSched {
   int total_tiles;   // NT
   int workers_eff;   // W_eff <= workers
+  int unit_cost;     // E: width of a sequence boundary on the virtual line, in tiles
+  int virt_total;    // NT + E (batch - 1)
+  int batch;
+  const int* prefix; // shared memory, batch + 1 entries
 };
 
 // Exclusive prefix of per-sequence tile counts into s_prefix[0..batch]
@@ -23,7 +32,7 @@ struct SlimSched {
 // t_cap also raises SLIM_ERR_CAPACITY in *status.
 __device__ __forceinline__ SlimSched slim_sched_build(const int32_t* __restrict__ lengths, int batch,
                                                       int t_cap, int workers, int min_tiles,
-                                                      int* s_prefix, int* status) {
+                                                      int* s_prefix, int* status, int unit_cost = 0) {
   const int tid = threadIdx.x + threadIdx.y * blockDim.x;
   const int nthr = blockDim.x * blockDim.y;
   for (int b = tid; b < batch; b += nthr) {
@@ -55,16 +64,25 @@ __device__ __forceinline__ SlimSched slim_sched_build(const int32_t* __restrict_
   int we = s.total_tiles / (min_tiles > 0 ? min_tiles : 1);
   if (we < 1) we = 1;
   s.workers_eff = we < workers ? we : workers;
+  s.unit_cost = unit_cost;
+  s.virt_total = s.total_tiles + unit_cost * (batch - 1);
+  s.batch = batch;
+  s.prefix = s_prefix;
   return s;
 }
 
+// First tile of worker w (w = workers_eff gives total_tiles).  A worker's range
+// [start(w), start(w+1)) may be empty.
 __device__ __forceinline__ int slim_worker_start(const SlimSched& s, int w) {
-  return (int)(((long long)w * s.total_tiles) / s.workers_eff);
-}
-
-// Worker that owns global tile g (0 <= g < total_tiles).
-__device__ __forceinline__ int slim_worker_of_tile(const SlimSched& s, int g) {
-  return (int)((((long long)g + 1) * s.workers_eff - 1) / s.total_tiles);
+  const int v = (int)(((long long)w * s.virt_total) / s.workers_eff);
+  // sequence whose virtual span [prefix[b] + E b, prefix[b+1] + E (b+1)) holds v
+  int lo = 0, hi = s.batch;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (s.prefix[mid] + s.unit_cost * mid <= v) lo = mid; else hi = mid;
+  }
+  const int t = v - s.unit_cost * lo;
+  return t < s.prefix[lo + 1] ? t : s.prefix[lo + 1];
 }
 
 // Sequence that owns global tile g: prefix[b] <= g < prefix[b+1].
@@ -75,4 +93,11 @@ __device__ __forceinline__ int slim_seq_of_tile(const int* s_prefix, int batch, 
     if (s_prefix[mid] <= g) lo = mid; else hi = mid;
   }
   return lo;
+}
+
+// Worker that owns global tile g (0 <= g < total_tiles): the largest w with start(w) <= g.
+__device__ __forceinline__ int slim_worker_of_tile(const SlimSched& s, int g) {
+  const int b = slim_seq_of_tile(s.prefix, s.batch, g);
+  const long long v = (long long)g + (long long)s.unit_cost * b;
+  return (int)(((v + 1) * s.workers_eff - 1) / s.virt_total);
 }

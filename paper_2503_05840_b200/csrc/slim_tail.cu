@@ -36,8 +36,7 @@ __global__ void __launch_bounds__(256) slim_tail1_kernel(SlimDecodeParams p, int
   const int BT = bg_count * BPT;
   const WT* __restrict__ W = reinterpret_cast<const WT*>(p.wkv) + ((size_t)h * d + j0) * dk;
 
-  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles,
-                                        s_prefix, p.status);
+  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
   const int c = tid % dk, bg = tid / dk;          // blockDim.x == dk * bg_count
 
   for (int b0 = 0; b0 < p.batch; b0 += BT) {

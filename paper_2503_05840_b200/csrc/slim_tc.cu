@@ -126,32 +126,25 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
     fence_mbar_init();
   }
   for (int i = tid; i < TC_NP * TC_P_BYTES / 16; i += blockDim.x) sts128_zero(p_stage0 + 16 * i);
-  fence_proxy_async();
   if (warp == mma_warp) tmem_alloc(smem_u32(s_tmem), (uint32_t)g.tmem_cols);
-  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status);
-  const bool have_work = sc.total_tiles > 0 && w < sc.workers_eff;
-  const int g_begin = have_work ? slim_worker_start(sc, w) : 0;
-  const int g_end = have_work ? slim_worker_start(sc, w + 1) : 0;
-  if (rank == 0 && have_work) {                   // clear the redo flags of this worker's units
-    const int b_lo = slim_seq_of_tile(s_prefix, p.batch, g_begin), b_hi = slim_seq_of_tile(s_prefix, p.batch, g_end - 1);
-    for (int b = b_lo + tid; b <= b_hi; b += blockDim.x) p.unit_flags[w + b] = 0;
-  }
-  // The first loads need only this CTA's barriers (ready since the __syncthreads inside
-  // slim_sched_build): start them before the cluster-wide set-up finishes.
-  const int pre_issued = have_work ? min(g.ns, g_end - g_begin) : 0;
-  if (warp == producer_warp && lane == 0) {
-    for (int it = 0; it < pre_issued; ++it) {
-      const int gg = g_begin + it, b = slim_seq_of_tile(s_prefix, p.batch, gg);
-      mbar_arrive_expect_tx(bar_k_full + 8 * it, (uint32_t)g.stage_bytes);
-      tma_load_3d(k_stage0 + (uint32_t)it * g.stage_bytes, &tmap, bar_k_full + 8 * it, 0,
-                  b * p.t_cap + (gg - s_prefix[b]) * SLIM_TT, (int)rank * g.nc64);
-    }
-  }
+  // Cluster-wide rendezvous first, while nothing is in flight (a cluster barrier that has
+  // to wait behind outstanding TMA loads costs several microseconds): after it the peer's
+  // barriers and P tiles may be written.
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
+  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
+  const bool in_range = sc.total_tiles > 0 && w < sc.workers_eff;
+  const int g_begin = in_range ? slim_worker_start(sc, w) : 0;
+  const int g_end = in_range ? slim_worker_start(sc, w + 1) : 0;
+  const bool have_work = g_end > g_begin;
+  if (have_work) {                                // clear this CTA's redo flags of the worker's units
+    const int b_lo = slim_seq_of_tile(s_prefix, p.batch, g_begin), b_hi = slim_seq_of_tile(s_prefix, p.batch, g_end - 1);
+    for (int b = b_lo + tid; b <= b_hi; b += blockDim.x) p.unit_flags[2 * (w + b) + (int)rank] = 0;
+  }
+  __syncthreads();
 
   if (have_work) {
     if (warp < g.nswl) {
@@ -305,7 +298,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
               lsum = 0.f;
             }
             float x = sv - mref;
-            if (valid && x > TC_XMAX) { p.unit_flags[unit] = 1; *p.any_flag = 1; x = TC_XMAX; }
+            if (valid && x > TC_XMAX) { p.unit_flags[2 * unit + (int)rank] = 1; *p.any_flag = 1; x = TC_XMAX; }
             const float pf = valid ? ex2_approx(x) : 0.f;
             const __nv_bfloat16 pb = __float2bfloat16_rn(pf);
             if ((jl % DUP) == 0) lsum += __bfloat162float(pb);
@@ -394,7 +387,6 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           const int seg_end = min(g_end, s_prefix[b + 1]);
           const int tile0 = gg - s_prefix[b], ntile = seg_end - gg;
           for (int kt = 0; kt < ntile; ++kt, ++it) {
-            if (it < pre_issued) continue;          // issued during set-up
             const int st = it % g.ns;
             ok = mbar_wait<false>(bar_k_empty + 8 * st, ((it / g.ns) & 1) ^ 1, s_abort, p.status);
             if (!ok) break;
