@@ -41,6 +41,8 @@ slim_exact_kernel(SlimDecodeParams p, int only_flagged) {
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int w = blockIdx.y;
+  slim_pdl_trigger();
+  slim_pdl_wait();
   if (only_flagged && *p.any_flag == 0) return;         // nothing was flagged in this decode
   const int col0 = blockIdx.x * (GEN_THREADS * COLS);
   const KT* __restrict__ Kc = reinterpret_cast<const KT*>(p.k);
@@ -393,8 +395,7 @@ cudaError_t launch_exact(const SlimDecodeParams& p, int only_flagged, cudaStream
     if (e != cudaSuccess) return e;
   }
   dim3 grid(dsplit, p.workers);
-  kern<<<grid, GEN_THREADS, smem, st>>>(p, only_flagged);
-  return cudaGetLastError();
+  return slim_launch_pdl(kern, grid, dim3(GEN_THREADS), smem, st, p, only_flagged);
 }
 
 template <typename KT>

@@ -103,3 +103,26 @@ cudaError_t slim_proj_make_wmap(slim_ctx* ctx);
 cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, unsigned char* u_tiled, float* o_part,
                              cudaStream_t st);
 cudaError_t slim_launch_sum_slices(const float* o_part, float* o, int n, int nsplit, cudaStream_t st);
+
+// ---- programmatic dependent launch ---------------------------------------------
+// The kernels of one decode step run back to back on one stream.  Launched with
+// slim_launch_pdl, a kernel may be scheduled while its predecessor is still
+// finishing; it must execute slim_pdl_wait() before it touches anything a
+// predecessor wrote (the wait returns once the predecessor grid has completed and
+// its memory is visible).  slim_pdl_trigger() lets the successor's launch begin.
+#ifdef __CUDACC__
+__device__ __forceinline__ void slim_pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void slim_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t slim_launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                   Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+#endif

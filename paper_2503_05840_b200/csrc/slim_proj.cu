@@ -56,6 +56,8 @@ slim_combine_kernel(const SlimDecodeParams p, unsigned char* __restrict__ u_tile
   const int tid = threadIdx.x, lane = tid & 31;
   const int h = blockIdx.x, b = blockIdx.y, bg = b / PJ_BG, n = b % PJ_BG;
   const int d = p.d, H = p.H;
+  slim_pdl_trigger();
+  slim_pdl_wait();
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) *p.any_flag = 0;   // the redo kernel has consumed it
 
   const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
@@ -143,10 +145,12 @@ slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned cha
     fence_mbar_init();
   }
   if (warp == 1) tmem_alloc(smem_u32(s_tmem), tmem_cols);
+  slim_pdl_trigger();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
+  slim_pdl_wait();                                             // u tiles come from the combine kernel
   const int row0 = js * g.nst * PJ_ROWS;                      // first row of W_KV,h of this CTA
 
   if (warp == 0 && lane == 0) {
@@ -278,13 +282,12 @@ cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, uns
   {
     dim3 grid(p.H, g.nbg * PJ_BG);
     const size_t smem = sizeof(float) * p.workers + sizeof(int) * (2 + p.batch + 1) + 16;
-    slim_combine_kernel<<<grid, 256, smem, st>>>(p, u_tiled, g.hp);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = slim_launch_pdl(slim_combine_kernel, grid, dim3(256), smem, st, p, u_tiled, g.hp);
     if (e != cudaSuccess) return e;
   }
   CUtensorMap map;
   memcpy(&map, ctx->wmap, sizeof(map));
   dim3 grid(g.hg, g.jsplit, g.nbg);
-  slim_proj_tc_kernel<<<grid, 128, proj_smem_bytes(g), st>>>(map, u_tiled, o_part, g, p.d, p.d_k, p.batch, p.status);
-  return cudaGetLastError();
+  return slim_launch_pdl(slim_proj_tc_kernel, grid, dim3(128), proj_smem_bytes(g), st, map, (const unsigned char*)u_tiled, o_part,
+                         g, p.d, p.d_k, p.batch, p.status);
 }

@@ -29,6 +29,8 @@ __global__ void __launch_bounds__(256) slim_tail1_kernel(SlimDecodeParams p, int
   int* s_wn = s_wlo + BT_MAX;                                   // [BT]
   int* s_prefix = s_wn + BT_MAX;                                // [batch+1]
 
+  slim_pdl_trigger();
+  slim_pdl_wait();
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nwarp = blockDim.x >> 5;
   const int h = blockIdx.x, js = blockIdx.y;
   const int d = p.d, H = p.H, dk = p.d_k;
@@ -119,6 +121,8 @@ __global__ void __launch_bounds__(256) slim_tail1_kernel(SlimDecodeParams p, int
 
 __global__ void __launch_bounds__(256) slim_tail2_kernel(const float* __restrict__ o_part, float* __restrict__ o,
                                                          int n, int nsplit) {
+  slim_pdl_trigger();
+  slim_pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   float a = 0.f;
@@ -130,6 +134,8 @@ template <typename KT>
 __global__ void slim_append_kernel(KT* __restrict__ cache, const KT* __restrict__ k_new,
                                    const int32_t* __restrict__ positions, int d, int t_cap, int n_new,
                                    int* status) {
+  slim_pdl_trigger();
+  slim_pdl_wait();
   const int b = blockIdx.x, r = blockIdx.y;
   const int pos = positions[b];
   if (pos < 0 || pos + n_new > t_cap) {
@@ -149,8 +155,7 @@ size_t slim_tail_opart_floats(int d, int batch) {
 }
 
 cudaError_t slim_launch_sum_slices(const float* o_part, float* o, int n, int nsplit, cudaStream_t st) {
-  slim_tail2_kernel<<<(n + 255) / 256, 256, 0, st>>>(o_part, o, n, nsplit);
-  return cudaGetLastError();
+  return slim_launch_pdl(slim_tail2_kernel, dim3((n + 255) / 256), dim3(256), 0, st, o_part, o, n, nsplit);
 }
 
 cudaError_t slim_launch_tail(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st) {
@@ -187,10 +192,8 @@ cudaError_t slim_launch_append(const slim_ctx* ctx, const slim_cache* c, const v
                                const int32_t* positions, int n_new, cudaStream_t st) {
   dim3 grid(c->batch, n_new);
   if (ctx->dtype == SLIM_BF16)
-    slim_append_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((__nv_bfloat16*)c->k, (const __nv_bfloat16*)k_new,
-                                                            positions, ctx->d, c->t_cap, n_new, ctx->status);
-  else
-    slim_append_kernel<float><<<grid, 256, 0, st>>>((float*)c->k, (const float*)k_new, positions, ctx->d,
-                                                    c->t_cap, n_new, ctx->status);
-  return cudaGetLastError();
+    return slim_launch_pdl(slim_append_kernel<__nv_bfloat16>, grid, dim3(256), 0, st, (__nv_bfloat16*)c->k,
+                           (const __nv_bfloat16*)k_new, positions, ctx->d, c->t_cap, n_new, ctx->status);
+  return slim_launch_pdl(slim_append_kernel<float>, grid, dim3(256), 0, st, (float*)c->k, (const float*)k_new, positions,
+                         ctx->d, c->t_cap, n_new, ctx->status);
 }

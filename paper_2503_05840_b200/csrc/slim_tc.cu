@@ -135,6 +135,8 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
+  slim_pdl_trigger();
+  slim_pdl_wait();          // lengths, q and the newest key rows may come from the kernels before this one
   const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
   const bool in_range = sc.total_tiles > 0 && w < sc.workers_eff;
   const int g_begin = in_range ? slim_worker_start(sc, w) : 0;
@@ -591,10 +593,12 @@ cudaError_t slim_launch_tc(const slim_ctx* ctx, const slim_cache* c, const SlimD
   cfg.blockDim = dim3((g.nswl + 2) * 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr; cfg.numAttrs = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 2;
   CUtensorMap map;
   memcpy(&map, c->tmap, sizeof(map));
   return cudaLaunchKernelEx(&cfg, kern, map, p, g);
