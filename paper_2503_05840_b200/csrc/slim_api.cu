@@ -164,7 +164,7 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
   cudaMemset(c->status, 0, sizeof(int));
   if (cudaMalloc(&c->any_flag, sizeof(int)) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
   cudaMemset(c->any_flag, 0, sizeof(int));
-  if (cudaMalloc(&c->wkv, esize(dtype) * (size_t)d * d) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
+  if (cudaMalloc(&c->wkv, esize(dtype) * (size_t)d * d + 256) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
   if (rope_theta != 0.0) {
     const int half = d_k / 2;
     std::vector<float2> off((size_t)SLIM_TT * half);
@@ -179,6 +179,7 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
       return SLIM_ERR_CUDA;
     }
   }
+  cudaMemset(c->wkv, 0, esize(dtype) * (size_t)d * d + 256);
   c->proj_ok = prop.major == 10 ? slim_proj_shape_ok(d, H, d_k, dtype) : 0;
   if (c->proj_ok && slim_proj_make_wmap(c) != cudaSuccess) { cudaGetLastError(); c->proj_ok = 0; }
   {

@@ -1,4 +1,4 @@
-// Tail of the decode step on the tensor cores (bf16 caches, d_k = 64 or 128):
+// Tail of the decode step on the tensor cores (bf16 caches, d_k = 64, 96 or 128):
 //
 //   slim_combine_kernel   log-sum-exp combine of the context-split partials:
 //                         u[b][h][:] = sum_s w_s U_s[h][:] / sum_s w_s l_s over the
@@ -13,7 +13,8 @@
 //                         weights used MN-major, B = the u tiles, D in tensor
 //                         memory.  N = 32 per head (16 sequences x {hi, lo}); for
 //                         d_k = 64 two heads share an instruction (M = 2 x 64,
-//                         N = 2 x 32) and the off-diagonal quadrants are ignored.
+//                         N = 2 x 32) and the off-diagonal quadrants are ignored; for
+//                         d_k = 96 the accumulator rows 96..127 are ignored.
 //                         A CTA owns (head group, slice of the d rows of W_KV,h,
 //                         16-sequence group) and writes a projection slice that
 //                         slim_tail2_kernel sums in a fixed order.
@@ -35,7 +36,7 @@ constexpr int PJ_NS = 4;                       // stages
 constexpr int PJ_BG = 16;                      // sequences per MMA (N = 32 per head: hi and lo)
 
 struct ProjGeom {
-  int hp;        // heads per MMA: 1 (d_k = 128) or 2 (d_k = 64)
+  int hp;        // heads per MMA: 1 (d_k = 96, 128) or 2 (d_k = 64)
   int hg;        // head groups = H / hp
   int jsplit;    // slices of the d rows of W_KV,h
   int nst;       // stages per CTA = d / 64 / jsplit
@@ -97,10 +98,27 @@ slim_combine_kernel(const SlimDecodeParams p, unsigned char* __restrict__ u_tile
     float acc[8];
 #pragma unroll
     for (int x = 0; x < 8; ++x) acc[x] = 0.f;
-    for (int i = 0; i < wn; ++i) {
+    const float* Ub = p.part_u + ((size_t)(wlo + b) * H + h) * d + j0;        // unit i lives H*d floats further
+    const size_t ustride = (size_t)H * d;
+    int i = 0;
+    for (; i + 4 <= wn; i += 4) {                // four units' loads in flight
+      float4 a[4], c[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float4* U = reinterpret_cast<const float4*>(Ub + (size_t)(i + k) * ustride);
+        a[k] = __ldcs(U); c[k] = __ldcs(U + 1);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float wg = s_w[i + k];
+        acc[0] = fmaf(wg, a[k].x, acc[0]); acc[1] = fmaf(wg, a[k].y, acc[1]); acc[2] = fmaf(wg, a[k].z, acc[2]); acc[3] = fmaf(wg, a[k].w, acc[3]);
+        acc[4] = fmaf(wg, c[k].x, acc[4]); acc[5] = fmaf(wg, c[k].y, acc[5]); acc[6] = fmaf(wg, c[k].z, acc[6]); acc[7] = fmaf(wg, c[k].w, acc[7]);
+      }
+    }
+    for (; i < wn; ++i) {
       const float wg = s_w[i];
-      const float4* U = reinterpret_cast<const float4*>(p.part_u + ((size_t)(wlo + i + b) * H + h) * d + j0);
-      const float4 a = __ldg(U), c = __ldg(U + 1);
+      const float4* U = reinterpret_cast<const float4*>(Ub + (size_t)i * ustride);
+      const float4 a = __ldcs(U), c = __ldcs(U + 1);
       acc[0] = fmaf(wg, a.x, acc[0]); acc[1] = fmaf(wg, a.y, acc[1]); acc[2] = fmaf(wg, a.z, acc[2]); acc[3] = fmaf(wg, a.w, acc[3]);
       acc[4] = fmaf(wg, c.x, acc[4]); acc[5] = fmaf(wg, c.y, acc[5]); acc[6] = fmaf(wg, c.z, acc[6]); acc[7] = fmaf(wg, c.w, acc[7]);
     }
@@ -228,7 +246,7 @@ slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned cha
 
 ProjGeom make_proj_geom(int d, int H, int d_k, int batch) {
   ProjGeom g;
-  g.hp = 128 / d_k;
+  g.hp = d_k == 64 ? 2 : 1;
   g.hg = H / g.hp;
   const int stages = d / PJ_ROWS;
   int js = 1;
@@ -247,8 +265,8 @@ size_t proj_smem_bytes(const ProjGeom& g) { return 1024 + (size_t)PJ_NS * (PJ_W_
 
 int slim_proj_shape_ok(int d, int H, int d_k, int dtype) {
   if (dtype != SLIM_BF16) return 0;
-  if (d_k != 64 && d_k != 128) return 0;
-  if (d % PJ_ROWS != 0 || H % (128 / d_k) != 0) return 0;
+  if (d_k != 64 && d_k != 96 && d_k != 128) return 0;
+  if (d % PJ_ROWS != 0 || (d_k == 64 && (H & 1))) return 0;
   return 1;
 }
 
@@ -262,9 +280,11 @@ cudaError_t slim_proj_make_wmap(slim_ctx* ctx) {
   const int d = ctx->d, d_k = ctx->d_k, H = ctx->H;
   unsigned long long dims[3], strides[2];
   unsigned int box[3] = {64, PJ_ROWS, 2};
-  if (d_k == 128) {          // (64 columns, H*d rows, 2 column halves)
+  if (d_k != 64) {           // (64 columns, H*d rows, 2 column halves).  With d_k = 96 the second half runs
+                             // 32 columns into the next row: finite weights that land in ignored accumulator
+                             // rows (the W_KV allocation is padded so the very last row stays in bounds).
     dims[0] = 64; dims[1] = (unsigned long long)H * d; dims[2] = 2;
-    strides[0] = 256; strides[1] = 128;
+    strides[0] = (unsigned long long)d_k * 2; strides[1] = 128;
   } else {                   // d_k = 64: (64 columns, d rows, H heads)
     dims[0] = 64; dims[1] = d; dims[2] = H;
     strides[0] = 128; strides[1] = (unsigned long long)d * 128;

@@ -144,7 +144,15 @@ __global__ void slim_append_kernel(KT* __restrict__ cache, const KT* __restrict_
   }
   const KT* src = k_new + ((size_t)b * n_new + r) * d;
   KT* dst = cache + ((size_t)b * t_cap + pos + r) * d;
-  for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = src[e];
+  // rows are 16-byte aligned when d * sizeof(KT) is a multiple of 16 and the buffers are
+  const size_t bytes = (size_t)d * sizeof(KT);
+  if ((bytes & 15) == 0 && (((uintptr_t)src | (uintptr_t)dst) & 15) == 0) {
+    const uint4* s4 = reinterpret_cast<const uint4*>(src);
+    uint4* d4 = reinterpret_cast<uint4*>(dst);
+    for (int e = threadIdx.x; e < (int)(bytes >> 4); e += blockDim.x) d4[e] = __ldg(s4 + e);
+  } else {
+    for (int e = threadIdx.x; e < d; e += blockDim.x) dst[e] = src[e];
+  }
 }
 
 }  // namespace
