@@ -148,6 +148,14 @@ slim_status slim_decode_static_ws(slim_ctx* ctx, const void* q, const slim_cache
  * SLIM_ERR_CAPACITY or SLIM_ERR_TIMEOUT) and clears it.                        */
 slim_status slim_device_status(slim_ctx* ctx, void* stream);
 
+/* Self-test of the bounded device-side waits every TMA / tcgen05 kernel relies on: runs
+ * a one-CTA kernel that waits on a barrier nothing completes.  The wait must give up after
+ * its limit (about two seconds), the kernel must return normally, and the sticky device
+ * status must read SLIM_ERR_TIMEOUT afterwards.  Returns SLIM_OK if the kernel gave up as
+ * designed (the caller then reads and clears the status with slim_device_status); the CUDA
+ * context stays usable.  Synchronises `stream`.                                       */
+slim_status slim_selftest_bounded_wait(slim_ctx* ctx, void* stream);
+
 /* Kernel timing for roofline reports.  While enabled, slim_decode records CUDA
  * events on its stream before the main (K-reading) kernel, after it, and after
  * the combine/projection tail.  slim_profile_read waits for the last decode of

@@ -35,6 +35,7 @@ SIGNATURES = {
     "slim_static_workspace_max": (c_size_t, []),
     "slim_decode_static_ws": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "slim_device_status": (c_int, [c_void_p, c_void_p]),
+    "slim_selftest_bounded_wait": (c_int, [c_void_p, c_void_p]),
     "slim_profile_enable": (c_int, [c_void_p, c_int]),
     "slim_profile_read": (c_int, [c_void_p, POINTER(ctypes.c_float), POINTER(ctypes.c_float)]),
     "slim_set_path": (c_int, [c_void_p, c_int]),
@@ -165,6 +166,10 @@ def slim_decode_static_ws(ctx: int, q, cache: int, lengths, o, stream: int = 0) 
 
 def slim_device_status(ctx: int, stream: int = 0) -> int:
     return lib().slim_device_status(c_void_p(ctx), c_void_p(stream))
+
+
+def slim_selftest_bounded_wait(ctx: int, stream: int = 0) -> None:
+    _check(lib().slim_selftest_bounded_wait(c_void_p(ctx), c_void_p(stream)), "slim_selftest_bounded_wait")
 
 
 def slim_profile_enable(ctx: int, enable: bool) -> None:

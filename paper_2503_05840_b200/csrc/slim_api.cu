@@ -382,6 +382,18 @@ slim_status slim_device_status(slim_ctx* ctx, void* stream) {
   return (slim_status)v;
 }
 
+slim_status slim_selftest_bounded_wait(slim_ctx* ctx, void* stream) {
+  if (!ctx) return SLIM_ERR_INVALID_ARG;
+  // any_flag doubles as the kernel's "gave up" word; it is 0 between decodes
+  cudaStream_t st = (cudaStream_t)stream;
+  if (slim_launch_wait_selftest(ctx->status, ctx->any_flag, st) != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
+  if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
+  int gave_up = 0;
+  if (cudaMemcpy(&gave_up, ctx->any_flag, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return SLIM_ERR_CUDA;
+  cudaMemset(ctx->any_flag, 0, sizeof(int));
+  return gave_up ? SLIM_OK : SLIM_ERR_CUDA;
+}
+
 slim_status slim_profile_enable(slim_ctx* ctx, int enable) {
   if (!ctx) return SLIM_ERR_INVALID_ARG;
   if (enable && !ctx->prof_ev[0]) {

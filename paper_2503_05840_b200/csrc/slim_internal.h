@@ -89,6 +89,7 @@ cudaError_t slim_wkv_store(const double* X, int d, int H, int d_k, int dtype, vo
 int  slim_tc_shape_ok(int d, int H, int d_k, int dtype);
 int  slim_tc_workers(const slim_ctx* ctx);
 cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c);
+cudaError_t slim_launch_wait_selftest(int* status, int* gave_up, cudaStream_t st);
 cudaError_t slim_launch_tc(const slim_ctx* ctx, const slim_cache* c, const SlimDecodeParams& p, cudaStream_t st);
 
 // 3-D tiled tensor map with 128-byte swizzle over bf16 data (driver entry point looked up once)

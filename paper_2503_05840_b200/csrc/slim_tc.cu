@@ -511,6 +511,25 @@ constexpr int TC_SMEM_LIMIT = 227 * 1024;
 
 }  // namespace
 
+namespace {
+// A CTA waits on an mbarrier that nothing ever arrives at: the bounded wait has to give up,
+// report SLIM_ERR_TIMEOUT through the status word and let the kernel return normally.
+__global__ void slim_wait_selftest_kernel(int* status, int* gave_up) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  const uint32_t b = smem_u32(&bar);
+  if (threadIdx.x == 0) { mbar_init(b, 1); abort_flag = 0; fence_mbar_init(); }
+  __syncthreads();
+  const bool ok = mbar_wait<false>(b, 0, &abort_flag, status);
+  if (threadIdx.x == 0) *gave_up = ok ? 0 : 1;
+}
+}  // namespace
+
+cudaError_t slim_launch_wait_selftest(int* status, int* gave_up, cudaStream_t st) {
+  slim_wait_selftest_kernel<<<1, 64, 0, st>>>(status, gave_up);
+  return cudaGetLastError();
+}
+
 int slim_tc_shape_ok(int d, int H, int d_k, int dtype) {
   if (dtype != SLIM_BF16) return 0;
   if (d_k != 64 && d_k != 96 && d_k != 128) return 0;

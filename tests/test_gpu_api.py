@@ -248,3 +248,26 @@ def test_scores_far_above_the_first_tile_are_handled():
                 assert so.err_rms_norm(got[b], ref[b]) <= 2e-2, f"path {path} seq {b}"
     finally:
         layer.close()
+
+
+def test_bounded_wait_gives_up_reports_timeout_and_context_survives():
+    # a wait that nothing completes must run out, not hang: status TIMEOUT, then normal work again
+    cfg = synth.SlimConfig("wait", 256, 2, 128, 2, 64, 1, 1.0e4, "bf16")
+    L = synth.make_layer(cfg, 5)
+    layer = SlimLayer(cfg.d, cfg.H, cfg.d_k, cfg.rope_theta, "bf16", cfg.batch, cfg.context, DEV)
+    try:
+        layer.k.copy_(to_device_keys(L.K, "bf16", DEV))
+        W_KV = so.oracle_wkv(L.W_K, L.W_V)
+        layer.set_wkv(W_KV)
+        q = to_device_keys(L.q, "bf16", DEV)
+        ld = torch.from_numpy(L.lengths).to(DEV)
+        before = layer.decode(q, ld).clone()
+        assert layer.device_status() == B.SLIM_OK
+        B.slim_selftest_bounded_wait(layer.ctx, torch.cuda.current_stream().cuda_stream)
+        assert layer.device_status() == B.SLIM_ERR_TIMEOUT
+        assert layer.device_status() == B.SLIM_OK
+        after = layer.decode(q, ld).clone()
+        assert layer.device_status() == B.SLIM_OK
+        assert torch.equal(before, after)
+    finally:
+        layer.close()

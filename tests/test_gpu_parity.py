@@ -154,3 +154,22 @@ def test_config2_codellama_shape_one_layer_sampled_sequences():
 
 def test_config4_long_context_full():
     _run_device_case(synth.CONFIGS[4], 4, [0])
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3, 4, 5, 6])
+def test_random_ragged_batches(seed):
+    """Random batch sizes and lengths (zeros, single rows, tile edges): exercises the
+    stream-K schedule (empty worker ranges, many units per sequence, sequence groups of
+    the projection that are only partly filled)."""
+    g = np.random.default_rng(seed)
+    d, H, d_k, theta = [(512, 4, 128, 1.0e6), (256, 4, 64, 0.0), (384, 4, 96, 1.0e4)][seed % 3]
+    batch = int(g.integers(1, 40))
+    t_cap = int(g.integers(40, 700))
+    lengths = g.integers(0, t_cap + 1, size=batch).astype(np.int32)
+    lengths[g.integers(0, batch)] = t_cap
+    if batch > 2:
+        lengths[g.integers(0, batch)] = 0
+        lengths[g.integers(0, batch)] = 1
+    cfg = synth.SlimConfig("ragged", d, H, d_k, batch, t_cap, 1, theta, "bf16")
+    L = synth.make_layer(cfg, 9000 + seed, lengths=lengths)
+    _run_host_case(cfg, L)
