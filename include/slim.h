@@ -84,6 +84,18 @@ void        slim_destroy(slim_ctx* ctx);
 slim_status slim_set_weights(slim_ctx* ctx, const void* W_K, const void* W_V, int host_dtype,
                              double* wkv_out, double* residual_out);
 
+/* Non-square projections (section "Support for non-square weight matrices", Option 1):
+ * the model width d_model is smaller than e = H*d_k, W_K and W_V are [d_model][e] (host,
+ * row-major) and K = X W_K is e wide.  Forms the right inverse
+ * W_K^{-1} = W_K^T (W_K W_K^T)^{-1} in float64 (LU solve of the d_model x d_model system)
+ * and stores W_KV = W_K^{-1} W_V, an [e][e] matrix, so that K W_KV = V for every K in the
+ * row space of W_K.  The ctx must have been created with d = e; caches, slim_append_k and
+ * slim_decode are used unchanged.  wkv_out (may be NULL) receives the [e][e] float64
+ * W_KV, residual_out (may be NULL) max |W_K W_KV - W_V|.  SLIM_ERR_SINGULAR if W_K does
+ * not have full row rank.  Synchronous.                                              */
+slim_status slim_set_weights_nonsquare(slim_ctx* ctx, const void* W_K, const void* W_V, int d_model,
+                                       int host_dtype, double* wkv_out, double* residual_out);
+
 /* Load a precomputed W_KV (the paper stores it in the parameter file in place
  * of W_V, Eq. 6).  W_KV: host, row-major [d][d].  Synchronous.                 */
 slim_status slim_set_wkv(slim_ctx* ctx, const void* W_KV, int host_dtype);

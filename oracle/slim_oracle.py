@@ -18,6 +18,10 @@ Paper passages followed (arxiv 2503.05840):
                         rotated after they are read
   Appendix "MHA complexity"     OP counts 2 n d_k (scores) and 2 n d
                         (weighted sum of K) per head
+  Section "Support for non-square weight matrices", Option 1
+                        right inverse W_K^{-1} = W_K^T (W_K W_K^T)^{-1} for
+                        W_K in R^{d x e}, e = d_k h > d;  W_KV = W_K^{-1} W_V
+                        is e x e
 
 Readings where the paper is silent (the CUDA path takes the same ones):
   * RoPE pairs element j with j + d_k/2 inside a head, frequency
@@ -118,6 +122,19 @@ def oracle_wkv(W_K: np.ndarray, W_V: np.ndarray) -> np.ndarray:
     return np.linalg.solve(W_K, W_V)
 
 
+def oracle_wkv_right_inverse(W_K: np.ndarray, W_V: np.ndarray) -> np.ndarray:
+    """Non-square projections, Option 1: W_K, W_V are [d, e] with e > d.
+    W_K^{-1} = W_K^T (W_K W_K^T)^{-1} (so that W_K W_K^{-1} = I_d) and
+    W_KV = W_K^{-1} W_V, an [e, e] matrix.  float64; the d x d inverse is
+    applied as a linear solve."""
+    W_K = np.asarray(W_K, dtype=F64)
+    W_V = np.asarray(W_V, dtype=F64)
+    if W_K.ndim != 2 or W_K.shape != W_V.shape or W_K.shape[0] > W_K.shape[1]:
+        raise ValueError("W_K and W_V must be [d, e] with e >= d")
+    G = W_K @ W_K.T                                   # d x d
+    return W_K.T @ np.linalg.solve(G, W_V)            # e x e
+
+
 # --------------------------------------------------------------------------
 # Eq. 4, 5, 2: vanilla MHA decode with an explicit V cache
 # --------------------------------------------------------------------------
@@ -127,14 +144,15 @@ def oracle_vanilla(X: np.ndarray, W_Q: np.ndarray, W_K: np.ndarray, W_V: np.ndar
     over all T = len(X) tokens.  X: [T, d].  If q is given it replaces
     X[-1] W_Q (used where the query carries a bias)."""
     X = np.asarray(X, dtype=F64)
-    T, d = X.shape
-    d_k = d // H
+    T = X.shape[0]
+    e = np.asarray(W_K).shape[1]                 # width of K and V: d for square MHA, d_k h > d otherwise
+    d_k = e // H
     K = X @ np.asarray(W_K, dtype=F64)           # Eq. 4
     V = X @ np.asarray(W_V, dtype=F64)           # Eq. 5
     if q is None:
         q = X[-1] @ np.asarray(W_Q, dtype=F64)   # Eq. 4, one query row
     q = np.asarray(q, dtype=F64)
-    out = np.empty(d, dtype=F64)
+    out = np.empty(e, dtype=F64)
     for i in range(H):
         sl = slice(i * d_k, (i + 1) * d_k)
         s = attention_weights(q[sl], K[:, sl], rope_theta)

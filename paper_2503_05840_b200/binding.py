@@ -25,6 +25,7 @@ SIGNATURES = {
     "slim_create": (c_int, [POINTER(c_void_p), c_int, c_int, c_int, c_double, c_int]),
     "slim_destroy": (None, [c_void_p]),
     "slim_set_weights": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_void_p, POINTER(c_double)]),
+    "slim_set_weights_nonsquare": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_int, c_void_p, POINTER(c_double)]),
     "slim_set_wkv": (c_int, [c_void_p, c_void_p, c_int]),
     "slim_cache_bytes": (c_size_t, [c_void_p, c_int, c_int]),
     "slim_workspace_bytes": (c_size_t, [c_void_p, c_int, c_int]),
@@ -118,6 +119,19 @@ def slim_set_weights(ctx: int, W_K, W_V, want_wkv: bool = False):
     out = np.empty(a.shape, dtype=np.float64) if want_wkv else None
     res = c_double(0.0)
     _check(lib().slim_set_weights(c_void_p(ctx), _ptr(a), _ptr(b), dt, _ptr(out), byref(res)), "slim_set_weights")
+    return res.value, out
+
+
+def slim_set_weights_nonsquare(ctx: int, W_K, W_V, want_wkv: bool = False):
+    """W_K, W_V: [d_model, e] with e = H d_k > d_model.  Returns (residual, W_KV [e, e] float64 or None)."""
+    a = np.ascontiguousarray(W_K, dtype=np.float64)
+    b = np.ascontiguousarray(W_V, dtype=np.float64)
+    assert a.shape == b.shape and a.ndim == 2
+    d_model, e = a.shape
+    out = np.empty((e, e), dtype=np.float64) if want_wkv else None
+    res = c_double(0.0)
+    _check(lib().slim_set_weights_nonsquare(c_void_p(ctx), _ptr(a), _ptr(b), d_model, SLIM_HOST_F64, _ptr(out), byref(res)),
+           "slim_set_weights_nonsquare")
     return res.value, out
 
 

@@ -247,6 +247,46 @@ slim_status slim_set_weights(slim_ctx* ctx, const void* W_K, const void* W_V, in
   return st;
 }
 
+slim_status slim_set_weights_nonsquare(slim_ctx* ctx, const void* W_K, const void* W_V, int d_model, int host_dtype,
+                                       double* wkv_out, double* residual_out) {
+  if (!ctx || !W_K || !W_V || (host_dtype != SLIM_HOST_F32 && host_dtype != SLIM_HOST_F64)) return SLIM_ERR_INVALID_ARG;
+  const int e = ctx->d;                                  // width of K and V: e = H d_k
+  if (d_model <= 0 || d_model > e) return SLIM_ERR_INVALID_ARG;
+  const size_t de = (size_t)d_model * e, ee = (size_t)e * e, dd = (size_t)d_model * d_model;
+  double *Wk = nullptr, *Wv = nullptr, *G = nullptr, *Y = nullptr, *X = nullptr, *R = nullptr;
+  slim_status st = upload_f64(W_K, host_dtype, de, &Wk);
+  if (st == SLIM_OK) st = upload_f64(W_V, host_dtype, de, &Wv);
+  if (st == SLIM_OK && (cudaMalloc(&G, sizeof(double) * dd) != cudaSuccess || cudaMalloc(&Y, sizeof(double) * de) != cudaSuccess ||
+                        cudaMalloc(&X, sizeof(double) * ee) != cudaSuccess))
+    st = SLIM_ERR_OOM;
+  int info = 0;
+  if (st == SLIM_OK) {
+    // right inverse: W_K^{-1} = W_K^T (W_K W_K^T)^{-1};  W_KV = W_K^{-1} W_V = W_K^T [ (W_K W_K^T)^{-1} W_V ]
+    cudaError_t ce = slim_dgemm(Wk, Wk, G, d_model, d_model, e, 0, 1);                       // G = W_K W_K^T
+    if (ce == cudaSuccess) ce = cudaMemcpy(Y, Wv, sizeof(double) * de, cudaMemcpyDeviceToDevice);
+    if (ce == cudaSuccess) ce = slim_wkv_solve_rhs(G, Y, d_model, e, &info);                  // G Y = W_V
+    if (ce == cudaSuccess && info == 0) ce = slim_dgemm(Wk, Y, X, e, e, d_model, 1, 0);       // W_KV = W_K^T Y
+    if (ce == cudaErrorMemoryAllocation) st = SLIM_ERR_OOM;
+    else if (ce != cudaSuccess) st = SLIM_ERR_CUDA;
+    else if (info != 0) st = SLIM_ERR_SINGULAR;
+  }
+  if (st == SLIM_OK && residual_out) {                   // max | W_K W_KV - W_V |
+    if (cudaMalloc(&R, sizeof(double) * de) != cudaSuccess) st = SLIM_ERR_OOM;
+    else if (slim_dgemm(Wk, X, R, d_model, e, e, 0, 0) != cudaSuccess || slim_absdiff_max(R, Wv, de, residual_out) != cudaSuccess)
+      st = SLIM_ERR_CUDA;
+  }
+  if (st == SLIM_OK && wkv_out && cudaMemcpy(wkv_out, X, sizeof(double) * ee, cudaMemcpyDeviceToHost) != cudaSuccess) st = SLIM_ERR_CUDA;
+  if (st == SLIM_OK) {
+    if (slim_wkv_store(X, ctx->d, ctx->H, ctx->d_k, ctx->dtype, ctx->wkv) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess)
+      st = SLIM_ERR_CUDA;
+    else
+      ctx->has_weights = 1;
+  }
+  cudaFree(Wk); cudaFree(Wv); cudaFree(G); cudaFree(Y); cudaFree(X); cudaFree(R);
+  if (st != SLIM_OK) cudaGetLastError();
+  return st;
+}
+
 slim_status slim_set_wkv(slim_ctx* ctx, const void* W_KV, int host_dtype) {
   if (!ctx || !W_KV || (host_dtype != SLIM_HOST_F32 && host_dtype != SLIM_HOST_F64)) return SLIM_ERR_INVALID_ARG;
   double* X = nullptr;

@@ -82,6 +82,11 @@ cudaError_t slim_launch_append(const slim_ctx* ctx, const slim_cache* c, const v
 // fp64 solve W_K X = W_V on the device; A and B are device row-major [n][n]
 // float64, both overwritten; X is returned in B.  info: 0 ok, 1 singular.
 cudaError_t slim_wkv_solve(double* A, double* B, int n, int* info_host);
+// same with an n x m right-hand side B (row-major), X returned in B
+cudaError_t slim_wkv_solve_rhs(double* A, double* B, int n, int m, int* info_host);
+// C[M x N] = op(A) op(B) in float64 on the device (row-major, t* = 1 transposes); max |A - B|
+cudaError_t slim_dgemm(const double* A, const double* B, double* C, int M, int N, int K, int ta, int tb);
+cudaError_t slim_absdiff_max(const double* A, const double* B, size_t n, double* res_host);
 cudaError_t slim_wkv_residual(const double* Wk, const double* X, const double* Wv, int n, double* res_host);
 cudaError_t slim_wkv_store(const double* X, int d, int H, int d_k, int dtype, void* dst);
 

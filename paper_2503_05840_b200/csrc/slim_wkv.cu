@@ -1,7 +1,10 @@
 // Eq. 6 on the device in float64:  solve W_K X = W_V  (X = W_KV) by blocked LU
 // with partial pivoting on the augmented matrix M = [W_K | W_V] (n x 2n),
 // followed by a blocked back substitution.  Offline set-up work; written for
-// clarity and a few seconds at n = 4096, not for peak FP64 rate.
+// clarity and a few seconds at n = 4096, not for peak FP64 rate.  The right-hand
+// side may have any number of columns m (M is n x (n + m)): the non-square case
+// (section "Support for non-square weight matrices", Option 1) solves
+// (W_K W_K^T) Y = W_V with n = d_model and m = e.
 #include "slim_internal.h"
 
 namespace {
@@ -143,13 +146,13 @@ __global__ void __launch_bounds__(256) lu_gemm_kernel(double* __restrict__ M, in
 }
 
 // --- X[k0:k0+kb, :] = U11^{-1} Y[k0:k0+kb, :] (upper, non-unit), thread per column of the right half
-__global__ void lu_trsm_upper_kernel(double* __restrict__ M, int ld, int n, int k0, int kb) {
+__global__ void lu_trsm_upper_kernel(double* __restrict__ M, int ld, int n, int k0, int kb) {   // rhs columns [n, ld)
   __shared__ double s_U[NB][NB + 1];
   for (int e = threadIdx.x; e < kb * kb; e += blockDim.x)
     s_U[e / kb][e % kb] = M[(size_t)(k0 + e / kb) * ld + k0 + e % kb];
   __syncthreads();
   const int c = n + blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= 2 * n) return;
+  if (c >= ld) return;
   double x[NB];
 #pragma unroll
   for (int rr = 0; rr < NB; ++rr) {
@@ -165,19 +168,74 @@ __global__ void lu_trsm_upper_kernel(double* __restrict__ M, int ld, int n, int 
   }
 }
 
-__global__ void pack_aug_kernel(const double* __restrict__ A, const double* __restrict__ B, double* __restrict__ M, int n) {
+// M = [A | B]: A is n x n, B is n x m
+__global__ void pack_aug_kernel(const double* __restrict__ A, const double* __restrict__ B, double* __restrict__ M, int n, int m) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= (size_t)n * n) return;
-  const size_t r = i / n, c = i % n;
-  M[r * 2 * n + c] = A[i];
-  M[r * 2 * n + n + c] = B[i];
+  const size_t ld = (size_t)n + m;
+  if (i >= (size_t)n * ld) return;
+  const size_t r = i / ld, c = i % ld;
+  M[i] = c < (size_t)n ? A[r * n + c] : B[r * m + (c - n)];
 }
 
-__global__ void unpack_x_kernel(const double* __restrict__ M, double* __restrict__ X, int n) {
+__global__ void unpack_x_kernel(const double* __restrict__ M, double* __restrict__ X, int n, int m) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= (size_t)n * n) return;
-  const size_t r = i / n, c = i % n;
-  X[i] = M[r * 2 * n + n + c];
+  if (i >= (size_t)n * m) return;
+  const size_t r = i / m, c = i % m;
+  X[i] = M[r * ((size_t)n + m) + n + c];
+}
+
+// C[M x N] = op(A) op(B), float64, 64 x 64 tiles.  op(A) is M x K: A is [M][K] (ta = 0) or [K][M]
+// (ta = 1); op(B) is K x N: B is [K][N] (tb = 0) or [N][K] (tb = 1).  Row-major, dense.
+__global__ void __launch_bounds__(256) dgemm_kernel(const double* __restrict__ A, const double* __restrict__ B,
+                                                    double* __restrict__ C, int Mr, int Nc, int Kd, int ta, int tb) {
+  __shared__ double s_A[64][NB + 1];
+  __shared__ double s_B[NB][64 + 1];
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int rb = blockIdx.y * 64, cb = blockIdx.x * 64;
+  double acc[4][4] = {};
+  for (int k0 = 0; k0 < Kd; k0 += NB) {
+    for (int e = threadIdx.x; e < 64 * NB; e += 256) {
+      const int r = e / NB, k = e % NB;
+      double v = 0.0;
+      if (rb + r < Mr && k0 + k < Kd) v = ta ? A[(size_t)(k0 + k) * Mr + rb + r] : A[(size_t)(rb + r) * Kd + k0 + k];
+      s_A[r][k] = v;
+    }
+    for (int e = threadIdx.x; e < NB * 64; e += 256) {
+      const int k = e / 64, c = e % 64;
+      double v = 0.0;
+      if (cb + c < Nc && k0 + k < Kd) v = tb ? B[(size_t)(cb + c) * Kd + k0 + k] : B[(size_t)(k0 + k) * Nc + cb + c];
+      s_B[k][c] = v;
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int k = 0; k < NB; ++k) {
+      double a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { a[i] = s_A[ty * 4 + i][k]; b[i] = s_B[k][tx * 4 + i]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fma(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int r = rb + ty * 4 + i, c = cb + tx * 4 + j;
+      if (r < Mr && c < Nc) C[(size_t)r * Nc + c] = acc[i][j];
+    }
+}
+
+__global__ void absdiff_max_kernel(const double* __restrict__ A, const double* __restrict__ B, size_t n, double* out) {
+  double m = 0.0;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    m = fmax(m, fabs(A[i] - B[i]));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0)
+    atomicMax(reinterpret_cast<unsigned long long*>(out), (unsigned long long)__double_as_longlong(m));
 }
 
 __global__ void absmax_kernel(const double* __restrict__ A, size_t n, double* out) {
@@ -249,15 +307,17 @@ __global__ void store_wkv_kernel(const double* __restrict__ X, WT* __restrict__ 
 
 }  // namespace
 
-cudaError_t slim_wkv_solve(double* A, double* B, int n, int* info_host) {
+cudaError_t slim_wkv_solve(double* A, double* B, int n, int* info_host) { return slim_wkv_solve_rhs(A, B, n, n, info_host); }
+
+cudaError_t slim_wkv_solve_rhs(double* A, double* B, int n, int m, int* info_host) {
   double* M = nullptr; int* piv = nullptr; double* scal = nullptr;   // scal: [0] = max|A| bits, [1] = info
-  const int ld = 2 * n;
+  const int ld = n + m;
   CK(cudaMalloc(&M, sizeof(double) * (size_t)n * ld));
   CK(cudaMalloc(&piv, sizeof(int) * n));
   CK(cudaMalloc(&scal, 16));
   CK(cudaMemset(scal, 0, 16));
   const size_t nn = (size_t)n * n;
-  pack_aug_kernel<<<(unsigned)((nn + 255) / 256), 256>>>(A, B, M, n);
+  pack_aug_kernel<<<(unsigned)(((size_t)n * ld + 255) / 256), 256>>>(A, B, M, n, m);
   absmax_kernel<<<256, 256>>>(A, nn, scal);
   double amax = 0.0;
   CK(cudaMemcpy(&amax, scal, sizeof(double), cudaMemcpyDeviceToHost));
@@ -279,13 +339,13 @@ cudaError_t slim_wkv_solve(double* A, double* B, int n, int* info_host) {
   const int nblk = (n + NB - 1) / NB;
   for (int blk = nblk - 1; blk >= 0; --blk) {
     const int k0 = blk * NB, kb = (n - k0 < NB) ? n - k0 : NB;
-    lu_trsm_upper_kernel<<<(n + 127) / 128, 128>>>(M, ld, n, k0, kb);
+    lu_trsm_upper_kernel<<<(m + 127) / 128, 128>>>(M, ld, n, k0, kb);
     if (k0 > 0) {
-      dim3 g((n + 63) / 64, (k0 + 63) / 64);
+      dim3 g((m + 63) / 64, (k0 + 63) / 64);
       lu_gemm_kernel<<<g, 256>>>(M, ld, 0, k0, n, ld, k0, kb);
     }
   }
-  unpack_x_kernel<<<(unsigned)((nn + 255) / 256), 256>>>(M, B, n);
+  unpack_x_kernel<<<(unsigned)(((size_t)n * m + 255) / 256), 256>>>(M, B, n, m);
   CK(cudaGetLastError());
   CK(cudaMemcpy(info_host, info, sizeof(int), cudaMemcpyDeviceToHost));
   cudaFree(M); cudaFree(piv); cudaFree(scal);
@@ -311,4 +371,21 @@ cudaError_t slim_wkv_store(const double* X, int d, int H, int d_k, int dtype, vo
   else
     store_wkv_kernel<float><<<(unsigned)((nn + 255) / 256), 256>>>(X, (float*)dst, d, H, d_k);
   return cudaGetLastError();
+}
+
+cudaError_t slim_dgemm(const double* A, const double* B, double* C, int M, int N, int K, int ta, int tb) {
+  dim3 g((N + 63) / 64, (M + 63) / 64);
+  dgemm_kernel<<<g, 256>>>(A, B, C, M, N, K, ta, tb);
+  return cudaGetLastError();
+}
+
+cudaError_t slim_absdiff_max(const double* A, const double* B, size_t n, double* res_host) {
+  double* out = nullptr;
+  cudaError_t e = cudaMalloc(&out, sizeof(double));
+  if (e != cudaSuccess) return e;
+  cudaMemset(out, 0, sizeof(double));
+  absdiff_max_kernel<<<256, 256>>>(A, B, n, out);
+  e = cudaMemcpy(res_host, out, sizeof(double), cudaMemcpyDeviceToHost);
+  cudaFree(out);
+  return e;
 }

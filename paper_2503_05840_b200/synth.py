@@ -109,6 +109,22 @@ def make_weights(d: int, seed: int):
     return W_Q, W_K, W_V, Qo, s
 
 
+def make_weights_nonsquare(d_model: int, e: int, seed: int):
+    """Non-square projections [d_model, e], e > d_model: W_K = diag(s) Q[:d_model, :] with Q an
+    e x e Haar-orthogonal matrix and s ~ U[0.5, 2] (orthogonal rows, cond <= 4);
+    W_V, W_Q ~ N(0, 1/d_model).  Returns (W_Q, W_K, W_V, Qrows, s) in float64."""
+    g = _rng(seed)
+    G = g.standard_normal((e, e))
+    Qo, R = np.linalg.qr(G)
+    Qo = Qo * np.sign(np.diag(R))[None, :]
+    Qrows = Qo[:d_model, :]
+    s = g.uniform(0.5, 2.0, size=d_model)
+    W_K = s[:, None] * Qrows
+    W_V = g.standard_normal((d_model, e)) / np.sqrt(d_model)
+    W_Q = g.standard_normal((d_model, e)) / np.sqrt(d_model)
+    return W_Q, W_K, W_V, Qrows, s
+
+
 def make_lengths(cfg: SlimConfig, seed: int) -> np.ndarray:
     if cfg.ragged_min and cfg.ragged_min < cfg.context:
         g = _rng(seed ^ 0x5EED)

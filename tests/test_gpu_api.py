@@ -271,3 +271,41 @@ def test_bounded_wait_gives_up_reports_timeout_and_context_survives():
         assert torch.equal(before, after)
     finally:
         layer.close()
+
+
+def test_nonsquare_weights_right_inverse_matches_oracle_and_decodes():
+    # d_model = 192 < e = H d_k = 512: W_KV is e x e (non-square section, Option 1)
+    d_model, e, H, d_k, T = 192, 512, 4, 128, 300
+    W_Q, W_K, W_V, Qrows, s = synth.make_weights_nonsquare(d_model, e, 21)
+    g = np.random.default_rng(2)
+    lengths = np.array([T, 77], dtype=np.int32)
+    layer = SlimLayer(e, H, d_k, 1.0e4, "bf16", 2, T, DEV)
+    try:
+        with torch.cuda.device(DEV):
+            res, wkv = B.slim_set_weights_nonsquare(layer.ctx, W_K, W_V, want_wkv=True)
+        ref = so.oracle_wkv_right_inverse(W_K, W_V)
+        assert np.allclose(wkv, ref, rtol=1e-8, atol=1e-10)
+        assert np.allclose(wkv, Qrows.T @ (W_V / s[:, None]), rtol=1e-8, atol=1e-10)
+        assert res < 1e-10
+        K = np.zeros((2, T, e), dtype=np.float32); q = np.zeros((2, e), dtype=np.float32)
+        Xs = []
+        for b in range(2):
+            X = g.standard_normal((int(lengths[b]), d_model)); Xs.append(X)
+            K[b, :lengths[b]] = synth.round_to_bf16(X @ W_K); q[b] = synth.round_to_bf16(X[-1] @ W_Q)
+        layer.k.copy_(to_device_keys(K, "bf16", DEV))
+        got = layer.decode(to_device_keys(q, "bf16", DEV), torch.from_numpy(lengths).to(DEV)).cpu().numpy().astype(np.float64)
+        assert layer.device_status() == B.SLIM_OK
+        for b in range(2):
+            slim = so.oracle_slim(q[b], K[b, :lengths[b]], ref, H, 1.0e4)
+            assert so.err_rms_norm(got[b], slim) <= 2e-2
+            # and, up to the bf16 rounding of K and q, the vanilla result with an explicit V = X W_V
+            van = so.oracle_vanilla(Xs[b], W_Q, W_K, W_V, H, 1.0e4)
+            assert so.err_rms_norm(got[b], van) <= 5e-2
+        # a rank-deficient W_K has no right inverse
+        bad = W_K.copy(); bad[1] = bad[0]
+        with pytest.raises(B.SlimError) as ei:
+            with torch.cuda.device(DEV):
+                B.slim_set_weights_nonsquare(layer.ctx, bad, W_V)
+        assert ei.value.status == B.SLIM_ERR_SINGULAR
+    finally:
+        layer.close()

@@ -324,3 +324,46 @@ def test_error_norms():
     assert abs(so.err_fp32_norm(got, ref) - 0.1) < 1e-15
     got2 = ref + np.array([0.3, 0.0, 0.0, 0.0])
     assert abs(so.err_fp32_norm(got2, ref) - 0.1) < 1e-15   # relative to |ref_i| = 3
+
+
+# ---- non-square projections, Option 1 (right inverse) -----------------------
+def test_right_inverse_hand_example_1x2():
+    # W_K = [3 4]: W_K W_K^T = 25, right inverse = [3 4]^T / 25; W_V = [1 2]
+    W_K = np.array([[3.0, 4.0]]); W_V = np.array([[1.0, 2.0]])
+    W_KV = so.oracle_wkv_right_inverse(W_K, W_V)
+    assert np.allclose(W_KV, np.array([[3.0, 6.0], [4.0, 8.0]]) / 25.0, rtol=0, atol=1e-15)
+    for x in (1.0, -2.5):
+        assert np.allclose((x * W_K) @ W_KV, x * W_V)          # K W_KV = V
+
+
+def test_right_inverse_properties_and_closed_form():
+    from paper_2503_05840_b200 import synth
+    d, e = 6, 16
+    W_Q, W_K, W_V, Qrows, s = synth.make_weights_nonsquare(d, e, 11)
+    W_KV = so.oracle_wkv_right_inverse(W_K, W_V)
+    assert W_KV.shape == (e, e)
+    assert np.allclose(W_K @ W_KV, W_V, rtol=1e-12, atol=1e-13)                   # W_K W_K^{-1} W_V = W_V
+    assert np.allclose(W_KV, Qrows.T @ (W_V / s[:, None]), rtol=1e-11, atol=1e-13)  # rows of W_K are s_i q_i
+    Rinv = so.oracle_wkv_right_inverse(W_K, np.eye(d) @ W_K)                      # W_K^{-1} W_K: projector on the row space
+    assert np.allclose(Rinv, Rinv.T, atol=1e-12) and np.allclose(Rinv @ Rinv, Rinv, atol=1e-12)
+    assert abs(np.trace(Rinv) - d) < 1e-10
+    X = np.random.default_rng(0).standard_normal((9, d))
+    assert np.allclose((X @ W_K) @ W_KV, X @ W_V, rtol=1e-11, atol=1e-12)          # V from K for any input
+
+
+def test_right_inverse_reduces_to_the_inverse_for_square_weights():
+    g = np.random.default_rng(3)
+    W_K = g.standard_normal((7, 7)) + 3 * np.eye(7); W_V = g.standard_normal((7, 7))
+    assert np.allclose(so.oracle_wkv_right_inverse(W_K, W_V), so.oracle_wkv(W_K, W_V), rtol=1e-9, atol=1e-11)
+
+
+def test_slim_equals_vanilla_with_nonsquare_projections():
+    from paper_2503_05840_b200 import synth
+    d, e, H, T = 6, 16, 2, 13
+    W_Q, W_K, W_V, _, _ = synth.make_weights_nonsquare(d, e, 5)
+    X = np.random.default_rng(1).standard_normal((T, d))
+    for theta in (0.0, 1.0e4):
+        van = so.oracle_vanilla(X, W_Q, W_K, W_V, H, theta)
+        slim = so.oracle_slim(X[-1] @ W_Q, X @ W_K, so.oracle_wkv_right_inverse(W_K, W_V), H, theta)
+        assert van.shape == (e,)
+        assert np.allclose(slim, van, rtol=1e-10, atol=1e-12)
