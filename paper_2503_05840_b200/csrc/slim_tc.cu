@@ -424,8 +424,9 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           const int ntile = seg_end - gg;
           for (int kt = 0; kt < ntile; ++kt, ++it) {
             const int st = it % g.ns, ps = it % TC_NP;
-            ok = mbar_wait<false>(bar_k_full + 8 * st, (it / g.ns) & 1, s_abort, p.status);
-            if (ok) ok = mbar_wait<true>(bar_p_full + 8 * ps, (it / TC_NP) & 1, s_abort, p.status);
+            // p_full alone is enough: every local score warp arrives on it after it has seen
+            // k_full of this stage, so the keys have landed (and are ordered before this wait).
+            ok = mbar_wait<true>(bar_p_full + 8 * ps, (it / TC_NP) & 1, s_abort, p.status);
             if (ok && kt == 0 && uc > 0) ok = mbar_wait<false>(bar_u_empty, (uc - 1) & 1, s_abort, p.status);
             if (!ok) break;
             fence_proxy_async_smem();        // P pieces and zero-filled key rows -> tensor-core reads
