@@ -18,6 +18,11 @@ Paper passages followed (arxiv 2503.05840):
                         rotated after they are read
   Appendix "MHA complexity"     OP counts 2 n d_k (scores) and 2 n d
                         (weighted sum of K) per head
+  Section "Support for non-square weight matrices", Option 2 (X-cache) and
+  section "Support for encoder-decoder transformers", Option 2 (E-cache)
+                        A_i = ((x_n W_Q,i + b) W_K,i^T) X^T; the values are
+                        recomputed as well: head_i = [softmax(.) X] W_V,i.
+                        No RoPE in this scheme.
   Section "Support for non-square weight matrices", Option 1
                         right inverse W_K^{-1} = W_K^T (W_K W_K^T)^{-1} for
                         W_K in R^{d x e}, e = d_k h > d;  W_KV = W_K^{-1} W_V
@@ -195,6 +200,27 @@ def oracle_slim_option1(q: np.ndarray, K: np.ndarray, W_KV: np.ndarray, H: int,
         s = attention_weights(q[sl], K[:, sl], rope_theta)
         V_i = K @ W_KV[:, sl]                                # Eq. 6
         out[sl] = s @ V_i
+    return out
+
+
+def oracle_xcache(q: np.ndarray, X: np.ndarray, W_K: np.ndarray, W_V: np.ndarray, H: int) -> np.ndarray:
+    """X-cache / E-cache scheme for one decode token.  q: [e] = x_n W_Q (+ query bias),
+    X: [T, d] cached layer inputs (or encoder outputs), W_K, W_V: [d, e].  Per head i:
+    q~_i = q_i W_K,i^T (a d-vector), A_i = q~_i X^T, s_i = softmax(A_i / sqrt(d_k)),
+    u_i = s_i X, head_i = u_i W_V,i.  Returns concat(head_1 .. head_h), [e]."""
+    q = np.asarray(q, dtype=F64)
+    X = np.asarray(X, dtype=F64)
+    W_K = np.asarray(W_K, dtype=F64)
+    W_V = np.asarray(W_V, dtype=F64)
+    e = W_K.shape[1]
+    d_k = e // H
+    out = np.empty(e, dtype=F64)
+    for i in range(H):
+        sl = slice(i * d_k, (i + 1) * d_k)
+        qt = q[sl] @ W_K[:, sl].T                     # [d]
+        s = softmax(X @ qt / math.sqrt(d_k))          # [T]
+        u = s @ X                                     # [d]
+        out[sl] = u @ W_V[:, sl]                      # [d_k]
     return out
 
 

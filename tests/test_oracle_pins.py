@@ -367,3 +367,41 @@ def test_slim_equals_vanilla_with_nonsquare_projections():
         slim = so.oracle_slim(X[-1] @ W_Q, X @ W_K, so.oracle_wkv_right_inverse(W_K, W_V), H, theta)
         assert van.shape == (e,)
         assert np.allclose(slim, van, rtol=1e-10, atol=1e-12)
+
+
+# ---- X-cache / E-cache scheme (non-square Option 2, encoder-decoder Option 2) ----
+def test_xcache_equals_vanilla_square_and_nonsquare_with_query_bias():
+    from paper_2503_05840_b200 import synth
+    g = np.random.default_rng(4)
+    for d, e, H, T in ((8, 8, 2, 11), (6, 16, 4, 9)):
+        if d == e:
+            W_Q, W_K, W_V, _, _ = synth.make_weights(d, 3)
+        else:
+            W_Q, W_K, W_V, _, _ = synth.make_weights_nonsquare(d, e, 3)
+        X = g.standard_normal((T, d))
+        bias = g.standard_normal(e)
+        q = X[-1] @ W_Q + bias
+        van = so.oracle_vanilla(X, W_Q, W_K, W_V, H, 0.0, q=q)       # explicit K and V, same biased query
+        xc = so.oracle_xcache(q, X, W_K, W_V, H)
+        assert np.allclose(xc, van, rtol=1e-11, atol=1e-13)
+
+
+def test_xcache_single_token_and_identical_rows():
+    g = np.random.default_rng(6)
+    d, H = 8, 2
+    W_K = g.standard_normal((d, d)); W_V = g.standard_normal((d, d))
+    x0 = g.standard_normal(d); q = g.standard_normal(d)
+    assert np.allclose(so.oracle_xcache(q, x0[None, :], W_K, W_V, H), x0 @ W_V)          # T = 1: the value row
+    X = np.tile(x0, (7, 1))
+    assert np.allclose(so.oracle_xcache(q, X, W_K, W_V, H), x0 @ W_V)                    # uniform softmax
+
+
+def test_xcache_two_tokens_closed_form():
+    # one head, d = 2: scores a_t = (q W_K^T) . x_t / sqrt(2); output = sigma(a0 - a1) v0 + (1 - sigma) v1
+    W_K = np.array([[1.0, 2.0], [0.5, -1.0]]); W_V = np.array([[2.0, 0.0], [1.0, 3.0]])
+    X = np.array([[1.0, 0.0], [0.0, 2.0]]); q = np.array([0.3, -0.7])
+    qt = q @ W_K.T
+    a = X @ qt / np.sqrt(2.0)
+    sig = 1.0 / (1.0 + np.exp(-(a[0] - a[1])))
+    want = sig * (X[0] @ W_V) + (1 - sig) * (X[1] @ W_V)
+    assert np.allclose(so.oracle_xcache(q, X, W_K, W_V, 1), want, rtol=1e-13)
