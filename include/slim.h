@@ -156,6 +156,22 @@ size_t      slim_static_workspace_max(void);
 slim_status slim_decode_static_ws(slim_ctx* ctx, const void* q, const slim_cache* cache,
                                   const int32_t* lengths, float* o, void* stream);
 
+/* X-cache / E-cache scheme (section "Support for non-square weight matrices", Option 2, and
+ * section "Support for encoder-decoder transformers", Option 2): the cache holds the layer
+ * inputs X (or the encoder output E, which all decoder layers may share: wrap the same
+ * storage with slim_cache_create for every layer's ctx) instead of keys.  Per head
+ *   A_i = ((x_n W_Q,i + b) W_K,i^T) X^T,   head_i = [softmax(A_i / sqrt(d_k)) X] W_V,i.
+ * No RoPE (the ctx must have rope_theta = 0); square projections (d = H*d_k) only.
+ *   slim_xcache_set_weights   W_K, W_V host row-major [d][d]; W_K is kept in float32 for the
+ *                             per-token query transform, W_V replaces W_KV in the projection
+ *   slim_xcache_decode        as slim_decode: q = x_n W_Q (+ bias) [batch][d], `cache` holds
+ *                             X rows; workspace >= slim_xcache_workspace_bytes
+ * This variant runs on the CUDA-core kernels (dense scores), not on the TMA/tcgen05 path. */
+slim_status slim_xcache_set_weights(slim_ctx* ctx, const void* W_K, const void* W_V, int host_dtype);
+size_t      slim_xcache_workspace_bytes(const slim_ctx* ctx, int batch, int t_cap);
+slim_status slim_xcache_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,
+                               float* o, void* workspace, void* stream);
+
 /* Synchronises `stream`, returns the sticky device status (SLIM_OK,
  * SLIM_ERR_CAPACITY or SLIM_ERR_TIMEOUT) and clears it.                        */
 slim_status slim_device_status(slim_ctx* ctx, void* stream);

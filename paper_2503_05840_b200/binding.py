@@ -35,6 +35,9 @@ SIGNATURES = {
     "slim_decode": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "slim_static_workspace_max": (c_size_t, []),
     "slim_decode_static_ws": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "slim_xcache_set_weights": (c_int, [c_void_p, c_void_p, c_void_p, c_int]),
+    "slim_xcache_workspace_bytes": (c_size_t, [c_void_p, c_int, c_int]),
+    "slim_xcache_decode": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "slim_device_status": (c_int, [c_void_p, c_void_p]),
     "slim_selftest_bounded_wait": (c_int, [c_void_p, c_void_p]),
     "slim_profile_enable": (c_int, [c_void_p, c_int]),
@@ -176,6 +179,21 @@ def slim_decode_static_ws(ctx: int, q, cache: int, lengths, o, stream: int = 0) 
     """slim_decode with the library's built-in scratch: for callers that must not allocate."""
     _check(lib().slim_decode_static_ws(c_void_p(ctx), _ptr(q), c_void_p(cache), _ptr(lengths), _ptr(o),
                                        c_void_p(stream)), "slim_decode_static_ws")
+
+
+def slim_xcache_set_weights(ctx: int, W_K, W_V) -> None:
+    a = np.ascontiguousarray(W_K, dtype=np.float64)
+    b = np.ascontiguousarray(W_V, dtype=np.float64)
+    _check(lib().slim_xcache_set_weights(c_void_p(ctx), _ptr(a), _ptr(b), SLIM_HOST_F64), "slim_xcache_set_weights")
+
+
+def slim_xcache_workspace_bytes(ctx: int, batch: int, t_cap: int) -> int:
+    return lib().slim_xcache_workspace_bytes(c_void_p(ctx), batch, t_cap)
+
+
+def slim_xcache_decode(ctx: int, q, cache: int, lengths, o, workspace, stream: int = 0) -> None:
+    _check(lib().slim_xcache_decode(c_void_p(ctx), _ptr(q), c_void_p(cache), _ptr(lengths), _ptr(o), _ptr(workspace),
+                                    c_void_p(stream)), "slim_xcache_decode")
 
 
 def slim_device_status(ctx: int, stream: int = 0) -> int:

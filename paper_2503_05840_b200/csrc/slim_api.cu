@@ -201,6 +201,7 @@ void slim_destroy(slim_ctx* ctx) {
   cudaFree(ctx->rope_base);
   cudaFree(ctx->status);
   cudaFree(ctx->any_flag);
+  cudaFree(ctx->xc_wk);
   for (int i = 0; i < 3; ++i)
     if (ctx->prof_ev[i]) cudaEventDestroy(ctx->prof_ev[i]);
   delete ctx;
@@ -287,6 +288,23 @@ slim_status slim_set_weights_nonsquare(slim_ctx* ctx, const void* W_K, const voi
   return st;
 }
 
+slim_status slim_xcache_set_weights(slim_ctx* ctx, const void* W_K, const void* W_V, int host_dtype) {
+  if (!ctx || !W_K || !W_V || (host_dtype != SLIM_HOST_F32 && host_dtype != SLIM_HOST_F64)) return SLIM_ERR_INVALID_ARG;
+  if (ctx->rope_theta != 0.0) return SLIM_ERR_UNSUPPORTED;          // the scheme has no place for RoPE
+  const size_t nn = (size_t)ctx->d * ctx->d;
+  std::vector<float> wk(nn);
+  if (host_dtype == SLIM_HOST_F64) { const double* s = static_cast<const double*>(W_K); for (size_t i = 0; i < nn; ++i) wk[i] = (float)s[i]; }
+  else std::memcpy(wk.data(), W_K, sizeof(float) * nn);
+  if (!ctx->xc_wk && cudaMalloc(&ctx->xc_wk, sizeof(float) * nn) != cudaSuccess) { ctx->xc_wk = nullptr; cudaGetLastError(); return SLIM_ERR_OOM; }
+  if (cudaMemcpy(ctx->xc_wk, wk.data(), sizeof(float) * nn, cudaMemcpyHostToDevice) != cudaSuccess) return SLIM_ERR_CUDA;
+  return slim_set_wkv(ctx, W_V, host_dtype);                        // the projection uses W_V,i in place of W_KV,i
+}
+
+size_t slim_xcache_workspace_bytes(const slim_ctx* ctx, int batch, int t_cap) {
+  const size_t base = slim_workspace_bytes(ctx, batch, t_cap);
+  return base ? base + align256(sizeof(float) * (size_t)batch * ctx->H * ctx->d) : 0;
+}
+
 slim_status slim_set_wkv(slim_ctx* ctx, const void* W_KV, int host_dtype) {
   if (!ctx || !W_KV || (host_dtype != SLIM_HOST_F32 && host_dtype != SLIM_HOST_F64)) return SLIM_ERR_INVALID_ARG;
   double* X = nullptr;
@@ -342,12 +360,14 @@ slim_status slim_append_k(slim_ctx* ctx, slim_cache* cache, const void* k_new, c
   return SLIM_OK;
 }
 
-slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,
-                        float* o, void* workspace, void* stream) {
+namespace {
+slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths, float* o,
+                        void* workspace, void* stream, bool xcache) {
   if (!ctx || !q || !cache || !lengths || !o || !workspace || cache->ctx != ctx) return SLIM_ERR_INVALID_ARG;
   if (((uintptr_t)workspace & 255) || ((uintptr_t)q & 15) || ((uintptr_t)o & 15)) return SLIM_ERR_INVALID_ARG;
   if (!ctx->has_weights) return SLIM_ERR_NO_WEIGHTS;
-  int path = path_in_use(ctx);
+  int path = xcache ? (int)SLIM_PATH_GENERIC : path_in_use(ctx);
+  if (xcache && !ctx->xc_wk) return SLIM_ERR_NO_WEIGHTS;
   if (path < 0) return SLIM_ERR_UNSUPPORTED;
   if (path == SLIM_PATH_TC && !cache->has_tmap) {
     if (ctx->path_req == SLIM_PATH_TC) return SLIM_ERR_UNSUPPORTED;
@@ -377,6 +397,9 @@ slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   if (path == SLIM_PATH_TC) {
     e = slim_launch_tc(ctx, cache, p, st);
     if (e == cudaSuccess) e = slim_launch_exact_flagged(ctx, p, st);
+  } else if (xcache) {
+    e = slim_launch_generic_xcache(ctx, p, reinterpret_cast<float*>(ws + L.scores), ctx->xc_wk,
+                                   reinterpret_cast<float*>(ws + L.total), st);
   } else {
     e = slim_launch_generic(ctx, p, reinterpret_cast<float*>(ws + L.scores), st);
   }
@@ -393,6 +416,17 @@ slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   if (ctx->prof_on) { cudaEventRecord(ctx->prof_ev[2], st); ctx->prof_valid = 1; }
   if (e != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
   return SLIM_OK;
+}
+}  // namespace
+
+slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,
+                        float* o, void* workspace, void* stream) {
+  return decode_impl(ctx, q, cache, lengths, o, workspace, stream, false);
+}
+
+slim_status slim_xcache_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,
+                               float* o, void* workspace, void* stream) {
+  return decode_impl(ctx, q, cache, lengths, o, workspace, stream, true);
 }
 
 size_t slim_static_workspace_max(void) { return SLIM_STATIC_WS_BYTES; }

@@ -385,6 +385,86 @@ slim_accum_kernel(SlimDecodeParams p, const float* __restrict__ scores) {
   }
 }
 
+
+// ---------------------------------------------------------------------------
+// X-cache / E-cache scheme (non-square Option 2, encoder-decoder Option 2): the cache
+// holds the layer inputs X and the softmax arguments come from a dense d-wide query per
+// head, A_i = ((x_n W_Q,i + b) W_K,i^T) X^T.
+// ---------------------------------------------------------------------------
+// q~[b][h][j] = qscale * sum_c q[b][h d_k + c] W_K[j][h d_k + c]      (one warp per j)
+template <typename KT>
+__global__ void __launch_bounds__(GEN_THREADS)
+slim_xq_kernel(SlimDecodeParams p, const float* __restrict__ W_K, float* __restrict__ qt) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* s_q = reinterpret_cast<float*>(smem_raw);                   // [d_k]
+  const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int d = p.d, dk = p.d_k;
+  const KT* Q = reinterpret_cast<const KT*>(p.q) + (size_t)b * d + h * dk;
+  for (int c = tid; c < dk; c += GEN_THREADS) s_q[c] = ld_k(Q + c) * p.qscale;
+  __syncthreads();
+  for (int j = wid; j < d; j += GEN_THREADS / 32) {
+    const float* w = W_K + (size_t)j * d + h * dk;
+    float a = 0.f;
+    for (int c = lane; c < dk; c += 32) a = fmaf(s_q[c], __ldg(w + c), a);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if (lane == 0) qt[((size_t)b * p.H + h) * d + j] = a;
+  }
+}
+
+// scores[b][h][t] = q~[b][h][:] . X[b][t][:]   CTA = (32-row tile, sequence); thread = (row, head group)
+constexpr int XS_ROWS = 32, XS_DC = 128;
+template <typename KT>
+__global__ void __launch_bounds__(GEN_THREADS)
+slim_xscores_kernel(SlimDecodeParams p, const float* __restrict__ qt, float* __restrict__ scores) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* s_x = reinterpret_cast<float*>(smem_raw);                   // [32][XS_DC + 1]
+  float* s_qt = s_x + XS_ROWS * (XS_DC + 1) + 3;                     // [H][XS_DC], 16-byte aligned below
+  s_qt = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(s_qt) + 15) & ~(uintptr_t)15);
+  const int b = blockIdx.y, t0 = blockIdx.x * XS_ROWS, tid = threadIdx.x, tx = tid & 31, ty = tid >> 5;
+  const int d = p.d, H = p.H;
+  const int len = min(max(p.lengths[b], 0), p.t_cap);
+  if (t0 >= len) return;
+  const KT* __restrict__ X = reinterpret_cast<const KT*>(p.k) + ((size_t)b * p.t_cap + t0) * d;
+  const float* __restrict__ Qb = qt + (size_t)b * H * d;
+  float acc[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+  for (int j0 = 0; j0 < d; j0 += XS_DC) {
+    const int dc = min(XS_DC, d - j0);
+    for (int e = tid; e < XS_ROWS * XS_DC; e += GEN_THREADS) {
+      const int r = e / XS_DC, k = e % XS_DC;
+      s_x[r * (XS_DC + 1) + k] = (k < dc && t0 + r < len) ? ld_k(X + (size_t)r * d + j0 + k) : 0.f;   // rows past the end may hold anything
+    }
+    for (int e = tid; e < H * XS_DC; e += GEN_THREADS) {
+      const int hh = e / XS_DC, k = e % XS_DC;
+      s_qt[e] = k < dc ? __ldg(Qb + (size_t)hh * d + j0 + k) : 0.f;
+    }
+    __syncthreads();
+    const float* xr = s_x + tx * (XS_DC + 1);
+    for (int k = 0; k < XS_DC; k += 4) {
+      const float x0 = xr[k], x1 = xr[k + 1], x2 = xr[k + 2], x3 = xr[k + 3];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int hh = ty + 8 * i;
+        if (hh < H) {
+          const float4 q4 = *reinterpret_cast<const float4*>(s_qt + hh * XS_DC + k);
+          acc[i] = fmaf(x0, q4.x, acc[i]); acc[i] = fmaf(x1, q4.y, acc[i]);
+          acc[i] = fmaf(x2, q4.z, acc[i]); acc[i] = fmaf(x3, q4.w, acc[i]);
+        }
+      }
+    }
+    __syncthreads();
+  }
+  if (t0 + tx < len) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int hh = ty + 8 * i;
+      if (hh < H) scores[((size_t)b * H + hh) * p.t_cap + t0 + tx] = acc[i];
+    }
+  }
+}
+
 template <typename KT, int HP, int COLS>
 cudaError_t launch_exact(const SlimDecodeParams& p, int only_flagged, cudaStream_t st) {
   const int dsplit = (p.d + GEN_THREADS * COLS - 1) / (GEN_THREADS * COLS);
@@ -399,9 +479,21 @@ cudaError_t launch_exact(const SlimDecodeParams& p, int only_flagged, cudaStream
 }
 
 template <typename KT>
-cudaError_t launch_two_pass(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, cudaStream_t st) {
+cudaError_t launch_two_pass(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, cudaStream_t st,
+                            const float* xc_wk = nullptr, float* xc_qt = nullptr) {
   constexpr int VEC = Vec<KT>::N;
-  {
+  if (xc_wk) {        // X-cache scheme: dense per-head queries instead of the per-head key slices
+    slim_xq_kernel<KT><<<dim3(p.H, p.batch), GEN_THREADS, sizeof(float) * p.d_k, st>>>(p, xc_wk, xc_qt);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const size_t smem = sizeof(float) * (XS_ROWS * (XS_DC + 1) + 8 + (size_t)p.H * XS_DC);
+    auto kern = slim_xscores_kernel<KT>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<dim3((p.t_cap + XS_ROWS - 1) / XS_ROWS, p.batch), GEN_THREADS, smem, st>>>(p, xc_qt, scores);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  } else {
     const size_t smem = sizeof(float) * (p.d + SLIM_TT * (p.d / (2 * VEC))) + sizeof(int) * (p.batch + 1);
     auto kern = slim_scores_kernel<KT>;
     if (smem > 48 * 1024) {
@@ -428,6 +520,12 @@ cudaError_t launch_two_pass(const slim_ctx* ctx, const SlimDecodeParams& p, floa
 }
 
 }  // namespace
+
+cudaError_t slim_launch_generic_xcache(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, const float* W_K,
+                                       float* qt, cudaStream_t st) {
+  return p.dtype == SLIM_BF16 ? launch_two_pass<__nv_bfloat16>(ctx, p, scores, st, W_K, qt)
+                              : launch_two_pass<float>(ctx, p, scores, st, W_K, qt);
+}
 
 int slim_generic_dsplit(const slim_ctx* ctx) { return (ctx->d + GEN_THREADS - 1) / GEN_THREADS; }
 

@@ -59,6 +59,7 @@ struct slim_ctx {
   int prof_on, prof_valid;
   cudaEvent_t prof_ev[3];
   int proj_ok;                   // tensor-core combine + projection usable for this shape
+  float* xc_wk;                  // X-cache scheme: device fp32 W_K [d][d] (NULL until slim_xcache_set_weights)
   int* any_flag;                 // device: 1 while some unit of the current decode is flagged for the exact redo
   alignas(64) unsigned char wmap[128];   // CUtensorMap over W_KV for the projection kernel
 };
@@ -75,6 +76,8 @@ struct slim_cache {
 int  slim_generic_workers(const slim_ctx* ctx);
 int  slim_generic_dsplit(const slim_ctx* ctx);
 cudaError_t slim_launch_generic(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, cudaStream_t st);
+cudaError_t slim_launch_generic_xcache(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, const float* W_K,
+                                       float* qt, cudaStream_t st);
 cudaError_t slim_launch_exact_flagged(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st);
 cudaError_t slim_launch_tail(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st);
 cudaError_t slim_launch_append(const slim_ctx* ctx, const slim_cache* c, const void* k_new,
