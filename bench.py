@@ -42,6 +42,8 @@ def parse():
     ap.add_argument("--path", default="auto", choices=["auto", "generic", "tc"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--variant", default="kcache", choices=["kcache", "xcache"],
+                    help="xcache: the X/E-cache scheme, one cache shared by all layers (configs without RoPE)")
     return ap.parse_args()
 
 
@@ -191,10 +193,66 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_xcache(args):
+    """X/E-cache scheme on a config without RoPE: one cache of layer inputs shared by all layers,
+    per layer slim_xcache_decode.  Reported beside the K-cache numbers; not the default line."""
+    import torch
+    from paper_2503_05840_b200 import binding as B
+    from paper_2503_05840_b200 import build as _build
+    from paper_2503_05840_b200 import synth
+    _build.build()
+    cfg = synth.CONFIGS[args.config]
+    assert cfg.rope_theta == 0.0, "the X-cache scheme has no RoPE: use --config 0 or 3"
+    layers_n = args.layers or cfg.layers
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    g = torch.Generator(device=dev); g.manual_seed(synth.layer_seed(args.config, 0))
+    X = torch.randn((cfg.batch, cfg.context, cfg.d), generator=g, device=dev, dtype=torch.float32).to(tdt)
+    lengths = torch.full((cfg.batch,), cfg.context, dtype=torch.int32, device=dev)
+    q = torch.randn((layers_n, cfg.batch, cfg.d), generator=g, device=dev, dtype=torch.float32).to(tdt)
+    o = torch.empty((layers_n, cfg.batch, cfg.d), dtype=torch.float32, device=dev)
+    ctxs, caches = [], []
+    ws = None
+    for li in range(layers_n):
+        ctx = B.slim_create(cfg.d, cfg.H, cfg.d_k, 0.0, B.SLIM_BF16 if cfg.dtype == "bf16" else B.SLIM_F32)
+        W_Q, W_K, W_V, _, _ = synth.make_weights_torch(cfg.d, synth.layer_seed(args.config, li), dev)
+        B.slim_xcache_set_weights(ctx, W_K.cpu().numpy(), W_V.cpu().numpy())
+        ctxs.append(ctx); caches.append(B.slim_cache_create(ctx, X, cfg.batch, cfg.context))
+        if ws is None:
+            ws = torch.empty(B.slim_xcache_workspace_bytes(ctx, cfg.batch, cfg.context), dtype=torch.uint8, device=dev)
+    st = torch.cuda.current_stream().cuda_stream
+
+    def step():
+        for li in range(layers_n):
+            B.slim_xcache_decode(ctxs[li], q[li], caches[li], lengths, o[li], ws, st)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record(); torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    cache_bytes = X.numel() * X.element_size()
+    print(json.dumps({"metric": "decode_attention_tokens_per_s", "variant": "xcache", "value": cfg.batch / (ms * 1e-3),
+                      "unit": "tokens/s", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+                      "higher_is_better": True, "dtype": cfg.dtype, "data": "synthetic",
+                      "config": {"workload": f"config{args.config}:{cfg.name} (X/E-cache scheme)", "layers": layers_n,
+                                 "batch": cfg.batch, "context": cfg.context, "d": cfg.d, "H": cfg.H, "d_k": cfg.d_k},
+                      "cache_bytes_shared_by_all_layers": cache_bytes,
+                      "kcache_bytes_equivalent": cache_bytes * layers_n,
+                      "device_status": int(B.slim_device_status(ctxs[0], st))}))
+
+
 def main():
     args = parse()
     if args.impl == "reference":
         return run_reference(args)
+    if args.variant == "xcache":
+        return run_xcache(args)
 
     import torch
     from paper_2503_05840_b200 import binding as B

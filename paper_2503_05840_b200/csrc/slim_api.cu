@@ -302,7 +302,7 @@ slim_status slim_xcache_set_weights(slim_ctx* ctx, const void* W_K, const void* 
 
 size_t slim_xcache_workspace_bytes(const slim_ctx* ctx, int batch, int t_cap) {
   const size_t base = slim_workspace_bytes(ctx, batch, t_cap);
-  return base ? base + align256(sizeof(float) * (size_t)batch * ctx->H * ctx->d) : 0;
+  return base ? base + align256(sizeof(float) * (size_t)batch * ctx->H * ctx->d) + align256(slim_xscores_qt_bytes(ctx->d, batch)) : 0;
 }
 
 slim_status slim_set_wkv(slim_ctx* ctx, const void* W_KV, int host_dtype) {
@@ -344,6 +344,11 @@ slim_status slim_cache_create(slim_ctx* ctx, slim_cache** out, void* k_storage, 
     if (slim_tc_make_tmap(ctx, c) == cudaSuccess) c->has_tmap = 1;
     else cudaGetLastError();
   }
+  c->has_xmap = 0;
+  if (ctx->proj_ok && slim_xscores_tc_ok(ctx)) {
+    if (slim_xscores_make_tmap(ctx, c) == cudaSuccess) c->has_xmap = 1;
+    else cudaGetLastError();
+  }
   *out = c;
   return SLIM_OK;
 }
@@ -366,7 +371,7 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   if (!ctx || !q || !cache || !lengths || !o || !workspace || cache->ctx != ctx) return SLIM_ERR_INVALID_ARG;
   if (((uintptr_t)workspace & 255) || ((uintptr_t)q & 15) || ((uintptr_t)o & 15)) return SLIM_ERR_INVALID_ARG;
   if (!ctx->has_weights) return SLIM_ERR_NO_WEIGHTS;
-  int path = xcache ? (int)SLIM_PATH_GENERIC : path_in_use(ctx);
+  int path = path_in_use(ctx);
   if (xcache && !ctx->xc_wk) return SLIM_ERR_NO_WEIGHTS;
   if (path < 0) return SLIM_ERR_UNSUPPORTED;
   if (path == SLIM_PATH_TC && !cache->has_tmap) {
@@ -391,17 +396,33 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   p.unit_flags = reinterpret_cast<int*>(ws + L.flags);
   p.u = reinterpret_cast<float*>(ws + L.o_part);
   p.o = o; p.status = ctx->status; p.any_flag = ctx->any_flag;
+  p.ext_scores = nullptr;
   cudaStream_t st = (cudaStream_t)stream;
   if (ctx->prof_on) cudaEventRecord(ctx->prof_ev[0], st);
   cudaError_t e;
-  if (path == SLIM_PATH_TC) {
+  float* scores = reinterpret_cast<float*>(ws + L.scores);
+  if (xcache) {
+    // dense scores first; then P.X on the tensor cores where the shape allows it (an argument that
+    // overflows its reference exponent triggers the CUDA-core accumulation as the exact redo)
+    if (cache->has_xmap && !getenv("SLIM_XSCORES_CUDA"))
+      e = slim_launch_xscores_tc(ctx, cache, p, ctx->xc_wk,
+                                 reinterpret_cast<unsigned char*>(ws + L.total + align256(sizeof(float) * (size_t)p.batch * p.H * p.d)), scores, st);
+    else
+      e = slim_launch_xcache_scores(ctx, p, scores, ctx->xc_wk, reinterpret_cast<float*>(ws + L.total), st);
+    if (e == cudaSuccess) {
+      if (path == SLIM_PATH_TC) {
+        p.ext_scores = scores;
+        e = slim_launch_tc(ctx, cache, p, st);
+        if (e == cudaSuccess) e = slim_launch_accum(ctx, p, scores, 0, st);
+      } else {
+        e = slim_launch_accum(ctx, p, scores, 1, st);
+      }
+    }
+  } else if (path == SLIM_PATH_TC) {
     e = slim_launch_tc(ctx, cache, p, st);
     if (e == cudaSuccess) e = slim_launch_exact_flagged(ctx, p, st);
-  } else if (xcache) {
-    e = slim_launch_generic_xcache(ctx, p, reinterpret_cast<float*>(ws + L.scores), ctx->xc_wk,
-                                   reinterpret_cast<float*>(ws + L.total), st);
   } else {
-    e = slim_launch_generic(ctx, p, reinterpret_cast<float*>(ws + L.scores), st);
+    e = slim_launch_generic(ctx, p, scores, st);
   }
   if (ctx->prof_on) cudaEventRecord(ctx->prof_ev[1], st);
   if (e == cudaSuccess) {

@@ -303,7 +303,7 @@ slim_scores_kernel(SlimDecodeParams p, float* __restrict__ scores) {
 // ---------------------------------------------------------------------------
 template <typename KT, int HP>
 __global__ void __launch_bounds__(GEN_THREADS, 2)
-slim_accum_kernel(SlimDecodeParams p, const float* __restrict__ scores) {
+slim_accum_kernel(SlimDecodeParams p, const float* __restrict__ scores, int only_if_flagged) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* s_P = reinterpret_cast<float*>(smem_raw);                  // [HP][TT]
   float* s_alpha = s_P + HP * SLIM_TT;                              // [HP]
@@ -312,6 +312,10 @@ slim_accum_kernel(SlimDecodeParams p, const float* __restrict__ scores) {
   int* s_prefix = reinterpret_cast<int*>(s_l + HP);                 // [batch+1]
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int w = blockIdx.y;
+  if (only_if_flagged) {
+    slim_pdl_wait();
+    if (*p.any_flag == 0) return;                     // nothing overflowed its reference exponent
+  }
   const int col = blockIdx.x * GEN_THREADS + tid;
   const KT* __restrict__ Kc = reinterpret_cast<const KT*>(p.k);
   const int d = p.d, H = p.H;
@@ -479,52 +483,59 @@ cudaError_t launch_exact(const SlimDecodeParams& p, int only_flagged, cudaStream
 }
 
 template <typename KT>
-cudaError_t launch_two_pass(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, cudaStream_t st,
-                            const float* xc_wk = nullptr, float* xc_qt = nullptr) {
+cudaError_t launch_scores(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, cudaStream_t st) {
   constexpr int VEC = Vec<KT>::N;
-  if (xc_wk) {        // X-cache scheme: dense per-head queries instead of the per-head key slices
-    slim_xq_kernel<KT><<<dim3(p.H, p.batch), GEN_THREADS, sizeof(float) * p.d_k, st>>>(p, xc_wk, xc_qt);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    const size_t smem = sizeof(float) * (XS_ROWS * (XS_DC + 1) + 8 + (size_t)p.H * XS_DC);
-    auto kern = slim_xscores_kernel<KT>;
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    kern<<<dim3((p.t_cap + XS_ROWS - 1) / XS_ROWS, p.batch), GEN_THREADS, smem, st>>>(p, xc_qt, scores);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-  } else {
-    const size_t smem = sizeof(float) * (p.d + SLIM_TT * (p.d / (2 * VEC))) + sizeof(int) * (p.batch + 1);
-    auto kern = slim_scores_kernel<KT>;
-    if (smem > 48 * 1024) {
-      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e != cudaSuccess) return e;
-    }
-    kern<<<4 * ctx->num_sms, GEN_THREADS, smem, st>>>(p, scores);
-    cudaError_t e = cudaGetLastError();
+  const size_t smem = sizeof(float) * (p.d + SLIM_TT * (p.d / (2 * VEC))) + sizeof(int) * (p.batch + 1);
+  auto kern = slim_scores_kernel<KT>;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
+  kern<<<4 * ctx->num_sms, GEN_THREADS, smem, st>>>(p, scores);
+  return cudaGetLastError();
+}
+
+template <typename KT>
+cudaError_t launch_xscores(const SlimDecodeParams& p, float* scores, const float* xc_wk, float* xc_qt, cudaStream_t st) {
+  slim_xq_kernel<KT><<<dim3(p.H, p.batch), GEN_THREADS, sizeof(float) * p.d_k, st>>>(p, xc_wk, xc_qt);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const size_t smem = sizeof(float) * (XS_ROWS * (XS_DC + 1) + 8 + (size_t)p.H * XS_DC);
+  auto kern = slim_xscores_kernel<KT>;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  kern<<<dim3((p.t_cap + XS_ROWS - 1) / XS_ROWS, p.batch), GEN_THREADS, smem, st>>>(p, xc_qt, scores);
+  return cudaGetLastError();
+}
+
+template <typename KT>
+cudaError_t launch_accum(const SlimDecodeParams& p, const float* scores, int only_if_flagged, cudaStream_t st) {
   const int dsplit = (p.d + GEN_THREADS - 1) / GEN_THREADS;
   dim3 grid(dsplit, p.workers);
   if (p.H <= 8) {
     const size_t smem = sizeof(float) * (8 * SLIM_TT + 3 * 8) + sizeof(int) * (p.batch + 1);
-    slim_accum_kernel<KT, 8><<<grid, GEN_THREADS, smem, st>>>(p, scores);
+    slim_accum_kernel<KT, 8><<<grid, GEN_THREADS, smem, st>>>(p, scores, only_if_flagged);
   } else if (p.H <= 32) {
     const size_t smem = sizeof(float) * (32 * SLIM_TT + 3 * 32) + sizeof(int) * (p.batch + 1);
-    slim_accum_kernel<KT, 32><<<grid, GEN_THREADS, smem, st>>>(p, scores);
+    slim_accum_kernel<KT, 32><<<grid, GEN_THREADS, smem, st>>>(p, scores, only_if_flagged);
   } else {
     const size_t smem = sizeof(float) * (64 * SLIM_TT + 3 * 64) + sizeof(int) * (p.batch + 1);
-    slim_accum_kernel<KT, 64><<<grid, GEN_THREADS, smem, st>>>(p, scores);
+    slim_accum_kernel<KT, 64><<<grid, GEN_THREADS, smem, st>>>(p, scores, only_if_flagged);
   }
   return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t slim_launch_generic_xcache(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, const float* W_K,
-                                       float* qt, cudaStream_t st) {
-  return p.dtype == SLIM_BF16 ? launch_two_pass<__nv_bfloat16>(ctx, p, scores, st, W_K, qt)
-                              : launch_two_pass<float>(ctx, p, scores, st, W_K, qt);
+cudaError_t slim_launch_xcache_scores(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, const float* W_K,
+                                      float* qt, cudaStream_t st) {
+  return p.dtype == SLIM_BF16 ? launch_xscores<__nv_bfloat16>(p, scores, W_K, qt, st)
+                              : launch_xscores<float>(p, scores, W_K, qt, st);
+}
+
+cudaError_t slim_launch_accum(const slim_ctx* ctx, const SlimDecodeParams& p, const float* scores, int whole, cudaStream_t st) {
+  return p.dtype == SLIM_BF16 ? launch_accum<__nv_bfloat16>(p, scores, whole ? 0 : 1, st)
+                              : launch_accum<float>(p, scores, whole ? 0 : 1, st);
 }
 
 int slim_generic_dsplit(const slim_ctx* ctx) { return (ctx->d + GEN_THREADS - 1) / GEN_THREADS; }
@@ -538,8 +549,9 @@ int slim_generic_workers(const slim_ctx* ctx) {
 }
 
 cudaError_t slim_launch_generic(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, cudaStream_t st) {
-  return p.dtype == SLIM_BF16 ? launch_two_pass<__nv_bfloat16>(ctx, p, scores, st)
-                              : launch_two_pass<float>(ctx, p, scores, st);
+  cudaError_t e = p.dtype == SLIM_BF16 ? launch_scores<__nv_bfloat16>(ctx, p, scores, st) : launch_scores<float>(ctx, p, scores, st);
+  if (e != cudaSuccess) return e;
+  return slim_launch_accum(ctx, p, scores, 1, st);
 }
 
 // Redo exactly the units whose flag is set (schedule taken from p.workers / p.min_tiles).

@@ -39,6 +39,7 @@ struct SlimDecodeParams {
   float* o;                      // [batch][d]
   int* status;                   // sticky device status word
   int* any_flag;                 // set to 1 by a kernel that flags a unit
+  const float* ext_scores;       // X-cache scheme: precomputed softmax arguments [batch][H][t_cap] (else NULL)
 };
 
 struct slim_ctx {
@@ -70,14 +71,20 @@ struct slim_cache {
   int batch, t_cap;
   alignas(64) unsigned char tmap[128];   // CUtensorMap for the tensor-core path
   int has_tmap;
+  alignas(64) unsigned char xmap[128];   // CUtensorMap for the dense X-cache scores (rows x 64 columns)
+  int has_xmap;
 };
 
 // ---- launchers implemented in the kernel translation units -----------------
 int  slim_generic_workers(const slim_ctx* ctx);
 int  slim_generic_dsplit(const slim_ctx* ctx);
 cudaError_t slim_launch_generic(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, cudaStream_t st);
-cudaError_t slim_launch_generic_xcache(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, const float* W_K,
-                                       float* qt, cudaStream_t st);
+// X-cache scheme: dense query transform + dense scores into `scores`; then either the CUDA-core
+// accumulation (whole = 1) or, after the tensor-core kernel, the same accumulation as an exact
+// redo that runs only if a unit was flagged (whole = 0)
+cudaError_t slim_launch_xcache_scores(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, const float* W_K,
+                                      float* qt, cudaStream_t st);
+cudaError_t slim_launch_accum(const slim_ctx* ctx, const SlimDecodeParams& p, const float* scores, int whole, cudaStream_t st);
 cudaError_t slim_launch_exact_flagged(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st);
 cudaError_t slim_launch_tail(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st);
 cudaError_t slim_launch_append(const slim_ctx* ctx, const slim_cache* c, const void* k_new,
@@ -135,3 +142,10 @@ inline cudaError_t slim_launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block
   return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 #endif
+
+// X-cache scheme: dense scores on the tensor cores (slim_xscores.cu)
+int    slim_xscores_tc_ok(const slim_ctx* ctx);
+size_t slim_xscores_qt_bytes(int d, int batch);
+cudaError_t slim_xscores_make_tmap(const slim_ctx* ctx, slim_cache* c);
+cudaError_t slim_launch_xscores_tc(const slim_ctx* ctx, const slim_cache* c, const SlimDecodeParams& p, const float* W_K,
+                                   unsigned char* qt_tiled, float* scores, cudaStream_t st);

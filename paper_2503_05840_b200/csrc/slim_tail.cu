@@ -33,6 +33,7 @@ __global__ void __launch_bounds__(256) slim_tail1_kernel(SlimDecodeParams p, int
   slim_pdl_wait();
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nwarp = blockDim.x >> 5;
   const int h = blockIdx.x, js = blockIdx.y;
+  if (h == 0 && js == 0 && tid == 0) *p.any_flag = 0;       // the redo kernel before this one has consumed it
   const int d = p.d, H = p.H, dk = p.d_k;
   const int j0 = js * JR, jn = min(JR, d - j0);
   const int BT = bg_count * BPT;

@@ -81,7 +81,9 @@ __host__ __device__ constexpr int tc_threads(int dk, int rt) {
 }
 
 // ------------------------------------------------------------------ the kernel
-template <int DK, bool ROPE, int RT>
+// EXT: the softmax arguments are read from p.ext_scores (X-cache scheme) instead of being
+// formed from the staged rows; the rest of the pipeline is the same.
+template <int DK, bool ROPE, int RT, bool EXT>
 __global__ void __launch_bounds__(tc_threads(DK, RT), 1)
 slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams p, const TcGeom g) {
   constexpr int PAIRS = DK / 2;                   // rotation pairs (j, j + DK/2) per head
@@ -241,7 +243,13 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
                 for (int e = lane; e < (SLIM_TT - nz) * 8; e += 32)
                   sts128_zero(kbase + (uint32_t)c64 * 2048u + (uint32_t)(nz + (e >> 3)) * 128u + (uint32_t)(e & 7) * 16u);
             }
-            // ---- a4: softmax arguments: this thread's partial sums for its RT rows ----
+            // ---- a4: softmax arguments ----
+            if (EXT) {
+              // X-cache scheme: the arguments were computed by the dense-score kernel (log2 domain)
+              if (head_valid && t0 + my_row < len)
+                sv = __ldg(p.ext_scores + ((size_t)b * p.H + my_n) * p.t_cap + t0 + my_row);
+            } else {
+            // this thread's partial sums for its RT rows
             float v[RT];
 #pragma unroll
             for (int i = 0; i < RT; ++i) v[i] = 0.f;
@@ -289,6 +297,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
                 }
               }
               sv = v[0];
+            }
             }
             const bool valid = head_valid && (t0 + my_row < len);
             // ---- a5: probabilities against the fixed reference of this unit ----
@@ -496,14 +505,26 @@ int tc_rows_per_thread(int d_k) {
   return want == 4 ? 4 : 8;
 }
 
-tc_kernel_t pick_kernel(int d_k, bool rope, int rt) {
+tc_kernel_t pick_kernel(int d_k, bool rope, int rt, bool ext = false) {
+  if (ext) {                                   // X-cache scheme: no RoPE
+    if (rope) return nullptr;
+    switch (d_k * 16 + rt) {
+      case 64 * 16 + 2: return slim_tc_kernel<64, false, 2, true>;
+      case 64 * 16 + 4: return slim_tc_kernel<64, false, 4, true>;
+      case 96 * 16 + 4: return slim_tc_kernel<96, false, 4, true>;
+      case 96 * 16 + 8: return slim_tc_kernel<96, false, 8, true>;
+      case 128 * 16 + 4: return slim_tc_kernel<128, false, 4, true>;
+      case 128 * 16 + 8: return slim_tc_kernel<128, false, 8, true>;
+      default: return nullptr;
+    }
+  }
   switch (d_k * 16 + rt) {
-    case 64 * 16 + 2: return rope ? slim_tc_kernel<64, true, 2> : slim_tc_kernel<64, false, 2>;
-    case 64 * 16 + 4: return rope ? slim_tc_kernel<64, true, 4> : slim_tc_kernel<64, false, 4>;
-    case 96 * 16 + 4: return rope ? slim_tc_kernel<96, true, 4> : slim_tc_kernel<96, false, 4>;
-    case 96 * 16 + 8: return rope ? slim_tc_kernel<96, true, 8> : slim_tc_kernel<96, false, 8>;
-    case 128 * 16 + 4: return rope ? slim_tc_kernel<128, true, 4> : slim_tc_kernel<128, false, 4>;
-    case 128 * 16 + 8: return rope ? slim_tc_kernel<128, true, 8> : slim_tc_kernel<128, false, 8>;
+    case 64 * 16 + 2: return rope ? slim_tc_kernel<64, true, 2, false> : slim_tc_kernel<64, false, 2, false>;
+    case 64 * 16 + 4: return rope ? slim_tc_kernel<64, true, 4, false> : slim_tc_kernel<64, false, 4, false>;
+    case 96 * 16 + 4: return rope ? slim_tc_kernel<96, true, 4, false> : slim_tc_kernel<96, false, 4, false>;
+    case 96 * 16 + 8: return rope ? slim_tc_kernel<96, true, 8, false> : slim_tc_kernel<96, false, 8, false>;
+    case 128 * 16 + 4: return rope ? slim_tc_kernel<128, true, 4, false> : slim_tc_kernel<128, false, 4, false>;
+    case 128 * 16 + 8: return rope ? slim_tc_kernel<128, true, 8, false> : slim_tc_kernel<128, false, 8, false>;
     default: return nullptr;
   }
 }
@@ -604,8 +625,13 @@ cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c) {
 
 cudaError_t slim_launch_tc(const slim_ctx* ctx, const slim_cache* c, const SlimDecodeParams& p, cudaStream_t st) {
   const int rt = tc_rows_per_thread(ctx->d_k);
-  tc_kernel_t kern = pick_kernel(ctx->d_k, ctx->rope_theta != 0.0, rt);
+  const bool ext = p.ext_scores != nullptr;
+  tc_kernel_t kern = pick_kernel(ctx->d_k, ctx->rope_theta != 0.0, rt, ext);
   if (!kern || !c->has_tmap) return cudaErrorNotSupported;
+  if (ext) {
+    cudaError_t ea = cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_LIMIT);
+    if (ea != cudaSuccess) return ea;
+  }
   const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, rt, TC_SMEM_LIMIT);
   const size_t smem = tc_smem_bytes(g, p.batch);
   cudaLaunchConfig_t cfg = {};
