@@ -166,7 +166,10 @@ slim_status slim_decode_static_ws(slim_ctx* ctx, const void* q, const slim_cache
  *                             per-token query transform, W_V replaces W_KV in the projection
  *   slim_xcache_decode        as slim_decode: q = x_n W_Q (+ bias) [batch][d], `cache` holds
  *                             X rows; workspace >= slim_xcache_workspace_bytes
- * This variant runs on the CUDA-core kernels (dense scores), not on the TMA/tcgen05 path. */
+ * bf16 caches with d % 64 == 0 and H <= 32 run on the tensor cores (dense scores: cache rows
+ * as a K-major TMA operand against bf16 hi/lo query tiles; weighted sum and projection: the
+ * kernels of slim_decode); other shapes use the CUDA-core kernels.  The cache is read twice
+ * per layer (scores, then the weighted sum).                                            */
 slim_status slim_xcache_set_weights(slim_ctx* ctx, const void* W_K, const void* W_V, int host_dtype);
 size_t      slim_xcache_workspace_bytes(const slim_ctx* ctx, int batch, int t_cap);
 slim_status slim_xcache_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,

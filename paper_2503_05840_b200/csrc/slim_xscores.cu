@@ -33,29 +33,42 @@ __host__ __device__ constexpr uint32_t idesc_kk(uint32_t n) {
 }
 
 // q~[b][h][j] = qscale sum_c q[b][h d_k + c] W_K[j][h d_k + c], written as bf16 hi / lo rows h and 32 + h
-// of the [64 x 16] tile of k-step j / 16 (one warp per j).
+// of the [64 x 16] tile of k-step j / 16.  CTA = (head, 64 rows j of W_K): the weight tile is read once
+// and used for every sequence of the batch.
+constexpr int XQ_J = 64, XQ_B = 16;
 __global__ void __launch_bounds__(256)
 slim_xq_tiled_kernel(SlimDecodeParams p, const float* __restrict__ W_K, unsigned char* __restrict__ qt_tiled) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  float* s_q = reinterpret_cast<float*>(smem_raw);                   // [d_k]
+  const int dk = p.d_k, d = p.d;
+  float* s_w = reinterpret_cast<float*>(smem_raw);                   // [XQ_J][dk + 1]
+  float* s_q = s_w + XQ_J * (dk + 1);                                // [XQ_B][dk]
   slim_pdl_wait();
-  const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  const int d = p.d, dk = p.d_k;
-  const __nv_bfloat16* Q = reinterpret_cast<const __nv_bfloat16*>(p.q) + (size_t)b * d + h * dk;
-  for (int c = tid; c < dk; c += 256) s_q[c] = __bfloat162float(Q[c]) * p.qscale;
-  __syncthreads();
-  unsigned char* dst = qt_tiled + (size_t)b * (d / 16) * 2048;
-  for (int j = wid; j < d; j += 8) {
-    const float* w = W_K + (size_t)j * d + h * dk;
-    float a = 0.f;
-    for (int c = lane; c < dk; c += 32) a = fmaf(s_q[c], __ldg(w + c), a);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-    if (lane == 0) {
+  const int h = blockIdx.x, j0 = blockIdx.y * XQ_J, tid = threadIdx.x;
+  for (int e = tid; e < XQ_J * dk; e += 256) {
+    const int j = e / dk, c = e % dk;
+    s_w[j * (dk + 1) + c] = (j0 + j < d) ? __ldg(W_K + (size_t)(j0 + j) * d + h * dk + c) : 0.f;
+  }
+  const int j = tid & (XQ_J - 1), bq = tid >> 6;                     // 4 sequences at a time per pass
+  for (int b0 = 0; b0 < p.batch; b0 += XQ_B) {
+    __syncthreads();
+    for (int e = tid; e < XQ_B * dk; e += 256) {
+      const int bb = e / dk, c = e % dk;
+      s_q[e] = (b0 + bb < p.batch)
+                   ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.q)[(size_t)(b0 + bb) * d + h * dk + c]) * p.qscale : 0.f;
+    }
+    __syncthreads();
+    for (int bb = bq; bb < XQ_B; bb += 4) {
+      const int b = b0 + bb;
+      if (b >= p.batch || j0 + j >= d) continue;
+      const float* w = s_w + j * (dk + 1);
+      const float* q = s_q + bb * dk;
+      float a = 0.f;
+#pragma unroll 8
+      for (int c = 0; c < dk; ++c) a = fmaf(q[c], w[c], a);
       const __nv_bfloat16 hi = __float2bfloat16_rn(a), lo = __float2bfloat16_rn(a - __bfloat162float(hi));
-      unsigned char* t = dst + (size_t)(j / 16) * 2048;
-      *reinterpret_cast<__nv_bfloat16*>(t + qt_offset(h, j & 15)) = hi;
-      *reinterpret_cast<__nv_bfloat16*>(t + qt_offset(32 + h, j & 15)) = lo;
+      unsigned char* t = qt_tiled + ((size_t)b * (d / 16) + (j0 + j) / 16) * 2048;
+      *reinterpret_cast<__nv_bfloat16*>(t + qt_offset(h, (j0 + j) & 15)) = hi;
+      *reinterpret_cast<__nv_bfloat16*>(t + qt_offset(32 + h, (j0 + j) & 15)) = lo;
     }
   }
 }
@@ -179,7 +192,7 @@ cudaError_t slim_xscores_make_tmap(const slim_ctx* ctx, slim_cache* c) {
 
 cudaError_t slim_launch_xscores_tc(const slim_ctx* ctx, const slim_cache* c, const SlimDecodeParams& p, const float* W_K,
                                    unsigned char* qt_tiled, float* scores, cudaStream_t st) {
-  slim_xq_tiled_kernel<<<dim3(p.H, p.batch), 256, sizeof(float) * p.d_k, st>>>(p, W_K, qt_tiled);
+  slim_xq_tiled_kernel<<<dim3(p.H, (p.d + XQ_J - 1) / XQ_J), 256, sizeof(float) * (XQ_J * (p.d_k + 1) + XQ_B * p.d_k), st>>>(p, W_K, qt_tiled);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   CUtensorMap map;
