@@ -40,6 +40,7 @@ def parse():
     ap.add_argument("--config", type=int, default=2, help="index into the five workload shapes")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (0 = the config's)")
     ap.add_argument("--path", default="auto", choices=["auto", "generic", "tc"])
+    ap.add_argument("--batch", type=int, default=0, help="override the batch size (0 = the config's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--variant", default="kcache", choices=["kcache", "xcache"],
@@ -202,6 +203,8 @@ def run_xcache(args):
     from paper_2503_05840_b200 import synth
     _build.build()
     cfg = synth.CONFIGS[args.config]
+    if args.batch:
+        cfg = cfg.scaled(batch=args.batch)
     assert cfg.rope_theta == 0.0, "the X-cache scheme has no RoPE: use --config 0 or 3"
     layers_n = args.layers or cfg.layers
     dev = "cuda:0"
@@ -276,6 +279,8 @@ def main():
     torch.cuda.set_device(local)
 
     cfg = synth.CONFIGS[args.config]
+    if args.batch:
+        cfg = cfg.scaled(batch=args.batch)
     layers_n = args.layers or cfg.layers
     cfg = cfg.scaled(layers=layers_n)
     path = {"auto": B.SLIM_PATH_AUTO, "generic": B.SLIM_PATH_GENERIC, "tc": B.SLIM_PATH_TC}[args.path]
