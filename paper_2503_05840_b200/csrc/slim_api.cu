@@ -186,10 +186,13 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
     const char* e = getenv("SLIM_TAIL");                 // "cuda" forces the CUDA-core tail (sweeps, tests)
     if (e && !strcmp(e, "cuda")) c->proj_ok = 0;
   }
-  c->tc_ok = prop.major == 10 ? slim_tc_shape_ok(d, H, d_k, dtype) : 0;
+  c->tc_ok = 0;
+  for (int cl = 1; cl <= 2; ++cl) {
+    c->tc_workers[cl - 1] = (prop.major == 10 && slim_tc_shape_ok(d, H, d_k, dtype, rope_theta != 0.0, cl)) ? slim_tc_workers(c, cl) : 0;
+    if (c->tc_workers[cl - 1] < 0) c->tc_workers[cl - 1] = 0;
+    if (c->tc_workers[cl - 1] > 0) c->tc_ok = 1;
+  }
   c->gen_workers = slim_generic_workers(c);
-  c->tc_workers = c->tc_ok ? slim_tc_workers(c) : 0;
-  if (c->tc_ok && c->tc_workers <= 0) c->tc_ok = 0;
   *out = c;
   return SLIM_OK;
 }
@@ -339,10 +342,13 @@ slim_status slim_cache_create(slim_ctx* ctx, slim_cache** out, void* k_storage, 
   if (st != SLIM_OK) return st;
   slim_cache* c = new (std::nothrow) slim_cache();
   if (!c) return SLIM_ERR_OOM;
-  c->ctx = ctx; c->k = k_storage; c->batch = batch; c->t_cap = t_cap; c->has_tmap = 0;
-  if (ctx->tc_ok) {
-    if (slim_tc_make_tmap(ctx, c) == cudaSuccess) c->has_tmap = 1;
-    else cudaGetLastError();
+  c->ctx = ctx; c->k = k_storage; c->batch = batch; c->t_cap = t_cap;
+  for (int cl = 1; cl <= 2; ++cl) {
+    c->has_tmap[cl - 1] = 0;
+    if (ctx->tc_workers[cl - 1] > 0) {
+      if (slim_tc_make_tmap(ctx, c, cl) == cudaSuccess) c->has_tmap[cl - 1] = 1;
+      else cudaGetLastError();
+    }
   }
   c->has_xmap = 0;
   if (ctx->proj_ok && slim_xscores_tc_ok(ctx)) {
@@ -374,7 +380,14 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   int path = path_in_use(ctx);
   if (xcache && !ctx->xc_wk) return SLIM_ERR_NO_WEIGHTS;
   if (path < 0) return SLIM_ERR_UNSUPPORTED;
-  if (path == SLIM_PATH_TC && !cache->has_tmap) {
+  // CTAs per worker: the pair when the kernel computes the scores, the lone CTA with external scores
+  int cl = 0;
+  if (path == SLIM_PATH_TC) {
+    const int pref = xcache ? 1 : 2, other = 3 - pref;
+    if (ctx->tc_workers[pref - 1] > 0 && cache->has_tmap[pref - 1]) cl = pref;
+    else if (ctx->tc_workers[other - 1] > 0 && cache->has_tmap[other - 1]) cl = other;
+  }
+  if (path == SLIM_PATH_TC && cl == 0) {
     if (ctx->path_req == SLIM_PATH_TC) return SLIM_ERR_UNSUPPORTED;
     path = SLIM_PATH_GENERIC;
   }
@@ -384,7 +397,8 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   p.d = ctx->d; p.H = ctx->H; p.d_k = ctx->d_k; p.half = ctx->d_k / 2;
   p.batch = cache->batch; p.t_cap = cache->t_cap;
   p.rope = ctx->rope_theta != 0.0; p.dtype = ctx->dtype;
-  p.workers = path == SLIM_PATH_TC ? ctx->tc_workers : ctx->gen_workers;
+  p.workers = path == SLIM_PATH_TC ? ctx->tc_workers[cl - 1] : ctx->gen_workers;
+  p.cl = cl;
   p.min_tiles = min_tiles_for(ctx);
   p.unit_cost = path == SLIM_PATH_TC ? (ctx->H + 3) / 4 : 0;   // measured: a drain costs about H/4 tiles
   p.qscale = (float)(1.4426950408889634 / std::sqrt((double)ctx->d_k));
@@ -526,7 +540,7 @@ long long slim_query(const slim_ctx* ctx, int key) {
       return 2 + (ctx->proj_ok ? 3 : 2);          // combine, projection, slice sum  |  combine+projection, slice sum
     case SLIM_Q_MAX_UNITS: return ctx->num_sms;   // + batch, known only per cache
     case SLIM_Q_NUM_SMS: return ctx->num_sms;
-    case SLIM_Q_WORKERS: return path == SLIM_PATH_TC ? ctx->tc_workers : ctx->gen_workers;
+    case SLIM_Q_WORKERS: return path == SLIM_PATH_TC ? (ctx->tc_workers[1] > 0 ? ctx->tc_workers[1] : ctx->tc_workers[0]) : ctx->gen_workers;
     default: return -1;
   }
 }

@@ -22,6 +22,7 @@ struct SlimDecodeParams {
   int rope;                      // 0 / 1
   int dtype;                     // slim_dtype
   int workers;                   // context-split workers (W)
+  int cl;                        // tensor-core path: CTAs per worker (1 or 2)
   int min_tiles;                 // a worker gets at least this many tiles if it gets any
   int unit_cost;                 // tiles of time that closing a unit costs a worker (schedule)
   float qscale;                  // log2(e) / sqrt(d_k)
@@ -54,8 +55,8 @@ struct slim_ctx {
   float2* rope_base;             // device table, grown by slim_cache_create
   int rope_base_tiles;
   int* status;                   // device status word
-  int tc_ok;                     // shape fits the tensor-core path
-  int tc_workers;                // clusters the tensor-core kernel runs
+  int tc_ok;                     // shape fits the tensor-core path with some cluster size
+  int tc_workers[2];             // workers of the tensor-core kernel with 1 / 2 CTAs per worker (0 = not usable)
   int gen_workers;
   int prof_on, prof_valid;
   cudaEvent_t prof_ev[3];
@@ -69,8 +70,8 @@ struct slim_cache {
   slim_ctx* ctx;
   void* k;
   int batch, t_cap;
-  alignas(64) unsigned char tmap[128];   // CUtensorMap for the tensor-core path
-  int has_tmap;
+  alignas(64) unsigned char tmap[2][128];   // CUtensorMaps of the tensor-core path for 1 / 2 CTAs per worker
+  int has_tmap[2];
   alignas(64) unsigned char xmap[128];   // CUtensorMap for the dense X-cache scores (rows x 64 columns)
   int has_xmap;
 };
@@ -101,9 +102,9 @@ cudaError_t slim_wkv_residual(const double* Wk, const double* X, const double* W
 cudaError_t slim_wkv_store(const double* X, int d, int H, int d_k, int dtype, void* dst);
 
 // tensor-core path (slim_tc.cu)
-int  slim_tc_shape_ok(int d, int H, int d_k, int dtype);
-int  slim_tc_workers(const slim_ctx* ctx);
-cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c);
+int  slim_tc_shape_ok(int d, int H, int d_k, int dtype, int rope, int cl);
+int  slim_tc_workers(const slim_ctx* ctx, int cl);
+cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c, int cl);
 cudaError_t slim_launch_wait_selftest(int* status, int* gave_up, cudaStream_t st);
 cudaError_t slim_launch_tc(const slim_ctx* ctx, const slim_cache* c, const SlimDecodeParams& p, cudaStream_t st);
 

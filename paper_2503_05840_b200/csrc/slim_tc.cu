@@ -31,6 +31,10 @@
 // At the end of a unit warps 0-3 read U from tensor memory and write the
 // partial (m_ref, l, U) for the log-sum-exp combine.
 //
+// Narrow shapes (d_k = 64 without RoPE, d <= 2048: the Whisper-like ones) run with one CTA per
+// worker (CL = 1): the whole key row and all heads live in one SM, the P exchange stays local and
+// twice as many workers share the context.
+//
 // Softmax reference.  m_ref of a (unit, head) is the maximum argument of the
 // unit's first tile and is never changed, so the accumulator is never rescaled.
 // 2^(s - m_ref) is exact in relative terms for any exponent below 2^127; a later
@@ -60,7 +64,8 @@ constexpr float TC_XMAX = 96.f;          // largest exponent accepted above m_re
 constexpr int TC_RESEED = 32;            // tiles between exact re-seeds of the stepped query rotation
 
 struct TcGeom {
-  int dsl;          // key columns per CTA (d / 2)
+  int cl;           // CTAs per worker
+  int dsl;          // key columns per CTA (d / cl)
   int nch;          // 128-column chunks per CTA
   int nc64;         // 64-column TMA chunks per CTA
   int hl;           // heads per CTA
@@ -75,16 +80,17 @@ struct TcGeom {
 // owns RT rows of the tile; 16 / RT row sets and JL lanes make one head.
 __host__ __device__ constexpr int tc_jl(int dk) { return dk / 16 <= 4 ? 4 : 8; }
 __host__ __device__ constexpr int tc_heads_per_warp(int dk, int rt) { return 32 / (tc_jl(dk) * (SLIM_TT / rt)); }
-__host__ __device__ constexpr int tc_threads(int dk, int rt) {
-  // up to 16 heads per CTA, at least four score/epilogue warps, plus the producer and MMA warps
-  return 32 * ((16 / tc_heads_per_warp(dk, rt) < 4 ? 4 : 16 / tc_heads_per_warp(dk, rt)) + 2);
+__host__ __device__ constexpr int tc_threads(int dk, int rt, int cl) {
+  // up to 32 / cl heads per CTA, at least four score/epilogue warps, plus the producer and MMA warps
+  return 32 * (((32 / cl) / tc_heads_per_warp(dk, rt) < 4 ? 4 : (32 / cl) / tc_heads_per_warp(dk, rt)) + 2);
 }
 
 // ------------------------------------------------------------------ the kernel
 // EXT: the softmax arguments are read from p.ext_scores (X-cache scheme) instead of being
 // formed from the staged rows; the rest of the pipeline is the same.
-template <int DK, bool ROPE, int RT, bool EXT>
-__global__ void __launch_bounds__(tc_threads(DK, RT), 1)
+// CL: CTAs per worker (cluster size), 2 or 1.
+template <int DK, bool ROPE, int RT, bool EXT, int CL>
+__global__ void __launch_bounds__(tc_threads(DK, RT, CL), 1)
 slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams p, const TcGeom g) {
   constexpr int PAIRS = DK / 2;                   // rotation pairs (j, j + DK/2) per head
   constexpr int OCT = PAIRS / 8;                  // 8-pair groups per head
@@ -113,7 +119,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t rank = cluster_ctarank();
-  const int w = blockIdx.x >> 1;                  // worker = cluster index
+  const int w = blockIdx.x / CL;                  // worker = cluster index
   const int producer_warp = g.nswl, mma_warp = g.nswl + 1;
 
   // ---- set-up -------------------------------------------------------------------
@@ -121,7 +127,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   if (tid == 0) {
     prefetch_tensormap(&tmap);
     for (int i = 0; i < g.ns; ++i) { mbar_init(bar_k_full + 8 * i, 1); mbar_init(bar_k_empty + 8 * i, g.nsw + 1); }
-    for (int i = 0; i < TC_NP; ++i) { mbar_init(bar_p_full + 8 * i, 1 + g.nsw); mbar_init(bar_p_empty + 8 * i, 2); }
+    for (int i = 0; i < TC_NP; ++i) { mbar_init(bar_p_full + 8 * i, 1 + g.nsw); mbar_init(bar_p_empty + 8 * i, CL); }
     mbar_init(bar_u_full, 1);
     mbar_init(bar_u_empty, nepi);
     *s_abort = 0;
@@ -326,7 +332,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
               if (lane < 4 * HW) {
                 const int hsel = lane >> 2, half = (lane >> 1) & 1, dest = lane & 1;
                 const int hl_s = HW * warp + hsel;
-                if (hl_s < g.hl) {
+                if (hl_s < g.hl && dest < CL) {
                   const uint4 pv = lds128(stg + (uint32_t)(hsel * 16 + half * 8) * 2u);
                   const int n_s = (int)rank * g.hl + hl_s;
                   const uint32_t dst = p_stage0 + (uint32_t)ps * TC_P_BYTES + p_offset(n_s & 31, half * 8);
@@ -445,7 +451,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             for (int c = 0; c < g.nch; ++c)
               umma_bf16(tmem_base + (uint32_t)(c * 32), desc_a(kbase + (uint32_t)c * 4096u), bd, umma_idesc(32), kt > 0 ? 1u : 0u);
             umma_commit(bar_k_empty + 8 * st);
-            umma_commit_pair(bar_p_empty + 8 * ps);
+            if (CL == 2) umma_commit_pair(bar_p_empty + 8 * ps); else umma_commit(bar_p_empty + 8 * ps);
             if (it + TC_NP < total_it) mbar_arrive_expect_tx(bar_p_full + 8 * ps, p_bytes);
             if (kt == ntile - 1) umma_commit(bar_u_full);
           }
@@ -467,12 +473,13 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
 }
 
 // ------------------------------------------------------------------ host side
-TcGeom make_geom(int d, int H, int d_k, int rt, int smem_limit) {
+TcGeom make_geom(int d, int H, int d_k, int rt, int cl, int smem_limit) {
   TcGeom g;
-  g.dsl = d / 2;
+  g.cl = cl;
+  g.dsl = d / cl;
   g.nch = g.dsl / 128;
   g.nc64 = g.dsl / 64;
-  g.hl = H / 2;
+  g.hl = H / cl;
   const int hw = tc_heads_per_warp(d_k, rt);
   g.nsw = (g.hl + hw - 1) / hw;
   g.nswl = g.nsw < 4 ? 4 : g.nsw;
@@ -505,26 +512,36 @@ int tc_rows_per_thread(int d_k) {
   return want == 4 ? 4 : 8;
 }
 
-tc_kernel_t pick_kernel(int d_k, bool rope, int rt, bool ext = false) {
-  if (ext) {                                   // X-cache scheme: no RoPE
-    if (rope) return nullptr;
-    switch (d_k * 16 + rt) {
-      case 64 * 16 + 2: return slim_tc_kernel<64, false, 2, true>;
-      case 64 * 16 + 4: return slim_tc_kernel<64, false, 4, true>;
-      case 96 * 16 + 4: return slim_tc_kernel<96, false, 4, true>;
-      case 96 * 16 + 8: return slim_tc_kernel<96, false, 8, true>;
-      case 128 * 16 + 4: return slim_tc_kernel<128, false, 4, true>;
-      case 128 * 16 + 8: return slim_tc_kernel<128, false, 8, true>;
-      default: return nullptr;
-    }
+// One CTA per worker (cl = 1) where a whole key row fits one SM's tensor memory and the kernel stays
+// under the register budget of its larger block (instantiated for d_k = 64 without RoPE).  Measured on
+// the Whisper-large shape: with scores computed in the kernel the CTA pair is faster (the score warps
+// of a lone CTA carry all heads); with external scores (X-cache scheme) the lone CTA is faster.
+bool tc_cl_ok(int d, int H, int d_k, bool rope, int cl) {
+  if (cl == 1) return d_k == 64 && !rope && d % 128 == 0 && d <= 2048 && H >= 1 && H <= 32;
+  return !(H & 1) && H <= 32 && H >= 2 && d % 256 == 0 && d <= 4096;   // d/2 in 128-column chunks, <= 512 TMEM columns
+}
+
+template <int DK, bool ROPE, int RT>
+tc_kernel_t pick_ext_cl(bool ext, int cl) {
+  if (cl == 1) {
+    if constexpr (DK == 64 && !ROPE && RT == 4) return ext ? slim_tc_kernel<DK, ROPE, RT, true, 1> : slim_tc_kernel<DK, ROPE, RT, false, 1>;
+    else return nullptr;
   }
+  if (ext) {
+    if constexpr (!ROPE) return slim_tc_kernel<DK, ROPE, RT, true, 2>;
+    else return nullptr;
+  }
+  return slim_tc_kernel<DK, ROPE, RT, false, 2>;
+}
+
+tc_kernel_t pick_kernel(int d_k, bool rope, int rt, bool ext, int cl) {
   switch (d_k * 16 + rt) {
-    case 64 * 16 + 2: return rope ? slim_tc_kernel<64, true, 2, false> : slim_tc_kernel<64, false, 2, false>;
-    case 64 * 16 + 4: return rope ? slim_tc_kernel<64, true, 4, false> : slim_tc_kernel<64, false, 4, false>;
-    case 96 * 16 + 4: return rope ? slim_tc_kernel<96, true, 4, false> : slim_tc_kernel<96, false, 4, false>;
-    case 96 * 16 + 8: return rope ? slim_tc_kernel<96, true, 8, false> : slim_tc_kernel<96, false, 8, false>;
-    case 128 * 16 + 4: return rope ? slim_tc_kernel<128, true, 4, false> : slim_tc_kernel<128, false, 4, false>;
-    case 128 * 16 + 8: return rope ? slim_tc_kernel<128, true, 8, false> : slim_tc_kernel<128, false, 8, false>;
+    case 64 * 16 + 2: return rope ? pick_ext_cl<64, true, 2>(ext, cl) : pick_ext_cl<64, false, 2>(ext, cl);
+    case 64 * 16 + 4: return rope ? pick_ext_cl<64, true, 4>(ext, cl) : pick_ext_cl<64, false, 4>(ext, cl);
+    case 96 * 16 + 4: return rope ? pick_ext_cl<96, true, 4>(ext, cl) : pick_ext_cl<96, false, 4>(ext, cl);
+    case 96 * 16 + 8: return rope ? pick_ext_cl<96, true, 8>(ext, cl) : pick_ext_cl<96, false, 8>(ext, cl);
+    case 128 * 16 + 4: return rope ? pick_ext_cl<128, true, 4>(ext, cl) : pick_ext_cl<128, false, 4>(ext, cl);
+    case 128 * 16 + 8: return rope ? pick_ext_cl<128, true, 8>(ext, cl) : pick_ext_cl<128, false, 8>(ext, cl);
     default: return nullptr;
   }
 }
@@ -552,19 +569,18 @@ cudaError_t slim_launch_wait_selftest(int* status, int* gave_up, cudaStream_t st
   return cudaGetLastError();
 }
 
-int slim_tc_shape_ok(int d, int H, int d_k, int dtype) {
+int slim_tc_shape_ok(int d, int H, int d_k, int dtype, int rope, int cl) {
   if (dtype != SLIM_BF16) return 0;
   if (d_k != 64 && d_k != 96 && d_k != 128) return 0;
-  if ((H & 1) || H > 32 || H < 2) return 0;
-  if (d % 256 != 0 || d > 4096) return 0;          // d/2 in 128-column chunks, <= 512 TMEM columns
-  return 1;
+  return tc_cl_ok(d, H, d_k, rope != 0, cl) ? 1 : 0;
 }
 
-int slim_tc_workers(const slim_ctx* ctx) {
+int slim_tc_workers(const slim_ctx* ctx, int cl) {
   const int rt = tc_rows_per_thread(ctx->d_k);
-  tc_kernel_t kern = pick_kernel(ctx->d_k, ctx->rope_theta != 0.0, rt);
+  const bool rope = ctx->rope_theta != 0.0;
+  tc_kernel_t kern = pick_kernel(ctx->d_k, rope, rt, false, cl);
   if (!kern) return 0;
-  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, rt, TC_SMEM_LIMIT);
+  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, rt, cl, TC_SMEM_LIMIT);
   if (g.ns < 2) return 0;
   const size_t smem = tc_smem_bytes(g, SLIM_MAX_BATCH);
   if (smem > (size_t)TC_SMEM_LIMIT) return 0;
@@ -573,19 +589,19 @@ int slim_tc_workers(const slim_ctx* ctx) {
     return 0;
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(2 * (ctx->num_sms / 2));
+  cfg.gridDim = dim3(cl * (ctx->num_sms / cl));
   cfg.blockDim = dim3((g.nswl + 2) * 32);
   cfg.dynamicSmemBytes = smem;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[0].val.clusterDim.x = cl; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
   int nclusters = 0;
   if (cudaOccupancyMaxActiveClusters(&nclusters, (const void*)kern, &cfg) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
-  const int cap = ctx->num_sms / 2;
+  const int cap = ctx->num_sms / cl;
   return nclusters < cap ? nclusters : cap;
 }
 
@@ -613,39 +629,40 @@ cudaError_t slim_tmap_encode_3d(void* out_map, void* base, const unsigned long l
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c) {
-  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, tc_rows_per_thread(ctx->d_k), TC_SMEM_LIMIT);
+cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c, int cl) {
+  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, tc_rows_per_thread(ctx->d_k), cl, TC_SMEM_LIMIT);
   // dim0: 64 contiguous elements; dim1: cache rows (stride d elements); dim2: 64-column chunks
   const unsigned long long dims[3] = {64, (unsigned long long)c->batch * (unsigned long long)c->t_cap,
                                       (unsigned long long)(ctx->d / 64)};
   const unsigned long long strides[2] = {(unsigned long long)ctx->d * 2, 128};
   const unsigned int box[3] = {64, SLIM_TT, (unsigned int)g.nc64};
-  return slim_tmap_encode_3d(c->tmap, c->k, dims, strides, box);
+  return slim_tmap_encode_3d(c->tmap[cl - 1], c->k, dims, strides, box);
 }
 
 cudaError_t slim_launch_tc(const slim_ctx* ctx, const slim_cache* c, const SlimDecodeParams& p, cudaStream_t st) {
   const int rt = tc_rows_per_thread(ctx->d_k);
   const bool ext = p.ext_scores != nullptr;
-  tc_kernel_t kern = pick_kernel(ctx->d_k, ctx->rope_theta != 0.0, rt, ext);
-  if (!kern || !c->has_tmap) return cudaErrorNotSupported;
+  const int cl = p.cl;
+  tc_kernel_t kern = pick_kernel(ctx->d_k, ctx->rope_theta != 0.0, rt, ext, cl);
+  if (!kern || cl < 1 || cl > 2 || !c->has_tmap[cl - 1]) return cudaErrorNotSupported;
   if (ext) {
     cudaError_t ea = cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_LIMIT);
     if (ea != cudaSuccess) return ea;
   }
-  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, rt, TC_SMEM_LIMIT);
+  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, rt, cl, TC_SMEM_LIMIT);
   const size_t smem = tc_smem_bytes(g, p.batch);
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(2 * p.workers);
+  cfg.gridDim = dim3(cl * p.workers);
   cfg.blockDim = dim3((g.nswl + 2) * 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[0].val.clusterDim.x = cl; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 2;
   CUtensorMap map;
-  memcpy(&map, c->tmap, sizeof(map));
+  memcpy(&map, c->tmap[cl - 1], sizeof(map));
   return cudaLaunchKernelEx(&cfg, kern, map, p, g);
 }
