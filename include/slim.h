@@ -112,6 +112,12 @@ size_t slim_workspace_bytes(const slim_ctx* ctx, int batch, int t_cap);
 slim_status slim_cache_create(slim_ctx* ctx, slim_cache** out, void* k_storage, int batch, int t_cap);
 void        slim_cache_destroy(slim_cache* cache);
 
+/* Prompt phase (Fig. 3(a)): the values of the n prompt tokens are formed once from their keys,
+ * V = K W_KV (Eq. 6), so that the prompt can be processed like vanilla attention while only K is
+ * kept.  K: device [n][d], ctx dtype, un-rotated keys; V: device [n][d] float32.  bf16 with
+ * d_k in {64, 96, 128} runs on the tensor cores (16-byte aligned K and V), else on CUDA cores. */
+slim_status slim_values_from_keys(slim_ctx* ctx, const void* K, int n, float* V, void* stream);
+
 /* Generate-phase cache update: for every sequence b write the n_new rows
  * k_new[b][0..n_new) (device, [batch][n_new][d], ctx dtype, un-rotated keys
  * k = x W_K) at rows positions[b] .. positions[b]+n_new-1 (device int32).

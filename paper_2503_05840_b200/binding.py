@@ -31,6 +31,7 @@ SIGNATURES = {
     "slim_workspace_bytes": (c_size_t, [c_void_p, c_int, c_int]),
     "slim_cache_create": (c_int, [c_void_p, POINTER(c_void_p), c_void_p, c_int, c_int]),
     "slim_cache_destroy": (None, [c_void_p]),
+    "slim_values_from_keys": (c_int, [c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
     "slim_append_k": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]),
     "slim_decode": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "slim_static_workspace_max": (c_size_t, []),
@@ -159,6 +160,10 @@ def slim_cache_create(ctx: int, k_storage, batch: int, t_cap: int) -> int:
 
 def slim_cache_destroy(cache: int) -> None:
     lib().slim_cache_destroy(c_void_p(cache))
+
+
+def slim_values_from_keys(ctx: int, K, n: int, V, stream: int = 0) -> None:
+    _check(lib().slim_values_from_keys(c_void_p(ctx), _ptr(K), n, _ptr(V), c_void_p(stream)), "slim_values_from_keys")
 
 
 def slim_append_k(ctx: int, cache: int, k_new, positions, n_new: int, stream: int = 0) -> None:

@@ -464,6 +464,13 @@ slim_status slim_xcache_decode(slim_ctx* ctx, const void* q, const slim_cache* c
   return decode_impl(ctx, q, cache, lengths, o, workspace, stream, true);
 }
 
+slim_status slim_values_from_keys(slim_ctx* ctx, const void* K, int n, float* V, void* stream) {
+  if (!ctx || !K || !V || n <= 0) return SLIM_ERR_INVALID_ARG;
+  if (!ctx->has_weights) return SLIM_ERR_NO_WEIGHTS;
+  if (slim_launch_values(ctx, K, n, V, (cudaStream_t)stream) != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
+  return SLIM_OK;
+}
+
 size_t slim_static_workspace_max(void) { return SLIM_STATIC_WS_BYTES; }
 
 slim_status slim_decode_static_ws(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,

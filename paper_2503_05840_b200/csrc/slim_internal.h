@@ -150,3 +150,6 @@ size_t slim_xscores_qt_bytes(int d, int batch);
 cudaError_t slim_xscores_make_tmap(const slim_ctx* ctx, slim_cache* c);
 cudaError_t slim_launch_xscores_tc(const slim_ctx* ctx, const slim_cache* c, const SlimDecodeParams& p, const float* W_K,
                                    unsigned char* qt_tiled, float* scores, cudaStream_t st);
+
+// prompt phase: V = K W_KV for n rows (slim_prompt.cu)
+cudaError_t slim_launch_values(const slim_ctx* ctx, const void* K, int n, float* V, cudaStream_t st);

@@ -1,0 +1,175 @@
+// Prompt phase of slim attention (Fig. 3(a)): the values of a whole prompt are formed once from
+// its keys, V = K W_KV (Eq. 6), after which the prompt is processed like vanilla attention.
+//
+//   slim_values_tc_kernel   bf16, d_k in {64, 96, 128}: CTA = (128 prompt rows, head group);
+//                           V[128 x N] += K_tile[128 x 16] W_KV,h[16 x N] per 16 columns of K on
+//                           tcgen05: A = key rows, K-major with 128-byte swizzle as TMA delivers
+//                           them; B = the W_KV tile, MN-major (the same TMA tiles the decode
+//                           projection uses); D in tensor memory (N = 128: one head of d_k = 128 or
+//                           96, or two heads of d_k = 64).
+//   slim_values_kernel      any dtype / shape: CUDA-core tiles.
+// Every mbarrier wait is bounded in time.
+#include <cstring>
+
+#include "slim_internal.h"
+#include "slim_ptx.cuh"
+
+namespace {
+using namespace slim_ptx;
+
+constexpr int PV_ROWS = 128;                       // prompt rows per CTA (MMA M)
+constexpr int PV_J = 64;                           // columns of K (rows of W_KV) per stage
+constexpr int PV_A_BYTES = PV_ROWS * PV_J * 2;     // 16 KB
+constexpr int PV_B_BYTES = PV_J * 128 * 2;         // two 64-column atoms x 64 rows x 128 B = 16 KB
+constexpr int PV_NS = 4;
+
+__global__ void __launch_bounds__(128)
+slim_values_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap wmap, float* __restrict__ V,
+                      const int n, const int d, const int d_k, const int hp, int* status) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw_u32 = smem_u32(smem_raw);
+  const uint32_t base = (raw_u32 + 1023u) & ~1023u;
+  unsigned char* sm = smem_raw + (base - raw_u32);
+  constexpr uint32_t stage_bytes = PV_A_BYTES + PV_B_BYTES;
+  const uint32_t bars = base + PV_NS * stage_bytes;
+  const uint32_t bar_full = bars, bar_empty = bars + 8 * PV_NS, bar_done = bars + 16 * PV_NS;
+  unsigned char* misc = sm + (bar_done + 8 - base);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 4);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int t0 = blockIdx.x * PV_ROWS, hg = blockIdx.y;
+  const int nst = d / PV_J;
+
+  if (tid == 0) {
+    prefetch_tensormap(&kmap);
+    prefetch_tensormap(&wmap);
+    for (int i = 0; i < PV_NS; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
+    mbar_init(bar_done, 1);
+    *s_abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(s_tmem), 128);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  slim_pdl_wait();
+
+  if (warp == 0 && lane == 0) {
+    int s = 0;
+    bool ok = true;
+    for (; s < nst; ++s) {
+      const int st = s % PV_NS;
+      ok = mbar_wait<false>(bar_empty + 8 * st, ((s / PV_NS) & 1) ^ 1, s_abort, status);
+      if (!ok) break;
+      const uint32_t dst = base + (uint32_t)st * stage_bytes;
+      mbar_arrive_expect_tx(bar_full + 8 * st, stage_bytes);
+      tma_load_3d(dst, &kmap, bar_full + 8 * st, s * PV_J, t0, 0);
+      if (hp == 1) tma_load_3d(dst + PV_A_BYTES, &wmap, bar_full + 8 * st, 0, hg * d + s * PV_J, 0);
+      else         tma_load_3d(dst + PV_A_BYTES, &wmap, bar_full + 8 * st, 0, s * PV_J, 2 * hg);
+    }
+    if (!ok) {
+      const int issued = s < PV_NS ? s : PV_NS;
+      for (int k = 0; k < issued; ++k) {
+        const int j = s - 1 - k, st = j % PV_NS;
+        const unsigned long long tt = globaltimer();
+        while (!mbar_try_wait(bar_full + 8 * st, (j / PV_NS) & 1) && globaltimer() - tt < SLIM_WAIT_NS) {}
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    bool ok = true;
+    for (int s = 0; s < nst && ok; ++s) {
+      const int st = s % PV_NS;
+      ok = mbar_wait<false>(bar_full + 8 * st, (s / PV_NS) & 1, s_abort, status);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t abase = base + (uint32_t)st * stage_bytes, bbase = abase + PV_A_BYTES;
+#pragma unroll
+      for (int kk = 0; kk < PV_J / 16; ++kk)
+        umma_bf16(tmem_base, desc_kmajor_sw128(abase + (uint32_t)kk * 32u), desc_a(bbase + (uint32_t)kk * 2048u, PV_J * 128),
+                  umma_idesc_major(128, 0, 1), (s | kk) ? 1u : 0u);
+      umma_commit(bar_empty + 8 * st);
+      if (s == nst - 1) umma_commit(bar_done);
+    }
+  }
+  __syncwarp();
+  {
+    bool ok = mbar_wait<false>(bar_done, 0, s_abort, status);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after();
+      const int row = t0 + warp * 32 + lane;                   // accumulator row = prompt row
+      const int ncols = hp == 2 ? 128 : d_k;                   // valid accumulator columns
+      float* out = V + (size_t)row * d + (size_t)hg * hp * d_k;
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, r);
+        if (row < n) {
+#pragma unroll
+          for (int c = 0; c < 32; c += 4)
+            if (c0 + c < ncols)
+              *reinterpret_cast<float4*>(out + c0 + c) = make_float4(__uint_as_float(r[c]), __uint_as_float(r[c + 1]),
+                                                                    __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 128);
+  }
+}
+
+// CUDA-core version: V[t][h d_k + c] = sum_j K[t][j] W[h][j][c]; 16 x 16 output tile per CTA.
+template <typename KT>
+__global__ void __launch_bounds__(256)
+slim_values_kernel(const KT* __restrict__ K, const KT* __restrict__ W, float* __restrict__ V, int n, int d, int d_k) {
+  __shared__ float s_k[16][17], s_w[16][17];
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int t = blockIdx.y * 16 + ty, col = blockIdx.x * 16 + tx;       // col = h d_k + c
+  const int h = col / d_k, c = col % d_k;
+  float acc = 0.f;
+  for (int j0 = 0; j0 < d; j0 += 16) {
+    s_k[ty][tx] = (t < n && j0 + tx < d) ? (float)K[(size_t)t * d + j0 + tx] : 0.f;
+    s_w[ty][tx] = (col < d && j0 + ty < d) ? (float)W[((size_t)h * d + j0 + ty) * d_k + c] : 0.f;
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < 16; ++j) acc = fmaf(s_k[ty][j], s_w[j][tx], acc);
+    __syncthreads();
+  }
+  if (t < n && col < d) V[(size_t)t * d + col] = acc;
+}
+
+constexpr size_t PV_SMEM = 1024 + (size_t)PV_NS * (PV_A_BYTES + PV_B_BYTES) + 16 * PV_NS + 8 + 16 + 64;
+
+}  // namespace
+
+cudaError_t slim_launch_values(const slim_ctx* ctx, const void* K, int n, float* V, cudaStream_t st) {
+  const int d = ctx->d, d_k = ctx->d_k, H = ctx->H;
+  if (ctx->proj_ok && ((uintptr_t)K & 15) == 0 && ((uintptr_t)V & 15) == 0) {
+    static bool attr_set = false;
+    if (!attr_set) {
+      cudaError_t e = cudaFuncSetAttribute((const void*)slim_values_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PV_SMEM);
+      if (e != cudaSuccess) return e;
+      attr_set = true;
+    }
+    CUtensorMap kmap, wmap;
+    const unsigned long long dims[3] = {(unsigned long long)d, (unsigned long long)n, 1};
+    const unsigned long long strides[2] = {(unsigned long long)d * 2, (unsigned long long)d * 2 * (unsigned long long)n};
+    const unsigned int box[3] = {PV_J, PV_ROWS, 1};
+    cudaError_t e = slim_tmap_encode_3d(&kmap, const_cast<void*>(K), dims, strides, box);
+    if (e != cudaSuccess) return e;
+    memcpy(&wmap, ctx->wmap, sizeof(wmap));
+    const int hp = d_k == 64 ? 2 : 1;
+    return slim_launch_pdl(slim_values_tc_kernel, dim3((n + PV_ROWS - 1) / PV_ROWS, H / hp), dim3(128), PV_SMEM, st, kmap, wmap, V, n,
+                           d, d_k, hp, ctx->status);
+  }
+  dim3 grid((d + 15) / 16, (n + 15) / 16);
+  if (ctx->dtype == SLIM_BF16)
+    slim_values_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)K, (const __nv_bfloat16*)ctx->wkv, V, n, d, d_k);
+  else
+    slim_values_kernel<float><<<grid, 256, 0, st>>>((const float*)K, (const float*)ctx->wkv, V, n, d, d_k);
+  return cudaGetLastError();
+}

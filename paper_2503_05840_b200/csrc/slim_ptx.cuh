@@ -138,6 +138,16 @@ __host__ __device__ constexpr uint32_t umma_idesc(uint32_t n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
+// K-major operand, 128-byte swizzle, as TMA delivers a [rows][64 elements] tile: 8-row groups
+// 1024 B apart; the 16-element k-step is selected by the start address (+32 B per step).
+__device__ __forceinline__ uint64_t desc_kmajor_sw128(uint32_t addr) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor with explicit operand majors (1 = MN-major): bf16 x bf16 -> f32, M = 128, N = n.
+__host__ __device__ constexpr uint32_t umma_idesc_major(uint32_t n, uint32_t a_mn, uint32_t b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn << 15) | (b_mn << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
 __device__ __forceinline__ uint32_t p_offset(int n, int k) {
   return (uint32_t)((n & 7) * 16 + (n >> 3) * 256 + (k >> 3) * 128 + (k & 7) * 2);
 }

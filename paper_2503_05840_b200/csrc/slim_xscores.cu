@@ -22,16 +22,6 @@ constexpr int XT_NS = 4;
 __device__ __forceinline__ uint32_t qt_offset(int n, int k) {     // K-major 8x8 core matrices, N = 64
   return (uint32_t)((n & 7) * 16 + (n >> 3) * 256 + (k >> 3) * 128 + (k & 7) * 2);
 }
-// A operand: 128 rows x 16 columns inside a [128 rows][64 columns] tile, K-major, 128-byte swizzle:
-// 8-row groups 1024 B apart; the k-step is selected by the start address (+32 B per step).
-__device__ __forceinline__ uint64_t desc_a_kmajor(uint32_t addr) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
-}
-// bf16 x bf16 -> f32, A and B K-major, M = 128, N = n
-__host__ __device__ constexpr uint32_t idesc_kk(uint32_t n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
-}
-
 // q~[b][h][j] = qscale sum_c q[b][h d_k + c] W_K[j][h d_k + c], written as bf16 hi / lo rows h and 32 + h
 // of the [64 x 16] tile of k-step j / 16.  CTA = (head, 64 rows j of W_K): the weight tile is read once
 // and used for every sequence of the batch.
@@ -138,7 +128,7 @@ slim_xscores_tc_kernel(const __grid_constant__ CUtensorMap xmap, const SlimDecod
       const uint32_t abase = base + (uint32_t)st * stage_bytes, bbase = abase + XT_A_BYTES;
 #pragma unroll
       for (int kk = 0; kk < XT_COLS / 16; ++kk)
-        umma_bf16(tmem_base, desc_a_kmajor(abase + (uint32_t)kk * 32u), desc_b(bbase + (uint32_t)kk * 2048u), idesc_kk(64),
+        umma_bf16(tmem_base, desc_kmajor_sw128(abase + (uint32_t)kk * 32u), desc_b(bbase + (uint32_t)kk * 2048u), umma_idesc_major(64, 0, 0),
                   (s | kk) ? 1u : 0u);
       umma_commit(bar_empty + 8 * st);
       if (s == nst - 1) umma_commit(bar_done);

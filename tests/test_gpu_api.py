@@ -309,3 +309,33 @@ def test_nonsquare_weights_right_inverse_matches_oracle_and_decodes():
         assert ei.value.status == B.SLIM_ERR_SINGULAR
     finally:
         layer.close()
+
+
+@pytest.mark.parametrize("d,H,d_k,dtype", [(512, 4, 128, "bf16"), (1280, 20, 64, "bf16"), (384, 4, 96, "bf16"), (256, 4, 64, "f32"), (192, 2, 96, "bf16")])
+def test_prompt_phase_values_from_keys(d, H, d_k, dtype):
+    # Fig. 3(a): V = K W_KV for a whole prompt; equals X W_V up to the rounding of the stored keys
+    n = 300
+    W_Q, W_K, W_V, _, _ = synth.make_weights(d, 300 + d)
+    X = np.random.default_rng(d).standard_normal((n, d))
+    K = synth.round_to_dtype(X @ W_K, dtype)
+    layer = SlimLayer(d, H, d_k, 0.0, dtype, 1, 16, DEV)
+    try:
+        layer.set_weights(W_K, W_V)
+        Kd = to_device_keys(K, dtype, DEV)
+        V = torch.full((n, d), float("nan"), dtype=torch.float32, device=DEV)
+        with torch.cuda.device(DEV):
+            B.slim_values_from_keys(layer.ctx, Kd, n, V, torch.cuda.current_stream().cuda_stream)
+        assert layer.device_status() == B.SLIM_OK
+        got = V.cpu().numpy().astype(np.float64)
+        assert np.all(np.isfinite(got))
+        ref = K.astype(np.float64) @ so.oracle_wkv(W_K, W_V)          # Eq. 6 on the stored keys
+        van = X @ W_V                                                  # Eq. 5
+        tol = 2e-2 if dtype == "bf16" else 1e-4
+        for t in (0, 1, 127, 128, 255, 299):
+            e = so.err_rms_norm(got[t], ref[t]) if dtype == "bf16" else so.err_fp32_norm(got[t], ref[t])
+            assert e <= tol, f"row {t}: {e:.3e}"
+            assert so.err_rms_norm(got[t], van[t]) <= (5e-2 if dtype == "bf16" else 1e-3)
+        worst = max(so.err_rms_norm(got[t], ref[t]) for t in range(n))
+        assert worst <= (2e-2 if dtype == "bf16" else 1e-4)
+    finally:
+        layer.close()
