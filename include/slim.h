@@ -110,6 +110,16 @@ size_t slim_workspace_bytes(const slim_ctx* ctx, int batch, int t_cap);
  * UN-ROTATED keys.  Builds the RoPE tables for positions < t_cap.  The storage
  * must outlive the cache object; its contents are not touched.                */
 slim_status slim_cache_create(slim_ctx* ctx, slim_cache** out, void* k_storage, int batch, int t_cap);
+/* Paged K-cache: the keys live in a caller-owned pool of num_pages pages of page_rows rows each
+ * (device, [num_pages][page_rows][d], ctx dtype, 16-byte aligned; page_rows a multiple of 16), and
+ * context row t of sequence b is row t % page_rows of page block_table[b][t / page_rows].
+ * block_table: device int32 [batch][max_pages], read by the kernels at every call (the caller may
+ * update it between calls); capacity per sequence t_cap = max_pages * page_rows.  A page id
+ * outside the pool raises SLIM_ERR_CAPACITY on the device.  slim_append_k and slim_decode take
+ * such a cache like a contiguous one (workspace: slim_workspace_bytes(ctx, batch, t_cap)); the
+ * X-cache calls do not.                                                               */
+slim_status slim_cache_create_paged(slim_ctx* ctx, slim_cache** out, void* pool, int num_pages, int page_rows,
+                                    const int32_t* block_table, int batch, int max_pages);
 void        slim_cache_destroy(slim_cache* cache);
 
 /* Prompt phase (Fig. 3(a)): the values of the n prompt tokens are formed once from their keys,

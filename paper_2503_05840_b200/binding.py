@@ -30,6 +30,7 @@ SIGNATURES = {
     "slim_cache_bytes": (c_size_t, [c_void_p, c_int, c_int]),
     "slim_workspace_bytes": (c_size_t, [c_void_p, c_int, c_int]),
     "slim_cache_create": (c_int, [c_void_p, POINTER(c_void_p), c_void_p, c_int, c_int]),
+    "slim_cache_create_paged": (c_int, [c_void_p, POINTER(c_void_p), c_void_p, c_int, c_int, c_void_p, c_int, c_int]),
     "slim_cache_destroy": (None, [c_void_p]),
     "slim_values_from_keys": (c_int, [c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
     "slim_append_k": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]),
@@ -155,6 +156,13 @@ def slim_workspace_bytes(ctx: int, batch: int, t_cap: int) -> int:
 def slim_cache_create(ctx: int, k_storage, batch: int, t_cap: int) -> int:
     h = c_void_p()
     _check(lib().slim_cache_create(c_void_p(ctx), byref(h), _ptr(k_storage), batch, t_cap), "slim_cache_create")
+    return h.value
+
+
+def slim_cache_create_paged(ctx: int, pool, num_pages: int, page_rows: int, block_table, batch: int, max_pages: int) -> int:
+    h = c_void_p()
+    _check(lib().slim_cache_create_paged(c_void_p(ctx), byref(h), _ptr(pool), num_pages, page_rows, _ptr(block_table), batch,
+                                         max_pages), "slim_cache_create_paged")
     return h.value
 
 

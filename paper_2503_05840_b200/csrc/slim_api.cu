@@ -343,6 +343,8 @@ slim_status slim_cache_create(slim_ctx* ctx, slim_cache** out, void* k_storage, 
   slim_cache* c = new (std::nothrow) slim_cache();
   if (!c) return SLIM_ERR_OOM;
   c->ctx = ctx; c->k = k_storage; c->batch = batch; c->t_cap = t_cap;
+  c->block_table = nullptr; c->page_rows = 0; c->max_pages = 0; c->num_pages = 0;
+  c->total_rows = (long long)batch * t_cap;
   for (int cl = 1; cl <= 2; ++cl) {
     c->has_tmap[cl - 1] = 0;
     if (ctx->tc_workers[cl - 1] > 0) {
@@ -355,6 +357,34 @@ slim_status slim_cache_create(slim_ctx* ctx, slim_cache** out, void* k_storage, 
     if (slim_xscores_make_tmap(ctx, c) == cudaSuccess) c->has_xmap = 1;
     else cudaGetLastError();
   }
+  *out = c;
+  return SLIM_OK;
+}
+
+slim_status slim_cache_create_paged(slim_ctx* ctx, slim_cache** out, void* pool, int num_pages, int page_rows,
+                                    const int32_t* block_table, int batch, int max_pages) {
+  if (!out) return SLIM_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!ctx || !pool || !block_table || num_pages <= 0 || page_rows <= 0 || batch <= 0 || max_pages <= 0) return SLIM_ERR_INVALID_ARG;
+  if (page_rows % SLIM_TT != 0 || batch > SLIM_MAX_BATCH || ((uintptr_t)pool & 15)) return SLIM_ERR_UNSUPPORTED;
+  if ((long long)num_pages * page_rows > 0x7fffffffLL - 64 || (long long)batch * max_pages * page_rows > 0x7fffffffLL - 64)
+    return SLIM_ERR_UNSUPPORTED;
+  const int t_cap = max_pages * page_rows;
+  slim_status st = grow_rope_base(ctx, t_cap);
+  if (st != SLIM_OK) return st;
+  slim_cache* c = new (std::nothrow) slim_cache();
+  if (!c) return SLIM_ERR_OOM;
+  c->ctx = ctx; c->k = pool; c->batch = batch; c->t_cap = t_cap;
+  c->block_table = block_table; c->page_rows = page_rows; c->max_pages = max_pages; c->num_pages = num_pages;
+  c->total_rows = (long long)num_pages * page_rows;
+  for (int cl = 1; cl <= 2; ++cl) {
+    c->has_tmap[cl - 1] = 0;
+    if (ctx->tc_workers[cl - 1] > 0) {
+      if (slim_tc_make_tmap(ctx, c, cl) == cudaSuccess) c->has_tmap[cl - 1] = 1;
+      else cudaGetLastError();
+    }
+  }
+  c->has_xmap = 0;                                     // the X-cache scheme takes contiguous caches only
   *out = c;
   return SLIM_OK;
 }
@@ -379,6 +409,7 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   if (!ctx->has_weights) return SLIM_ERR_NO_WEIGHTS;
   int path = path_in_use(ctx);
   if (xcache && !ctx->xc_wk) return SLIM_ERR_NO_WEIGHTS;
+  if (xcache && cache->block_table) return SLIM_ERR_UNSUPPORTED;
   if (path < 0) return SLIM_ERR_UNSUPPORTED;
   // CTAs per worker: the pair when the kernel computes the scores, the lone CTA with external scores
   int cl = 0;
@@ -411,6 +442,8 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   p.u = reinterpret_cast<float*>(ws + L.o_part);
   p.o = o; p.status = ctx->status; p.any_flag = ctx->any_flag;
   p.ext_scores = nullptr;
+  p.block_table = cache->block_table; p.page_rows = cache->page_rows; p.max_pages = cache->max_pages;
+  p.num_pages = cache->num_pages;
   cudaStream_t st = (cudaStream_t)stream;
   if (ctx->prof_on) cudaEventRecord(ctx->prof_ev[0], st);
   cudaError_t e;

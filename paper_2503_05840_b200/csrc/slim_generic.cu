@@ -94,7 +94,7 @@ slim_exact_kernel(SlimDecodeParams p, int only_flagged) {
 
     for (int tile = tile0; tile < tile1; ++tile) {
       const int t0 = tile * SLIM_TT;
-      const KT* __restrict__ Kt = Kc + ((size_t)b * p.t_cap + t0) * d;
+      const KT* __restrict__ Kt = Kc + (size_t)slim_cache_row(p, b, t0) * d;
 
       // ---- A: softmax arguments for all heads, rows of this tile ------------
       for (int pi = wid; pi < H * SLIM_TT; pi += GEN_THREADS / 32) {
@@ -261,7 +261,7 @@ slim_scores_kernel(SlimDecodeParams p, float* __restrict__ scores) {
     }
     for (int t = wid; t < SLIM_TT; t += GEN_THREADS / 32) {
       if (t0 + t >= len) continue;
-      const KT* kr = Kc + ((size_t)b * p.t_cap + t0 + t) * d;
+      const KT* kr = Kc + (size_t)(slim_cache_row(p, b, t0) + t) * d;
       for (int pv = lane; pv < npv; pv += 32) {
         const int h = pv / pv_per_head, j0 = (pv - h * pv_per_head) * VEC;
         float k1[VEC], k2[VEC];
@@ -338,7 +338,7 @@ slim_accum_kernel(SlimDecodeParams p, const float* __restrict__ scores, int only
     __syncthreads();
     for (int tile = tile0; tile < tile1; ++tile) {
       const int t0 = tile * SLIM_TT;
-      const KT* __restrict__ Kt = Kc + ((size_t)b * p.t_cap + t0) * d;
+      const KT* __restrict__ Kt = Kc + (size_t)slim_cache_row(p, b, t0) * d;
       float kv[SLIM_TT];
 #pragma unroll
       for (int t = 0; t < SLIM_TT; ++t) kv[t] = (col < d && t0 + t < len) ? ld_k(Kt + (size_t)t * d + col) : 0.f;

@@ -41,6 +41,8 @@ struct SlimDecodeParams {
   int* status;                   // sticky device status word
   int* any_flag;                 // set to 1 by a kernel that flags a unit
   const float* ext_scores;       // X-cache scheme: precomputed softmax arguments [batch][H][t_cap] (else NULL)
+  const int32_t* block_table;    // paged cache: [batch][max_pages] page ids (NULL = contiguous [batch][t_cap][d])
+  int page_rows, max_pages, num_pages;
 };
 
 struct slim_ctx {
@@ -69,7 +71,10 @@ struct slim_ctx {
 struct slim_cache {
   slim_ctx* ctx;
   void* k;
-  int batch, t_cap;
+  int batch, t_cap;              // paged: t_cap = max_pages * page_rows
+  const int32_t* block_table;    // paged: device [batch][max_pages]; NULL for a contiguous cache
+  int page_rows, max_pages, num_pages;
+  long long total_rows;          // rows of the storage: batch * t_cap, or num_pages * page_rows
   alignas(64) unsigned char tmap[2][128];   // CUtensorMaps of the tensor-core path for 1 / 2 CTAs per worker
   int has_tmap[2];
   alignas(64) unsigned char xmap[128];   // CUtensorMap for the dense X-cache scores (rows x 64 columns)

@@ -101,3 +101,15 @@ __device__ __forceinline__ int slim_worker_of_tile(const SlimSched& s, int g) {
   const long long v = (long long)g + (long long)s.unit_cost * b;
   return (int)(((v + 1) * s.workers_eff - 1) / s.virt_total);
 }
+
+// Row of the key storage that holds context row t0 of sequence b (t0 a multiple of SLIM_TT; a tile
+// never straddles pages because page_rows is a multiple of SLIM_TT).  A page id outside the pool
+// raises SLIM_ERR_CAPACITY and reads page 0.
+__device__ __forceinline__ long long slim_cache_row(const SlimDecodeParams& p, int b, int t0) {
+  if (p.block_table) {
+    int pg = p.block_table[(size_t)b * p.max_pages + t0 / p.page_rows];
+    if (pg < 0 || pg >= p.num_pages) { atomicMax(p.status, (int)SLIM_ERR_CAPACITY); pg = 0; }
+    return (long long)pg * p.page_rows + t0 % p.page_rows;
+  }
+  return (long long)b * p.t_cap + t0;
+}

@@ -134,7 +134,8 @@ __global__ void __launch_bounds__(256) slim_tail2_kernel(const float* __restrict
 template <typename KT>
 __global__ void slim_append_kernel(KT* __restrict__ cache, const KT* __restrict__ k_new,
                                    const int32_t* __restrict__ positions, int d, int t_cap, int n_new,
-                                   int* status) {
+                                   int* status, const int32_t* __restrict__ block_table, int page_rows, int max_pages,
+                                   int num_pages) {
   slim_pdl_trigger();
   slim_pdl_wait();
   const int b = blockIdx.x, r = blockIdx.y;
@@ -144,7 +145,16 @@ __global__ void slim_append_kernel(KT* __restrict__ cache, const KT* __restrict_
     return;
   }
   const KT* src = k_new + ((size_t)b * n_new + r) * d;
-  KT* dst = cache + ((size_t)b * t_cap + pos + r) * d;
+  size_t row = (size_t)b * t_cap + pos + r;
+  if (block_table) {                                // paged storage
+    const int pg = block_table[(size_t)b * max_pages + (pos + r) / page_rows];
+    if (pg < 0 || pg >= num_pages) {
+      if (threadIdx.x == 0) atomicMax(status, (int)SLIM_ERR_CAPACITY);
+      return;
+    }
+    row = (size_t)pg * page_rows + (pos + r) % page_rows;
+  }
+  KT* dst = cache + row * d;
   // rows are 16-byte aligned when d * sizeof(KT) is a multiple of 16 and the buffers are
   const size_t bytes = (size_t)d * sizeof(KT);
   if ((bytes & 15) == 0 && (((uintptr_t)src | (uintptr_t)dst) & 15) == 0) {
@@ -202,7 +212,8 @@ cudaError_t slim_launch_append(const slim_ctx* ctx, const slim_cache* c, const v
   dim3 grid(c->batch, n_new);
   if (ctx->dtype == SLIM_BF16)
     return slim_launch_pdl(slim_append_kernel<__nv_bfloat16>, grid, dim3(256), 0, st, (__nv_bfloat16*)c->k,
-                           (const __nv_bfloat16*)k_new, positions, ctx->d, c->t_cap, n_new, ctx->status);
+                           (const __nv_bfloat16*)k_new, positions, ctx->d, c->t_cap, n_new, ctx->status, c->block_table,
+                           c->page_rows, c->max_pages, c->num_pages);
   return slim_launch_pdl(slim_append_kernel<float>, grid, dim3(256), 0, st, (float*)c->k, (const float*)k_new, positions,
-                         ctx->d, c->t_cap, n_new, ctx->status);
+                         ctx->d, c->t_cap, n_new, ctx->status, c->block_table, c->page_rows, c->max_pages, c->num_pages);
 }

@@ -409,7 +409,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             if (!ok) break;
             mbar_arrive_expect_tx(bar_k_full + 8 * st, (uint32_t)g.stage_bytes);
             tma_load_3d(k_stage0 + (uint32_t)st * g.stage_bytes, &tmap, bar_k_full + 8 * st, 0,
-                        b * p.t_cap + (tile0 + kt) * SLIM_TT, (int)rank * g.nc64);
+                        (int)slim_cache_row(p, b, (tile0 + kt) * SLIM_TT), (int)rank * g.nc64);
           }
           gg = seg_end;
         }
@@ -632,8 +632,7 @@ cudaError_t slim_tmap_encode_3d(void* out_map, void* base, const unsigned long l
 cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c, int cl) {
   const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, tc_rows_per_thread(ctx->d_k), cl, TC_SMEM_LIMIT);
   // dim0: 64 contiguous elements; dim1: cache rows (stride d elements); dim2: 64-column chunks
-  const unsigned long long dims[3] = {64, (unsigned long long)c->batch * (unsigned long long)c->t_cap,
-                                      (unsigned long long)(ctx->d / 64)};
+  const unsigned long long dims[3] = {64, (unsigned long long)c->total_rows, (unsigned long long)(ctx->d / 64)};
   const unsigned long long strides[2] = {(unsigned long long)ctx->d * 2, 128};
   const unsigned int box[3] = {64, SLIM_TT, (unsigned int)g.nc64};
   return slim_tmap_encode_3d(c->tmap[cl - 1], c->k, dims, strides, box);
