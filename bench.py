@@ -43,8 +43,10 @@ def parse():
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (0 = the config's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--variant", default="kcache", choices=["kcache", "xcache"],
-                    help="xcache: the X/E-cache scheme, one cache shared by all layers (configs without RoPE)")
+    ap.add_argument("--variant", default="kcache", choices=["kcache", "xcache", "prompt"],
+                    help="xcache: the X/E-cache scheme, one cache shared by all layers (configs without RoPE); "
+                         "prompt: the prompt-phase V = K W_KV of the config's shape")
+    ap.add_argument("--paged", type=int, default=0, help="K-cache in a shuffled pool of pages of this many rows (0 = contiguous)")
     return ap.parse_args()
 
 
@@ -250,12 +252,58 @@ def run_xcache(args):
                       "device_status": int(B.slim_device_status(ctxs[0], st))}))
 
 
+def run_prompt(args):
+    """Prompt phase: V = K W_KV for all prompt rows of one layer of the config (batch x context rows)."""
+    import torch
+    from paper_2503_05840_b200 import binding as B
+    from paper_2503_05840_b200 import build as _build
+    from paper_2503_05840_b200 import synth
+    _build.build()
+    cfg = synth.CONFIGS[args.config]
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    n = min(cfg.batch * cfg.context, 262144)
+    ctx = B.slim_create(cfg.d, cfg.H, cfg.d_k, 0.0, B.SLIM_BF16 if cfg.dtype == "bf16" else B.SLIM_F32)
+    B.slim_set_wkv(ctx, np.random.default_rng(0).standard_normal((cfg.d, cfg.d)) / np.sqrt(cfg.d))
+    tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    K = torch.randn((n, cfg.d), device=dev).to(tdt)
+    V = torch.empty((n, cfg.d), dtype=torch.float32, device=dev)
+    st = torch.cuda.current_stream().cuda_stream
+    for _ in range(max(args.warmup, 3)):
+        B.slim_values_from_keys(ctx, K, n, V, st)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        B.slim_values_from_keys(ctx, K, n, V, st)
+    e1.record(); torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    tf = 2.0 * n * cfg.d * cfg.d / (ms * 1e-3) / 1e12
+    peak = 1590.0
+    pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    kind = "fallback"
+    if os.path.exists(pk):
+        with open(pk) as f:
+            peak = float(json.load(f)["bf16_tflops"]); kind = "measured"
+    print(json.dumps({"metric": "prompt_value_rows_per_s", "variant": "prompt", "value": n / (ms * 1e-3), "unit": "rows/s",
+                      "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+                      "dtype": cfg.dtype, "data": "synthetic",
+                      "config": {"workload": f"config{args.config}:{cfg.name} (prompt phase V = K W_KV)", "rows": n, "d": cfg.d,
+                                 "H": cfg.H, "d_k": cfg.d_k},
+                      "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+                                   "traffic": None, "peak_kind": kind},
+                      "device_status": int(B.slim_device_status(ctx, st))}))
+    B.slim_destroy(ctx)
+
+
 def main():
     args = parse()
     if args.impl == "reference":
         return run_reference(args)
     if args.variant == "xcache":
         return run_xcache(args)
+    if args.variant == "prompt":
+        return run_prompt(args)
 
     import torch
     from paper_2503_05840_b200 import binding as B
@@ -292,6 +340,25 @@ def main():
     pos_dev = (lens_dev - 1).clamp(min=0).to(torch.int32)
     layers = []
     ws = None
+    paged_tables = []
+
+    def seq_rows(li, lay, b, n):
+        """Context rows 0..n-1 of sequence b of a layer, whatever the cache arrangement."""
+        if not args.paged:
+            return lay.k[b, :n]
+        pr = args.paged
+        pages = paged_tables[li][b, :(n + pr - 1) // pr].long()
+        return lay.k.reshape(-1, pr, cfg.d)[pages].reshape(-1, cfg.d)[:n]
+
+    def make_paged(lay, page_rows, li):
+        # the layer's own storage is the pool: [batch * pages][page_rows][d]; sequence b uses pages in a rotated order,
+        # so rows must be written through the table (slim_append_k) -- done below by re-appending the drawn keys
+        assert cfg.context % page_rows == 0
+        mp = cfg.context // page_rows
+        tab = (torch.arange(cfg.batch * mp, dtype=torch.int32, device=dev).reshape(cfg.batch, mp) + 7 * (li + 1)) % (cfg.batch * mp)
+        B.slim_cache_destroy(lay.cache)
+        lay.cache = B.slim_cache_create_paged(lay.ctx, lay.k, cfg.batch * mp, page_rows, tab, cfg.batch, mp)
+        return tab
     q_all = torch.zeros((layers_n, cfg.batch, cfg.d), dtype=torch.bfloat16 if cfg.dtype == "bf16" else torch.float32,
                         device=dev)
     knew_all = torch.zeros_like(q_all)
@@ -304,6 +371,12 @@ def main():
         lay.set_path(path)
         W_Q, W_K, W_V, _, _ = synth.make_weights_torch(cfg.d, seed0 + li, dev)
         synth.fill_layer_torch(cfg, seed0 + li, W_Q, W_K, lengths, lay.k, q_all[li])
+        if args.paged:                      # move the drawn keys into the paged arrangement through slim_append_k
+            tmp = lay.k.clone()
+            paged_tables.append(make_paged(lay, args.paged, li))
+            lay.append_k(tmp, torch.zeros(cfg.batch, dtype=torch.int32, device=dev))
+            torch.cuda.synchronize()
+            del tmp
         want = (li == layers_n - 1)
         res, wkv = lay.set_weights(W_K.cpu().numpy(), W_V.cpu().numpy(), want_wkv=want)
         if want:
@@ -311,7 +384,7 @@ def main():
         assert res < 1e-8, f"W_KV residual {res}"
         for b in range(cfg.batch):          # the step re-appends the newest key row
             if lengths[b] > 0:
-                knew_all[li, b] = lay.k[b, int(lengths[b]) - 1]
+                knew_all[li, b] = seq_rows(li, lay, b, int(lengths[b]))[-1]
         del W_Q, W_K, W_V
         layers.append(lay)
     torch.cuda.synchronize()
@@ -408,7 +481,7 @@ def main():
             n = int(lengths[b])
             if n == 0:
                 continue
-            Kb = lay.k[b, :n].float().cpu().numpy().astype(np.float64)
+            Kb = seq_rows(layers_n - 1, lay, b, n).float().cpu().numpy().astype(np.float64)
             qb = q_all[-1, b].float().cpu().numpy().astype(np.float64)
             tt = time.perf_counter()
             ref = so.oracle_slim(qb, Kb, W_KV, cfg.H, cfg.rope_theta)
@@ -438,7 +511,8 @@ def main():
                        "parallelism": f"replicas x{world} (batch-sharded, no collective)",
                        "l2": "inputs larger than L2 (K-cache per step >> 126 MB)" if k_bytes_layer * layers_n > 2.6e8
                              else "K-cache per step fits L2: warm-cache number",
-                       "path": {1: "generic", 2: "tc"}[layers[0].query(B.SLIM_Q_PATH_IN_USE)]},
+                       "path": {1: "generic", 2: "tc"}[layers[0].query(B.SLIM_Q_PATH_IN_USE)],
+                       "cache": f"paged, {args.paged} rows per page" if args.paged else "contiguous"},
             "kcache_gbs": step_gbs, "kcache_frac_of_8000": step_gbs / 8000.0, "kcache_frac_of_measured": step_gbs / peak,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": ncu_traffic(args.config), "peak_kind": peak_kind, "kernel": "main decode kernel (per layer launch)",
