@@ -476,7 +476,6 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
     if (ctx->proj_ok) {
       float* o_part = reinterpret_cast<float*>(ws + L.o_part);
       e = slim_launch_proj(ctx, p, reinterpret_cast<unsigned char*>(ws + L.u_tiled), o_part, st);
-      if (e == cudaSuccess) e = slim_launch_sum_slices(o_part, o, p.batch * p.d, slim_proj_jsplit(ctx->d), st);
     } else {
       e = slim_launch_tail(ctx, p, st);
     }
@@ -577,7 +576,7 @@ long long slim_query(const slim_ctx* ctx, int key) {
   switch (key) {
     case SLIM_Q_PATH_IN_USE: return path;
     case SLIM_Q_LAUNCHES_PER_DECODE:              // main (tc: + exact redo; generic: scores + accum), then the tail
-      return 2 + (ctx->proj_ok ? 3 : 2);          // combine, projection, slice sum  |  combine+projection, slice sum
+      return 2 + 2;                               // combine, projection  |  combine+projection, slice sum
     case SLIM_Q_MAX_UNITS: return ctx->num_sms;   // + batch, known only per cache
     case SLIM_Q_NUM_SMS: return ctx->num_sms;
     case SLIM_Q_WORKERS: return path == SLIM_PATH_TC ? (ctx->tc_workers[1] > 0 ? ctx->tc_workers[1] : ctx->tc_workers[0]) : ctx->gen_workers;

@@ -16,8 +16,10 @@
 //                         N = 2 x 32) and the off-diagonal quadrants are ignored; for
 //                         d_k = 96 the accumulator rows 96..127 are ignored.
 //                         A CTA owns (head group, slice of the d rows of W_KV,h,
-//                         16-sequence group) and writes a projection slice that
-//                         slim_tail2_kernel sums in a fixed order.
+//                         16-sequence group); the CTAs of the row slices form a
+//                         cluster, leave their slice results in shared memory and
+//                         each adds, in slice order, a share of the output rows
+//                         through distributed shared memory (bitwise repeatable).
 //
 // Every mbarrier wait is bounded in time; a wait that runs out sets the device
 // status to SLIM_ERR_TIMEOUT and the CTA drains and exits.
@@ -139,7 +141,7 @@ slim_combine_kernel(const SlimDecodeParams p, unsigned char* __restrict__ u_tile
 
 __global__ void __launch_bounds__(128)
 slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned char* __restrict__ u_tiled,
-                    float* __restrict__ o_part, const ProjGeom g, const int d, const int d_k, const int batch,
+                    float* __restrict__ o, const ProjGeom g, const int d, const int d_k, const int batch,
                     int* status) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_u32 = smem_u32(smem_raw);
@@ -215,27 +217,38 @@ slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned cha
   }
   __syncwarp();
   // =========================== epilogue: all four warps ===========================
+  // This CTA's slice result [16 sequences][128 accumulator rows] goes to shared memory (the stage
+  // area is free once bar_done has completed); after a cluster barrier CTA r of the jsplit slices
+  // adds sequences [16 r / jsplit, 16 (r + 1) / jsplit) over all slices in slice order.
+  const int m = warp * 32 + lane;                             // accumulator row = TMEM lane
+  const int upper = g.hp == 2 ? (warp >> 1) : 0;              // d_k = 64: lanes 64..127 hold the second head
+  const int head = hg * g.hp + upper;
+  const int c = g.hp == 2 ? (m & 63) : m;
   {
     bool ok = mbar_wait<false>(bar_done, 0, s_abort, status);
     ok = __all_sync(0xffffffffu, ok);
+    uint32_t r[32];
+#pragma unroll
+    for (int n = 0; n < 32; ++n) r[n] = 0u;
     if (ok) {
       tc_fence_after();
-      const int m = warp * 32 + lane;                           // accumulator row = TMEM lane
-      const int upper = g.hp == 2 ? (warp >> 1) : 0;            // d_k = 64: lanes 64..127 hold the second head
-      const int head = hg * g.hp + upper;
-      const int c = g.hp == 2 ? (m & 63) : m;
-      uint32_t r[32];
       tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(32 * upper), r);
-      if (c < d_k) {
+    }
+    float* tile = reinterpret_cast<float*>(sm);
 #pragma unroll
-        for (int n = 0; n < PJ_BG; ++n) {
-          const int b = bg * PJ_BG + n;
-          if (b < batch)
-            o_part[((size_t)js * batch + b) * d + head * d_k + c] = __uint_as_float(r[n]) + __uint_as_float(r[PJ_BG + n]);
-        }
-      }
+    for (int n = 0; n < PJ_BG; ++n) tile[n * 128 + m] = __uint_as_float(r[n]) + __uint_as_float(r[PJ_BG + n]);
+  }
+  cluster_sync_all();
+  {
+    const int n_lo = (js * PJ_BG) / g.jsplit, n_hi = ((js + 1) * PJ_BG) / g.jsplit;
+    for (int n = n_lo; n < n_hi; ++n) {
+      const int b = bg * PJ_BG + n;
+      float a = 0.f;
+      for (int sl = 0; sl < g.jsplit; ++sl) a += ld_cluster_f32(mapa(base + (uint32_t)(n * 128 + m) * 4u, (uint32_t)sl));
+      if (b < batch && c < d_k) o[(size_t)b * d + head * d_k + c] = a;
     }
   }
+  cluster_sync_all();                                          // nobody leaves while its tile may still be read
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -307,7 +320,16 @@ cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, uns
   }
   CUtensorMap map;
   memcpy(&map, ctx->wmap, sizeof(map));
-  dim3 grid(g.hg, g.jsplit, g.nbg);
-  return slim_launch_pdl(slim_proj_tc_kernel, grid, dim3(128), proj_smem_bytes(g), st, map, (const unsigned char*)u_tiled, o_part,
-                         g, p.d, p.d_k, p.batch, p.status);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(g.hg, g.jsplit, g.nbg);
+  cfg.blockDim = dim3(128);
+  cfg.dynamicSmemBytes = proj_smem_bytes(g);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;            // the row slices of one output tile
+  attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = g.jsplit; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, slim_proj_tc_kernel, map, (const unsigned char*)u_tiled, p.o, g, p.d, p.d_k, p.batch, p.status);
 }
