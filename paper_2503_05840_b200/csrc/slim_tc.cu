@@ -184,7 +184,9 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
         }
       }
 
-      int it = 0, uc = 0;
+      // (st, kph): K stage and phase parity of tile `it`, stepped instead of divided
+      int it = 0, uc = 0, st = 0;
+      uint32_t kph = 0;
       bool ok = true;
       for (int gg = g_begin; gg < g_end && ok; ++uc) {
         const int b = slim_seq_of_tile(s_prefix, p.batch, gg);
@@ -221,9 +223,9 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
         for (int x = 0; x < 4; ++x) { Qa[x] = pack2(qh1[2 * x], qh1[2 * x + 1]); Qb[x] = pack2(qh2[2 * x], qh2[2 * x + 1]); }
         float mref = 0.f, lsum = 0.f;
 
-        for (int kt = 0; kt < ntile && ok; ++kt, ++it) {
+        for (int kt = 0; kt < ntile && ok; ++kt, ++it, st = (st + 1 == g.ns ? 0 : st + 1), kph ^= (st == 0)) {
           const int tile = tile0 + kt, t0 = tile * SLIM_TT;
-          const int st = it % g.ns, ps = it % TC_NP;
+          const int ps = it % TC_NP;
           const uint32_t kbase = k_stage0 + (uint32_t)st * g.stage_bytes;
           float sv = 0.f;
           if (scorer) {
@@ -239,9 +241,9 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
                 Qb[x] = pack2(qh1[2 * x] * s0 + qh2[2 * x] * c0, qh1[2 * x + 1] * s1 + qh2[2 * x + 1] * c1);
               }
             }
-            ok = mbar_wait<false>(bar_k_full + 8 * st, (it / g.ns) & 1, s_abort, p.status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+            // a wait that ran out is acted on after the vote below (until then the lanes only
+            // touch their own registers and this CTA's shared memory)
+            ok = mbar_wait<false>(bar_k_full + 8 * st, kph, s_abort, p.status);
             // rows at or beyond the sequence end must not reach the tensor core (0 x NaN)
             if (t0 + SLIM_TT > len) {
               const int nz = len - t0;
@@ -320,7 +322,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             const __nv_bfloat16 pb = __float2bfloat16_rn(pf);
             if ((jl % DUP) == 0) lsum += __bfloat162float(pb);
             // the P stage is free once the MMAs of tile it - TC_NP are done in both CTAs
-            ok = mbar_wait<false>(bar_p_empty + 8 * ps, ((it / TC_NP) & 1) ^ 1, s_abort, p.status);
+            ok = mbar_wait<false>(bar_p_empty + 8 * ps, ((it / TC_NP) & 1) ^ 1, s_abort, p.status) && ok;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             {
@@ -397,15 +399,15 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
     } else if (warp == producer_warp) {
       // =========================== TMA producer ===========================
       if (lane == 0) {
-        int it = 0;
+        int it = 0, st = 0;
+        uint32_t kph = 0;
         bool ok = true;
         for (int gg = g_begin; gg < g_end && ok;) {
           const int b = slim_seq_of_tile(s_prefix, p.batch, gg);
           const int seg_end = min(g_end, s_prefix[b + 1]);
           const int tile0 = gg - s_prefix[b], ntile = seg_end - gg;
-          for (int kt = 0; kt < ntile; ++kt, ++it) {
-            const int st = it % g.ns;
-            ok = mbar_wait<false>(bar_k_empty + 8 * st, ((it / g.ns) & 1) ^ 1, s_abort, p.status);
+          for (int kt = 0; kt < ntile; ++kt, ++it, st = (st + 1 == g.ns ? 0 : st + 1), kph ^= (st == 0)) {
+            ok = mbar_wait<false>(bar_k_empty + 8 * st, kph ^ 1, s_abort, p.status);
             if (!ok) break;
             mbar_arrive_expect_tx(bar_k_full + 8 * st, (uint32_t)g.stage_bytes);
             tma_load_3d(k_stage0 + (uint32_t)st * g.stage_bytes, &tmap, bar_k_full + 8 * st, 0,
@@ -426,7 +428,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
     } else if (warp == mma_warp) {
       // =========================== MMA issuer ===========================
       if (lane == 0) {
-        int it = 0, uc = 0;
+        int it = 0, uc = 0, st = 0;
         bool ok = true;
         // p_full of a tile completes on: this thread's arming arrival + the local score
         // warps' arrivals + 32 bytes per head shipped by the score warps of both CTAs
@@ -437,8 +439,8 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           const int b = slim_seq_of_tile(s_prefix, p.batch, gg);
           const int seg_end = min(g_end, s_prefix[b + 1]);
           const int ntile = seg_end - gg;
-          for (int kt = 0; kt < ntile; ++kt, ++it) {
-            const int st = it % g.ns, ps = it % TC_NP;
+          for (int kt = 0; kt < ntile; ++kt, ++it, st = (st + 1 == g.ns ? 0 : st + 1)) {
+            const int ps = it % TC_NP;
             // p_full alone is enough: every local score warp arrives on it after it has seen
             // k_full of this stage, so the keys have landed (and are ordered before this wait).
             ok = mbar_wait<true>(bar_p_full + 8 * ps, (it / TC_NP) & 1, s_abort, p.status);
