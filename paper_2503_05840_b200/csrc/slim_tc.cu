@@ -35,6 +35,16 @@
 // worker (CL = 1): the whole key row and all heads live in one SM, the P exchange stays local and
 // twice as many workers share the context.
 //
+// Two score-warp sets (SETS = 2, the narrow d_k = 64 shapes).  There a tile is so small that a score
+// warp's chain of dependent steps per tile (wait, shared-memory reads, dot products, shuffles,
+// exponent, staging, shipping), not its instruction count, sets the pace.  With two sets of score
+// warps, set s forms the probabilities of the tiles with kt mod 2 = s of every unit, so two tiles are
+// in the chain at once.  Every warp still waits on the barriers of the tiles it skips (each barrier
+// phase is seen in order by every waiter).  Set 0 owns the unit's first tile: it fixes m_ref and hands
+// it to set 1 through shared memory (barrier xm); set 1 hands its share of l back at the unit's end
+// (barrier xl); both hand-overs are strictly alternating, so the single slots are never overwritten
+// early.
+//
 // Softmax reference.  m_ref of a (unit, head) is the maximum argument of the
 // unit's first tile and is never changed, so the accumulator is never rescaled.
 // 2^(s - m_ref) is exact in relative terms for any exponent below 2^127; a later
@@ -69,8 +79,9 @@ struct TcGeom {
   int nch;          // 128-column chunks per CTA
   int nc64;         // 64-column TMA chunks per CTA
   int hl;           // heads per CTA
-  int nsw;          // score warps (tc_heads_per_warp heads each)
-  int nswl;         // launched score/epilogue warps = max(4, nsw)
+  int nsw;          // score warps of one set (tc_heads_per_warp heads each)
+  int sets;         // score-warp sets
+  int nswl;         // launched score/epilogue warps = max(4, nsw * sets)
   int ns;           // K stages
   int stage_bytes;  // 16 * dsl * 2
   int tmem_cols;    // power of two >= 32 * nch
@@ -80,17 +91,19 @@ struct TcGeom {
 // owns RT rows of the tile; 16 / RT row sets and JL lanes make one head.
 __host__ __device__ constexpr int tc_jl(int dk) { return dk / 16 <= 4 ? 4 : 8; }
 __host__ __device__ constexpr int tc_heads_per_warp(int dk, int rt) { return 32 / (tc_jl(dk) * (SLIM_TT / rt)); }
-__host__ __device__ constexpr int tc_threads(int dk, int rt, int cl) {
+constexpr int TC_SETS2_WARPS = 10;       // score warps of a two-set launch (both sets together), at most
+__host__ __device__ constexpr int tc_threads(int dk, int rt, int cl, int sets) {
   // up to 32 / cl heads per CTA, at least four score/epilogue warps, plus the producer and MMA warps
-  return 32 * (((32 / cl) / tc_heads_per_warp(dk, rt) < 4 ? 4 : (32 / cl) / tc_heads_per_warp(dk, rt)) + 2);
+  return sets == 2 ? 32 * (TC_SETS2_WARPS + 2)
+                   : 32 * (((32 / cl) / tc_heads_per_warp(dk, rt) < 4 ? 4 : (32 / cl) / tc_heads_per_warp(dk, rt)) + 2);
 }
 
 // ------------------------------------------------------------------ the kernel
 // EXT: the softmax arguments are read from p.ext_scores (X-cache scheme) instead of being
 // formed from the staged rows; the rest of the pipeline is the same.
-// CL: CTAs per worker (cluster size), 2 or 1.
-template <int DK, bool ROPE, int RT, bool EXT, int CL>
-__global__ void __launch_bounds__(tc_threads(DK, RT, CL), 1)
+// CL: CTAs per worker (cluster size), 2 or 1.  SETS: score-warp sets, 1 or 2.
+template <int DK, bool ROPE, int RT, bool EXT, int CL, int SETS>
+__global__ void __launch_bounds__(tc_threads(DK, RT, CL, SETS), 1)
 slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams p, const TcGeom g) {
   constexpr int PAIRS = DK / 2;                   // rotation pairs (j, j + DK/2) per head
   constexpr int OCT = PAIRS / 8;                  // 8-pair groups per head
@@ -112,10 +125,13 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   const uint32_t bar_k_full = bars, bar_k_empty = bars + 8 * TC_MAX_NS;
   const uint32_t bar_p_full = bars + 16 * TC_MAX_NS, bar_p_empty = bar_p_full + 8 * TC_NP;
   const uint32_t bar_u_full = bar_p_empty + 8 * TC_NP, bar_u_empty = bar_u_full + 8;
-  unsigned char* misc = sm + (bar_u_empty + 8 - base);
+  const uint32_t bar_xm = bar_u_empty + 8, bar_xl = bar_xm + 8;
+  unsigned char* misc = sm + (bar_xl + 8 - base);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc);
   volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 4);
-  int* s_prefix = reinterpret_cast<int*>(misc + 8);
+  float* s_xm = reinterpret_cast<float*>(misc + 8);          // m_ref per local head, set 0 -> set 1
+  float* s_xl = s_xm + 32;                                   // l per local head, set 1 -> set 0
+  int* s_prefix = reinterpret_cast<int*>(misc + 8 + 256);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t rank = cluster_ctarank();
@@ -130,6 +146,8 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
     for (int i = 0; i < TC_NP; ++i) { mbar_init(bar_p_full + 8 * i, 1 + g.nsw); mbar_init(bar_p_empty + 8 * i, CL); }
     mbar_init(bar_u_full, 1);
     mbar_init(bar_u_empty, nepi);
+    mbar_init(bar_xm, g.nsw);
+    mbar_init(bar_xl, g.nsw);
     *s_abort = 0;
     fence_mbar_init();
   }
@@ -159,9 +177,11 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   if (have_work) {
     if (warp < g.nswl) {
       // =========================== score / epilogue warps ===========================
-      const bool scorer = warp < g.nsw;
+      const bool scorer = warp < g.nsw * SETS;
+      const int wset = (SETS == 2 && warp >= g.nsw) ? 1 : 0;     // this warp's set
+      const int wis = warp - wset * g.nsw;                       // warp within the set
       const int jl = lane % JL, rp = (lane / JL) % RP, hw = lane / HL;
-      const int hl = HW * warp + hw;                             // head within this CTA
+      const int hl = HW * wis + hw;                              // head within this CTA
       const bool head_valid = scorer && hl < g.hl;
       const bool active = head_valid && jl < OCT;
       const int my_n = (int)rank * g.hl + hl;                    // global head
@@ -222,14 +242,34 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
 #pragma unroll
         for (int x = 0; x < 4; ++x) { Qa[x] = pack2(qh1[2 * x], qh1[2 * x + 1]); Qb[x] = pack2(qh2[2 * x], qh2[2 * x + 1]); }
         float mref = 0.f, lsum = 0.f;
+        bool have_mref = false;
 
         for (int kt = 0; kt < ntile && ok; ++kt, ++it, st = (st + 1 == g.ns ? 0 : st + 1), kph ^= (st == 0)) {
           const int tile = tile0 + kt, t0 = tile * SLIM_TT;
           const int ps = it % TC_NP;
           const uint32_t kbase = k_stage0 + (uint32_t)st * g.stage_bytes;
           float sv = 0.f;
-          if (scorer) {
-            if (ROPE && active && (kt % TC_RESEED) == 0) {
+          // set s forms the probabilities of the tiles with kt mod 2 = s and only waits on the others
+          const bool mine = SETS == 1 || (kt & 1) == wset;
+          if (scorer && !mine) {
+            ok = mbar_wait<false>(bar_k_full + 8 * st, kph, s_abort, p.status);
+            ok = mbar_wait<false>(bar_p_empty + 8 * ps, ((it / TC_NP) & 1) ^ 1, s_abort, p.status) && ok;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (ROPE && active && SETS == 2) {
+              // keep the stepped rotation in step with the tiles: RT row steps of RP rows = one tile
+#pragma unroll
+              for (int i = 0; i < RT; ++i)
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                  const f32x2 na = fma2(Qb[x], stn[x], mul2(Qa[x], stc[x]));
+                  Qb[x] = fma2(Qa[x], sts[x], mul2(Qb[x], stc[x]));
+                  Qa[x] = na;
+                }
+            }
+          }
+          if (scorer && mine) {
+            if (ROPE && active && ((kt >> (SETS - 1)) % (TC_RESEED / SETS)) == 0) {
               // exact Q at this thread's first row of the tile (position t0 + rp)
 #pragma unroll
               for (int x = 0; x < 4; ++x) {
@@ -247,7 +287,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             // rows at or beyond the sequence end must not reach the tensor core (0 x NaN)
             if (t0 + SLIM_TT > len) {
               const int nz = len - t0;
-              for (int c64 = warp; c64 < g.nc64; c64 += g.nsw)
+              for (int c64 = wis; c64 < g.nc64; c64 += g.nsw)
                 for (int e = lane; e < (SLIM_TT - nz) * 8; e += 32)
                   sts128_zero(kbase + (uint32_t)c64 * 2048u + (uint32_t)(nz + (e >> 3)) * 128u + (uint32_t)(e & 7) * 16u);
             }
@@ -315,6 +355,16 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
               for (int o = 1; o < HL; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
               mref = mx;
               lsum = 0.f;
+              if (SETS == 2) {
+                if (head_valid && (lane % HL) == 0) s_xm[hl] = mref;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_xm);
+              }
+            } else if (SETS == 2 && kt == 1) {
+              ok = mbar_wait<false>(bar_xm, uc & 1, s_abort, p.status) && ok;
+              have_mref = true;
+              mref = head_valid ? s_xm[hl] : 0.f;
+              lsum = 0.f;
             }
             float x = sv - mref;
             if (valid && x > TC_XMAX) { p.unit_flags[2 * unit + (int)rank] = 1; *p.any_flag = 1; x = TC_XMAX; }
@@ -328,12 +378,12 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             {
               // stage this warp's probabilities in the K-major order of the P tile, then ship
               // them in 16-byte pieces (8 rows of one head) to both CTAs
-              const uint32_t stg = stg0 + (uint32_t)warp * 128u + (uint32_t)(it & 1) * 64u;
+              const uint32_t stg = stg0 + (uint32_t)warp * 128u + (uint32_t)((kt >> (SETS - 1)) & 1) * 64u;
               if ((jl % DUP) == 0) sts_u16(stg + (uint32_t)(hw * 16 + my_row) * 2u, __bfloat16_as_ushort(pb));
               __syncwarp();
               if (lane < 4 * HW) {
                 const int hsel = lane >> 2, half = (lane >> 1) & 1, dest = lane & 1;
-                const int hl_s = HW * warp + hsel;
+                const int hl_s = HW * wis + hsel;
                 if (hl_s < g.hl && dest < CL) {
                   const uint4 pv = lds128(stg + (uint32_t)(hsel * 16 + half * 8) * 2u);
                   const int n_s = (int)rank * g.hl + hl_s;
@@ -356,7 +406,21 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
         if (scorer) {
 #pragma unroll
           for (int o = 1; o < HL; o <<= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
-          if (head_valid && (lane % HL) == 0) {
+          if (SETS == 2) {
+            if (wset == 1) {
+              // a unit of one tile never showed m_ref to this set: take the hand-over all the same
+              if (!have_mref) ok = mbar_wait<false>(bar_xm, uc & 1, s_abort, p.status);
+              if (head_valid && (lane % HL) == 0) s_xl[hl] = ntile > 1 ? lsum : 0.f;
+              __syncwarp();
+              if (lane == 0) mbar_arrive(bar_xl);
+            } else {
+              ok = mbar_wait<false>(bar_xl, uc & 1, s_abort, p.status);
+              if (head_valid) lsum += s_xl[hl];
+            }
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+          }
+          if (wset == 0 && head_valid && (lane % HL) == 0) {
             p.part_m[(size_t)unit * p.H + my_n] = mref;
             p.part_l[(size_t)unit * p.H + my_n] = lsum;
           }
@@ -475,16 +539,17 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
 }
 
 // ------------------------------------------------------------------ host side
-TcGeom make_geom(int d, int H, int d_k, int rt, int cl, int smem_limit) {
+TcGeom make_geom(int d, int H, int d_k, int rt, int cl, int sets, int smem_limit) {
   TcGeom g;
   g.cl = cl;
+  g.sets = sets;
   g.dsl = d / cl;
   g.nch = g.dsl / 128;
   g.nc64 = g.dsl / 64;
   g.hl = H / cl;
   const int hw = tc_heads_per_warp(d_k, rt);
   g.nsw = (g.hl + hw - 1) / hw;
-  g.nswl = g.nsw < 4 ? 4 : g.nsw;
+  g.nswl = g.nsw * sets < 4 ? 4 : g.nsw * sets;
   g.stage_bytes = SLIM_TT * g.dsl * 2;
   int ns = (smem_limit - 16 * 1024) / g.stage_bytes;
   g.ns = ns > TC_MAX_NS ? TC_MAX_NS : ns;
@@ -495,13 +560,23 @@ TcGeom make_geom(int d, int H, int d_k, int rt, int cl, int smem_limit) {
 }
 
 size_t tc_smem_bytes(const TcGeom& g, int batch) {
-  size_t need = 1024 + (size_t)g.ns * g.stage_bytes + TC_NP * TC_P_BYTES + TC_MAX_SW * 128 + 16 * TC_MAX_NS + 16 * TC_NP + 16 + 8 +
+  size_t need = 1024 + (size_t)g.ns * g.stage_bytes + TC_NP * TC_P_BYTES + TC_MAX_SW * 128 + 16 * TC_MAX_NS + 16 * TC_NP + 32 + 8 + 256 +
                 sizeof(int) * (batch + 1) + 64;
   const size_t floor_bytes = 120 * 1024;         // one CTA per SM: tensor memory is not shared
   return need < floor_bytes ? floor_bytes : need;
 }
 
 typedef void (*tc_kernel_t)(const CUtensorMap, const SlimDecodeParams, const TcGeom);
+
+// Two score-warp sets where a tile is small (d_k = 64, scores formed in the kernel, CTA pair) and both
+// sets fit the block.  SLIM_TC_SETS=1 switches them off for comparisons.
+int tc_sets(int H, int d_k, int rt, bool ext, int cl) {
+  const char* e = getenv("SLIM_TC_SETS");
+  if (e && atoi(e) == 1) return 1;
+  if (d_k != 64 || rt != 4 || ext || cl != 2) return 1;
+  const int hw = tc_heads_per_warp(d_k, rt), nsw = (H / cl + hw - 1) / hw;
+  return 2 * nsw <= TC_SETS2_WARPS ? 2 : 1;
+}
 
 // Rows per thread and tile.  Measured on the d = 4096 / 32-head shape: 8 rows per
 // thread (8 score warps) beats 4 rows (16 warps); the stepped query rotation is
@@ -524,26 +599,30 @@ bool tc_cl_ok(int d, int H, int d_k, bool rope, int cl) {
 }
 
 template <int DK, bool ROPE, int RT>
-tc_kernel_t pick_ext_cl(bool ext, int cl) {
+tc_kernel_t pick_ext_cl(bool ext, int cl, int sets) {
+  if (sets == 2) {
+    if constexpr (DK == 64 && RT == 4) return (!ext && cl == 2) ? slim_tc_kernel<DK, ROPE, RT, false, 2, 2> : nullptr;
+    else return nullptr;
+  }
   if (cl == 1) {
-    if constexpr (DK == 64 && !ROPE && RT == 4) return ext ? slim_tc_kernel<DK, ROPE, RT, true, 1> : slim_tc_kernel<DK, ROPE, RT, false, 1>;
+    if constexpr (DK == 64 && !ROPE && RT == 4) return ext ? slim_tc_kernel<DK, ROPE, RT, true, 1, 1> : slim_tc_kernel<DK, ROPE, RT, false, 1, 1>;
     else return nullptr;
   }
   if (ext) {
-    if constexpr (!ROPE) return slim_tc_kernel<DK, ROPE, RT, true, 2>;
+    if constexpr (!ROPE) return slim_tc_kernel<DK, ROPE, RT, true, 2, 1>;
     else return nullptr;
   }
-  return slim_tc_kernel<DK, ROPE, RT, false, 2>;
+  return slim_tc_kernel<DK, ROPE, RT, false, 2, 1>;
 }
 
-tc_kernel_t pick_kernel(int d_k, bool rope, int rt, bool ext, int cl) {
+tc_kernel_t pick_kernel(int d_k, bool rope, int rt, bool ext, int cl, int sets) {
   switch (d_k * 16 + rt) {
-    case 64 * 16 + 2: return rope ? pick_ext_cl<64, true, 2>(ext, cl) : pick_ext_cl<64, false, 2>(ext, cl);
-    case 64 * 16 + 4: return rope ? pick_ext_cl<64, true, 4>(ext, cl) : pick_ext_cl<64, false, 4>(ext, cl);
-    case 96 * 16 + 4: return rope ? pick_ext_cl<96, true, 4>(ext, cl) : pick_ext_cl<96, false, 4>(ext, cl);
-    case 96 * 16 + 8: return rope ? pick_ext_cl<96, true, 8>(ext, cl) : pick_ext_cl<96, false, 8>(ext, cl);
-    case 128 * 16 + 4: return rope ? pick_ext_cl<128, true, 4>(ext, cl) : pick_ext_cl<128, false, 4>(ext, cl);
-    case 128 * 16 + 8: return rope ? pick_ext_cl<128, true, 8>(ext, cl) : pick_ext_cl<128, false, 8>(ext, cl);
+    case 64 * 16 + 2: return rope ? pick_ext_cl<64, true, 2>(ext, cl, sets) : pick_ext_cl<64, false, 2>(ext, cl, sets);
+    case 64 * 16 + 4: return rope ? pick_ext_cl<64, true, 4>(ext, cl, sets) : pick_ext_cl<64, false, 4>(ext, cl, sets);
+    case 96 * 16 + 4: return rope ? pick_ext_cl<96, true, 4>(ext, cl, sets) : pick_ext_cl<96, false, 4>(ext, cl, sets);
+    case 96 * 16 + 8: return rope ? pick_ext_cl<96, true, 8>(ext, cl, sets) : pick_ext_cl<96, false, 8>(ext, cl, sets);
+    case 128 * 16 + 4: return rope ? pick_ext_cl<128, true, 4>(ext, cl, sets) : pick_ext_cl<128, false, 4>(ext, cl, sets);
+    case 128 * 16 + 8: return rope ? pick_ext_cl<128, true, 8>(ext, cl, sets) : pick_ext_cl<128, false, 8>(ext, cl, sets);
     default: return nullptr;
   }
 }
@@ -580,9 +659,10 @@ int slim_tc_shape_ok(int d, int H, int d_k, int dtype, int rope, int cl) {
 int slim_tc_workers(const slim_ctx* ctx, int cl) {
   const int rt = tc_rows_per_thread(ctx->d_k);
   const bool rope = ctx->rope_theta != 0.0;
-  tc_kernel_t kern = pick_kernel(ctx->d_k, rope, rt, false, cl);
+  const int sets = tc_sets(ctx->H, ctx->d_k, rt, false, cl);
+  tc_kernel_t kern = pick_kernel(ctx->d_k, rope, rt, false, cl, sets);
   if (!kern) return 0;
-  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, rt, cl, TC_SMEM_LIMIT);
+  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, rt, cl, sets, TC_SMEM_LIMIT);
   if (g.ns < 2) return 0;
   const size_t smem = tc_smem_bytes(g, SLIM_MAX_BATCH);
   if (smem > (size_t)TC_SMEM_LIMIT) return 0;
@@ -632,7 +712,7 @@ cudaError_t slim_tmap_encode_3d(void* out_map, void* base, const unsigned long l
 }
 
 cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c, int cl) {
-  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, tc_rows_per_thread(ctx->d_k), cl, TC_SMEM_LIMIT);
+  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, tc_rows_per_thread(ctx->d_k), cl, 1, TC_SMEM_LIMIT);
   // dim0: 64 contiguous elements; dim1: cache rows (stride d elements); dim2: 64-column chunks
   const unsigned long long dims[3] = {64, (unsigned long long)c->total_rows, (unsigned long long)(ctx->d / 64)};
   const unsigned long long strides[2] = {(unsigned long long)ctx->d * 2, 128};
@@ -644,13 +724,14 @@ cudaError_t slim_launch_tc(const slim_ctx* ctx, const slim_cache* c, const SlimD
   const int rt = tc_rows_per_thread(ctx->d_k);
   const bool ext = p.ext_scores != nullptr;
   const int cl = p.cl;
-  tc_kernel_t kern = pick_kernel(ctx->d_k, ctx->rope_theta != 0.0, rt, ext, cl);
+  const int sets = tc_sets(ctx->H, ctx->d_k, rt, ext, cl);
+  tc_kernel_t kern = pick_kernel(ctx->d_k, ctx->rope_theta != 0.0, rt, ext, cl, sets);
   if (!kern || cl < 1 || cl > 2 || !c->has_tmap[cl - 1]) return cudaErrorNotSupported;
   if (ext) {
     cudaError_t ea = cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_LIMIT);
     if (ea != cudaSuccess) return ea;
   }
-  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, rt, cl, TC_SMEM_LIMIT);
+  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, rt, cl, sets, TC_SMEM_LIMIT);
   const size_t smem = tc_smem_bytes(g, p.batch);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(cl * p.workers);

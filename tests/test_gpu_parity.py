@@ -94,6 +94,14 @@ def test_single_sequence_lengths(T):
     _run_host_case(cfg, L)
 
 
+def test_long_sequence_narrow_heads_rope():
+    """d_k = 64 with RoPE and one long sequence: every worker walks dozens of tiles of one unit, so the
+    two score-warp sets alternate over many tiles and the stepped query rotation is re-seeded."""
+    cfg = synth.SlimConfig("long-narrow", 256, 4, 64, 1, 100000, 1, 1.0e4, "bf16")
+    L = synth.make_layer(cfg, 4242, lengths=np.array([100000], dtype=np.int32))
+    _run_host_case(cfg, L)
+
+
 def test_config0_whisper_tiny_shape_full():
     cfg = synth.CONFIGS[0]
     _run_host_case(cfg, synth.make_layer(cfg, synth.layer_seed(0, 0)))
