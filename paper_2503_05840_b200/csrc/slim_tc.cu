@@ -66,7 +66,6 @@
 namespace {
 using namespace slim_ptx;
 
-constexpr int TC_NP = 4;                 // P-tile stages
 constexpr int TC_P_BYTES = 1024;         // [32 heads][16 rows] bf16
 constexpr int TC_MAX_NS = 8;             // K stages
 constexpr int TC_MAX_SW = 16;            // score warps
@@ -120,11 +119,11 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   unsigned char* sm = smem_raw + (base - raw_u32);
   const uint32_t k_stage0 = base;
   const uint32_t p_stage0 = base + (uint32_t)g.ns * g.stage_bytes;
-  const uint32_t stg0 = p_stage0 + TC_NP * TC_P_BYTES;            // per-warp P staging: 2 x 64 B
+  const uint32_t stg0 = p_stage0 + TC_MAX_NS * TC_P_BYTES;            // per-warp P staging: 2 x 64 B
   const uint32_t bars = stg0 + TC_MAX_SW * 128;
   const uint32_t bar_k_full = bars, bar_k_empty = bars + 8 * TC_MAX_NS;
-  const uint32_t bar_p_full = bars + 16 * TC_MAX_NS, bar_p_empty = bar_p_full + 8 * TC_NP;
-  const uint32_t bar_u_full = bar_p_empty + 8 * TC_NP, bar_u_empty = bar_u_full + 8;
+  const uint32_t bar_p_full = bars + 16 * TC_MAX_NS, bar_p_empty = bar_p_full + 8 * TC_MAX_NS;
+  const uint32_t bar_u_full = bar_p_empty + 8 * TC_MAX_NS, bar_u_empty = bar_u_full + 8;
   const uint32_t bar_xm = bar_u_empty + 8, bar_xl = bar_xm + 8;
   unsigned char* misc = sm + (bar_xl + 8 - base);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc);
@@ -142,8 +141,14 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   const int nepi = (g.nswl / 4) * 4;              // warps that drain the accumulator at a unit's end
   if (tid == 0) {
     prefetch_tensormap(&tmap);
-    for (int i = 0; i < g.ns; ++i) { mbar_init(bar_k_full + 8 * i, 1); mbar_init(bar_k_empty + 8 * i, g.nsw + 1); }
-    for (int i = 0; i < TC_NP; ++i) { mbar_init(bar_p_full + 8 * i, 1 + g.nsw); mbar_init(bar_p_empty + 8 * i, CL); }
+    // Stage i holds the keys AND the probabilities of the tiles it, it + ns, ...: one commit of the
+    // MMA thread (p_empty, to both CTAs) frees both.  k_empty counts the score warps that are done
+    // reading the keys; p_full counts the local score warps, each of which also announces the bytes
+    // that it and its twin in the other CTA ship into this CTA's P tile.
+    for (int i = 0; i < g.ns; ++i) {
+      mbar_init(bar_k_full + 8 * i, 1); mbar_init(bar_k_empty + 8 * i, g.nsw);
+      mbar_init(bar_p_full + 8 * i, g.nsw); mbar_init(bar_p_empty + 8 * i, CL);
+    }
     mbar_init(bar_u_full, 1);
     mbar_init(bar_u_empty, nepi);
     mbar_init(bar_xm, g.nsw);
@@ -151,7 +156,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
     *s_abort = 0;
     fence_mbar_init();
   }
-  for (int i = tid; i < TC_NP * TC_P_BYTES / 16; i += blockDim.x) sts128_zero(p_stage0 + 16 * i);
+  for (int i = tid; i < TC_MAX_NS * TC_P_BYTES / 16; i += blockDim.x) sts128_zero(p_stage0 + 16 * i);
   if (warp == mma_warp) tmem_alloc(smem_u32(s_tmem), (uint32_t)g.tmem_cols);
   // Cluster-wide rendezvous first, while nothing is in flight (a cluster barrier that has
   // to wait behind outstanding TMA loads costs several microseconds): after it the peer's
@@ -194,6 +199,9 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
         koff[hf] = (uint32_t)(col >> 6) * 2048u;
         kunit[hf] = (uint32_t)((col & 63) >> 3);
       }
+      // bytes that this warp and its twin in the other CTA(s) ship into one P tile: 32 per head
+      const int nvalid = min(HW, max(g.hl - HW * wis, 0));
+      const uint32_t p_bytes_w = (uint32_t)(CL * 32 * nvalid);
       // e^{i RP theta}: one step of this thread's rows
       f32x2 stc[4], sts[4], stn[4];
       if (ROPE && active) {
@@ -246,14 +254,13 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
 
         for (int kt = 0; kt < ntile && ok; ++kt, ++it, st = (st + 1 == g.ns ? 0 : st + 1), kph ^= (st == 0)) {
           const int tile = tile0 + kt, t0 = tile * SLIM_TT;
-          const int ps = it % TC_NP;
           const uint32_t kbase = k_stage0 + (uint32_t)st * g.stage_bytes;
           float sv = 0.f;
           // set s forms the probabilities of the tiles with kt mod 2 = s and only waits on the others
           const bool mine = SETS == 1 || (kt & 1) == wset;
           if (scorer && !mine) {
             ok = mbar_wait<false>(bar_k_full + 8 * st, kph, s_abort, p.status);
-            ok = mbar_wait<false>(bar_p_empty + 8 * ps, ((it / TC_NP) & 1) ^ 1, s_abort, p.status) && ok;
+            ok = mbar_wait<false>(bar_p_empty + 8 * st, kph ^ 1, s_abort, p.status) && ok;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             if (ROPE && active && SETS == 2) {
@@ -371,8 +378,8 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             const float pf = valid ? ex2_approx(x) : 0.f;
             const __nv_bfloat16 pb = __float2bfloat16_rn(pf);
             if ((jl % DUP) == 0) lsum += __bfloat162float(pb);
-            // the P stage is free once the MMAs of tile it - TC_NP are done in both CTAs
-            ok = mbar_wait<false>(bar_p_empty + 8 * ps, ((it / TC_NP) & 1) ^ 1, s_abort, p.status) && ok;
+            // the P stage is free once the MMAs of tile it - ns are done in both CTAs
+            ok = mbar_wait<false>(bar_p_empty + 8 * st, kph ^ 1, s_abort, p.status) && ok;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             {
@@ -387,8 +394,8 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
                 if (hl_s < g.hl && dest < CL) {
                   const uint4 pv = lds128(stg + (uint32_t)(hsel * 16 + half * 8) * 2u);
                   const int n_s = (int)rank * g.hl + hl_s;
-                  const uint32_t dst = p_stage0 + (uint32_t)ps * TC_P_BYTES + p_offset(n_s & 31, half * 8);
-                  st_async_v4(mapa(dst, dest), pv, mapa(bar_p_full + 8 * ps, dest));
+                  const uint32_t dst = p_stage0 + (uint32_t)st * TC_P_BYTES + p_offset(n_s & 31, half * 8);
+                  st_async_v4(mapa(dst, dest), pv, mapa(bar_p_full + 8 * st, dest));
                 }
               }
             }
@@ -396,7 +403,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             // MMA thread, whose proxy fence orders it before the tensor-core reads.
             __syncwarp();
             if (lane == 0) {
-              mbar_arrive(bar_p_full + 8 * ps);
+              mbar_arrive_expect_tx(bar_p_full + 8 * st, p_bytes_w);
               mbar_arrive(bar_k_empty + 8 * st);
             }
           }
@@ -471,7 +478,9 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           const int seg_end = min(g_end, s_prefix[b + 1]);
           const int tile0 = gg - s_prefix[b], ntile = seg_end - gg;
           for (int kt = 0; kt < ntile; ++kt, ++it, st = (st + 1 == g.ns ? 0 : st + 1), kph ^= (st == 0)) {
-            ok = mbar_wait<false>(bar_k_empty + 8 * st, kph ^ 1, s_abort, p.status);
+            // free once the score warps have read the keys and the tensor core has consumed them
+            ok = mbar_wait<false>(bar_k_empty + 8 * st, kph ^ 1, s_abort, p.status) &&
+                 mbar_wait<false>(bar_p_empty + 8 * st, kph ^ 1, s_abort, p.status);
             if (!ok) break;
             mbar_arrive_expect_tx(bar_k_full + 8 * st, (uint32_t)g.stage_bytes);
             tma_load_3d(k_stage0 + (uint32_t)st * g.stage_bytes, &tmap, bar_k_full + 8 * st, 0,
@@ -493,32 +502,27 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
       // =========================== MMA issuer ===========================
       if (lane == 0) {
         int it = 0, uc = 0, st = 0;
+        uint32_t kph = 0;
         bool ok = true;
-        // p_full of a tile completes on: this thread's arming arrival + the local score
-        // warps' arrivals + 32 bytes per head shipped by the score warps of both CTAs
-        const int total_it = g_end - g_begin;
-        const uint32_t p_bytes = (uint32_t)p.H * 32u;
-        for (int i = 0; i < TC_NP && i < total_it; ++i) mbar_arrive_expect_tx(bar_p_full + 8 * i, p_bytes);
+        // p_full of a tile completes on the local score warps' arrivals + the 32 bytes per head
+        // shipped by the score warps of both CTAs (announced by the local ones)
         for (int gg = g_begin; gg < g_end && ok; ++uc) {
           const int b = slim_seq_of_tile(s_prefix, p.batch, gg);
           const int seg_end = min(g_end, s_prefix[b + 1]);
           const int ntile = seg_end - gg;
-          for (int kt = 0; kt < ntile; ++kt, ++it, st = (st + 1 == g.ns ? 0 : st + 1)) {
-            const int ps = it % TC_NP;
+          for (int kt = 0; kt < ntile; ++kt, ++it, st = (st + 1 == g.ns ? 0 : st + 1), kph ^= (st == 0)) {
             // p_full alone is enough: every local score warp arrives on it after it has seen
             // k_full of this stage, so the keys have landed (and are ordered before this wait).
-            ok = mbar_wait<true>(bar_p_full + 8 * ps, (it / TC_NP) & 1, s_abort, p.status);
+            ok = mbar_wait<true>(bar_p_full + 8 * st, kph, s_abort, p.status);
             if (ok && kt == 0 && uc > 0) ok = mbar_wait<false>(bar_u_empty, (uc - 1) & 1, s_abort, p.status);
             if (!ok) break;
             fence_proxy_async_smem();        // P pieces and zero-filled key rows -> tensor-core reads
             tc_fence_after();
-            const uint64_t bd = desc_b(p_stage0 + (uint32_t)ps * TC_P_BYTES);
+            const uint64_t bd = desc_b(p_stage0 + (uint32_t)st * TC_P_BYTES);
             const uint32_t kbase = k_stage0 + (uint32_t)st * g.stage_bytes;
             for (int c = 0; c < g.nch; ++c)
               umma_bf16(tmem_base + (uint32_t)(c * 32), desc_a(kbase + (uint32_t)c * 4096u), bd, umma_idesc(32), kt > 0 ? 1u : 0u);
-            umma_commit(bar_k_empty + 8 * st);
-            if (CL == 2) umma_commit_pair(bar_p_empty + 8 * ps); else umma_commit(bar_p_empty + 8 * ps);
-            if (it + TC_NP < total_it) mbar_arrive_expect_tx(bar_p_full + 8 * ps, p_bytes);
+            if (CL == 2) umma_commit_pair(bar_p_empty + 8 * st); else umma_commit(bar_p_empty + 8 * st);
             if (kt == ntile - 1) umma_commit(bar_u_full);
           }
           gg = seg_end;
@@ -560,7 +564,7 @@ TcGeom make_geom(int d, int H, int d_k, int rt, int cl, int sets, int smem_limit
 }
 
 size_t tc_smem_bytes(const TcGeom& g, int batch) {
-  size_t need = 1024 + (size_t)g.ns * g.stage_bytes + TC_NP * TC_P_BYTES + TC_MAX_SW * 128 + 16 * TC_MAX_NS + 16 * TC_NP + 32 + 8 + 256 +
+  size_t need = 1024 + (size_t)g.ns * g.stage_bytes + TC_MAX_NS * TC_P_BYTES + TC_MAX_SW * 128 + 32 * TC_MAX_NS + 32 + 8 + 256 +
                 sizeof(int) * (batch + 1) + 64;
   const size_t floor_bytes = 120 * 1024;         // one CTA per SM: tensor memory is not shared
   return need < floor_bytes ? floor_bytes : need;
