@@ -506,6 +506,11 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
         bool ok = true;
         // p_full of a tile completes on the local score warps' arrivals + the 32 bytes per head
         // shipped by the score warps of both CTAs (announced by the local ones)
+        // operand descriptors of stage 0 as (low, high) words; a stage or a chunk further on only
+        // moves the start-address field (all of shared memory stays below its 18-bit range)
+        const uint64_t ad0 = desc_a(k_stage0), bd0 = desc_b(p_stage0);
+        const uint32_t a_lo = (uint32_t)ad0, a_hi = (uint32_t)(ad0 >> 32), b_lo = (uint32_t)bd0, b_hi = (uint32_t)(bd0 >> 32);
+        const uint32_t a_step = (uint32_t)g.stage_bytes >> 4;
         for (int gg = g_begin; gg < g_end && ok; ++uc) {
           const int b = slim_seq_of_tile(s_prefix, p.batch, gg);
           const int seg_end = min(g_end, s_prefix[b + 1]);
@@ -518,10 +523,16 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             if (!ok) break;
             fence_proxy_async_smem();        // P pieces and zero-filled key rows -> tensor-core reads
             tc_fence_after();
-            const uint64_t bd = desc_b(p_stage0 + (uint32_t)st * TC_P_BYTES);
-            const uint32_t kbase = k_stage0 + (uint32_t)st * g.stage_bytes;
-            for (int c = 0; c < g.nch; ++c)
-              umma_bf16(tmem_base + (uint32_t)(c * 32), desc_a(kbase + (uint32_t)c * 4096u), bd, umma_idesc(32), kt > 0 ? 1u : 0u);
+            // One instruction per 128-column chunk.  The tensor core takes one of these every ~65
+            // clocks; this thread's own instructions between two of them must stay below that, so
+            // the descriptors are stepped as 32-bit words instead of being rebuilt.
+            {
+              const uint32_t acc = kt > 0 ? 1u : 0u;
+              uint32_t al = a_lo + (uint32_t)st * a_step, dcol = tmem_base;
+              const uint32_t bl = b_lo + (uint32_t)st * (TC_P_BYTES >> 4);
+              for (int c = 0; c < g.nch; ++c, al += 4096u >> 4, dcol += 32u)
+                umma_bf16_words(dcol, al, a_hi, bl, b_hi, umma_idesc(32), acc);
+            }
             if (CL == 2) umma_commit_pair(bar_p_empty + 8 * st); else umma_commit(bar_p_empty + 8 * st);
             if (kt == ntile - 1) umma_commit(bar_u_full);
           }
