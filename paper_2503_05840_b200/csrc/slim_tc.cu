@@ -38,12 +38,11 @@
 // Two score-warp sets (SETS = 2, the narrow d_k = 64 shapes).  There a tile is so small that a score
 // warp's chain of dependent steps per tile (wait, shared-memory reads, dot products, shuffles,
 // exponent, staging, shipping), not its instruction count, sets the pace.  With two sets of score
-// warps, set s forms the probabilities of the tiles with kt mod 2 = s of every unit, so two tiles are
-// in the chain at once.  Every warp still waits on the barriers of the tiles it skips (each barrier
-// phase is seen in order by every waiter).  Set 0 owns the unit's first tile: it fixes m_ref and hands
-// it to set 1 through shared memory (barrier xm); set 1 hands its share of l back at the unit's end
-// (barrier xl); both hand-overs are strictly alternating, so the single slots are never overwritten
-// early.
+// warps, set s forms the probabilities of the worker's tiles number s, s + 2, ... (counted through all
+// its units), so two tiles are in the chain at once and a set only ever meets the stages of its own
+// parity.  The set that has a unit's first tile fixes m_ref and hands it to the other through shared
+// memory (barrier xm); the other hands its share of l back at the unit's end (barrier xl).  Both
+// sets wait on both barriers in every unit, which orders the re-use of the two slots.
 //
 // Softmax reference.  m_ref of a (unit, head) is the maximum argument of the
 // unit's first tile and is never changed, so the accumulator is never rescaled.
@@ -212,8 +211,11 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
         }
       }
 
-      // (st, kph): K stage and phase parity of tile `it`, stepped instead of divided
-      int it = 0, uc = 0, st = 0;
+      // Tile number `it` of the worker (counted through all its units) belongs to set it mod SETS, so
+      // a set meets only the stages of its own parity (ns is even then) and sees each of their
+      // barrier phases in order.  (st, kph): stage and phase parity of this set's next tile it_own,
+      // stepped instead of divided.
+      int it_base = 0, it_own = wset, uc = 0, st = wset;
       uint32_t kph = 0;
       bool ok = true;
       for (int gg = g_begin; gg < g_end && ok; ++uc) {
@@ -250,32 +252,16 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
 #pragma unroll
         for (int x = 0; x < 4; ++x) { Qa[x] = pack2(qh1[2 * x], qh1[2 * x + 1]); Qb[x] = pack2(qh2[2 * x], qh2[2 * x + 1]); }
         float mref = 0.f, lsum = 0.f;
-        bool have_mref = false;
+        // this set's first tile of the unit; the set that has the unit's first tile owns m_ref
+        const int kt0 = SETS == 1 ? 0 : it_own - it_base;
+        const bool owner = kt0 == 0;
 
-        for (int kt = 0; kt < ntile && ok; ++kt, ++it, st = (st + 1 == g.ns ? 0 : st + 1), kph ^= (st == 0)) {
+        for (int kt = kt0; kt < ntile && ok; kt += SETS, it_own += SETS, st += SETS) {
+          if (st >= g.ns) { st -= g.ns; kph ^= 1u; }
           const int tile = tile0 + kt, t0 = tile * SLIM_TT;
           const uint32_t kbase = k_stage0 + (uint32_t)st * g.stage_bytes;
           float sv = 0.f;
-          // set s forms the probabilities of the tiles with kt mod 2 = s and only waits on the others
-          const bool mine = SETS == 1 || (kt & 1) == wset;
-          if (scorer && !mine) {
-            ok = mbar_wait<false>(bar_k_full + 8 * st, kph, s_abort, p.status);
-            ok = mbar_wait<false>(bar_p_empty + 8 * st, kph ^ 1, s_abort, p.status) && ok;
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            if (ROPE && active && SETS == 2) {
-              // keep the stepped rotation in step with the tiles: RT row steps of RP rows = one tile
-#pragma unroll
-              for (int i = 0; i < RT; ++i)
-#pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                  const f32x2 na = fma2(Qb[x], stn[x], mul2(Qa[x], stc[x]));
-                  Qb[x] = fma2(Qa[x], sts[x], mul2(Qb[x], stc[x]));
-                  Qa[x] = na;
-                }
-            }
-          }
-          if (scorer && mine) {
+          if (scorer) {
             if (ROPE && active && ((kt >> (SETS - 1)) % (TC_RESEED / SETS)) == 0) {
               // exact Q at this thread's first row of the tile (position t0 + rp)
 #pragma unroll
@@ -369,7 +355,6 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
               }
             } else if (SETS == 2 && kt == 1) {
               ok = mbar_wait<false>(bar_xm, uc & 1, s_abort, p.status) && ok;
-              have_mref = true;
               mref = head_valid ? s_xm[hl] : 0.f;
               lsum = 0.f;
             }
@@ -406,6 +391,17 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
               mbar_arrive_expect_tx(bar_p_full + 8 * st, p_bytes_w);
               mbar_arrive(bar_k_empty + 8 * st);
             }
+            if (ROPE && active && SETS == 2) {
+              // the other set's tile: RT row steps of RP rows keep the stepped rotation in step
+#pragma unroll
+              for (int i = 0; i < RT; ++i)
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                  const f32x2 na = fma2(Qb[x], stn[x], mul2(Qa[x], stc[x]));
+                  Qb[x] = fma2(Qa[x], sts[x], mul2(Qb[x], stc[x]));
+                  Qa[x] = na;
+                }
+            }
           }
         }
         if (!ok) break;
@@ -414,20 +410,23 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
 #pragma unroll
           for (int o = 1; o < HL; o <<= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
           if (SETS == 2) {
-            if (wset == 1) {
-              // a unit of one tile never showed m_ref to this set: take the hand-over all the same
-              if (!have_mref) ok = mbar_wait<false>(bar_xm, uc & 1, s_abort, p.status);
-              if (head_valid && (lane % HL) == 0) s_xl[hl] = ntile > 1 ? lsum : 0.f;
+            // Both sets wait on both hand-over barriers in every unit, so each warp sees every
+            // phase of them, whichever role its set had.
+            if (!owner) {
+              if (kt0 >= ntile) ok = mbar_wait<false>(bar_xm, uc & 1, s_abort, p.status);   // no tile of this unit
+              if (head_valid && (lane % HL) == 0) s_xl[hl] = lsum;
               __syncwarp();
               if (lane == 0) mbar_arrive(bar_xl);
-            } else {
-              ok = mbar_wait<false>(bar_xl, uc & 1, s_abort, p.status);
+            }
+            ok = mbar_wait<false>(bar_xl, uc & 1, s_abort, p.status) && ok;
+            if (owner) {
+              ok = mbar_wait<false>(bar_xm, uc & 1, s_abort, p.status) && ok;
               if (head_valid) lsum += s_xl[hl];
             }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
           }
-          if (wset == 0 && head_valid && (lane % HL) == 0) {
+          if (owner && head_valid && (lane % HL) == 0) {
             p.part_m[(size_t)unit * p.H + my_n] = mref;
             p.part_l[(size_t)unit * p.H + my_n] = lsum;
           }
@@ -466,6 +465,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           if (lane == 0) mbar_arrive(bar_u_empty);
         }
         gg = seg_end;
+        it_base += ntile;
       }
     } else if (warp == producer_warp) {
       // =========================== TMA producer ===========================
@@ -568,6 +568,7 @@ TcGeom make_geom(int d, int H, int d_k, int rt, int cl, int sets, int smem_limit
   g.stage_bytes = SLIM_TT * g.dsl * 2;
   int ns = (smem_limit - 16 * 1024) / g.stage_bytes;
   g.ns = ns > TC_MAX_NS ? TC_MAX_NS : ns;
+  if (sets == 2) g.ns &= ~1;                     // each set keeps to the stages of its own parity
   int cols = 32;
   while (cols < 32 * g.nch) cols <<= 1;
   g.tmem_cols = cols;
