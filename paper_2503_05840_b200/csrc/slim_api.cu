@@ -431,7 +431,12 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   p.workers = path == SLIM_PATH_TC ? ctx->tc_workers[cl - 1] : ctx->gen_workers;
   p.cl = cl;
   p.min_tiles = min_tiles_for(ctx);
-  p.unit_cost = path == SLIM_PATH_TC ? (ctx->H + 3) / 4 : 0;   // measured: a drain costs about H/4 tiles
+  // measured: closing a unit (accumulator drain + pipeline restart) costs a worker about H/4 + 4 tiles
+  p.unit_cost = path == SLIM_PATH_TC ? (ctx->H + 3) / 4 + 4 : 0;
+  if (path == SLIM_PATH_TC) {
+    const char* e = getenv("SLIM_TC_UNIT_COST");                // override for sweeps
+    if (e && atoi(e) >= 0 && atoi(e) <= 64) p.unit_cost = atoi(e);
+  }
   p.qscale = (float)(1.4426950408889634 / std::sqrt((double)ctx->d_k));
   p.q = q; p.k = cache->k; p.lengths = lengths;
   p.rope_base = ctx->rope_base; p.rope_off = ctx->rope_off; p.wkv = ctx->wkv;
