@@ -53,7 +53,7 @@ def parse():
 # DRAM bytes (read + write) of one main-kernel launch on the benchmarked workload, from an
 # ncu capture (profiles/), keyed by the hash of the kernel source it was taken with.  A kernel
 # that has changed since reports no traffic.
-NCU_TRAFFIC = {"0d387b6eb135fe38": 1636450000 + 10277632}
+NCU_TRAFFIC = {"93f963936855f9ab": 1636465000 + 10541056}
 
 
 def ncu_traffic(config_index, layers_ignored=None):
