@@ -170,14 +170,28 @@ slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned cha
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
-  slim_pdl_wait();                                             // u tiles come from the combine kernel
   const int row0 = js * g.nst * PJ_ROWS;                      // first row of W_KV,h of this CTA
+  // The weights do not depend on the kernels before this one: the producer starts the W_KV tiles
+  // of the first stages before the dependency wait, so they stream in while the combine kernel
+  // still runs; the u tiles of those stages follow after the wait (same barrier, one byte count).
+  const int npre = g.nst < PJ_NS ? g.nst : PJ_NS;
+  if (warp == 0 && lane == 0) {
+    for (int s = 0; s < npre; ++s) {
+      const uint32_t dst = base + (uint32_t)s * stage_bytes;
+      mbar_arrive_expect_tx(bar_full + 8 * s, stage_bytes);
+      if (g.hp == 1) tma_load_3d(dst, &wmap, bar_full + 8 * s, 0, hg * d + row0 + s * PJ_ROWS, 0);
+      else           tma_load_3d(dst, &wmap, bar_full + 8 * s, 0, row0 + s * PJ_ROWS, 2 * hg);
+    }
+  }
+  slim_pdl_wait();                                             // u tiles come from the combine kernel
 
   if (warp == 0 && lane == 0) {
     // =========================== producer ===========================
     const unsigned char* usrc = u_tiled + ((size_t)(bg * g.hg + hg) * (d / 16) + row0 / 16) * ((size_t)1024 * g.hp);
     int s = 0;
     bool ok = true;
+    for (; s < npre; ++s)
+      bulk_load(base + (uint32_t)s * stage_bytes + PJ_W_BYTES, usrc + (size_t)s * g.u_bytes, (uint32_t)g.u_bytes, bar_full + 8 * s);
     for (; s < g.nst; ++s) {
       const int st = s % PJ_NS;
       ok = mbar_wait<false>(bar_empty + 8 * st, ((s / PJ_NS) & 1) ^ 1, s_abort, status);
