@@ -102,6 +102,20 @@ def test_long_sequence_narrow_heads_rope():
     _run_host_case(cfg, L)
 
 
+@pytest.mark.parametrize("theta", [0.0, 1.0e4])
+def test_many_short_sequences_narrow_heads(theta):
+    """Dozens of sequences of one to three tiles with d_k = 64: few workers, each walking many units, most
+    of them a single tile, so the two score-warp sets swap the m_ref role from unit to unit and one
+    set often has no tile of a unit at all."""
+    g = np.random.default_rng(77)
+    lengths = g.integers(1, 17, size=48).astype(np.int32)
+    lengths[::5] = g.integers(17, 49, size=len(lengths[::5]))
+    lengths[7] = 0
+    cfg = synth.SlimConfig("short-narrow", 256, 4, 64, len(lengths), 48, 1, theta, "bf16")
+    L = synth.make_layer(cfg, 5150, lengths=lengths)
+    _run_host_case(cfg, L)
+
+
 def test_config0_whisper_tiny_shape_full():
     cfg = synth.CONFIGS[0]
     _run_host_case(cfg, synth.make_layer(cfg, synth.layer_seed(0, 0)))
