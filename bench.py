@@ -417,7 +417,7 @@ def main():
     for _ in range(max(args.warmup, 3)):
         step()
     for lay in layers[:1]:
-        assert lay.device_status() == B.SLIM_OK
+        assert lay.device_status() == B.SLIM_OK, f"device status {lay.device_status()} after warm-up"
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -497,7 +497,7 @@ def main():
                          f"{dt:.1f} s), scaled by rows to {int(np.sum(lengths))} rows x {layers_n} layers",
                "parity_err_on_sample": worst}
 
-    status = layers[0].device_status()
+    status = max(int(lay.device_status()) for lay in layers)      # worst status over all layers
     if rank == 0:
         launches = sum(1 + lay.query(B.SLIM_Q_LAUNCHES_PER_DECODE) for lay in layers)
         line = {
