@@ -31,31 +31,36 @@ slim_xq_tiled_kernel(SlimDecodeParams p, const float* __restrict__ W_K, unsigned
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int dk = p.d_k, d = p.d;
   float* s_w = reinterpret_cast<float*>(smem_raw);                   // [XQ_J][dk + 1]
-  float* s_q = s_w + XQ_J * (dk + 1);                                // [XQ_B][dk]
+  float* s_q = s_w + XQ_J * (dk + 1);                                // [dk][XQ_B]
   slim_pdl_wait();
   const int h = blockIdx.x, j0 = blockIdx.y * XQ_J, tid = threadIdx.x;
   for (int e = tid; e < XQ_J * dk; e += 256) {
     const int j = e / dk, c = e % dk;
     s_w[j * (dk + 1) + c] = (j0 + j < d) ? __ldg(W_K + (size_t)(j0 + j) * d + h * dk + c) : 0.f;
   }
-  const int j = tid & (XQ_J - 1), bq = tid >> 6;                     // 4 sequences at a time per pass
+  const int j = tid & (XQ_J - 1), bq = tid >> 6;                     // a thread: row j, sequences 4 bq .. 4 bq + 3 of a pass
   for (int b0 = 0; b0 < p.batch; b0 += XQ_B) {
     __syncthreads();
-    for (int e = tid; e < XQ_B * dk; e += 256) {
+    for (int e = tid; e < XQ_B * dk; e += 256) {                     // s_q[c][bb]: four sequences of one c in 16 bytes
       const int bb = e / dk, c = e % dk;
-      s_q[e] = (b0 + bb < p.batch)
-                   ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.q)[(size_t)(b0 + bb) * d + h * dk + c]) * p.qscale : 0.f;
+      s_q[c * XQ_B + bb] = (b0 + bb < p.batch)
+                               ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.q)[(size_t)(b0 + bb) * d + h * dk + c]) * p.qscale : 0.f;
     }
     __syncthreads();
-    for (int bb = bq; bb < XQ_B; bb += 4) {
-      const int b = b0 + bb;
-      if (b >= p.batch || j0 + j >= d) continue;
-      const float* w = s_w + j * (dk + 1);
-      const float* q = s_q + bb * dk;
-      float a = 0.f;
+    if (j0 + j >= d) continue;
+    const float* w = s_w + j * (dk + 1);
+    float a[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 8
-      for (int c = 0; c < dk; ++c) a = fmaf(q[c], w[c], a);
-      const __nv_bfloat16 hi = __float2bfloat16_rn(a), lo = __float2bfloat16_rn(a - __bfloat162float(hi));
+    for (int c = 0; c < dk; ++c) {
+      const float wc = w[c];
+      const float4 qv = *reinterpret_cast<const float4*>(s_q + c * XQ_B + 4 * bq);
+      a[0] = fmaf(qv.x, wc, a[0]); a[1] = fmaf(qv.y, wc, a[1]); a[2] = fmaf(qv.z, wc, a[2]); a[3] = fmaf(qv.w, wc, a[3]);
+    }
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const int b = b0 + 4 * bq + x;
+      if (b >= p.batch) continue;
+      const __nv_bfloat16 hi = __float2bfloat16_rn(a[x]), lo = __float2bfloat16_rn(a[x] - __bfloat162float(hi));
       unsigned char* t = qt_tiled + ((size_t)b * (d / 16) + (j0 + j) / 16) * 2048;
       *reinterpret_cast<__nv_bfloat16*>(t + qt_offset(h, (j0 + j) & 15)) = hi;
       *reinterpret_cast<__nv_bfloat16*>(t + qt_offset(32 + h, (j0 + j) & 15)) = lo;
