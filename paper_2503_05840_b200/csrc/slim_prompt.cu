@@ -21,7 +21,7 @@ constexpr int PV_ROWS = 128;                       // prompt rows per CTA (MMA M
 constexpr int PV_J = 64;                           // columns of K (rows of W_KV) per stage
 constexpr int PV_A_BYTES = PV_ROWS * PV_J * 2;     // 16 KB
 constexpr int PV_B_BYTES = PV_J * 128 * 2;         // two 64-column atoms x 64 rows x 128 B = 16 KB
-constexpr int PV_NS = 4;
+constexpr int PV_NS = 3;                          // 97 KB per CTA: two CTAs per SM, one's epilogue under the other's MMAs
 
 __global__ void __launch_bounds__(128)
 slim_values_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap wmap, float* __restrict__ V,
@@ -37,7 +37,8 @@ slim_values_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc);
   volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 4);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int t0 = blockIdx.x * PV_ROWS, hg = blockIdx.y;
+  // head groups vary fastest: the CTAs in flight share a few key tiles and all of W_KV (L2-resident)
+  const int t0 = blockIdx.y * PV_ROWS, hg = blockIdx.x;
   const int nst = d / PV_J;
 
   if (tid == 0) {
@@ -78,16 +79,20 @@ slim_values_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     }
   } else if (warp == 1 && lane == 0) {
     bool ok = true;
-    for (int s = 0; s < nst && ok; ++s) {
-      const int st = s % PV_NS;
-      ok = mbar_wait<false>(bar_full + 8 * st, (s / PV_NS) & 1, s_abort, status);
+    // descriptors of stage 0 as words; a stage or a k-step only moves the start-address field
+    const uint64_t ad0 = desc_kmajor_sw128(base), bd0 = desc_a(base + PV_A_BYTES, PV_J * 128);
+    const uint32_t a_lo0 = (uint32_t)ad0, a_hi = (uint32_t)(ad0 >> 32), b_lo0 = (uint32_t)bd0, b_hi = (uint32_t)(bd0 >> 32);
+    int st = 0;
+    uint32_t ph = 0;
+    for (int s = 0; s < nst && ok; ++s, st = (st + 1 == PV_NS ? 0 : st + 1), ph ^= (st == 0)) {
+      ok = mbar_wait<false>(bar_full + 8 * st, ph, s_abort, status);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t abase = base + (uint32_t)st * stage_bytes, bbase = abase + PV_A_BYTES;
+      const uint32_t a_lo = a_lo0 + (uint32_t)st * (stage_bytes >> 4), b_lo = b_lo0 + (uint32_t)st * (stage_bytes >> 4);
 #pragma unroll
       for (int kk = 0; kk < PV_J / 16; ++kk)
-        umma_bf16(tmem_base, desc_kmajor_sw128(abase + (uint32_t)kk * 32u), desc_a(bbase + (uint32_t)kk * 2048u, PV_J * 128),
-                  umma_idesc_major(128, 0, 1), (s | kk) ? 1u : 0u);
+        umma_bf16_words(tmem_base, a_lo + (uint32_t)kk * (32u >> 4), a_hi, b_lo + (uint32_t)kk * (2048u >> 4), b_hi,
+                        umma_idesc_major(128, 0, 1), (s | kk) ? 1u : 0u);
       umma_commit(bar_empty + 8 * st);
       if (s == nst - 1) umma_commit(bar_done);
     }
@@ -163,7 +168,7 @@ cudaError_t slim_launch_values(const slim_ctx* ctx, const void* K, int n, float*
     if (e != cudaSuccess) return e;
     memcpy(&wmap, ctx->wmap, sizeof(wmap));
     const int hp = d_k == 64 ? 2 : 1;
-    return slim_launch_pdl(slim_values_tc_kernel, dim3((n + PV_ROWS - 1) / PV_ROWS, H / hp), dim3(128), PV_SMEM, st, kmap, wmap, V, n,
+    return slim_launch_pdl(slim_values_tc_kernel, dim3(H / hp, (n + PV_ROWS - 1) / PV_ROWS), dim3(128), PV_SMEM, st, kmap, wmap, V, n,
                            d, d_k, hp, ctx->status);
   }
   dim3 grid((d + 15) / 16, (n + 15) / 16);
