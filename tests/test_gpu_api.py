@@ -221,10 +221,12 @@ def test_row_permutation_invariance_without_rope_and_identical_keys():
         layer.close()
 
 
-def test_scores_far_above_the_first_tile_are_handled():
+@pytest.mark.parametrize("d,H,d_k", [(512, 4, 128), (256, 4, 64)])
+def test_scores_far_above_the_first_tile_are_handled(d, H, d_k):
     # later keys score much higher than the first tile's: exercises the
-    # reference-exponent handling of every path (and its exact redo, if any).
-    cfg = synth.SlimConfig("ramp", 512, 4, 128, 2, 400, 1, 0.0, "bf16")
+    # reference-exponent handling of every path (and its exact redo, if any);
+    # d_k = 64 runs the kernel with two score-warp sets, either of which may raise the flag.
+    cfg = synth.SlimConfig("ramp", d, H, d_k, 2, 400, 1, 0.0, "bf16")
     L = synth.make_layer(cfg, 77)
     K = L.K.copy()
     q = L.q.copy()
