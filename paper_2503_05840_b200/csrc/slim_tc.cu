@@ -189,7 +189,12 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
       const bool head_valid = scorer && hl < g.hl;
       const bool active = head_valid && jl < OCT;
       const int my_n = (int)rank * g.hl + hl;                    // global head
-      const int my_row = rp + RP * (jl / DUP);                   // row whose argument this lane ends up with
+      // Row i of this thread's RT rows.  Without RoPE nothing ties a thread to equidistant rows, and for
+      // d_k = 64 (a head's half is 64 bytes, half a swizzled line) the rows read by one load instruction
+      // are then chosen two swizzle phases apart, so that the 32 lanes cover all banks (no conflicts).
+      constexpr bool SPREAD = !ROPE && DK == 64 && RT == 4;
+      auto row_of = [&](const int i) { return SPREAD ? 2 * rp + (i & 1) + 8 * (i >> 1) : rp + RP * i; };
+      const int my_row = row_of(jl / DUP);                       // row whose argument this lane ends up with
       // byte offsets of this thread's two 16-byte key units (first / second half of the head)
       uint32_t koff[2], kunit[2];
 #pragma unroll
@@ -297,7 +302,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             if (active) {
 #pragma unroll
               for (int i = 0; i < RT; ++i) {
-                const int row = rp + RP * i;
+                const int row = row_of(i);
                 const uint32_t rbase = kbase + (uint32_t)row * 128u;
                 const uint32_t sw = (uint32_t)(row & 7);
                 const uint4 ka = lds128(rbase + koff[0] + ((kunit[0] ^ sw) << 4));
