@@ -110,6 +110,10 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   constexpr int DUP = JL / RT;                    // lanes that end up with the same row's sum
   constexpr int HL = JL * RP;                     // lanes per head
   constexpr int HW = 32 / HL;                     // heads per warp
+  // PAIR (with the two score-warp sets, stage count even): stages 2k and 2k + 1 are freed together by
+  // one commit on p_empty[k]; the MMA thread then takes two tiles per turn of its loop where it can,
+  // which halves its waits, fences, commits and loop bookkeeping per tile.
+  constexpr bool PAIR = SETS == 2;
   static_assert(RT <= JL && HL <= 32 && HW == tc_heads_per_warp(DK, RT), "lane mapping");
 
   extern __shared__ unsigned char smem_raw[];
@@ -369,7 +373,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             const __nv_bfloat16 pb = __float2bfloat16_rn(pf);
             if ((jl % DUP) == 0) lsum += __bfloat162float(pb);
             // the P stage is free once the MMAs of tile it - ns are done in both CTAs
-            ok = mbar_wait<false>(bar_p_empty + 8 * st, kph ^ 1, s_abort, p.status) && ok;
+            ok = mbar_wait<false>(bar_p_empty + 8 * (PAIR ? st >> 1 : st), kph ^ 1, s_abort, p.status) && ok;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             {
@@ -485,7 +489,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           for (int kt = 0; kt < ntile; ++kt, ++it, st = (st + 1 == g.ns ? 0 : st + 1), kph ^= (st == 0)) {
             // free once the score warps have read the keys and the tensor core has consumed them
             ok = mbar_wait<false>(bar_k_empty + 8 * st, kph ^ 1, s_abort, p.status) &&
-                 mbar_wait<false>(bar_p_empty + 8 * st, kph ^ 1, s_abort, p.status);
+                 mbar_wait<false>(bar_p_empty + 8 * (PAIR ? st >> 1 : st), kph ^ 1, s_abort, p.status);
             if (!ok) break;
             mbar_arrive_expect_tx(bar_k_full + 8 * st, (uint32_t)g.stage_bytes);
             tma_load_3d(k_stage0 + (uint32_t)st * g.stage_bytes, &tmap, bar_k_full + 8 * st, 0,
@@ -520,10 +524,13 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           const int b = slim_seq_of_tile(s_prefix, p.batch, gg);
           const int seg_end = min(g_end, s_prefix[b + 1]);
           const int ntile = seg_end - gg;
-          for (int kt = 0; kt < ntile; ++kt, ++it, st = (st + 1 == g.ns ? 0 : st + 1), kph ^= (st == 0)) {
+          for (int kt = 0; kt < ntile;) {
+            // two tiles in one turn: the even stage of a pair with the odd one behind it, same unit
+            const bool two = PAIR && (st & 1) == 0 && kt + 1 < ntile;
             // p_full alone is enough: every local score warp arrives on it after it has seen
             // k_full of this stage, so the keys have landed (and are ordered before this wait).
             ok = mbar_wait<true>(bar_p_full + 8 * st, kph, s_abort, p.status);
+            if (ok && two) ok = mbar_wait<true>(bar_p_full + 8 * (st + 1), kph, s_abort, p.status);
             if (ok && kt == 0 && uc > 0) ok = mbar_wait<false>(bar_u_empty, (uc - 1) & 1, s_abort, p.status);
             if (!ok) break;
             fence_proxy_async_smem();        // P pieces and zero-filled key rows -> tensor-core reads
@@ -537,9 +544,22 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
               const uint32_t bl = b_lo + (uint32_t)st * (TC_P_BYTES >> 4);
               for (int c = 0; c < g.nch; ++c, al += 4096u >> 4, dcol += 32u)
                 umma_bf16_words(dcol, al, a_hi, bl, b_hi, umma_idesc(32), acc);
+              if (two) {
+                al = a_lo + (uint32_t)(st + 1) * a_step; dcol = tmem_base;
+                for (int c = 0; c < g.nch; ++c, al += 4096u >> 4, dcol += 32u)
+                  umma_bf16_words(dcol, al, a_hi, bl + (TC_P_BYTES >> 4), b_hi, umma_idesc(32), 1u);
+              }
             }
-            if (CL == 2) umma_commit_pair(bar_p_empty + 8 * st); else umma_commit(bar_p_empty + 8 * st);
-            if (kt == ntile - 1) umma_commit(bar_u_full);
+            const int last = two ? st + 1 : st;
+            if (!PAIR) {
+              if (CL == 2) umma_commit_pair(bar_p_empty + 8 * st); else umma_commit(bar_p_empty + 8 * st);
+            } else if (last & 1) {               // the odd stage closes the pair (the even one is older)
+              if (CL == 2) umma_commit_pair(bar_p_empty + 8 * (last >> 1)); else umma_commit(bar_p_empty + 8 * (last >> 1));
+            }
+            const int adv = two ? 2 : 1;
+            kt += adv; it += adv; st += adv;
+            if (st >= g.ns) { st -= g.ns; kph ^= 1u; }
+            if (kt == ntile) umma_commit(bar_u_full);
           }
           gg = seg_end;
         }
