@@ -176,11 +176,6 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   const int g_begin = in_range ? slim_worker_start(sc, w) : 0;
   const int g_end = in_range ? slim_worker_start(sc, w + 1) : 0;
   const bool have_work = g_end > g_begin;
-  if (have_work) {                                // clear this CTA's redo flags of the worker's units
-    const int b_lo = slim_seq_of_tile(s_prefix, p.batch, g_begin), b_hi = slim_seq_of_tile(s_prefix, p.batch, g_end - 1);
-    for (int b = b_lo + tid; b <= b_hi; b += blockDim.x) p.unit_flags[2 * (w + b) + (int)rank] = 0;
-  }
-  __syncthreads();
 
   if (have_work) {
     if (warp < g.nswl) {
@@ -482,6 +477,14 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
         int it = 0, st = 0;
         uint32_t kph = 0;
         bool ok = true;
+        {
+          // Clear this CTA's redo flags of the worker's units.  A score warp can only raise one after
+          // it has seen a k_full phase, which takes this thread's arming arrival (a release) below:
+          // the clears are ordered before any such store.
+          const int b_lo = slim_seq_of_tile(s_prefix, p.batch, g_begin), b_hi = slim_seq_of_tile(s_prefix, p.batch, g_end - 1);
+          for (int b = b_lo; b <= b_hi; ++b) p.unit_flags[2 * (w + b) + (int)rank] = 0;
+          __threadfence_block();
+        }
         for (int gg = g_begin; gg < g_end && ok;) {
           const int b = slim_seq_of_tile(s_prefix, p.batch, gg);
           const int seg_end = min(g_end, s_prefix[b + 1]);
