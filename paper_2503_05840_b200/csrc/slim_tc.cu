@@ -69,7 +69,7 @@ constexpr int TC_P_BYTES = 1024;         // [32 heads][16 rows] bf16
 constexpr int TC_MAX_NS = 8;             // K stages
 constexpr int TC_MAX_SW = 16;            // score warps
 constexpr float TC_XMAX = 96.f;          // largest exponent accepted above m_ref
-constexpr int TC_RESEED = 32;            // tiles between exact re-seeds of the stepped query rotation
+constexpr int TC_RESEED = 64;            // tiles between exact re-seeds of the stepped query rotation
 
 struct TcGeom {
   int cl;           // CTAs per worker
