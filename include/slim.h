@@ -22,6 +22,11 @@
  *     by slim_device_status.
  *   - No call falls back to the CPU.  Without a usable CUDA device every
  *     compute call returns SLIM_ERR_CUDA.
+ *   - A context is not re-entrant on the device: decode calls of one context
+ *     share its status word and redo flag, and calls given the same workspace
+ *     share its partials.  Enqueue the calls of one context (and of contexts
+ *     that share a workspace) on one stream, or order them with events; host
+ *     threads must not call into one context at the same time.
  */
 #ifndef SLIM_H_
 #define SLIM_H_
