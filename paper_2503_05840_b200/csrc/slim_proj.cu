@@ -139,6 +139,120 @@ slim_combine_kernel(const SlimDecodeParams p, unsigned char* __restrict__ u_tile
   }
 }
 
+// The same for small batches, where a sequence has many units and few (head, sequence) pairs exist:
+// grid.z CTAs share the d / 8 column groups of a pair, a CTA takes G of them per pass and spreads the
+// units over UL = 256 / G thread rows, whose sums meet in shared memory.
+__global__ void __launch_bounds__(256)
+slim_combine_split_kernel(const SlimDecodeParams p, unsigned char* __restrict__ u_tiled, const int hp, const int G) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* s_w = reinterpret_cast<float*>(smem_raw);                 // [workers]
+  int* s_info = reinterpret_cast<int*>(s_w + p.workers);           // wlo, wn
+  int* s_prefix = s_info + 2;                                      // [batch+1]
+  // [UL - 1][G][8] floats (7 KB at most) behind the prefix, 16-byte aligned
+  float* s_red = reinterpret_cast<float*>(smem_raw + ((sizeof(float) * p.workers + sizeof(int) * (2 + p.batch + 1) + 15) & ~(size_t)15));
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int h = blockIdx.x, b = blockIdx.y, bg = b / PJ_BG, n = b % PJ_BG;
+  const int d = p.d, H = p.H;
+  slim_pdl_trigger();
+  slim_pdl_wait();
+  if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) *p.any_flag = 0;   // the redo kernel has consumed it
+
+  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
+  if (tid < 32) {
+    int wlo = 0, wn = 0;
+    if (b < p.batch && s_prefix[b + 1] > s_prefix[b]) {
+      wlo = slim_worker_of_tile(sc, s_prefix[b]);
+      wn = slim_worker_of_tile(sc, s_prefix[b + 1] - 1) - wlo + 1;
+      float M = -INFINITY;
+      for (int i = lane; i < wn; i += 32) {
+        const size_t ui = (size_t)(wlo + i + b) * H + h;
+        M = fmaxf(M, p.part_m[ui] + log2f(p.part_l[ui]));
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+      float L = 0.f;
+      for (int i = lane; i < wn; i += 32) {
+        const size_t ui = (size_t)(wlo + i + b) * H + h;
+        const float wg = exp2f(p.part_m[ui] - M);
+        s_w[i] = wg;
+        L += wg * p.part_l[ui];
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+      const float inv = 1.f / L;
+      __syncwarp();
+      for (int i = lane; i < wn; i += 32) s_w[i] *= inv;
+    }
+    if (lane == 0) { s_info[0] = wlo; s_info[1] = wn; }
+  }
+  __syncthreads();
+  const int wlo = s_info[0], wn = s_info[1];
+  const size_t tile_bytes = (size_t)1024 * hp;
+  unsigned char* dst_h = u_tiled + ((size_t)(bg * (H / hp) + h / hp) * (d / 16)) * tile_bytes + (size_t)(h % hp) * 1024;
+  const int UL = 256 / G, gi = tid % G, ul = tid / G;
+  const size_t ustride = (size_t)H * d;                                       // unit i lives H*d floats further
+  for (int jg0 = blockIdx.z * G; jg0 < d / 8; jg0 += gridDim.z * G) {
+    const int jg = jg0 + gi, j0 = jg * 8;
+    const bool live = jg < d / 8;
+    float acc[8];
+#pragma unroll
+    for (int x = 0; x < 8; ++x) acc[x] = 0.f;
+    const float* Ub = p.part_u + ((size_t)(wlo + b) * H + h) * d + j0;
+    int i = ul;
+    if (live) {
+      for (; i + 3 * UL < wn; i += 4 * UL) {      // four units' loads in flight
+        float4 a[4], c[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float4* U = reinterpret_cast<const float4*>(Ub + (size_t)(i + k * UL) * ustride);
+          a[k] = __ldcs(U); c[k] = __ldcs(U + 1);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float wg = s_w[i + k * UL];
+          acc[0] = fmaf(wg, a[k].x, acc[0]); acc[1] = fmaf(wg, a[k].y, acc[1]); acc[2] = fmaf(wg, a[k].z, acc[2]); acc[3] = fmaf(wg, a[k].w, acc[3]);
+          acc[4] = fmaf(wg, c[k].x, acc[4]); acc[5] = fmaf(wg, c[k].y, acc[5]); acc[6] = fmaf(wg, c[k].z, acc[6]); acc[7] = fmaf(wg, c[k].w, acc[7]);
+        }
+      }
+      for (; i < wn; i += UL) {
+        const float wg = s_w[i];
+        const float4* U = reinterpret_cast<const float4*>(Ub + (size_t)i * ustride);
+        const float4 a = __ldcs(U), c = __ldcs(U + 1);
+        acc[0] = fmaf(wg, a.x, acc[0]); acc[1] = fmaf(wg, a.y, acc[1]); acc[2] = fmaf(wg, a.z, acc[2]); acc[3] = fmaf(wg, a.w, acc[3]);
+        acc[4] = fmaf(wg, c.x, acc[4]); acc[5] = fmaf(wg, c.y, acc[5]); acc[6] = fmaf(wg, c.z, acc[6]); acc[7] = fmaf(wg, c.w, acc[7]);
+      }
+    }
+    if (UL > 1) {                        // thread row 0 adds the other rows' sums in row order
+      __syncthreads();                            // the last pass has been read
+      if (ul > 0) {
+        float4* r = reinterpret_cast<float4*>(s_red + ((size_t)(ul - 1) * G + gi) * 8);
+        r[0] = make_float4(acc[0], acc[1], acc[2], acc[3]); r[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+      }
+      __syncthreads();
+      if (ul == 0) {
+        for (int u2 = 1; u2 < UL; ++u2) {
+          const float4* r = reinterpret_cast<const float4*>(s_red + ((size_t)(u2 - 1) * G + gi) * 8);
+          const float4 a = r[0], c = r[1];
+          acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w; acc[4] += c.x; acc[5] += c.y; acc[6] += c.z; acc[7] += c.w;
+        }
+      }
+    }
+    if (ul != 0 || !live) continue;
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const __nv_bfloat16 h0 = __float2bfloat16_rn(acc[2 * x]), h1 = __float2bfloat16_rn(acc[2 * x + 1]);
+      const __nv_bfloat16 l0 = __float2bfloat16_rn(acc[2 * x] - __bfloat162float(h0));
+      const __nv_bfloat16 l1 = __float2bfloat16_rn(acc[2 * x + 1] - __bfloat162float(h1));
+      hi[x] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+      lo[x] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+    }
+    unsigned char* t = dst_h + (size_t)(j0 / 16) * tile_bytes;
+    *reinterpret_cast<uint4*>(t + u_offset(n, j0 & 15)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    *reinterpret_cast<uint4*>(t + u_offset(PJ_BG + n, j0 & 15)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+  }
+}
+
 __global__ void __launch_bounds__(128)
 slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned char* __restrict__ u_tiled,
                     float* __restrict__ o, const ProjGeom g, const int d, const int d_k, const int batch,
@@ -327,9 +441,23 @@ cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, uns
                              cudaStream_t st) {
   const ProjGeom g = make_proj_geom(p.d, p.H, p.d_k, p.batch);
   {
-    dim3 grid(p.H, g.nbg * PJ_BG);
-    const size_t smem = sizeof(float) * p.workers + sizeof(int) * (2 + p.batch + 1) + 16;
-    cudaError_t e = slim_launch_pdl(slim_combine_kernel, grid, dim3(256), smem, st, p, u_tiled, g.hp);
+    // Small batches: no CTAs for the padding sequences of a 16-sequence group (their columns of the
+    // projection's B operand stay unwritten and only feed outputs that are never stored), and slices
+    // of the columns across grid.z so that ~2 CTAs per SM exist.
+    const int ngroups = p.d / 8;
+    int nslice = 1;
+    while (nslice < 16 && (long long)p.H * p.batch * nslice < 2 * 148 && ngroups / (2 * nslice) >= 32) nslice <<= 1;
+    cudaError_t e;
+    if (nslice > 1) {
+      int G = 256;
+      while (G > 32 && G / 2 * nslice >= ngroups) G >>= 1;
+      const size_t smem = sizeof(float) * p.workers + sizeof(int) * (2 + p.batch + 1) + 16 + sizeof(float) * 7 * 256;
+      e = slim_launch_pdl(slim_combine_split_kernel, dim3(p.H, p.batch, nslice), dim3(256), smem, st, p, u_tiled, g.hp, G);
+    } else {
+      dim3 grid(p.H, g.nbg * PJ_BG);
+      const size_t smem = sizeof(float) * p.workers + sizeof(int) * (2 + p.batch + 1) + 16;
+      e = slim_launch_pdl(slim_combine_kernel, grid, dim3(256), smem, st, p, u_tiled, g.hp);
+    }
     if (e != cudaSuccess) return e;
   }
   CUtensorMap map;
