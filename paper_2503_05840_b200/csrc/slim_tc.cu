@@ -169,7 +169,6 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
-  slim_pdl_trigger();
   slim_pdl_wait();          // lengths, q and the newest key rows may come from the kernels before this one
   const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
   const bool in_range = sc.total_tiles > 0 && w < sc.workers_eff;
@@ -566,9 +565,14 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           }
           gg = seg_end;
         }
+        // Every tile of this CTA is with the tensor core: from here on the kernels behind this one may
+        // take their places on the SMs (they still wait for this grid to finish before they read its
+        // results).  Letting them in at the start of this kernel was measured ~1 % slower per step.
+        slim_pdl_trigger();
       }
     }
   }
+  slim_pdl_trigger();
 
   // ---- teardown: nobody may still write into a CTA that has left ------------------
   __syncwarp();
