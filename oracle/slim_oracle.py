@@ -297,7 +297,7 @@ def oracle_slim_loops(q, K, W_KV, H: int, rope_theta: float = 0.0):
 
 
 # --------------------------------------------------------------------------
-# Error norms used by the parity tests (stated in the benchmark spec's tolerances)
+# Error norms used by the parity tests (the two stated tolerances: fp32 and bf16 caches)
 # --------------------------------------------------------------------------
 def err_fp32_norm(got: np.ndarray, ref: np.ndarray) -> float:
     """max_i |got_i - ref_i| / max(|ref_i|, RMS(ref)) over one output row."""

@@ -154,11 +154,12 @@ constexpr size_t PV_SMEM = 1024 + (size_t)PV_NS * (PV_A_BYTES + PV_B_BYTES) + 16
 cudaError_t slim_launch_values(const slim_ctx* ctx, const void* K, int n, float* V, cudaStream_t st) {
   const int d = ctx->d, d_k = ctx->d_k, H = ctx->H;
   if (ctx->proj_ok && ((uintptr_t)K & 15) == 0 && ((uintptr_t)V & 15) == 0) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    // function attributes are kept per device: opt in once on each device this is called on
+    static bool attr_set[64] = {};
+    if (ctx->device < 0 || ctx->device >= 64 || !attr_set[ctx->device]) {
       cudaError_t e = cudaFuncSetAttribute((const void*)slim_values_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PV_SMEM);
       if (e != cudaSuccess) return e;
-      attr_set = true;
+      if (ctx->device >= 0 && ctx->device < 64) attr_set[ctx->device] = true;
     }
     CUtensorMap kmap, wmap;
     const unsigned long long dims[3] = {(unsigned long long)d, (unsigned long long)n, 1};

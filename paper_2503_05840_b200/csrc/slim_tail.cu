@@ -140,7 +140,7 @@ __global__ void slim_append_kernel(KT* __restrict__ cache, const KT* __restrict_
   slim_pdl_wait();
   const int b = blockIdx.x, r = blockIdx.y;
   const int pos = positions[b];
-  if (pos < 0 || pos + n_new > t_cap) {
+  if (pos < 0 || pos > t_cap - n_new) {            // (n_new <= t_cap is checked on the host; no overflow for any pos)
     if (threadIdx.x == 0) atomicMax(status, (int)SLIM_ERR_CAPACITY);
     return;
   }

@@ -481,7 +481,10 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           // it has seen a k_full phase, which takes this thread's arming arrival (a release) below:
           // the clears are ordered before any such store.
           const int b_lo = slim_seq_of_tile(s_prefix, p.batch, g_begin), b_hi = slim_seq_of_tile(s_prefix, p.batch, g_end - 1);
-          for (int b = b_lo; b <= b_hi; ++b) p.unit_flags[2 * (w + b) + (int)rank] = 0;
+          for (int b = b_lo; b <= b_hi; ++b) {
+            p.unit_flags[2 * (w + b) + (int)rank] = 0;
+            if (CL == 1) p.unit_flags[2 * (w + b) + 1] = 0;        // a lone CTA owns both words of its units
+          }
           __threadfence_block();
         }
         for (int gg = g_begin; gg < g_end && ok;) {

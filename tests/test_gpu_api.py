@@ -133,6 +133,20 @@ def test_append_beyond_capacity_sets_status_and_writes_nothing():
         layer.close()
 
 
+def test_append_at_a_huge_position_is_refused_not_wrapped():
+    """A garbage position near INT_MAX must not wrap around the capacity check (the comparison is made
+    without adding to the position): status CAPACITY, no row written."""
+    layer = SlimLayer(64, 2, 32, 0.0, "f32", 2, 8, DEV)
+    try:
+        layer.k.fill_(7.0)
+        k_new = torch.ones((2, 2, 64), device=DEV)
+        layer.append_k(k_new, torch.tensor([2**31 - 1, 2**31 - 2], dtype=torch.int32, device=DEV))
+        assert layer.device_status() == B.SLIM_ERR_CAPACITY
+        assert torch.all(layer.k == 7.0)
+    finally:
+        layer.close()
+
+
 def test_length_beyond_capacity_is_clamped_and_reported():
     cfg = synth.SlimConfig("cap", 128, 2, 64, 1, 40, 1, 0.0, "f32")
     L = synth.make_layer(cfg, 3)

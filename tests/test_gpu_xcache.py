@@ -92,3 +92,56 @@ def test_xcache_needs_its_weights_and_refuses_rope():
             assert ei.value.status == B.SLIM_ERR_UNSUPPORTED
         finally:
             B.slim_destroy(ctx)
+
+
+def _xcache_device_case(d, H, d_k, batch, t_cap, lengths, sample, seed):
+    """Inputs drawn on the device (bf16), weights from the seeded host recipe; the stored bits of
+    the sampled sequences go back to the host for the oracle."""
+    with torch.cuda.device(DEV):
+        g = torch.Generator(device=DEV); g.manual_seed(seed)
+        storage = torch.randn((batch, t_cap, d), generator=g, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+        W_Q, W_K, W_V, _, _ = synth.make_weights(d, seed)
+        bias = np.random.default_rng(seed).standard_normal(d) * 0.1
+        lens = torch.from_numpy(lengths).to(DEV)
+        x_last = storage[torch.arange(batch, device=DEV), (lens.long() - 1).clamp(min=0)].double()
+        q = (x_last @ torch.from_numpy(W_Q).to(DEV) + torch.from_numpy(bias).to(DEV)).to(torch.bfloat16)
+        for b in range(batch):
+            if lengths[b] < t_cap:
+                storage[b, int(lengths[b]):] = float("nan")         # rows past the end must not matter
+        lay = XLayer(d, H, d_k, "bf16", batch, t_cap, storage)
+        try:
+            B.slim_xcache_set_weights(lay.ctx, W_K, W_V)
+            got = lay.decode(q, lens).cpu().numpy().astype(np.float64)
+            assert B.slim_device_status(lay.ctx, torch.cuda.current_stream().cuda_stream) == B.SLIM_OK
+            assert np.all(np.isfinite(got))
+            worst = 0.0
+            for b in sample:
+                n = int(lengths[b])
+                if n == 0:
+                    assert np.all(got[b] == 0)
+                    continue
+                ref = so.oracle_xcache(q[b].float().cpu().numpy(), storage[b, :n].float().cpu().numpy(), W_K, W_V, H)
+                e = so.err_rms_norm(got[b], ref)
+                worst = max(worst, e)
+                assert e <= TOL["bf16"], f"seq {b}: {e:.3e}"
+            return worst
+        finally:
+            lay.close()
+
+
+def test_xcache_whisper_large_shape_full_batch_sampled_sequences():
+    """The shape the X-cache variant is benchmarked on (batch 64, 1500 encoder rows, d = 1280, 20 heads):
+    the dense query transform walks the batch in four passes of 16 sequences; one sequence of each pass
+    and both ends of the batch are checked."""
+    lengths = np.full(64, 1500, dtype=np.int32)
+    worst = _xcache_device_case(1280, 20, 64, 64, 1500, lengths, [0, 15, 16, 37, 48, 63], 3003)
+    print(f"X-cache, Whisper-large shape: worst error {worst:.3e}")
+
+
+def test_xcache_batch_above_sixteen_small_ragged():
+    """More than 16 sequences at a small size: several passes of the query transform, ragged lengths,
+    an empty sequence and single rows; every sequence is checked."""
+    g = np.random.default_rng(5)
+    lengths = g.integers(1, 120, size=40).astype(np.int32)
+    lengths[[3, 17, 33]] = [0, 1, 119]
+    _xcache_device_case(256, 4, 64, 40, 119, lengths, list(range(40)), 3004)

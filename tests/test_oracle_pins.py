@@ -405,3 +405,60 @@ def test_xcache_two_tokens_closed_form():
     sig = 1.0 / (1.0 + np.exp(-(a[0] - a[1])))
     want = sig * (X[0] @ W_V) + (1 - sig) * (X[1] @ W_V)
     assert np.allclose(so.oracle_xcache(q, X, W_K, W_V, 1), want, rtol=1e-13)
+
+
+# ---- head -> column-block mapping for more than one head (Eq. 4 / 5 / 2: head i owns the
+# ---- i-th block of d_k consecutive columns of Q, K, V) -------------------------------------
+def _two_head_hand_case():
+    """d = 4, H = 2 (d_k = 2), T = 2, no RoPE; every number typed in.  With W_Q = W_K = I the keys
+    are the inputs and q is the last input row.  Head 0 (columns 0, 1) sees two equal scores
+    (q.k0 = q.k1 = 1), so it blends the values 1/2 : 1/2.  Head 1 (columns 2, 3) sees
+    q.(k1 - k0) / sqrt(2) = sqrt(2) (sqrt(2) - c) / sqrt(2) = ln 3 with c = sqrt(2) - ln 3, so it
+    blends 1/4 : 3/4.  A head that took columns (0, 2) or (1, 3) instead would get other scores."""
+    r2, c = math.sqrt(2.0), math.sqrt(2.0) - math.log(3.0)
+    X = np.array([[1.0, 5.0, c, 7.0],
+                  [1.0, 0.0, r2, 0.0]])
+    W_V = np.array([[1.0, 2.0, 0.0, 1.0],
+                    [0.0, 1.0, 1.0, 0.0],
+                    [2.0, 0.0, 1.0, 1.0],
+                    [1.0, 1.0, 0.0, 2.0]])
+    # value rows by hand: v0 = x0 W_V, v1 = x1 W_V
+    v0 = np.array([8.0 + 2.0 * c, 14.0, 5.0 + c, 15.0 + c])
+    v1 = np.array([1.0 + 2.0 * r2, 2.0, r2, 1.0 + r2])
+    expect = np.array([0.5 * v0[0] + 0.5 * v1[0], 0.5 * v0[1] + 0.5 * v1[1],       # head 0: columns 0, 1
+                       0.25 * v0[2] + 0.75 * v1[2], 0.25 * v0[3] + 0.75 * v1[3]])  # head 1: columns 2, 3
+    return X, W_V, expect
+
+
+def test_two_heads_hand_computed_column_blocks():
+    X, W_V, expect = _two_head_hand_case()
+    I4 = np.eye(4)
+    assert np.allclose(so.oracle_vanilla(X, I4, I4, W_V, 2, 0.0), expect, rtol=1e-13)
+    # slim attention on scaled keys: W_K = diag(2, 1, 1, 1/2), W_Q = W_K^{-1} (every q.k product is
+    # unchanged), and W_KV = W_K^{-1} W_V typed row by row
+    D = np.array([2.0, 1.0, 1.0, 0.5])
+    K = X * D[None, :]
+    q = X[1] / D
+    W_KV = np.array([[0.5, 1.0, 0.0, 0.5],
+                     [0.0, 1.0, 1.0, 0.0],
+                     [2.0, 0.0, 1.0, 1.0],
+                     [2.0, 2.0, 0.0, 4.0]])
+    assert np.allclose(so.oracle_slim(q, K, W_KV, 2, 0.0), expect, rtol=1e-13)
+    assert np.allclose(so.oracle_slim_option1(q, K, W_KV, 2, 0.0), expect, rtol=1e-13)
+    assert np.allclose(so.oracle_slim_loops(q, K, W_KV, 2, 0.0)[0], expect, rtol=1e-13)
+    assert np.allclose(so.oracle_slim_batch(q[None, :], K[None, :, :], [2], W_KV, 2, 0.0)[0], expect, rtol=1e-13)
+    # X-cache scheme with the same scaled projections: q = x_n W_Q, cache holds X
+    assert np.allclose(so.oracle_xcache(q, X, np.diag(D), W_V, 2), expect, rtol=1e-13)
+
+
+def test_two_head_pin_catches_a_strided_head_slice():
+    # the same arithmetic with head i = columns i, i + H, ... (a plausible mistake that every
+    # single-head pin and the slim == vanilla identity would let through)
+    X, W_V, expect = _two_head_hand_case()
+    V = X @ W_V
+    out = np.empty(4)
+    for i in range(2):
+        cols = [i, i + 2]
+        s = so.softmax(X[:, cols] @ X[1, cols] / math.sqrt(2.0))
+        out[cols] = s @ V[:, cols]
+    assert np.max(np.abs(out - expect)) > 1e-2
