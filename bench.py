@@ -296,10 +296,23 @@ def run_prompt(args):
     B.slim_destroy(ctx)
 
 
+def _rank_entry(rank, world, argv):
+    """Body of one spawned replica: the launcher environment is set, run the benchmark as that rank."""
+    sys.argv = [os.path.abspath(__file__)] + list(argv)
+    main()
+
+
 def main():
     args = parse()
     if args.impl == "reference":
         return run_reference(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.variant == "kcache":
+        # no launcher around us: start one process per GPU ourselves (same rendezvous a launcher would set up)
+        from paper_2503_05840_b200 import replicas
+        import torch
+        if torch.cuda.device_count() < args.gpus:
+            raise SystemExit(f"--gpus {args.gpus} asked for, {torch.cuda.device_count()} CUDA device(s) visible")
+        return replicas.spawn_replicas(_rank_entry, args.gpus, (sys.argv[1:],))
     if args.variant == "xcache":
         return run_xcache(args)
     if args.variant == "prompt":
@@ -321,6 +334,7 @@ def main():
     if world > 1:
         import torch.distributed as dist
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("NCCL_DEBUG", "INFO")           # the rank count of the job shows in NCCL's own log (stderr)
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
         dist.barrier()
     dev = f"cuda:{local}"
@@ -393,8 +407,7 @@ def main():
 
     def step():
         for li, lay in enumerate(layers):
-            lay.append_k(knew_all[li].unsqueeze(1), pos_dev)
-            lay.decode(q_all[li], lens_dev, o_all[li])
+            lay.decode_step(q_all[li], knew_all[li], lens_dev, o_all[li])
 
     def barrier():
         if dist is not None:
@@ -413,6 +426,17 @@ def main():
         barrier()
         return ms
 
+    def timed_blocks(fn, steps):
+        """The timed region: `steps` steps bracketed by barrier + synchronize.  A region under a second
+        is repeated (up to 5 blocks of `steps` steps, back to back) and the median block is reported,
+        so that one slow or fast block (clock ramp, a neighbour on the host) does not decide the line."""
+        first = timed(fn, steps)
+        blocks = [first]
+        if first < 1000.0:
+            n_more = int(min(4, max(0, 2000.0 // max(first, 1.0))))
+            blocks += [timed(fn, steps) for _ in range(n_more)]
+        return float(np.median(blocks)), blocks
+
     # ---- device-resident timing ------------------------------------------------
     for _ in range(max(args.warmup, 3)):
         step()
@@ -423,25 +447,26 @@ def main():
         sampler.start()
         time.sleep(0.25)
     t0 = time.time()
-    ms_total = timed(step, args.steps)
-    t1 = time.time()
-    clocks = sampler.stop(t0, t1) if rank == 0 else None
+    ms_total, ms_blocks = timed_blocks(step, args.steps)
     ms_step = ms_total / args.steps
     tokens = cfg.batch * world
     value = replicas.job_throughput(cfg.batch, world, ms_step)
 
-    # ---- attribution pass: CUDA events around the main kernel of every decode ----
+    # ---- attribution inside a sustained loop: the library records CUDA events around the main
+    # kernel and the tail of every decode; the loop runs like the timed one (no synchronisation
+    # between steps, same clocks and power state) and the events of its last step are read once,
+    # after it.  The events cost a little, so this loop's own step time is reported beside it.
     for lay in layers:
         lay.profile(True)
-    main_ms, tail_ms, n_launch = 0.0, 0.0, 0
-    for _ in range(min(args.steps, 5)):
-        step()
-        for lay in layers:
-            a, b = lay.profile_read()
-            main_ms += a; tail_ms += b; n_launch += 1
+    ms_prof = timed(step, args.steps) / args.steps
+    main_list, tail_list = [], []
     for lay in layers:
+        a, b = lay.profile_read()
+        main_list.append(a); tail_list.append(b)
         lay.profile(False)
-    main_ms /= n_launch; tail_ms /= n_launch
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1) if rank == 0 else None
+    main_ms, tail_ms = float(np.mean(main_list)), float(np.mean(tail_list))
     k_bytes_layer = synth.kcache_bytes_per_step(cfg.scaled(layers=1), lengths)
     peak, peak_kind = measured_peaks()
     achieved = k_bytes_layer / (main_ms * 1e-3) / 1e9
@@ -474,8 +499,7 @@ def main():
                 ev_h2d_end.record(h2d_s)
             for li, lay in enumerate(layers):
                 stream.wait_event(ev_in[li])
-                lay.append_k(knew_all[li].unsqueeze(1), pos_dev)
-                lay.decode(q_all[li], lens_dev, o_all[li])
+                lay.decode_step(q_all[li], knew_all[li], lens_dev, o_all[li])
                 ev_dec[li].record(stream)
                 d2h_s.wait_event(ev_dec[li])
                 with torch.cuda.stream(d2h_s):
@@ -486,7 +510,7 @@ def main():
 
         for _ in range(3):
             step_e2e()
-        ms_e2e = timed(step_e2e, args.steps) / args.steps
+        ms_e2e = timed_blocks(step_e2e, args.steps)[0] / args.steps
         assert torch.equal(o_host, o_all.cpu()), "end-to-end outputs differ from the resident ones"
         e2e = {"value": tokens / (ms_e2e * 1e-3), "unit": "tokens/s",
                "h2d_bytes_per_step": int(q_host.numel() * q_host.element_size() * 2),
@@ -517,14 +541,17 @@ def main():
             if dt > 20.0:
                 break
         per_step = dt * (float(np.sum(lengths)) / rows_done) * layers_n      # all sequences, all layers
+        tol = 2e-2 if cfg.dtype == "bf16" else 1e-4
+        parity_ok = worst <= tol
         cpu = {"value": cfg.batch / per_step, "unit": "tokens/s", "cores": host_threads(), "kind": "oracle",
+               "parity_tolerance": tol, "parity": "green" if parity_ok else "FAILED",
                "sample": f"oracle_slim on layer {layers_n - 1}, {n_seq} full sequences ({rows_done} context rows, "
                          f"{dt:.1f} s), scaled by rows to {int(np.sum(lengths))} rows x {layers_n} layers",
                "parity_err_on_sample": worst}
 
     status = max(int(lay.device_status()) for lay in layers)      # worst status over all layers
     if rank == 0:
-        launches = sum(1 + lay.query(B.SLIM_Q_LAUNCHES_PER_DECODE) for lay in layers)
+        launches = sum(lay.query(B.SLIM_Q_LAUNCHES_PER_DECODE) for lay in layers)
         line = {
             "metric": "decode_attention_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
@@ -541,7 +568,10 @@ def main():
             "kcache_gbs": step_gbs, "kcache_frac_of_8000": step_gbs / 8000.0, "kcache_frac_of_measured": step_gbs / peak,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": ncu_traffic(args.config), "peak_kind": peak_kind, "kernel": "main decode kernel (per layer launch)",
-                         "main_ms": main_ms, "tail_ms": tail_ms, "bytes_per_launch": k_bytes_layer},
+                         "main_ms": main_ms, "tail_ms": tail_ms, "bytes_per_launch": k_bytes_layer,
+                         "timing": "CUDA events recorded by the library inside a sustained loop of the same step "
+                                   "(last step, mean over layers); that loop ran at %.4f ms per step" % ms_prof},
+            "ms_per_step_blocks": [b / args.steps for b in ms_blocks],
             "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": launches, "clocks": clocks,
             "device_status": int(status), "setup_s": t_setup,
         }
@@ -549,6 +579,9 @@ def main():
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
+    if cpu is not None and cpu["parity"] != "green":
+        raise SystemExit(f"parity check against the oracle FAILED on the timed workload: {cpu['parity_err_on_sample']:.3e} "
+                         f"> {cpu['parity_tolerance']}")
 
 
 if __name__ == "__main__":

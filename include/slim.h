@@ -64,7 +64,7 @@ typedef enum {
 /* Keys for slim_query. */
 typedef enum {
   SLIM_Q_PATH_IN_USE = 0,        /* slim_path that slim_decode will take             */
-  SLIM_Q_LAUNCHES_PER_DECODE = 1,/* kernels one slim_decode enqueues                 */
+  SLIM_Q_LAUNCHES_PER_DECODE = 1,/* kernels the last decode call of this ctx enqueued (counted) */
   SLIM_Q_MAX_UNITS = 2,          /* upper bound of (sequence, context-split) units   */
   SLIM_Q_NUM_SMS = 3,
   SLIM_Q_WORKERS = 4             /* context-split workers of the path in use         */
@@ -153,6 +153,22 @@ slim_status slim_append_k(slim_ctx* ctx, slim_cache* cache, const void* k_new,
 slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache,
                         const int32_t* lengths, float* o, void* workspace, void* stream);
 
+/* One generate-phase step of a layer in a single call: the cache update and the attention
+ * (introduction, "one new K-vector per iteration": the newest key is appended, then the token
+ * attends over all cached keys, itself included; Eq. 7 Option 2).
+ *   k_new    device [batch][d], ctx dtype, un-rotated key row x_n W_K of every sequence, 16-byte
+ *            aligned; it is written to cache row lengths[b]-1 before that row is read
+ *   lengths  device int32 [batch]: the context lengths AFTER the update.  lengths[b] == 0 writes
+ *            nothing and gives a zero output row; lengths[b] > t_cap writes nothing, is clamped
+ *            and reported as SLIM_ERR_CAPACITY
+ *   other arguments and the result as for slim_decode.
+ * Equivalent to slim_append_k(k_new, positions = lengths-1, n_new = 1) followed by slim_decode.
+ * On the tensor-core path the row is written by the decode kernel itself (by the CTA pair that
+ * reads the sequence's last tile, ahead of its first load), so no append kernel runs; other
+ * paths launch the append kernel first.                                                 */
+slim_status slim_decode_step(slim_ctx* ctx, const void* q, const void* k_new, slim_cache* cache,
+                             const int32_t* lengths, float* o, void* workspace, void* stream);
+
 /* slim_decode for callers that cannot allocate device memory.  (The paper has no
  * counterpart; this is a convenience of the library.)  Some hosts of this code must
  * not call cudaMalloc or any allocator while they run: a serving loop whose memory
@@ -170,9 +186,11 @@ slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache,
  *     up the array's device address (once per device); make that first call before
  *     starting any stream capture.
  *   - All calls on a device share the one array, and it keeps whatever the previous
- *     call left.  The kernels write every word before they read it, so nothing needs
- *     clearing, but two calls whose kernels overlap on the GPU (different streams,
- *     different ctx objects) race on it: run them one after another.              */
+ *     call left.  Nothing needs clearing: every word that can reach a stored output is
+ *     written earlier in the same call (words of padding sequences of a 16-sequence
+ *     group may be read unwritten, but only feed outputs that are never stored).  Two
+ *     calls whose kernels overlap on the GPU (different streams, different ctx objects)
+ *     race on it: run them one after another.                                      */
 size_t      slim_static_workspace_max(void);
 slim_status slim_decode_static_ws(slim_ctx* ctx, const void* q, const slim_cache* cache,
                                   const int32_t* lengths, float* o, void* stream);

@@ -35,6 +35,7 @@ SIGNATURES = {
     "slim_values_from_keys": (c_int, [c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
     "slim_append_k": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]),
     "slim_decode": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "slim_decode_step": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "slim_static_workspace_max": (c_size_t, []),
     "slim_decode_static_ws": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "slim_xcache_set_weights": (c_int, [c_void_p, c_void_p, c_void_p, c_int]),
@@ -182,6 +183,12 @@ def slim_append_k(ctx: int, cache: int, k_new, positions, n_new: int, stream: in
 def slim_decode(ctx: int, q, cache: int, lengths, o, workspace, stream: int = 0) -> None:
     _check(lib().slim_decode(c_void_p(ctx), _ptr(q), c_void_p(cache), _ptr(lengths), _ptr(o), _ptr(workspace),
                              c_void_p(stream)), "slim_decode")
+
+
+def slim_decode_step(ctx: int, q, k_new, cache: int, lengths, o, workspace, stream: int = 0) -> None:
+    """Cache update (k_new at row lengths[b]-1) and decode in one call."""
+    _check(lib().slim_decode_step(c_void_p(ctx), _ptr(q), _ptr(k_new), c_void_p(cache), _ptr(lengths), _ptr(o),
+                                  _ptr(workspace), c_void_p(stream)), "slim_decode_step")
 
 
 def slim_static_workspace_max() -> int:

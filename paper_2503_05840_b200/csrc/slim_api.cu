@@ -160,6 +160,16 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
   c->d = d; c->H = H; c->d_k = d_k; c->dtype = dtype; c->rope_theta = rope_theta;
   c->device = dev; c->num_sms = prop.multiProcessorCount;
   c->path_req = SLIM_PATH_AUTO;
+  {
+    // tuning switches for sweeps and tests: the environment is read here, once per context, never on
+    // the decode path
+    const char* e;
+    c->opt_tc_sets1 = ((e = getenv("SLIM_TC_SETS")) && atoi(e) == 1) ? 1 : 0;
+    c->opt_tc_rt = (e = getenv("SLIM_TC_RT")) ? atoi(e) : 0;
+    c->opt_unit_cost = ((e = getenv("SLIM_TC_UNIT_COST")) && atoi(e) >= 0 && atoi(e) <= 64) ? atoi(e) : -1;
+    c->opt_xscores_cuda = getenv("SLIM_XSCORES_CUDA") ? 1 : 0;
+    c->opt_legacy_flow = getenv("SLIM_TC_LEGACY") ? 1 : 0;
+  }
   if (cudaMalloc(&c->status, sizeof(int)) != cudaSuccess) { delete c; return SLIM_ERR_OOM; }
   cudaMemset(c->status, 0, sizeof(int));
   if (cudaMalloc(&c->any_flag, sizeof(int)) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
@@ -396,14 +406,15 @@ slim_status slim_append_k(slim_ctx* ctx, slim_cache* cache, const void* k_new, c
   if (!ctx || !cache || !k_new || !positions || cache->ctx != ctx) return SLIM_ERR_INVALID_ARG;
   if (n_new <= 0 || n_new > 65535) return SLIM_ERR_INVALID_ARG;
   if (n_new > cache->t_cap) return SLIM_ERR_CAPACITY;
-  if (slim_launch_append(ctx, cache, k_new, positions, n_new, (cudaStream_t)stream) != cudaSuccess)
+  if (slim_launch_append(ctx, cache, k_new, positions, n_new, 0, (cudaStream_t)stream) != cudaSuccess)
     return SLIM_ERR_CUDA;
   return SLIM_OK;
 }
 
 namespace {
+// k_new != NULL: the generate-phase step (newest key rows written at lengths[b] - 1 first)
 slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths, float* o,
-                        void* workspace, void* stream, bool xcache) {
+                        void* workspace, void* stream, bool xcache, const void* k_new = nullptr) {
   if (!ctx || !q || !cache || !lengths || !o || !workspace || cache->ctx != ctx) return SLIM_ERR_INVALID_ARG;
   if (((uintptr_t)workspace & 255) || ((uintptr_t)q & 15) || ((uintptr_t)o & 15)) return SLIM_ERR_INVALID_ARG;
   if (!ctx->has_weights) return SLIM_ERR_NO_WEIGHTS;
@@ -433,10 +444,7 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   p.min_tiles = min_tiles_for(ctx);
   // measured: closing a unit (accumulator drain + pipeline restart) costs a worker about H/4 + 4 tiles
   p.unit_cost = path == SLIM_PATH_TC ? (ctx->H + 3) / 4 + 4 : 0;
-  if (path == SLIM_PATH_TC) {
-    const char* e = getenv("SLIM_TC_UNIT_COST");                // override for sweeps
-    if (e && atoi(e) >= 0 && atoi(e) <= 64) p.unit_cost = atoi(e);
-  }
+  if (path == SLIM_PATH_TC && ctx->opt_unit_cost >= 0) p.unit_cost = ctx->opt_unit_cost;      // override for sweeps
   p.qscale = (float)(1.4426950408889634 / std::sqrt((double)ctx->d_k));
   p.q = q; p.k = cache->k; p.lengths = lengths;
   p.rope_base = ctx->rope_base; p.rope_off = ctx->rope_off; p.wkv = ctx->wkv;
@@ -449,14 +457,25 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   p.ext_scores = nullptr;
   p.block_table = cache->block_table; p.page_rows = cache->page_rows; p.max_pages = cache->max_pages;
   p.num_pages = cache->num_pages;
+  // K-cache path on the tensor cores: the decode kernel writes the newest key rows itself, and a sequence
+  // with a flagged unit is recomputed by the combine kernel (no append kernel, no redo kernel)
+  const bool tc_kcache = !xcache && path == SLIM_PATH_TC && !ctx->opt_legacy_flow;
+  p.k_new = tc_kcache ? k_new : nullptr;
+  p.redo_in_combine = (tc_kcache && ctx->proj_ok) ? 1 : 0;
   cudaStream_t st = (cudaStream_t)stream;
+  int launches = 0;
+  if (k_new && !p.k_new) {                           // no fused update on this path: the append kernel first
+    if (slim_launch_append(ctx, cache, k_new, lengths, 1, 1, st) != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
+    ++launches;
+  }
   if (ctx->prof_on) cudaEventRecord(ctx->prof_ev[0], st);
   cudaError_t e;
   float* scores = reinterpret_cast<float*>(ws + L.scores);
   if (xcache) {
     // dense scores first; then P.X on the tensor cores where the shape allows it (an argument that
     // overflows its reference exponent triggers the CUDA-core accumulation as the exact redo)
-    if (cache->has_xmap && !getenv("SLIM_XSCORES_CUDA"))
+    launches += 2;                                   // query transform + dense scores
+    if (cache->has_xmap && !ctx->opt_xscores_cuda)
       e = slim_launch_xscores_tc(ctx, cache, p, ctx->xc_wk,
                                  reinterpret_cast<unsigned char*>(ws + L.total + align256(sizeof(float) * (size_t)p.batch * p.H * p.d)), scores, st);
     else
@@ -466,25 +485,32 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
         p.ext_scores = scores;
         e = slim_launch_tc(ctx, cache, p, st);
         if (e == cudaSuccess) e = slim_launch_accum(ctx, p, scores, 0, st);
+        launches += 2;
       } else {
         e = slim_launch_accum(ctx, p, scores, 1, st);
+        launches += 1;
       }
     }
   } else if (path == SLIM_PATH_TC) {
     e = slim_launch_tc(ctx, cache, p, st);
-    if (e == cudaSuccess) e = slim_launch_exact_flagged(ctx, p, st);
+    ++launches;
+    if (e == cudaSuccess && !p.redo_in_combine) { e = slim_launch_exact_flagged(ctx, p, st); ++launches; }
   } else {
     e = slim_launch_generic(ctx, p, scores, st);
+    launches += 2;                                   // scores, accumulation
   }
   if (ctx->prof_on) cudaEventRecord(ctx->prof_ev[1], st);
   if (e == cudaSuccess) {
     if (ctx->proj_ok) {
       float* o_part = reinterpret_cast<float*>(ws + L.o_part);
       e = slim_launch_proj(ctx, p, reinterpret_cast<unsigned char*>(ws + L.u_tiled), o_part, st);
+      launches += 2;                                 // combine, projection
     } else {
       e = slim_launch_tail(ctx, p, st);
+      launches += 2;                                 // combine + projection slices, slice sum
     }
   }
+  ctx->launches_last = launches;
   if (ctx->prof_on) { cudaEventRecord(ctx->prof_ev[2], st); ctx->prof_valid = 1; }
   if (e != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
   return SLIM_OK;
@@ -494,6 +520,12 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
 slim_status slim_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,
                         float* o, void* workspace, void* stream) {
   return decode_impl(ctx, q, cache, lengths, o, workspace, stream, false);
+}
+
+slim_status slim_decode_step(slim_ctx* ctx, const void* q, const void* k_new, slim_cache* cache, const int32_t* lengths,
+                             float* o, void* workspace, void* stream) {
+  if (!k_new || ((uintptr_t)k_new & 15)) return SLIM_ERR_INVALID_ARG;
+  return decode_impl(ctx, q, cache, lengths, o, workspace, stream, false, k_new);
 }
 
 slim_status slim_xcache_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,
@@ -521,8 +553,8 @@ slim_status slim_decode_static_ws(slim_ctx* ctx, const void* q, const slim_cache
   void* ws = nullptr;
   const slim_status st = static_ws_address(dev, &ws);
   if (st != SLIM_OK) return st;
-  // Nothing in the scratch has to start at zero: every word the kernels read was written
-  // earlier in the same call (partials, redo flags, projection slices).
+  // Nothing in the scratch has to start at zero: every word that reaches a stored output was
+  // written earlier in the same call (partials, redo flags, projection operand tiles).
   return slim_decode(ctx, q, cache, lengths, o, ws, stream);
 }
 
@@ -580,8 +612,8 @@ long long slim_query(const slim_ctx* ctx, int key) {
   const int path = path_in_use(ctx);
   switch (key) {
     case SLIM_Q_PATH_IN_USE: return path;
-    case SLIM_Q_LAUNCHES_PER_DECODE:              // main (tc: + exact redo; generic: scores + accum), then the tail
-      return 2 + 2;                               // combine, projection  |  combine+projection, slice sum
+    case SLIM_Q_LAUNCHES_PER_DECODE:              // counted by the last decode call of this ctx (0 before the first)
+      return ctx->launches_last;
     case SLIM_Q_MAX_UNITS: return ctx->num_sms;   // + batch, known only per cache
     case SLIM_Q_NUM_SMS: return ctx->num_sms;
     case SLIM_Q_WORKERS: return path == SLIM_PATH_TC ? (ctx->tc_workers[1] > 0 ? ctx->tc_workers[1] : ctx->tc_workers[0]) : ctx->gen_workers;

@@ -43,6 +43,8 @@ struct SlimDecodeParams {
   const float* ext_scores;       // X-cache scheme: precomputed softmax arguments [batch][H][t_cap] (else NULL)
   const int32_t* block_table;    // paged cache: [batch][max_pages] page ids (NULL = contiguous [batch][t_cap][d])
   int page_rows, max_pages, num_pages;
+  const void* k_new;             // tensor-core path: [batch][d] newest key rows, written at row lengths[b]-1 before the read (or NULL)
+  int redo_in_combine;           // 1: the combine kernel recomputes the sequences that have a flagged unit (no redo kernel runs)
 };
 
 struct slim_ctx {
@@ -65,6 +67,13 @@ struct slim_ctx {
   int proj_ok;                   // tensor-core combine + projection usable for this shape
   float* xc_wk;                  // X-cache scheme: device fp32 W_K [d][d] (NULL until slim_xcache_set_weights)
   int* any_flag;                 // device: 1 while some unit of the current decode is flagged for the exact redo
+  int launches_last;             // kernels the last decode call enqueued
+  // tuning switches, read from the environment once, by slim_create (sweeps and tests only)
+  int opt_tc_sets1;              // SLIM_TC_SETS=1: never use two score-warp sets
+  int opt_tc_rt;                 // SLIM_TC_RT: rows per thread and tile (0 = default)
+  int opt_unit_cost;             // SLIM_TC_UNIT_COST: boundary cost of the schedule in tiles (-1 = default)
+  int opt_xscores_cuda;          // SLIM_XSCORES_CUDA: dense X-cache scores on CUDA cores
+  int opt_legacy_flow;           // SLIM_TC_LEGACY: append and exact redo as kernels of their own (for side-by-side timing)
   alignas(64) unsigned char wmap[128];   // CUtensorMap over W_KV for the projection kernel
 };
 
@@ -93,8 +102,9 @@ cudaError_t slim_launch_xcache_scores(const slim_ctx* ctx, const SlimDecodeParam
 cudaError_t slim_launch_accum(const slim_ctx* ctx, const SlimDecodeParams& p, const float* scores, int whole, cudaStream_t st);
 cudaError_t slim_launch_exact_flagged(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st);
 cudaError_t slim_launch_tail(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st);
+// pos_is_length = 1: positions[b] holds the length AFTER the append (row positions[b]-1 is written; 0 writes nothing)
 cudaError_t slim_launch_append(const slim_ctx* ctx, const slim_cache* c, const void* k_new,
-                               const int32_t* positions, int n_new, cudaStream_t st);
+                               const int32_t* positions, int n_new, int pos_is_length, cudaStream_t st);
 // fp64 solve W_K X = W_V on the device; A and B are device row-major [n][n]
 // float64, both overwritten; X is returned in B.  info: 0 ok, 1 singular.
 cudaError_t slim_wkv_solve(double* A, double* B, int n, int* info_host);

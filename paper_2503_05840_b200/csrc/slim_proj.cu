@@ -28,14 +28,15 @@
 #include "slim_internal.h"
 #include "slim_sched.cuh"
 #include "slim_ptx.cuh"
+#include "slim_combine.cuh"
 
 namespace {
 using namespace slim_ptx;
+using slim_comb::PJ_BG;
 
 constexpr int PJ_ROWS = 64;                    // rows of W_KV,h per stage (4 MMA k-steps)
 constexpr int PJ_W_BYTES = PJ_ROWS * 128 * 2;  // two 64-column atoms x 64 rows x 128 B
 constexpr int PJ_NS = 4;                       // stages
-constexpr int PJ_BG = 16;                      // sequences per MMA (N = 32 per head: hi and lo)
 
 struct ProjGeom {
   int hp;        // heads per MMA: 1 (d_k = 96, 128) or 2 (d_k = 64)
@@ -46,55 +47,52 @@ struct ProjGeom {
   int u_bytes;   // bytes of u per stage = 4 k-steps x hp x 1 KB
 };
 
-__device__ __forceinline__ uint32_t u_offset(int n, int k) {      // K-major 8x8 core matrices, N = 32
-  return (uint32_t)((n & 7) * 16 + (n >> 3) * 256 + (k >> 3) * 128 + (k & 7) * 2);
+// weights [workers], info [4], prefix [batch + 1]; behind them, 16-byte aligned, the scratch of the exact path
+__device__ __forceinline__ size_t exact_scratch_offset(const SlimDecodeParams& p) {
+  return (sizeof(float) * p.workers + sizeof(int) * (4 + p.batch + 1) + 15) & ~(size_t)15;
 }
 
-__global__ void __launch_bounds__(256)
-slim_combine_kernel(const SlimDecodeParams p, unsigned char* __restrict__ u_tiled, const int hp) {
+// Units of sequence b and their weights for head h (warp 0 of the CTA):
+// s_info = (first worker, unit count, 1 if a unit of the sequence is flagged for the exact recomputation)
+__device__ __forceinline__ void combine_prologue(const SlimDecodeParams& p, const SlimSched& sc, const int* s_prefix, int b, int h,
+                                                 float* s_w, int* s_info, int lane) {
+  int wlo = 0, wn = 0, flagged = 0;
+  if (b < p.batch && s_prefix[b + 1] > s_prefix[b]) {
+    wlo = slim_worker_of_tile(sc, s_prefix[b]);
+    wn = slim_worker_of_tile(sc, s_prefix[b + 1] - 1) - wlo + 1;
+    if (p.redo_in_combine) {
+      for (int i = lane; i < 2 * wn; i += 32) flagged |= p.unit_flags[2 * (wlo + b) + i];
+      flagged = __any_sync(0xffffffffu, flagged != 0) ? 1 : 0;
+    }
+    if (!flagged) slim_comb::weights_warp(p.part_m, p.part_l, wlo + b, wn, p.H, h, s_w, lane);
+  }
+  if (lane == 0) { s_info[0] = wlo; s_info[1] = wn; s_info[2] = flagged; }
+}
+
+// (launch bounds: the register budget of the hot loop; the exact path, a call, may spill under it)
+__global__ void __launch_bounds__(256, 4)
+slim_combine_kernel(const __grid_constant__ SlimDecodeParams p, unsigned char* __restrict__ u_tiled, const int hp) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* s_w = reinterpret_cast<float*>(smem_raw);                 // [workers]
-  int* s_info = reinterpret_cast<int*>(s_w + p.workers);           // wlo, wn
-  int* s_prefix = s_info + 2;                                      // [batch+1]
+  int* s_info = reinterpret_cast<int*>(s_w + p.workers);           // wlo, wn, flagged
+  int* s_prefix = s_info + 4;                                      // [batch+1]
   const int tid = threadIdx.x, lane = tid & 31;
-  const int h = blockIdx.x, b = blockIdx.y, bg = b / PJ_BG, n = b % PJ_BG;
+  const int h = blockIdx.x, b = blockIdx.y;
   const int d = p.d, H = p.H;
   slim_pdl_trigger();
   slim_pdl_wait();
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) *p.any_flag = 0;   // the redo kernel has consumed it
 
   const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
-  if (tid < 32) {
-    int wlo = 0, wn = 0;
-    if (b < p.batch && s_prefix[b + 1] > s_prefix[b]) {
-      wlo = slim_worker_of_tile(sc, s_prefix[b]);
-      wn = slim_worker_of_tile(sc, s_prefix[b + 1] - 1) - wlo + 1;
-      float M = -INFINITY;
-      for (int i = lane; i < wn; i += 32) {
-        const size_t ui = (size_t)(wlo + i + b) * H + h;
-        M = fmaxf(M, p.part_m[ui] + log2f(p.part_l[ui]));
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-      float L = 0.f;
-      for (int i = lane; i < wn; i += 32) {
-        const size_t ui = (size_t)(wlo + i + b) * H + h;
-        const float wg = exp2f(p.part_m[ui] - M);
-        s_w[i] = wg;
-        L += wg * p.part_l[ui];
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
-      const float inv = 1.f / L;
-      __syncwarp();
-      for (int i = lane; i < wn; i += 32) s_w[i] *= inv;
-    }
-    if (lane == 0) { s_info[0] = wlo; s_info[1] = wn; }
-  }
+  if (tid < 32) combine_prologue(p, sc, s_prefix, b, h, s_w, s_info, lane);
   __syncthreads();
   const int wlo = s_info[0], wn = s_info[1];
-  const size_t tile_bytes = (size_t)1024 * hp;
-  unsigned char* dst_h = u_tiled + ((size_t)(bg * (H / hp) + h / hp) * (d / 16)) * tile_bytes + (size_t)(h % hp) * 1024;
+  if (s_info[2]) {                               // a flagged unit: this (head, sequence) is recomputed exactly
+    float* s_x = reinterpret_cast<float*>(smem_raw + exact_scratch_offset(p));
+    for (int jg0 = 0; jg0 < d / 8; jg0 += blockDim.x)
+      slim_comb::exact_groups(p, u_tiled, hp, b, h, jg0, min((int)blockDim.x, d / 8 - jg0), s_x);
+    return;
+  }
   for (int jg = tid; jg < d / 8; jg += blockDim.x) {
     const int j0 = jg * 8;
     float acc[8];
@@ -124,71 +122,37 @@ slim_combine_kernel(const SlimDecodeParams p, unsigned char* __restrict__ u_tile
       acc[0] = fmaf(wg, a.x, acc[0]); acc[1] = fmaf(wg, a.y, acc[1]); acc[2] = fmaf(wg, a.z, acc[2]); acc[3] = fmaf(wg, a.w, acc[3]);
       acc[4] = fmaf(wg, c.x, acc[4]); acc[5] = fmaf(wg, c.y, acc[5]); acc[6] = fmaf(wg, c.z, acc[6]); acc[7] = fmaf(wg, c.w, acc[7]);
     }
-    uint32_t hi[4], lo[4];
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      const __nv_bfloat16 h0 = __float2bfloat16_rn(acc[2 * x]), h1 = __float2bfloat16_rn(acc[2 * x + 1]);
-      const __nv_bfloat16 l0 = __float2bfloat16_rn(acc[2 * x] - __bfloat162float(h0));
-      const __nv_bfloat16 l1 = __float2bfloat16_rn(acc[2 * x + 1] - __bfloat162float(h1));
-      hi[x] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-      lo[x] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
-    }
-    unsigned char* t = dst_h + (size_t)(j0 / 16) * tile_bytes;
-    *reinterpret_cast<uint4*>(t + u_offset(n, j0 & 15)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-    *reinterpret_cast<uint4*>(t + u_offset(PJ_BG + n, j0 & 15)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    slim_comb::store_u8(u_tiled, d, H, hp, b, h, j0, acc);
   }
 }
 
 // The same for small batches, where a sequence has many units and few (head, sequence) pairs exist:
 // grid.z CTAs share the d / 8 column groups of a pair, a CTA takes G of them per pass and spreads the
 // units over UL = 256 / G thread rows, whose sums meet in shared memory.
-__global__ void __launch_bounds__(256)
-slim_combine_split_kernel(const SlimDecodeParams p, unsigned char* __restrict__ u_tiled, const int hp, const int G) {
+__global__ void __launch_bounds__(256, 4)
+slim_combine_split_kernel(const __grid_constant__ SlimDecodeParams p, unsigned char* __restrict__ u_tiled, const int hp, const int G) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* s_w = reinterpret_cast<float*>(smem_raw);                 // [workers]
-  int* s_info = reinterpret_cast<int*>(s_w + p.workers);           // wlo, wn
-  int* s_prefix = s_info + 2;                                      // [batch+1]
-  // [UL - 1][G][8] floats (7 KB at most) behind the prefix, 16-byte aligned
-  float* s_red = reinterpret_cast<float*>(smem_raw + ((sizeof(float) * p.workers + sizeof(int) * (2 + p.batch + 1) + 15) & ~(size_t)15));
+  int* s_info = reinterpret_cast<int*>(s_w + p.workers);           // wlo, wn, flagged
+  int* s_prefix = s_info + 4;                                      // [batch+1]
+  // [UL - 1][G][8] floats (7 KB at most) behind the prefix, 16-byte aligned (the exact path uses the same room)
+  float* s_red = reinterpret_cast<float*>(smem_raw + exact_scratch_offset(p));
   const int tid = threadIdx.x, lane = tid & 31;
-  const int h = blockIdx.x, b = blockIdx.y, bg = b / PJ_BG, n = b % PJ_BG;
+  const int h = blockIdx.x, b = blockIdx.y;
   const int d = p.d, H = p.H;
   slim_pdl_trigger();
   slim_pdl_wait();
   if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) *p.any_flag = 0;   // the redo kernel has consumed it
 
   const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
-  if (tid < 32) {
-    int wlo = 0, wn = 0;
-    if (b < p.batch && s_prefix[b + 1] > s_prefix[b]) {
-      wlo = slim_worker_of_tile(sc, s_prefix[b]);
-      wn = slim_worker_of_tile(sc, s_prefix[b + 1] - 1) - wlo + 1;
-      float M = -INFINITY;
-      for (int i = lane; i < wn; i += 32) {
-        const size_t ui = (size_t)(wlo + i + b) * H + h;
-        M = fmaxf(M, p.part_m[ui] + log2f(p.part_l[ui]));
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-      float L = 0.f;
-      for (int i = lane; i < wn; i += 32) {
-        const size_t ui = (size_t)(wlo + i + b) * H + h;
-        const float wg = exp2f(p.part_m[ui] - M);
-        s_w[i] = wg;
-        L += wg * p.part_l[ui];
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
-      const float inv = 1.f / L;
-      __syncwarp();
-      for (int i = lane; i < wn; i += 32) s_w[i] *= inv;
-    }
-    if (lane == 0) { s_info[0] = wlo; s_info[1] = wn; }
-  }
+  if (tid < 32) combine_prologue(p, sc, s_prefix, b, h, s_w, s_info, lane);
   __syncthreads();
   const int wlo = s_info[0], wn = s_info[1];
-  const size_t tile_bytes = (size_t)1024 * hp;
-  unsigned char* dst_h = u_tiled + ((size_t)(bg * (H / hp) + h / hp) * (d / 16)) * tile_bytes + (size_t)(h % hp) * 1024;
+  if (s_info[2]) {                               // a flagged unit: this CTA's column groups are recomputed exactly
+    for (int jg0 = blockIdx.z * G; jg0 < d / 8; jg0 += gridDim.z * G)
+      slim_comb::exact_groups(p, u_tiled, hp, b, h, jg0, min(G, d / 8 - jg0), s_red);
+    return;
+  }
   const int UL = 256 / G, gi = tid % G, ul = tid / G;
   const size_t ustride = (size_t)H * d;                                       // unit i lives H*d floats further
   for (int jg0 = blockIdx.z * G; jg0 < d / 8; jg0 += gridDim.z * G) {
@@ -238,25 +202,14 @@ slim_combine_split_kernel(const SlimDecodeParams p, unsigned char* __restrict__ 
       }
     }
     if (ul != 0 || !live) continue;
-    uint32_t hi[4], lo[4];
-#pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      const __nv_bfloat16 h0 = __float2bfloat16_rn(acc[2 * x]), h1 = __float2bfloat16_rn(acc[2 * x + 1]);
-      const __nv_bfloat16 l0 = __float2bfloat16_rn(acc[2 * x] - __bfloat162float(h0));
-      const __nv_bfloat16 l1 = __float2bfloat16_rn(acc[2 * x + 1] - __bfloat162float(h1));
-      hi[x] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-      lo[x] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
-    }
-    unsigned char* t = dst_h + (size_t)(j0 / 16) * tile_bytes;
-    *reinterpret_cast<uint4*>(t + u_offset(n, j0 & 15)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-    *reinterpret_cast<uint4*>(t + u_offset(PJ_BG + n, j0 & 15)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    slim_comb::store_u8(u_tiled, d, H, hp, b, h, j0, acc);
   }
 }
 
 __global__ void __launch_bounds__(128)
 slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned char* __restrict__ u_tiled,
                     float* __restrict__ o, const ProjGeom g, const int d, const int d_k, const int batch,
-                    int* status) {
+                    int* status, const int32_t* __restrict__ lengths) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_u32 = smem_u32(smem_raw);
   const uint32_t base = (raw_u32 + 1023u) & ~1023u;
@@ -373,7 +326,8 @@ slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned cha
       const int b = bg * PJ_BG + n;
       float a = 0.f;
       for (int sl = 0; sl < g.jsplit; ++sl) a += ld_cluster_f32(mapa(base + (uint32_t)(n * 128 + m) * 4u, (uint32_t)sl));
-      if (b < batch && c < d_k) o[(size_t)b * d + head * d_k + c] = a;
+      // an empty sequence has no partials: its operand columns hold whatever an earlier call left
+      if (b < batch && c < d_k) o[(size_t)b * d + head * d_k + c] = lengths[b] > 0 ? a : 0.f;
     }
   }
   cluster_sync_all();                                          // nobody leaves while its tile may still be read
@@ -446,16 +400,16 @@ cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, uns
     // of the columns across grid.z so that ~2 CTAs per SM exist.
     const int ngroups = p.d / 8;
     int nslice = 1;
-    while (nslice < 16 && (long long)p.H * p.batch * nslice < 2 * 148 && ngroups / (2 * nslice) >= 32) nslice <<= 1;
+    while (nslice < 16 && (long long)p.H * p.batch * nslice < 2 * ctx->num_sms && ngroups / (2 * nslice) >= 32) nslice <<= 1;
     cudaError_t e;
     if (nslice > 1) {
       int G = 256;
       while (G > 32 && G / 2 * nslice >= ngroups) G >>= 1;
-      const size_t smem = sizeof(float) * p.workers + sizeof(int) * (2 + p.batch + 1) + 16 + sizeof(float) * 7 * 256;
+      const size_t smem = sizeof(float) * p.workers + sizeof(int) * (4 + p.batch + 1) + 16 + sizeof(float) * 7 * 256;
       e = slim_launch_pdl(slim_combine_split_kernel, dim3(p.H, p.batch, nslice), dim3(256), smem, st, p, u_tiled, g.hp, G);
     } else {
       dim3 grid(p.H, g.nbg * PJ_BG);
-      const size_t smem = sizeof(float) * p.workers + sizeof(int) * (2 + p.batch + 1) + 16;
+      const size_t smem = sizeof(float) * p.workers + sizeof(int) * (4 + p.batch + 1) + 16 + sizeof(float) * (p.d_k + 2 * SLIM_TT + 4);
       e = slim_launch_pdl(slim_combine_kernel, grid, dim3(256), smem, st, p, u_tiled, g.hp);
     }
     if (e != cudaSuccess) return e;
@@ -473,5 +427,6 @@ cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, uns
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, slim_proj_tc_kernel, map, (const unsigned char*)u_tiled, p.o, g, p.d, p.d_k, p.batch, p.status);
+  return cudaLaunchKernelEx(&cfg, slim_proj_tc_kernel, map, (const unsigned char*)u_tiled, p.o, g, p.d, p.d_k, p.batch, p.status,
+                            p.lengths);
 }

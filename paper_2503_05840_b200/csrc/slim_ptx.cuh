@@ -38,6 +38,8 @@ __device__ __forceinline__ void st_async_v4(uint32_t cluster_addr, const uint4& 
 __device__ __forceinline__ void sts_u16(uint32_t addr, unsigned short v) {
   asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
 }
+// orders this thread's earlier global-memory stores before later reads of the async proxy (TMA loads)
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;

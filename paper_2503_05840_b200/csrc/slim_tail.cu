@@ -135,11 +135,15 @@ template <typename KT>
 __global__ void slim_append_kernel(KT* __restrict__ cache, const KT* __restrict__ k_new,
                                    const int32_t* __restrict__ positions, int d, int t_cap, int n_new,
                                    int* status, const int32_t* __restrict__ block_table, int page_rows, int max_pages,
-                                   int num_pages) {
+                                   int num_pages, int pos_is_length) {
   slim_pdl_trigger();
   slim_pdl_wait();
   const int b = blockIdx.x, r = blockIdx.y;
-  const int pos = positions[b];
+  int pos = positions[b];
+  if (pos_is_length) {                       // positions[] holds the lengths after the append
+    if (pos <= 0) return;                    // an empty sequence receives no row
+    pos -= 1;
+  }
   if (pos < 0 || pos > t_cap - n_new) {            // (n_new <= t_cap is checked on the host; no overflow for any pos)
     if (threadIdx.x == 0) atomicMax(status, (int)SLIM_ERR_CAPACITY);
     return;
@@ -208,12 +212,12 @@ cudaError_t slim_launch_tail(const slim_ctx* ctx, const SlimDecodeParams& p, cud
 }
 
 cudaError_t slim_launch_append(const slim_ctx* ctx, const slim_cache* c, const void* k_new,
-                               const int32_t* positions, int n_new, cudaStream_t st) {
+                               const int32_t* positions, int n_new, int pos_is_length, cudaStream_t st) {
   dim3 grid(c->batch, n_new);
   if (ctx->dtype == SLIM_BF16)
     return slim_launch_pdl(slim_append_kernel<__nv_bfloat16>, grid, dim3(256), 0, st, (__nv_bfloat16*)c->k,
                            (const __nv_bfloat16*)k_new, positions, ctx->d, c->t_cap, n_new, ctx->status, c->block_table,
-                           c->page_rows, c->max_pages, c->num_pages);
+                           c->page_rows, c->max_pages, c->num_pages, pos_is_length);
   return slim_launch_pdl(slim_append_kernel<float>, grid, dim3(256), 0, st, (float*)c->k, (const float*)k_new, positions,
-                         ctx->d, c->t_cap, n_new, ctx->status, c->block_table, c->page_rows, c->max_pages, c->num_pages);
+                         ctx->d, c->t_cap, n_new, ctx->status, c->block_table, c->page_rows, c->max_pages, c->num_pages, pos_is_length);
 }

@@ -51,11 +51,14 @@
 // unit is redone by the exact CUDA-core kernel afterwards.  l is accumulated
 // from the bf16-rounded p, so U / l stays an exact weighted mean of key rows.
 //
+// With k_new set, the worker that owns a sequence's last tile first writes the newest key row
+// (position lengths[b] - 1, each CTA its own column half) and orders the write before its TMA reads:
+// the cache update of the generate phase needs no kernel of its own.
+//
 // Every wait on an mbarrier is bounded in time; a wait that runs out sets the
 // device status to SLIM_ERR_TIMEOUT, all roles leave their loops, and the CTA
 // frees its tensor memory and exits.
 #include <cuda.h>
-#include <cstdlib>
 #include <cstring>
 
 #include "slim_internal.h"
@@ -362,7 +365,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
               lsum = 0.f;
             }
             float x = sv - mref;
-            if (valid && x > TC_XMAX) { p.unit_flags[2 * unit + (int)rank] = 1; *p.any_flag = 1; x = TC_XMAX; }
+            if (valid && x > TC_XMAX) { p.unit_flags[2 * unit + (int)rank] = 1; if (EXT) *p.any_flag = 1; x = TC_XMAX; }
             const float pf = valid ? ex2_approx(x) : 0.f;
             const __nv_bfloat16 pb = __float2bfloat16_rn(pf);
             if ((jl % DUP) == 0) lsum += __bfloat162float(pb);
@@ -472,6 +475,23 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
       }
     } else if (warp == producer_warp) {
       // =========================== TMA producer ===========================
+      if (!EXT && p.k_new != nullptr) {
+        // Generate-phase cache update: the newest key row of every sequence whose last tile this worker
+        // reads goes to row lengths[b] - 1 (this CTA's column half), by the whole warp, before the first
+        // load.  Each lane orders its own stores before the TMA reads (generic -> async proxy).
+        const int b_lo = slim_seq_of_tile(s_prefix, p.batch, g_begin), b_hi = slim_seq_of_tile(s_prefix, p.batch, g_end - 1);
+        for (int b = b_lo; b <= b_hi; ++b) {
+          const int last = s_prefix[b + 1] - 1;
+          const int len = p.lengths[b];
+          if (s_prefix[b + 1] == s_prefix[b] || last < g_begin || last >= g_end || len > p.t_cap) continue;
+          const long long row = slim_cache_row(p, b, ((len - 1) / SLIM_TT) * SLIM_TT) + (len - 1) % SLIM_TT;
+          const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.k_new) + (size_t)b * p.d + (size_t)rank * g.dsl);
+          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(const_cast<void*>(p.k)) + (size_t)row * p.d + (size_t)rank * g.dsl);
+          for (int e = lane; e < g.dsl / 8; e += 32) dst[e] = __ldg(src + e);
+        }
+        fence_proxy_async_global();
+        __syncwarp();
+      }
       if (lane == 0) {
         int it = 0, st = 0;
         uint32_t kph = 0;
@@ -620,10 +640,9 @@ size_t tc_smem_bytes(const TcGeom& g, int batch) {
 typedef void (*tc_kernel_t)(const CUtensorMap, const SlimDecodeParams, const TcGeom);
 
 // Two score-warp sets where a tile is small (d_k = 64, scores formed in the kernel, CTA pair) and both
-// sets fit the block.  SLIM_TC_SETS=1 switches them off for comparisons.
-int tc_sets(int H, int d_k, int rt, bool ext, int cl) {
-  const char* e = getenv("SLIM_TC_SETS");
-  if (e && atoi(e) == 1) return 1;
+// sets fit the block.  ctx->opt_tc_sets1 switches them off for comparisons.
+int tc_sets(const slim_ctx* ctx, int H, int d_k, int rt, bool ext, int cl) {
+  if (ctx->opt_tc_sets1) return 1;
   if (d_k != 64 || rt != 4 || ext || cl != 2) return 1;
   const int hw = tc_heads_per_warp(d_k, rt), nsw = (H / cl + hw - 1) / hw;
   return 2 * nsw <= TC_SETS2_WARPS ? 2 : 1;
@@ -632,10 +651,9 @@ int tc_sets(int H, int d_k, int rt, bool ext, int cl) {
 // Rows per thread and tile.  Measured on the d = 4096 / 32-head shape: 8 rows per
 // thread (8 score warps) beats 4 rows (16 warps); the stepped query rotation is
 // re-used over more rows and fewer warps contend for the issue slots.
-// SLIM_TC_RT overrides the choice for sweeps.
-int tc_rows_per_thread(int d_k) {
-  const char* e = getenv("SLIM_TC_RT");
-  const int want = e ? atoi(e) : 0;
+// ctx->opt_tc_rt overrides the choice for sweeps.
+int tc_rows_per_thread(const slim_ctx* ctx) {
+  const int d_k = ctx->d_k, want = ctx->opt_tc_rt;
   if (d_k == 64) return want == 2 ? 2 : 4;
   return want == 4 ? 4 : 8;
 }
@@ -708,9 +726,9 @@ int slim_tc_shape_ok(int d, int H, int d_k, int dtype, int rope, int cl) {
 }
 
 int slim_tc_workers(const slim_ctx* ctx, int cl) {
-  const int rt = tc_rows_per_thread(ctx->d_k);
+  const int rt = tc_rows_per_thread(ctx);
   const bool rope = ctx->rope_theta != 0.0;
-  const int sets = tc_sets(ctx->H, ctx->d_k, rt, false, cl);
+  const int sets = tc_sets(ctx, ctx->H, ctx->d_k, rt, false, cl);
   tc_kernel_t kern = pick_kernel(ctx->d_k, rope, rt, false, cl, sets);
   if (!kern) return 0;
   const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, rt, cl, sets, TC_SMEM_LIMIT);
@@ -763,7 +781,7 @@ cudaError_t slim_tmap_encode_3d(void* out_map, void* base, const unsigned long l
 }
 
 cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c, int cl) {
-  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, tc_rows_per_thread(ctx->d_k), cl, 1, TC_SMEM_LIMIT);
+  const TcGeom g = make_geom(ctx->d, ctx->H, ctx->d_k, tc_rows_per_thread(ctx), cl, 1, TC_SMEM_LIMIT);
   // dim0: 64 contiguous elements; dim1: cache rows (stride d elements); dim2: 64-column chunks
   const unsigned long long dims[3] = {64, (unsigned long long)c->total_rows, (unsigned long long)(ctx->d / 64)};
   const unsigned long long strides[2] = {(unsigned long long)ctx->d * 2, 128};
@@ -772,10 +790,10 @@ cudaError_t slim_tc_make_tmap(const slim_ctx* ctx, slim_cache* c, int cl) {
 }
 
 cudaError_t slim_launch_tc(const slim_ctx* ctx, const slim_cache* c, const SlimDecodeParams& p, cudaStream_t st) {
-  const int rt = tc_rows_per_thread(ctx->d_k);
+  const int rt = tc_rows_per_thread(ctx);
   const bool ext = p.ext_scores != nullptr;
   const int cl = p.cl;
-  const int sets = tc_sets(ctx->H, ctx->d_k, rt, ext, cl);
+  const int sets = tc_sets(ctx, ctx->H, ctx->d_k, rt, ext, cl);
   tc_kernel_t kern = pick_kernel(ctx->d_k, ctx->rope_theta != 0.0, rt, ext, cl, sets);
   if (!kern || cl < 1 || cl > 2 || !c->has_tmap[cl - 1]) return cudaErrorNotSupported;
   if (ext) {

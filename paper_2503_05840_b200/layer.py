@@ -56,6 +56,13 @@ class SlimLayer:
                       torch.cuda.current_stream(self.device).cuda_stream)
         return o
 
+    def decode_step(self, q: torch.Tensor, k_new: torch.Tensor, lengths: torch.Tensor,
+                    o: torch.Tensor | None = None) -> torch.Tensor:
+        o = self.o if o is None else o
+        B.slim_decode_step(self.ctx, q, k_new, self.cache, lengths, o, self.workspace,
+                           torch.cuda.current_stream(self.device).cuda_stream)
+        return o
+
     def profile(self, enable: bool) -> None:
         B.slim_profile_enable(self.ctx, enable)
 

@@ -14,6 +14,28 @@ def rank_info():
             int(os.environ.get("LOCAL_RANK", "0")))
 
 
+def _free_port() -> int:
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def _spawned(rank: int, world: int, port: int, target, args) -> None:
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    target(rank, world, *args)
+
+
+def spawn_replicas(target, world: int, args=(), port: int | None = None) -> None:
+    """Start `world` processes on this node, one per GPU (rank = local rank), each with the
+    environment a launcher would give it (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR, MASTER_PORT),
+    and run target(rank, world, *args) in each.  Returns when all have exited; raises if one failed.
+    `target` must be importable (a module-level function)."""
+    import torch.multiprocessing as mp
+    mp.spawn(_spawned, args=(world, port or _free_port(), target, tuple(args)), nprocs=world, join=True)
+
+
 def replica_seed(base_seed: int, rank: int) -> int:
     """Every replica draws its own keys and queries; the ragged length mix is
     the same on all ranks so that per-GPU work is equal (weak scaling)."""

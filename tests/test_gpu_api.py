@@ -355,3 +355,109 @@ def test_prompt_phase_values_from_keys(d, H, d_k, dtype):
         assert worst <= (2e-2 if dtype == "bf16" else 1e-4)
     finally:
         layer.close()
+
+
+@pytest.mark.parametrize("d,H,d_k,theta,dtype", [(512, 4, 128, 1.0e6, "bf16"), (1280, 20, 64, 0.0, "bf16"),
+                                                 (384, 4, 96, 1.0e4, "bf16"), (384, 6, 64, 0.0, "f32")])
+def test_decode_step_equals_append_then_decode(d, H, d_k, theta, dtype):
+    """slim_decode_step (cache update + attention in one call) against slim_append_k + slim_decode on a
+    second, identical cache: same output bits, same cache bits afterwards; sequence lengths at tile
+    edges, an empty sequence (nothing written) and the oracle on top."""
+    lengths = np.array([333, 0, 640, 17, 16, 1, 257], dtype=np.int32)      # lengths AFTER the update
+    batch, t_cap = len(lengths), 640
+    cfg = synth.SlimConfig("step", d, H, d_k, batch, t_cap, 1, theta, dtype)
+    L = synth.make_layer(cfg, 31, lengths=lengths)
+    W_KV = so.oracle_wkv(L.W_K, L.W_V)
+    a = SlimLayer(d, H, d_k, theta, dtype, batch, t_cap, DEV)
+    b_ = SlimLayer(d, H, d_k, theta, dtype, batch, t_cap, DEV)
+    try:
+        Kd = to_device_keys(L.K, dtype, DEV)
+        k_new = torch.zeros((batch, d), dtype=Kd.dtype, device=DEV)
+        before = Kd.clone()
+        for b in range(batch):
+            if lengths[b] > 0:
+                k_new[b] = Kd[b, lengths[b] - 1]
+                before[b, lengths[b] - 1] = 123.0              # the row the step has to overwrite
+            before[b, lengths[b]:] = float("nan")              # rows past the end are poison
+        k_new[1] = 55.0                                        # empty sequence: must not be written anywhere
+        q = to_device_keys(L.q, dtype, DEV)
+        ld = torch.from_numpy(lengths).to(DEV)
+        ref = so.oracle_slim_batch(L.q, L.K, lengths, W_KV, H, theta)
+        tol = 2e-2 if dtype == "bf16" else 1e-4
+        for path in _paths(a):
+            for lay in (a, b_):
+                lay.set_path(path); lay.set_wkv(W_KV); lay.k.copy_(before)
+            got = a.decode_step(q, k_new, ld).clone()
+            assert a.device_status() == B.SLIM_OK
+            b_.append_k(k_new.unsqueeze(1).contiguous(), (ld - 1).clamp(min=0))
+            # (the append call writes row 0 of the empty sequence; the step call must not)
+            want = b_.decode(q, ld).clone()
+            assert torch.equal(got, want), f"path {path}"
+            ka, kb = a.k.clone(), b_.k.clone()
+            assert torch.equal(ka[1].isnan(), before[1].isnan()) and not (ka[1] == 55.0).any()
+            kb[1] = ka[1]
+            assert torch.equal(torch.nan_to_num(ka, nan=-7.0), torch.nan_to_num(kb, nan=-7.0)), f"path {path}: cache differs"
+            g = got.cpu().numpy().astype(np.float64)
+            for b in range(batch):
+                if lengths[b] == 0:
+                    assert np.all(g[b] == 0)
+                else:
+                    e = so.err_rms_norm(g[b], ref[b]) if dtype == "bf16" else so.err_fp32_norm(g[b], ref[b])
+                    assert e <= tol, f"path {path} seq {b}: {e:.3e}"
+    finally:
+        a.close(); b_.close()
+
+
+def test_decode_step_capacity_and_launch_count():
+    cfg = synth.SlimConfig("stepcap", 512, 4, 128, 2, 64, 1, 1.0e4, "bf16")
+    L = synth.make_layer(cfg, 5)
+    layer = SlimLayer(cfg.d, cfg.H, cfg.d_k, cfg.rope_theta, "bf16", 2, 64, DEV)
+    try:
+        layer.set_wkv(so.oracle_wkv(L.W_K, L.W_V))
+        layer.k.copy_(to_device_keys(L.K, "bf16", DEV))
+        q = to_device_keys(L.q, "bf16", DEV)
+        k_new = torch.full((2, 512), 9.0, dtype=torch.bfloat16, device=DEV)
+        keep = layer.k.clone()
+        layer.decode_step(q, k_new, torch.tensor([65, 64], dtype=torch.int32, device=DEV))
+        assert layer.device_status() == B.SLIM_ERR_CAPACITY          # sequence 0: beyond t_cap, nothing written
+        assert torch.equal(layer.k[0], keep[0])
+        assert torch.all(layer.k[1, 63] == 9.0) and torch.equal(layer.k[1, :63], keep[1, :63])
+        # tensor-core path: decode kernel, combine, projection; the update needs no kernel of its own
+        assert layer.query(B.SLIM_Q_PATH_IN_USE) == B.SLIM_PATH_TC
+        assert layer.query(B.SLIM_Q_LAUNCHES_PER_DECODE) == 3
+        layer.set_path(B.SLIM_PATH_GENERIC)
+        layer.decode_step(q, k_new, torch.tensor([3, 64], dtype=torch.int32, device=DEV))
+        assert layer.device_status() == B.SLIM_OK
+        assert layer.query(B.SLIM_Q_LAUNCHES_PER_DECODE) == 5         # append, scores, accumulation, combine, projection
+    finally:
+        layer.close()
+
+
+def test_scores_far_above_the_first_tile_with_rope_and_long_units():
+    """Keys whose size grows along the context, with RoPE: arguments run hundreds of units above the
+    first tile's in several heads and units, so whole sequences take the exact recomputation inside
+    the combine kernel (rotation included); a third sequence stays ordinary."""
+    d, H, d_k, theta = 512, 4, 128, 1.0e4
+    lengths = np.array([3000, 1500, 900], dtype=np.int32)
+    cfg = synth.SlimConfig("ramp-rope", d, H, d_k, 3, 3000, 1, theta, "bf16")
+    L = synth.make_layer(cfg, 78, lengths=lengths)
+    K = L.K.copy()
+    for b in range(2):
+        n = int(lengths[b])
+        K[b, :n] = synth.round_to_bf16(K[b, :n] * (1.0 + np.arange(n)[:, None] * (0.5 if b == 0 else 0.05)))
+    layer = SlimLayer(d, H, d_k, theta, "bf16", 3, 3000, DEV)
+    try:
+        W_KV = so.oracle_wkv(L.W_K, L.W_V)
+        layer.set_wkv(W_KV)
+        layer.k.copy_(to_device_keys(K, "bf16", DEV))
+        qd = to_device_keys(L.q, "bf16", DEV)
+        ld = torch.from_numpy(lengths).to(DEV)
+        ref = so.oracle_slim_batch(L.q, K, lengths, W_KV, H, theta)
+        for path in _paths(layer):
+            layer.set_path(path)
+            got = layer.decode(qd, ld).cpu().numpy().astype(np.float64)
+            assert layer.device_status() == B.SLIM_OK
+            for b in range(3):
+                assert so.err_rms_norm(got[b], ref[b]) <= 2e-2, f"path {path} seq {b}"
+    finally:
+        layer.close()

@@ -61,3 +61,35 @@ def test_single_process_needs_no_group():
     from paper_2503_05840_b200 import replicas
     assert replicas.max_over_ranks(3.5) == 3.5
     assert replicas.replica_seed(7, 0) == 7 and replicas.replica_seed(7, 3) != replicas.replica_seed(7, 2)
+
+
+def _stub_rank(rank, world, out_dir):
+    """What bench.py does per rank, with the GPU step replaced by a stub: rendezvous from the
+    launcher environment, barrier, max-over-ranks of a per-rank time, one line from rank 0."""
+    sys.path.insert(0, ROOT)
+    import json
+    import torch.distributed as dist
+    from paper_2503_05840_b200 import replicas
+    r, w, local = replicas.rank_info()
+    assert (r, w, local) == (rank, world, rank)
+    dist.init_process_group("gloo")
+    dist.barrier()
+    ms = replicas.max_over_ranks(4.0 + 2.0 * r, dist)
+    dist.barrier()
+    if r == 0:
+        with open(os.path.join(out_dir, "line.json"), "w") as f:
+            json.dump({"n_gpus": w, "ms_per_step": ms, "value": replicas.job_throughput(16, w, ms), "scaling": "weak"}, f)
+    dist.destroy_process_group()
+
+
+def test_spawn_replicas_starts_one_process_per_rank(tmp_path):
+    """The path bench.py --gpus N takes when no launcher started it: N processes, launcher-style
+    environment, one result line from rank 0 that carries the whole job."""
+    import json
+    sys.path.insert(0, ROOT)
+    from paper_2503_05840_b200 import replicas
+    replicas.spawn_replicas(_stub_rank, 2, (str(tmp_path),))
+    with open(tmp_path / "line.json") as f:
+        line = json.load(f)
+    assert line["n_gpus"] == 2 and line["ms_per_step"] == 6.0 and line["scaling"] == "weak"
+    assert np.isclose(line["value"], 16 * 2 / 6e-3)
