@@ -28,6 +28,13 @@ Paper passages followed (arxiv 2503.05840):
                         W_K in R^{d x e}, e = d_k h > d;  W_KV = W_K^{-1} W_V
                         is e x e
 
+  Appendix "Taking advantage of softmax sparsities" with appendix "Support for
+  RoPE", Option 2     the cache holds RoPE'd keys; attention scores below a
+                        threshold are skipped in the weighted sum, and only the
+                        key rows that are kept are RoPE-decoded before they
+                        enter it (oracle_rotated_cache).  Not exact: the skipped
+                        scores are simply left out, nothing is renormalised.
+
 Readings where the paper is silent (the CUDA path takes the same ones):
   * RoPE pairs element j with j + d_k/2 inside a head, frequency
     theta_j = rope_theta ** (-2 j / d_k), angle = position * theta_j;
@@ -222,6 +229,41 @@ def oracle_xcache(q: np.ndarray, X: np.ndarray, W_K: np.ndarray, W_V: np.ndarray
         u = s @ X                                     # [d]
         out[sl] = u @ W_V[:, sl]                      # [d_k]
     return out
+
+
+def oracle_rotated_cache(q: np.ndarray, K_rot: np.ndarray, W_KV: np.ndarray, H: int, rope_theta: float,
+                         threshold: float):
+    """Sparsity appendix + RoPE appendix Option 2.  K_rot: [T, d] keys stored ALREADY rotated
+    (head slice i of row t encoded at position t).  Per head i:
+      s = softmax(RoPE_{T-1}(q_i) . K_rot,i^T / sqrt(d_k))         (no rotation at read time)
+      keep = { t : s_t > threshold }                               (scores at or below it are skipped)
+      u_i = sum_{t in keep} s_t * RoPE-decode_t(K_rot[t, :])       (full-width row, every head slice decoded)
+      head_i = u_i W_KV,i
+    The kept scores are used as they are (the paper skips vectors, it does not renormalise), so with
+    threshold < min s the result is oracle_slim on the raw keys, and the error of a larger threshold is
+    bounded by the skipped probability mass times the largest value row.
+    Returns (out [d], kept [H] number of rows decoded per head)."""
+    q = np.asarray(q, dtype=F64)
+    K_rot = np.asarray(K_rot, dtype=F64)
+    W_KV = np.asarray(W_KV, dtype=F64)
+    T, d = K_rot.shape
+    d_k = d // H
+    pos = np.arange(T)
+    out = np.empty(d, dtype=F64)
+    kept = np.zeros(H, dtype=np.int64)
+    for i in range(H):
+        sl = slice(i * d_k, (i + 1) * d_k)
+        qr = rope_encode(q[sl], T - 1, rope_theta)
+        s = softmax(K_rot[:, sl] @ qr / math.sqrt(d_k))                 # [T]
+        keep = np.nonzero(s > threshold)[0]
+        kept[i] = keep.size
+        u = np.zeros(d, dtype=F64)
+        if keep.size:
+            rows = K_rot[keep].reshape(keep.size, H, d_k)               # decode every head slice of the kept rows
+            raw = rope_decode(rows, pos[keep][:, None], rope_theta).reshape(keep.size, d)
+            u = s[keep] @ raw
+        out[sl] = u @ W_KV[:, sl]
+    return out, kept
 
 
 def oracle_slim_batch(q: np.ndarray, K: np.ndarray, lengths, W_KV: np.ndarray, H: int,

@@ -462,3 +462,86 @@ def test_two_head_pin_catches_a_strided_head_slice():
         s = so.softmax(X[:, cols] @ X[1, cols] / math.sqrt(2.0))
         out[cols] = s @ V[:, cols]
     assert np.max(np.abs(out - expect)) > 1e-2
+
+
+# ---- rotated-key cache with skipped scores (sparsity appendix + RoPE appendix Option 2) -------------
+def _rotated(K, H, theta):
+    T, d = K.shape
+    return so.rope_encode(K.reshape(T, H, d // H), np.arange(T)[:, None], theta).reshape(T, d)
+
+
+def test_rotated_cache_hand_case_one_row_skipped():
+    # one head of width 2, theta = 10000 (one frequency, angle = position): key 1 is stored rotated by
+    # 1 rad (typed with cos 1, sin 1), key 0 at position 0 is stored as it is.  q is chosen so that the
+    # rotated query is (1, 0): q = decode_1((1, 0)) = (cos 1, sin 1).  Scores: z0 = k0r[0]/sqrt 2,
+    # z1 = k1r[0]/sqrt 2 with k0r = (0, 3), k1r = (sqrt 2 ln 9, 5)  =>  z1 - z0 = ln 9, s = (0.1, 0.9).
+    c1, s1 = math.cos(1.0), math.sin(1.0)
+    q = np.array([c1, s1])
+    K_rot = np.array([[0.0, 3.0], [math.sqrt(2.0) * math.log(9.0), 5.0]])
+    W_KV = np.array([[1.0, 2.0], [3.0, 4.0]])
+    # raw keys by the decoding formulas: x1 = y1 cos - y2 sin, x2 = y1 sin + y2 cos
+    k0 = K_rot[0]
+    k1 = np.array([K_rot[1][0] * c1 - K_rot[1][1] * s1, K_rot[1][0] * s1 + K_rot[1][1] * c1])
+    v0, v1 = k0 @ W_KV, k1 @ W_KV
+    full, kept = so.oracle_rotated_cache(q, K_rot, W_KV, 1, 10000.0, threshold=0.0)
+    assert kept[0] == 2 and np.allclose(full, 0.1 * v0 + 0.9 * v1, rtol=1e-12)
+    cut, kept = so.oracle_rotated_cache(q, K_rot, W_KV, 1, 10000.0, threshold=0.5)
+    assert kept[0] == 1 and np.allclose(cut, 0.9 * v1, rtol=1e-12)          # skipped, not renormalised
+    none, kept = so.oracle_rotated_cache(q, K_rot, W_KV, 1, 10000.0, threshold=0.95)
+    assert kept[0] == 0 and np.all(none == 0)
+
+
+@pytest.mark.parametrize("theta", [0.0, 1.0e4, 1.0e6])
+def test_rotated_cache_without_skipping_is_vanilla_attention(theta):
+    T, d, H = 37, 32, 4
+    X, W_Q, W_K, W_V = _rand_case(31, T, d, H)
+    K = X @ W_K
+    out, kept = so.oracle_rotated_cache(X[-1] @ W_Q, _rotated(K, H, theta), so.oracle_wkv(W_K, W_V), H, theta, threshold=-1.0)
+    ref = so.oracle_vanilla(X, W_Q, W_K, W_V, H, theta)
+    assert np.all(kept == T)
+    assert np.max(np.abs(out - ref)) <= 1e-10 * np.max(np.abs(ref))
+
+
+def test_rotated_cache_error_is_bounded_by_the_skipped_mass_and_work_shrinks():
+    # peaked attention: a few keys aligned with the query.  For every head the error of the skipped
+    # sum is at most (skipped probability mass) x (largest value row norm), and the rows decoded are
+    # exactly those above the threshold (complexity factor 1 / (1 - S) of the sparsity appendix).
+    g = np.random.default_rng(12)
+    T, d, H, theta = 200, 16, 2, 1.0e4
+    X, W_Q, W_K, W_V = _rand_case(32, T, d, H)
+    K = X @ W_K
+    q = X[-1] @ W_Q * 6.0
+    W_KV = so.oracle_wkv(W_K, W_V)
+    K_rot = _rotated(K, H, theta)
+    exact = so.oracle_slim(q, K, W_KV, H, theta)
+    V = K @ W_KV
+    d_k = d // H
+    for thr in (1e-4, 1e-2, 0.2):
+        out, kept = so.oracle_rotated_cache(q, K_rot, W_KV, H, theta, thr)
+        for i in range(H):
+            sl = slice(i * d_k, (i + 1) * d_k)
+            s = so.attention_weights(q[sl], K[:, sl], theta)
+            assert kept[i] == int(np.sum(s > thr))
+            skipped = float(np.sum(s[s <= thr]))
+            bound = skipped * np.max(np.linalg.norm(V[:, sl], axis=1))
+            assert np.linalg.norm(out[sl] - exact[sl]) <= bound + 1e-12
+    # S = 0.8 exactly: ten keys, two of them carry everything above the threshold
+    qh = np.array([1.0, 0.0]); Kh = np.zeros((10, 2)); Kh[[3, 7], 0] = 20.0
+    _, kept = so.oracle_rotated_cache(qh, Kh, np.eye(2), 1, 0.0, threshold=1e-3)
+    assert kept[0] == 2                                  # 1 / (1 - 0.8) = 5 times fewer rows in the weighted sum
+
+
+def test_rotated_cache_pin_catches_a_missing_decode():
+    # the same sum with the kept rows used as stored (still rotated) must differ
+    T, d, H, theta = 20, 8, 2, 1.0e4
+    X, W_Q, W_K, W_V = _rand_case(33, T, d, H)
+    K = X @ W_K; q = X[-1] @ W_Q; W_KV = so.oracle_wkv(W_K, W_V)
+    K_rot = _rotated(K, H, theta)
+    good, _ = so.oracle_rotated_cache(q, K_rot, W_KV, H, theta, -1.0)
+    bad = so.oracle_slim(q, K, W_KV, H, theta) * 0
+    d_k = d // H
+    for i in range(H):
+        sl = slice(i * d_k, (i + 1) * d_k)
+        s = so.attention_weights(q[sl], K[:, sl], theta)
+        bad[sl] = (s @ K_rot) @ W_KV[:, sl]
+    assert np.max(np.abs(good - bad)) > 1e-3 * np.max(np.abs(good))
