@@ -133,6 +133,19 @@ void        slim_cache_destroy(slim_cache* cache);
  * d_k in {64, 96, 128} runs on the tensor cores (16-byte aligned K and V), else on CUDA cores. */
 slim_status slim_values_from_keys(slim_ctx* ctx, const void* K, int n, float* V, void* stream);
 
+/* Prompt phase in one call (Fig. 3(a)): the prompt's keys are stored in the K-cache AND their values
+ * V = K W_KV (Eq. 6) are returned, from one pass over the keys.
+ *   k_new      device [batch][n_new][d], ctx dtype, un-rotated keys of the prompt tokens
+ *   positions  device int32 [batch]: first cache row of sequence b (0 for a fresh prompt)
+ *   V          device [batch][n_new][d] float32
+ * Equivalent to slim_append_k(k_new, positions, n_new) + slim_values_from_keys on the same rows; a
+ * sequence whose rows would pass t_cap is left unwritten (device status SLIM_ERR_CAPACITY), its
+ * values are still returned.  On the tensor-core path (bf16, d_k in {64, 96, 128}, 16-byte aligned
+ * buffers) both happen in one kernel: otherwise idle warps of the GEMM CTAs store the rows while the
+ * same CTAs stream them, so the keys are read from HBM once.  Contiguous and paged caches.      */
+slim_status slim_prefill(slim_ctx* ctx, slim_cache* cache, const void* k_new, const int32_t* positions,
+                         int n_new, float* V, void* stream);
+
 /* Generate-phase cache update: for every sequence b write the n_new rows
  * k_new[b][0..n_new) (device, [batch][n_new][d], ctx dtype, un-rotated keys
  * k = x W_K) at rows positions[b] .. positions[b]+n_new-1 (device int32).

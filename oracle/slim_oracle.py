@@ -147,6 +147,12 @@ def oracle_wkv_right_inverse(W_K: np.ndarray, W_V: np.ndarray) -> np.ndarray:
     return W_K.T @ np.linalg.solve(G, W_V)            # e x e
 
 
+def oracle_prompt_values(K: np.ndarray, W_KV: np.ndarray) -> np.ndarray:
+    """Prompt phase (Fig. 3(a), Eq. 6): the values of all prompt tokens from their keys,
+    V = K W_KV.  K: [n, d] raw keys, returns [n, d]."""
+    return np.asarray(K, dtype=F64) @ np.asarray(W_KV, dtype=F64)
+
+
 # --------------------------------------------------------------------------
 # Eq. 4, 5, 2: vanilla MHA decode with an explicit V cache
 # --------------------------------------------------------------------------

@@ -33,6 +33,7 @@ SIGNATURES = {
     "slim_cache_create_paged": (c_int, [c_void_p, POINTER(c_void_p), c_void_p, c_int, c_int, c_void_p, c_int, c_int]),
     "slim_cache_destroy": (None, [c_void_p]),
     "slim_values_from_keys": (c_int, [c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
+    "slim_prefill": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
     "slim_append_k": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p]),
     "slim_decode": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "slim_decode_step": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -173,6 +174,12 @@ def slim_cache_destroy(cache: int) -> None:
 
 def slim_values_from_keys(ctx: int, K, n: int, V, stream: int = 0) -> None:
     _check(lib().slim_values_from_keys(c_void_p(ctx), _ptr(K), n, _ptr(V), c_void_p(stream)), "slim_values_from_keys")
+
+
+def slim_prefill(ctx: int, cache: int, k_new, positions, n_new: int, V, stream: int = 0) -> None:
+    """Prompt phase: store the prompt's keys and return V = K W_KV in one call."""
+    _check(lib().slim_prefill(c_void_p(ctx), c_void_p(cache), _ptr(k_new), _ptr(positions), n_new, _ptr(V),
+                              c_void_p(stream)), "slim_prefill")
 
 
 def slim_append_k(ctx: int, cache: int, k_new, positions, n_new: int, stream: int = 0) -> None:

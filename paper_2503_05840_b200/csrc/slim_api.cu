@@ -540,6 +540,20 @@ slim_status slim_values_from_keys(slim_ctx* ctx, const void* K, int n, float* V,
   return SLIM_OK;
 }
 
+slim_status slim_prefill(slim_ctx* ctx, slim_cache* cache, const void* k_new, const int32_t* positions, int n_new,
+                         float* V, void* stream) {
+  if (!ctx || !cache || !k_new || !positions || !V || cache->ctx != ctx) return SLIM_ERR_INVALID_ARG;
+  if (n_new <= 0 || n_new > 65535) return SLIM_ERR_INVALID_ARG;
+  if (n_new > cache->t_cap) return SLIM_ERR_CAPACITY;
+  if ((long long)cache->batch * n_new > 0x7fffffffLL) return SLIM_ERR_UNSUPPORTED;
+  if (!ctx->has_weights) return SLIM_ERR_NO_WEIGHTS;
+  if (slim_launch_values(ctx, k_new, cache->batch * n_new, V, (cudaStream_t)stream, cache, positions, n_new) != cudaSuccess) {
+    cudaGetLastError();
+    return SLIM_ERR_CUDA;
+  }
+  return SLIM_OK;
+}
+
 size_t slim_static_workspace_max(void) { return SLIM_STATIC_WS_BYTES; }
 
 slim_status slim_decode_static_ws(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,

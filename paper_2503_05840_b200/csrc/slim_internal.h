@@ -167,4 +167,5 @@ cudaError_t slim_launch_xscores_tc(const slim_ctx* ctx, const slim_cache* c, con
                                    unsigned char* qt_tiled, float* scores, cudaStream_t st);
 
 // prompt phase: V = K W_KV for n rows (slim_prompt.cu)
-cudaError_t slim_launch_values(const slim_ctx* ctx, const void* K, int n, float* V, cudaStream_t st);
+cudaError_t slim_launch_values(const slim_ctx* ctx, const void* K, int n, float* V, cudaStream_t st,
+                               const slim_cache* cache = nullptr, const int32_t* positions = nullptr, int n_new = 0);

@@ -8,10 +8,15 @@
 //                           projection uses); D in tensor memory (N = 128: one head of d_k = 128 or
 //                           96, or two heads of d_k = 64).
 //   slim_values_kernel      any dtype / shape: CUDA-core tiles.
+// With a cache given (slim_prefill) the same launch also stores the prompt's keys: the CTAs of head
+// group 0 have two warps that idle while one thread loads and one issues the MMAs; those warps copy
+// the CTA's 128 key rows into the K-cache (rows positions[b] ..), reading them through L2 while the
+// TMA of the same CTA streams them, so the prompt's keys leave HBM once.
 // Every mbarrier wait is bounded in time.
 #include <cstring>
 
 #include "slim_internal.h"
+#include "slim_sched.cuh"
 #include "slim_ptx.cuh"
 
 namespace {
@@ -23,9 +28,11 @@ constexpr int PV_A_BYTES = PV_ROWS * PV_J * 2;     // 16 KB
 constexpr int PV_B_BYTES = PV_J * 128 * 2;         // two 64-column atoms x 64 rows x 128 B = 16 KB
 constexpr int PV_NS = 3;                          // 97 KB per CTA: two CTAs per SM, one's epilogue under the other's MMAs
 
+// cp (cache side of slim_prefill; cp.k == NULL: values only): the fields of SlimDecodeParams that address
+// cache rows, plus q = the prompt's keys [batch][n_new][d], lengths = first row per sequence, workers = n_new.
 __global__ void __launch_bounds__(128)
 slim_values_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap wmap, float* __restrict__ V,
-                      const int n, const int d, const int d_k, const int hp, int* status) {
+                      const int n, const int d, const int d_k, const int hp, int* status, const SlimDecodeParams cp) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_u32 = smem_u32(smem_raw);
   const uint32_t base = (raw_u32 + 1023u) & ~1023u;
@@ -76,6 +83,20 @@ slim_values_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         const unsigned long long tt = globaltimer();
         while (!mbar_try_wait(bar_full + 8 * st, (j / PV_NS) & 1) && globaltimer() - tt < SLIM_WAIT_NS) {}
       }
+    }
+  } else if (warp >= 2 && hg == 0 && cp.k != nullptr) {
+    // bulk append: prompt row r = b * n_new + i goes to cache row (b, positions[b] + i); a sequence whose
+    // rows would pass the capacity is left unwritten and reported
+    const int n_new = cp.workers, t64 = tid - 64;
+    const uint4* src = reinterpret_cast<const uint4*>(cp.q);
+    uint4* dst = reinterpret_cast<uint4*>(const_cast<void*>(cp.k));
+    const int vec_per_row = d / 8;
+    for (int r = t0; r < min(t0 + PV_ROWS, n); ++r) {
+      const int b = r / n_new, i = r - b * n_new;
+      const int pos = cp.lengths[b];
+      if (pos < 0 || pos > cp.t_cap - n_new) { if (t64 == 0) atomicMax(status, (int)SLIM_ERR_CAPACITY); continue; }
+      const long long row = slim_cache_row(cp, b, pos + i);
+      for (int e = t64; e < vec_per_row; e += 64) dst[(size_t)row * vec_per_row + e] = __ldg(src + (size_t)r * vec_per_row + e);
     }
   } else if (warp == 1 && lane == 0) {
     bool ok = true;
@@ -151,9 +172,25 @@ constexpr size_t PV_SMEM = 1024 + (size_t)PV_NS * (PV_A_BYTES + PV_B_BYTES) + 16
 
 }  // namespace
 
-cudaError_t slim_launch_values(const slim_ctx* ctx, const void* K, int n, float* V, cudaStream_t st) {
+// cache != NULL (slim_prefill): K is [batch][n_new][d] and its rows are also stored at positions[b] ..
+cudaError_t slim_launch_values(const slim_ctx* ctx, const void* K, int n, float* V, cudaStream_t st, const slim_cache* cache,
+                               const int32_t* positions, int n_new) {
   const int d = ctx->d, d_k = ctx->d_k, H = ctx->H;
-  if (ctx->proj_ok && ((uintptr_t)K & 15) == 0 && ((uintptr_t)V & 15) == 0) {
+  const bool tc = ctx->proj_ok && ((uintptr_t)K & 15) == 0 && ((uintptr_t)V & 15) == 0;
+  SlimDecodeParams cp;
+  memset(&cp, 0, sizeof(cp));
+  if (cache) {
+    if (!tc || ((uintptr_t)cache->k & 15)) {         // no fused store on this path: the append kernel first
+      cudaError_t e = slim_launch_append(ctx, cache, K, positions, n_new, 0, st);
+      if (e != cudaSuccess) return e;
+    } else {
+      cp.k = cache->k; cp.q = K; cp.lengths = positions; cp.workers = n_new; cp.d = d;
+      cp.batch = cache->batch; cp.t_cap = cache->t_cap; cp.status = ctx->status;
+      cp.block_table = cache->block_table; cp.page_rows = cache->page_rows; cp.max_pages = cache->max_pages;
+      cp.num_pages = cache->num_pages;
+    }
+  }
+  if (tc) {
     // function attributes are kept per device: opt in once on each device this is called on
     static bool attr_set[64] = {};
     if (ctx->device < 0 || ctx->device >= 64 || !attr_set[ctx->device]) {
@@ -170,7 +207,7 @@ cudaError_t slim_launch_values(const slim_ctx* ctx, const void* K, int n, float*
     memcpy(&wmap, ctx->wmap, sizeof(wmap));
     const int hp = d_k == 64 ? 2 : 1;
     return slim_launch_pdl(slim_values_tc_kernel, dim3(H / hp, (n + PV_ROWS - 1) / PV_ROWS), dim3(128), PV_SMEM, st, kmap, wmap, V, n,
-                           d, d_k, hp, ctx->status);
+                           d, d_k, hp, ctx->status, cp);
   }
   dim3 grid((d + 15) / 16, (n + 15) / 16);
   if (ctx->dtype == SLIM_BF16)

@@ -461,3 +461,63 @@ def test_scores_far_above_the_first_tile_with_rope_and_long_units():
                 assert so.err_rms_norm(got[b], ref[b]) <= 2e-2, f"path {path} seq {b}"
     finally:
         layer.close()
+
+
+@pytest.mark.parametrize("d,H,d_k,dtype,paged", [(512, 4, 128, "bf16", False), (1280, 20, 64, "bf16", False),
+                                                 (512, 4, 128, "bf16", True), (256, 4, 64, "f32", False)])
+def test_prefill_stores_the_keys_and_returns_their_values(d, H, d_k, dtype, paged):
+    """slim_prefill (Fig. 3(a) in one call): several 128-row tiles with a ragged last one, three
+    sequences, rows landing at different first positions; V against the oracle on every row, the
+    cache bit for bit against the keys, rows outside the prompt untouched, a sequence without room
+    refused."""
+    batch, n_new, t_cap = 3, 293, 640
+    g = np.random.default_rng(d + n_new)
+    W_Q, W_K, W_V, _, _ = synth.make_weights(d, 400 + d)
+    X = g.standard_normal((batch, n_new, d))
+    K = synth.round_to_dtype(X @ W_K, dtype)
+    W_KV = so.oracle_wkv(W_K, W_V)
+    layer = SlimLayer(d, H, d_k, 0.0, dtype, batch, t_cap, DEV)
+    try:
+        layer.set_weights(W_K, W_V)
+        Kd = to_device_keys(K, dtype, DEV)
+        pos = np.array([0, 100, 347], dtype=np.int32)
+        st = torch.cuda.current_stream().cuda_stream
+        cache, table = layer.cache, None
+        if paged:
+            pr = 32
+            mp = t_cap // pr
+            perm = g.permutation(batch * mp).astype(np.int32).reshape(batch, mp)
+            table = torch.from_numpy(perm).to(DEV)
+            cache = B.slim_cache_create_paged(layer.ctx, layer.k, batch * mp, pr, table, batch, mp)
+        layer.k.fill_(-3.0)
+        V = torch.full((batch, n_new, d), float("nan"), dtype=torch.float32, device=DEV)
+        with torch.cuda.device(DEV):
+            B.slim_prefill(layer.ctx, cache, Kd, torch.from_numpy(pos).to(DEV), n_new, V, st)
+        assert layer.device_status() == B.SLIM_OK
+        got = V.cpu().numpy().astype(np.float64)
+        tol = 2e-2 if dtype == "bf16" else 1e-4
+        for b in range(batch):
+            ref = so.oracle_prompt_values(K[b], W_KV)
+            worst = max((so.err_rms_norm(got[b, t], ref[t]) if dtype == "bf16" else so.err_fp32_norm(got[b, t], ref[t]))
+                        for t in range(n_new))
+            assert worst <= tol, f"sequence {b}: {worst:.3e}"
+        stored = layer.k.clone()
+        if paged:
+            rows = stored.reshape(batch * mp, pr, d)[table.long()].reshape(batch, t_cap, d)
+        else:
+            rows = stored
+        for b in range(batch):
+            assert torch.equal(rows[b, pos[b]:pos[b] + n_new], Kd[b]), f"sequence {b}: cache differs from the keys"
+            assert torch.all(rows[b, :pos[b]] == -3.0) and torch.all(rows[b, pos[b] + n_new:] == -3.0)
+        # no room for sequence 2: refused, nothing of it written, the other two stored
+        layer.k.fill_(-3.0)
+        with torch.cuda.device(DEV):
+            B.slim_prefill(layer.ctx, cache, Kd, torch.tensor([0, 0, 348], dtype=torch.int32, device=DEV), n_new, V, st)
+        assert layer.device_status() == B.SLIM_ERR_CAPACITY
+        stored = layer.k.clone()
+        rows = stored.reshape(batch * mp, pr, d)[table.long()].reshape(batch, t_cap, d) if paged else stored
+        assert torch.all(rows[2] == -3.0) and torch.equal(rows[1, :n_new], Kd[1])
+        if paged:
+            B.slim_cache_destroy(cache)
+    finally:
+        layer.close()

@@ -545,3 +545,12 @@ def test_rotated_cache_pin_catches_a_missing_decode():
         s = so.attention_weights(q[sl], K[:, sl], theta)
         bad[sl] = (s @ K_rot) @ W_KV[:, sl]
     assert np.max(np.abs(good - bad)) > 1e-3 * np.max(np.abs(good))
+
+
+def test_prompt_values_from_keys_are_the_vanilla_values():
+    # Fig. 3(a) / Eq. 6: V = K W_KV equals X W_V (Eq. 5) for every prompt row, and one row by hand
+    X, _, W_K, W_V = _rand_case(40, 11, 12, 3, well_conditioned=False)
+    V = so.oracle_prompt_values(X @ W_K, so.oracle_wkv(W_K, W_V))
+    assert np.allclose(V, X @ W_V, rtol=1e-9, atol=1e-11)
+    K = np.array([[1.0, 2.0], [0.0, -1.0]]); W = np.array([[3.0, 1.0], [2.0, 0.5]])
+    assert np.array_equal(so.oracle_prompt_values(K, W), np.array([[7.0, 2.0], [-2.0, -0.5]]))
