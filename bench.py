@@ -43,9 +43,10 @@ def parse():
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (0 = the config's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--variant", default="kcache", choices=["kcache", "xcache", "prompt"],
+    ap.add_argument("--variant", default="kcache", choices=["kcache", "xcache", "prompt", "fp8"],
                     help="xcache: the X/E-cache scheme, one cache shared by all layers (configs without RoPE); "
-                         "prompt: the prompt-phase V = K W_KV of the config's shape")
+                         "prompt: the prompt-phase V = K W_KV of the config's shape; "
+                         "fp8: the K-cache path with an 8-bit cache (CUDA-core kernels)")
     ap.add_argument("--paged", type=int, default=0, help="K-cache in a shuffled pool of pages of this many rows (0 = contiguous)")
     return ap.parse_args()
 
@@ -306,7 +307,7 @@ def main():
     args = parse()
     if args.impl == "reference":
         return run_reference(args)
-    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.variant == "kcache":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.variant in ("kcache", "fp8"):
         # no launcher around us: start one process per GPU ourselves (same rendezvous a launcher would set up)
         from paper_2503_05840_b200 import replicas
         import torch
@@ -345,6 +346,11 @@ def main():
         cfg = cfg.scaled(batch=args.batch)
     layers_n = args.layers or cfg.layers
     cfg = cfg.scaled(layers=layers_n)
+    fp8 = args.variant == "fp8"
+    cfg_draw = cfg                               # the keys are drawn in the config's own type ...
+    if fp8:
+        assert cfg.dtype == "bf16", "the 8-bit cache takes bf16 keys"
+        cfg = cfg.scaled(dtype="fp8")            # ... and quantised by the library when they are appended
     path = {"auto": B.SLIM_PATH_AUTO, "generic": B.SLIM_PATH_GENERIC, "tc": B.SLIM_PATH_TC}[args.path]
 
     # ---- set-up (untimed): per-layer weights, W_KV solve, K-cache fill -----------
@@ -358,6 +364,14 @@ def main():
 
     def seq_rows(li, lay, b, n):
         """Context rows 0..n-1 of sequence b of a layer, whatever the cache arrangement."""
+        if fp8:                                  # stored key = code * 2^exponent, decoded with the oracle's table of the format
+            from oracle import slim_oracle as so
+            nb = cfg.batch * cfg.context * cfg.d
+            codes = lay.k[:nb].view(cfg.batch, cfg.context, cfg.d)[b, :n].cpu().numpy()
+            off = (nb + 15) // 16 * 16
+            exps = lay.k[off:off + cfg.batch * cfg.context * cfg.H].view(torch.int8).view(cfg.batch, cfg.context, cfg.H)[b, :n].cpu().numpy()
+            vals = so.e4m3_decode_table()[codes].reshape(n, cfg.H, cfg.d_k) * np.exp2(exps.astype(np.float64))[:, :, None]
+            return torch.from_numpy(vals.reshape(n, cfg.d))
         if not args.paged:
             return lay.k[b, :n]
         pr = args.paged
@@ -373,7 +387,7 @@ def main():
         B.slim_cache_destroy(lay.cache)
         lay.cache = B.slim_cache_create_paged(lay.ctx, lay.k, cfg.batch * mp, page_rows, tab, cfg.batch, mp)
         return tab
-    q_all = torch.zeros((layers_n, cfg.batch, cfg.d), dtype=torch.bfloat16 if cfg.dtype == "bf16" else torch.float32,
+    q_all = torch.zeros((layers_n, cfg.batch, cfg.d), dtype=torch.float32 if cfg.dtype == "f32" else torch.bfloat16,
                         device=dev)
     knew_all = torch.zeros_like(q_all)
     o_all = torch.zeros((layers_n, cfg.batch, cfg.d), dtype=torch.float32, device=dev)
@@ -384,7 +398,17 @@ def main():
         ws = lay.workspace
         lay.set_path(path)
         W_Q, W_K, W_V, _, _ = synth.make_weights_torch(cfg.d, seed0 + li, dev)
-        synth.fill_layer_torch(cfg, seed0 + li, W_Q, W_K, lengths, lay.k, q_all[li])
+        if fp8:                             # bf16 keys into a scratch tensor, then through slim_append_k (which quantises)
+            tmp = torch.zeros((cfg.batch, cfg.context, cfg.d), dtype=torch.bfloat16, device=dev)
+            synth.fill_layer_torch(cfg_draw, seed0 + li, W_Q, W_K, lengths, tmp, q_all[li])
+            lay.append_k(tmp, torch.zeros(cfg.batch, dtype=torch.int32, device=dev))
+            for b in range(cfg.batch):
+                if lengths[b] > 0:
+                    knew_all[li, b] = tmp[b, int(lengths[b]) - 1]
+            torch.cuda.synchronize()
+            del tmp
+        else:
+            synth.fill_layer_torch(cfg, seed0 + li, W_Q, W_K, lengths, lay.k, q_all[li])
         if args.paged:                      # move the drawn keys into the paged arrangement through slim_append_k
             tmp = lay.k.clone()
             paged_tables.append(make_paged(lay, args.paged, li))
@@ -397,7 +421,7 @@ def main():
             wkv_last = wkv
         assert res < 1e-8, f"W_KV residual {res}"
         for b in range(cfg.batch):          # the step re-appends the newest key row
-            if lengths[b] > 0:
+            if lengths[b] > 0 and not fp8:
                 knew_all[li, b] = seq_rows(li, lay, b, int(lengths[b]))[-1]
         del W_Q, W_K, W_V
         layers.append(lay)
@@ -530,18 +554,18 @@ def main():
             n = int(lengths[b])
             if n == 0:
                 continue
-            Kb = seq_rows(layers_n - 1, lay, b, n).float().cpu().numpy().astype(np.float64)
+            Kb = seq_rows(layers_n - 1, lay, b, n).double().cpu().numpy()
             qb = q_all[-1, b].float().cpu().numpy().astype(np.float64)
             tt = time.perf_counter()
             ref = so.oracle_slim(qb, Kb, W_KV, cfg.H, cfg.rope_theta)
             dt += time.perf_counter() - tt
             rows_done += n; n_seq += 1
-            err = so.err_rms_norm(got_all[b], ref) if cfg.dtype == "bf16" else so.err_fp32_norm(got_all[b], ref)
+            err = so.err_fp32_norm(got_all[b], ref) if cfg.dtype == "f32" else so.err_rms_norm(got_all[b], ref)
             worst = max(worst, err)          # the same sample doubles as a live parity check of what was timed
             if dt > 20.0:
                 break
         per_step = dt * (float(np.sum(lengths)) / rows_done) * layers_n      # all sequences, all layers
-        tol = 2e-2 if cfg.dtype == "bf16" else 1e-4
+        tol = 1e-4 if cfg.dtype == "f32" else 2e-2
         parity_ok = worst <= tol
         cpu = {"value": cfg.batch / per_step, "unit": "tokens/s", "cores": host_threads(), "kind": "oracle",
                "parity_tolerance": tol, "parity": "green" if parity_ok else "FAILED",
@@ -555,9 +579,10 @@ def main():
         line = {
             "metric": "decode_attention_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": {"bf16": "bf16", "f32": "f32", "fp8": "f32 arithmetic on an e4m3 cache (bf16 queries and W_KV)"}[cfg.dtype],
             "data": "synthetic",
-            "config": {"workload": f"config{args.config}:{cfg.name}", "layers": layers_n, "batch_per_gpu": cfg.batch,
+            "config": {"workload": f"config{args.config}:{cfg.name}" + (" (8-bit K-cache)" if fp8 else ""), "layers": layers_n, "batch_per_gpu": cfg.batch,
                        "global_batch": tokens, "context": cfg.context, "sum_lengths": int(lengths.sum()),
                        "d": cfg.d, "H": cfg.H, "d_k": cfg.d_k, "rope_theta": cfg.rope_theta,
                        "parallelism": f"replicas x{world} (batch-sharded, no collective)",
@@ -567,7 +592,9 @@ def main():
                        "cache": f"paged, {args.paged} rows per page" if args.paged else "contiguous"},
             "kcache_gbs": step_gbs, "kcache_frac_of_8000": step_gbs / 8000.0, "kcache_frac_of_measured": step_gbs / peak,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": ncu_traffic(args.config), "peak_kind": peak_kind, "kernel": "main decode kernel (per layer launch)",
+                         "traffic": ncu_traffic(args.config) if not fp8 else None, "peak_kind": peak_kind,
+                         "kernel": "main decode kernel (per layer launch)" if not fp8 else
+                                   "score + accumulation kernels (CUDA cores; the 8-bit keys are read twice per layer)",
                          "main_ms": main_ms, "tail_ms": tail_ms, "bytes_per_launch": k_bytes_layer,
                          "timing": "CUDA events recorded by the library inside a sustained loop of the same step "
                                    "(last step, mean over layers); that loop ran at %.4f ms per step" % ms_prof},

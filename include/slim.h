@@ -51,7 +51,9 @@ typedef enum {
   SLIM_ERR_STATIC_WS = 9     /* slim_decode_static_ws: scratch need above the built-in maximum */
 } slim_status;
 
-typedef enum { SLIM_F32 = 0, SLIM_BF16 = 1 } slim_dtype;      /* cache / query dtype   */
+/* cache / query dtype.  SLIM_FP8: the cache holds 8-bit keys (1 byte per value, the paper's own byte
+ * accounting in its introduction), queries, new key rows and W_KV are bf16 -- see slim_cache_bytes. */
+typedef enum { SLIM_F32 = 0, SLIM_BF16 = 1, SLIM_FP8 = 2 } slim_dtype;
 typedef enum { SLIM_HOST_F32 = 0, SLIM_HOST_F64 = 1 } slim_host_dtype;
 
 /* Kernel selection for slim_decode (slim_set_path). */
@@ -106,7 +108,14 @@ slim_status slim_set_weights_nonsquare(slim_ctx* ctx, const void* W_K, const voi
 slim_status slim_set_wkv(slim_ctx* ctx, const void* W_KV, int host_dtype);
 
 /* Bytes of key storage for `batch` sequences of capacity t_cap, and of the
- * scratch workspace slim_decode needs for such a cache (0 on bad arguments).  */
+ * scratch workspace slim_decode needs for such a cache (0 on bad arguments).
+ * SLIM_FP8 caches: the storage holds the codes [batch][t_cap][d] (OCP FP8 E4M3, one byte per
+ * value) followed, at the next multiple of 16 bytes, by one int8 exponent per (row, head)
+ * [batch][t_cap][H]: the stored key is code * 2^exponent, the exponent being the smallest one
+ * for which the head slice of the row fits the E4M3 range (|value| <= 448), codes rounded to
+ * nearest even.  Such a cache is filled only through slim_append_k / slim_decode_step /
+ * slim_prefill (which quantise bf16 rows); it is contiguous (no paged variant), has no X-cache
+ * mode, and is read by the CUDA-core kernels.                                            */
 size_t slim_cache_bytes(const slim_ctx* ctx, int batch, int t_cap);
 size_t slim_workspace_bytes(const slim_ctx* ctx, int batch, int t_cap);
 

@@ -35,6 +35,10 @@ Paper passages followed (arxiv 2503.05840):
                         enter it (oracle_rotated_cache).  Not exact: the skipped
                         scores are simply left out, nothing is renormalised.
 
+  Introduction, memory-size example ("1 byte per value")  8-bit K-cache: the paper only counts
+                        the bytes; the format is a reading (e4m3_* and quantize_keys_e4m3 below):
+                        OCP FP8 E4M3 codes with one power-of-two exponent per (row, head)
+
 Readings where the paper is silent (the CUDA path takes the same ones):
   * RoPE pairs element j with j + d_k/2 inside a head, frequency
     theta_j = rope_theta ** (-2 j / d_k), angle = position * theta_j;
@@ -270,6 +274,69 @@ def oracle_rotated_cache(q: np.ndarray, K_rot: np.ndarray, W_KV: np.ndarray, H: 
             u = s[keep] @ raw
         out[sl] = u @ W_KV[:, sl]
     return out, kept
+
+
+# --------------------------------------------------------------------------
+# 8-bit K-cache: OCP FP8 E4M3 (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities,
+# S.1111.111 is NaN, largest finite value 448, subnormals k * 2^-9) with a power-of-two exponent per
+# (row, head).  Written from the published format definition.
+# --------------------------------------------------------------------------
+def e4m3_decode_table() -> np.ndarray:
+    """Value of each of the 256 codes (NaN for 0x7f and 0xff)."""
+    v = np.empty(256, dtype=F64)
+    for c in range(256):
+        sign = -1.0 if c & 0x80 else 1.0
+        ex, man = (c >> 3) & 0xF, c & 7
+        if ex == 0xF and man == 7:
+            v[c] = np.nan
+        elif ex == 0:
+            v[c] = sign * man * 2.0 ** -9                       # subnormal: 0.mmm * 2^-6
+        else:
+            v[c] = sign * (1.0 + man / 8.0) * 2.0 ** (ex - 7)
+    return v
+
+
+def e4m3_encode(x: np.ndarray) -> np.ndarray:
+    """Round to the nearest E4M3 value, ties to the even code, saturating at +-448.  Brute force over
+    the 127 finite magnitudes: the definition of rounding, not a bit trick."""
+    x = np.asarray(x, dtype=F64)
+    mags = e4m3_decode_table()[:0x7F]                            # codes 0x00 .. 0x7e, increasing in value
+    a = np.minimum(np.abs(x), 448.0)
+    hi = np.searchsorted(mags, a, side="left")                   # first code with value >= a
+    hi = np.minimum(hi, 0x7E)
+    lo = np.maximum(hi - 1, 0)
+    d_hi, d_lo = mags[hi] - a, a - mags[lo]
+    pick_lo = (d_lo < d_hi) | ((d_lo == d_hi) & (lo % 2 == 0))
+    code = np.where(pick_lo, lo, hi).astype(np.uint8)
+    return np.where(np.signbit(x), code | 0x80, code).astype(np.uint8)
+
+
+def quantize_keys_e4m3(K: np.ndarray, H: int):
+    """K: [T, d] key rows (bf16-representable values).  Per (row, head): exponent e = the smallest
+    integer with max|k| * 2^-e <= 448 (0 for an all-zero slice, clamped to [-126, 127]), codes =
+    e4m3_encode(k * 2^-e).  Returns (codes uint8 [T, d], exps int8 [T, H], dequantised keys [T, d])."""
+    K = np.asarray(K, dtype=F64)
+    T, d = K.shape
+    d_k = d // H
+    Kh = K.reshape(T, H, d_k)
+    amax = np.max(np.abs(Kh), axis=2)                            # [T, H]
+    e = np.zeros((T, H), dtype=np.int64)
+    nz = amax > 0
+    e[nz] = np.ceil(np.log2(amax[nz] / 448.0)).astype(np.int64)
+    # log2 can be off by one ulp at exact powers of two: fix up so that e is the smallest that fits
+    e = np.where(nz & (amax * np.exp2(-(e - 1).astype(F64)) <= 448.0), e - 1, e)
+    e = np.where(nz & (amax * np.exp2(-e.astype(F64)) > 448.0), e + 1, e)
+    e = np.clip(e, -126, 127)
+    scale = np.exp2(e.astype(F64))[:, :, None]
+    codes = e4m3_encode(Kh / scale)
+    deq = (e4m3_decode_table()[codes] * scale).reshape(T, d)
+    return codes.reshape(T, d), e.astype(np.int8), deq
+
+
+def oracle_slim_fp8(q: np.ndarray, K: np.ndarray, W_KV: np.ndarray, H: int, rope_theta: float = 0.0) -> np.ndarray:
+    """Slim attention over an 8-bit K-cache: the keys are quantised (quantize_keys_e4m3) and Eq. 7
+    Option 2 is evaluated on the stored (dequantised) keys."""
+    return oracle_slim(q, quantize_keys_e4m3(K, H)[2], W_KV, H, rope_theta)
 
 
 def oracle_slim_batch(q: np.ndarray, K: np.ndarray, lengths, W_KV: np.ndarray, H: int,

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libslim.so")
 
 SLIM_OK, SLIM_ERR_INVALID_ARG, SLIM_ERR_UNSUPPORTED, SLIM_ERR_SINGULAR, SLIM_ERR_CAPACITY, \
     SLIM_ERR_OOM, SLIM_ERR_CUDA, SLIM_ERR_TIMEOUT, SLIM_ERR_NO_WEIGHTS, SLIM_ERR_STATIC_WS = range(10)
-SLIM_F32, SLIM_BF16 = 0, 1
+SLIM_F32, SLIM_BF16, SLIM_FP8 = 0, 1, 2
 SLIM_HOST_F32, SLIM_HOST_F64 = 0, 1
 SLIM_PATH_AUTO, SLIM_PATH_GENERIC, SLIM_PATH_TC = 0, 1, 2
 SLIM_Q_PATH_IN_USE, SLIM_Q_LAUNCHES_PER_DECODE, SLIM_Q_MAX_UNITS, SLIM_Q_NUM_SMS, SLIM_Q_WORKERS = range(5)

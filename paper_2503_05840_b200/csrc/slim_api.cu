@@ -146,8 +146,10 @@ const char* slim_strerror(int status) {
 slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta, int dtype) {
   if (!out) return SLIM_ERR_INVALID_ARG;
   *out = nullptr;
-  if (d <= 0 || H <= 0 || d_k <= 0 || !(rope_theta >= 0.0) || (dtype != SLIM_F32 && dtype != SLIM_BF16))
+  if (d <= 0 || H <= 0 || d_k <= 0 || !(rope_theta >= 0.0) || (dtype != SLIM_F32 && dtype != SLIM_BF16 && dtype != SLIM_FP8))
     return SLIM_ERR_INVALID_ARG;
+  const int kdtype = dtype;
+  if (dtype == SLIM_FP8) dtype = SLIM_BF16;            // 8-bit cache; queries, new rows and W_KV are bf16
   if ((long long)H * d_k != d) return SLIM_ERR_UNSUPPORTED;       // Eq. 6 needs a square W_K
   if (H > SLIM_MAX_H || d_k > 256 || (d_k % 16) != 0 || d > 16384) return SLIM_ERR_UNSUPPORTED;
   int dev = 0;
@@ -157,7 +159,7 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
   slim_ctx* c = new (std::nothrow) slim_ctx();
   if (!c) return SLIM_ERR_OOM;
   std::memset(c, 0, sizeof(*c));
-  c->d = d; c->H = H; c->d_k = d_k; c->dtype = dtype; c->rope_theta = rope_theta;
+  c->d = d; c->H = H; c->d_k = d_k; c->dtype = dtype; c->kdtype = kdtype; c->rope_theta = rope_theta;
   c->device = dev; c->num_sms = prop.multiProcessorCount;
   c->path_req = SLIM_PATH_AUTO;
   {
@@ -198,7 +200,7 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
   }
   c->tc_ok = 0;
   for (int cl = 1; cl <= 2; ++cl) {
-    c->tc_workers[cl - 1] = (prop.major == 10 && slim_tc_shape_ok(d, H, d_k, dtype, rope_theta != 0.0, cl)) ? slim_tc_workers(c, cl) : 0;
+    c->tc_workers[cl - 1] = (prop.major == 10 && kdtype != SLIM_FP8 && slim_tc_shape_ok(d, H, d_k, dtype, rope_theta != 0.0, cl)) ? slim_tc_workers(c, cl) : 0;
     if (c->tc_workers[cl - 1] < 0) c->tc_workers[cl - 1] = 0;
     if (c->tc_workers[cl - 1] > 0) c->tc_ok = 1;
   }
@@ -304,6 +306,7 @@ slim_status slim_set_weights_nonsquare(slim_ctx* ctx, const void* W_K, const voi
 slim_status slim_xcache_set_weights(slim_ctx* ctx, const void* W_K, const void* W_V, int host_dtype) {
   if (!ctx || !W_K || !W_V || (host_dtype != SLIM_HOST_F32 && host_dtype != SLIM_HOST_F64)) return SLIM_ERR_INVALID_ARG;
   if (ctx->rope_theta != 0.0) return SLIM_ERR_UNSUPPORTED;          // the scheme has no place for RoPE
+  if (ctx->kdtype == SLIM_FP8) return SLIM_ERR_UNSUPPORTED;
   const size_t nn = (size_t)ctx->d * ctx->d;
   std::vector<float> wk(nn);
   if (host_dtype == SLIM_HOST_F64) { const double* s = static_cast<const double*>(W_K); for (size_t i = 0; i < nn; ++i) wk[i] = (float)s[i]; }
@@ -334,6 +337,8 @@ slim_status slim_set_wkv(slim_ctx* ctx, const void* W_KV, int host_dtype) {
 
 size_t slim_cache_bytes(const slim_ctx* ctx, int batch, int t_cap) {
   if (!ctx || batch <= 0 || t_cap <= 0) return 0;
+  if (ctx->kdtype == SLIM_FP8)                             // codes, then one exponent per (row, head)
+    return ((((size_t)batch * t_cap * ctx->d) + 15) & ~(size_t)15) + (size_t)batch * t_cap * ctx->H;
   return esize(ctx->dtype) * (size_t)batch * t_cap * ctx->d;
 }
 
@@ -353,6 +358,8 @@ slim_status slim_cache_create(slim_ctx* ctx, slim_cache** out, void* k_storage, 
   slim_cache* c = new (std::nothrow) slim_cache();
   if (!c) return SLIM_ERR_OOM;
   c->ctx = ctx; c->k = k_storage; c->batch = batch; c->t_cap = t_cap;
+  c->k_exp = ctx->kdtype == SLIM_FP8
+                 ? reinterpret_cast<signed char*>(k_storage) + ((((size_t)batch * t_cap * ctx->d) + 15) & ~(size_t)15) : nullptr;
   c->block_table = nullptr; c->page_rows = 0; c->max_pages = 0; c->num_pages = 0;
   c->total_rows = (long long)batch * t_cap;
   for (int cl = 1; cl <= 2; ++cl) {
@@ -363,7 +370,7 @@ slim_status slim_cache_create(slim_ctx* ctx, slim_cache** out, void* k_storage, 
     }
   }
   c->has_xmap = 0;
-  if (ctx->proj_ok && slim_xscores_tc_ok(ctx)) {
+  if (ctx->proj_ok && ctx->kdtype != SLIM_FP8 && slim_xscores_tc_ok(ctx)) {
     if (slim_xscores_make_tmap(ctx, c) == cudaSuccess) c->has_xmap = 1;
     else cudaGetLastError();
   }
@@ -377,6 +384,7 @@ slim_status slim_cache_create_paged(slim_ctx* ctx, slim_cache** out, void* pool,
   *out = nullptr;
   if (!ctx || !pool || !block_table || num_pages <= 0 || page_rows <= 0 || batch <= 0 || max_pages <= 0) return SLIM_ERR_INVALID_ARG;
   if (page_rows % SLIM_TT != 0 || batch > SLIM_MAX_BATCH || ((uintptr_t)pool & 15)) return SLIM_ERR_UNSUPPORTED;
+  if (ctx->kdtype == SLIM_FP8) return SLIM_ERR_UNSUPPORTED;
   if ((long long)num_pages * page_rows > 0x7fffffffLL - 64 || (long long)batch * max_pages * page_rows > 0x7fffffffLL - 64)
     return SLIM_ERR_UNSUPPORTED;
   const int t_cap = max_pages * page_rows;
@@ -384,7 +392,7 @@ slim_status slim_cache_create_paged(slim_ctx* ctx, slim_cache** out, void* pool,
   if (st != SLIM_OK) return st;
   slim_cache* c = new (std::nothrow) slim_cache();
   if (!c) return SLIM_ERR_OOM;
-  c->ctx = ctx; c->k = pool; c->batch = batch; c->t_cap = t_cap;
+  c->ctx = ctx; c->k = pool; c->k_exp = nullptr; c->batch = batch; c->t_cap = t_cap;
   c->block_table = block_table; c->page_rows = page_rows; c->max_pages = max_pages; c->num_pages = num_pages;
   c->total_rows = (long long)num_pages * page_rows;
   for (int cl = 1; cl <= 2; ++cl) {
@@ -438,7 +446,7 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   SlimDecodeParams p;
   p.d = ctx->d; p.H = ctx->H; p.d_k = ctx->d_k; p.half = ctx->d_k / 2;
   p.batch = cache->batch; p.t_cap = cache->t_cap;
-  p.rope = ctx->rope_theta != 0.0; p.dtype = ctx->dtype;
+  p.rope = ctx->rope_theta != 0.0; p.dtype = ctx->dtype; p.kdtype = ctx->kdtype; p.k_exp = cache->k_exp;
   p.workers = path == SLIM_PATH_TC ? ctx->tc_workers[cl - 1] : ctx->gen_workers;
   p.cl = cl;
   p.min_tiles = min_tiles_for(ctx);

@@ -15,15 +15,32 @@
 // slim_exact_kernel is the single-pass variant (scores recomputed per
 // d-slice).  It is only used to redo, exactly, the rare units the tensor-core
 // kernel flags because a softmax argument ran away from its reference.
+#include <cuda_fp8.h>
+
 #include "slim_internal.h"
 #include "slim_sched.cuh"
 
 namespace {
 
+// 8-bit cache (SLIM_FP8): elements are OCP E4M3 codes; the stored key is code * 2^exponent with one
+// exponent per (cache row, head).  ld_k returns the bare code value; k_scale the power of two.
+typedef unsigned char fp8code;
+__device__ __forceinline__ float fp8_value(fp8code c) {
+  return __half2float(__half(__nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)c, __NV_E4M3)));
+}
 __device__ __forceinline__ float ld_k(const float* p) { return __ldg(p); }
 __device__ __forceinline__ float ld_k(const __nv_bfloat16* p) {
   return __bfloat162float(__ldg(reinterpret_cast<const __nv_bfloat16*>(p)));
 }
+__device__ __forceinline__ float ld_k(const fp8code* p) { return fp8_value(__ldg(p)); }
+// 2^exponent of (row, head) of an fp8 cache; 1 for the other cache types
+__device__ __forceinline__ float k_scale(const SlimDecodeParams& p, long long row, int h) {
+  if (!p.k_exp) return 1.f;
+  return __int_as_float(((int)__ldg(p.k_exp + (size_t)row * p.H + h) + 127) << 23);
+}
+// query / weight element type that goes with a cache element type
+template <typename KT> struct QueryOf { typedef KT type; };
+template <> struct QueryOf<fp8code> { typedef __nv_bfloat16 type; };
 
 constexpr int GEN_THREADS = 256;
 
@@ -216,6 +233,16 @@ template <> struct Vec<__nv_bfloat16> {
   }
 };
 
+template <> struct Vec<fp8code> {
+  static constexpr int N = 8;
+  __device__ static void load(const fp8code* p, float (&v)[8]) {
+    const uint2 x = __ldg(reinterpret_cast<const uint2*>(p));
+    const uint32_t w[2] = {x.x, x.y};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = fp8_value((fp8code)((w[i >> 2] >> (8 * (i & 3))) & 0xffu));
+  }
+};
+
 // One CTA walks tiles g = blockIdx.x, blockIdx.x + gridDim.x, ...  A warp owns
 // rows of the tile; a lane owns "pair vectors": VEC consecutive elements j of
 // the first half of a head together with their partners j + d_k/2.
@@ -230,8 +257,9 @@ slim_scores_kernel(SlimDecodeParams p, float* __restrict__ scores) {
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int d = p.d, H = p.H, dk = p.d_k, half = p.half;
   const int npv = d / (2 * VEC), pv_per_head = half / VEC;
+  typedef typename QueryOf<KT>::type QT;
   const KT* __restrict__ Kc = reinterpret_cast<const KT*>(p.k);
-  const KT* __restrict__ Q = reinterpret_cast<const KT*>(p.q);
+  const QT* __restrict__ Q = reinterpret_cast<const QT*>(p.q);
 
   const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
   int cur_b = -1;
@@ -292,7 +320,7 @@ slim_scores_kernel(SlimDecodeParams p, float* __restrict__ scores) {
       if (t0 + t < len) {
         float a = 0.f;
         for (int x = 0; x < pv_per_head; ++x) a += s_part[t * npv + h * pv_per_head + x];
-        scores[((size_t)b * H + h) * p.t_cap + t0 + t] = a;
+        scores[((size_t)b * H + h) * p.t_cap + t0 + t] = a * k_scale(p, slim_cache_row(p, b, t0) + t, h);
       }
     }
   }
@@ -340,8 +368,10 @@ slim_accum_kernel(SlimDecodeParams p, const float* __restrict__ scores, int only
       const int t0 = tile * SLIM_TT;
       const KT* __restrict__ Kt = Kc + (size_t)slim_cache_row(p, b, t0) * d;
       float kv[SLIM_TT];
+      const long long row0 = slim_cache_row(p, b, t0);
 #pragma unroll
-      for (int t = 0; t < SLIM_TT; ++t) kv[t] = (col < d && t0 + t < len) ? ld_k(Kt + (size_t)t * d + col) : 0.f;
+      for (int t = 0; t < SLIM_TT; ++t)
+        kv[t] = (col < d && t0 + t < len) ? ld_k(Kt + (size_t)t * d + col) * k_scale(p, row0 + t, col / p.d_k) : 0.f;
       // ---- a5: online softmax, one warp per head ----
       for (int h = wid; h < H; h += GEN_THREADS / 32) {
         const float s = (lane < SLIM_TT && t0 + lane < len)
@@ -534,6 +564,7 @@ cudaError_t slim_launch_xcache_scores(const slim_ctx* ctx, const SlimDecodeParam
 }
 
 cudaError_t slim_launch_accum(const slim_ctx* ctx, const SlimDecodeParams& p, const float* scores, int whole, cudaStream_t st) {
+  if (p.kdtype == SLIM_FP8) return launch_accum<fp8code>(p, scores, whole ? 0 : 1, st);
   return p.dtype == SLIM_BF16 ? launch_accum<__nv_bfloat16>(p, scores, whole ? 0 : 1, st)
                               : launch_accum<float>(p, scores, whole ? 0 : 1, st);
 }
@@ -549,7 +580,8 @@ int slim_generic_workers(const slim_ctx* ctx) {
 }
 
 cudaError_t slim_launch_generic(const slim_ctx* ctx, const SlimDecodeParams& p, float* scores, cudaStream_t st) {
-  cudaError_t e = p.dtype == SLIM_BF16 ? launch_scores<__nv_bfloat16>(ctx, p, scores, st) : launch_scores<float>(ctx, p, scores, st);
+  cudaError_t e = p.kdtype == SLIM_FP8 ? launch_scores<fp8code>(ctx, p, scores, st)
+                  : p.dtype == SLIM_BF16 ? launch_scores<__nv_bfloat16>(ctx, p, scores, st) : launch_scores<float>(ctx, p, scores, st);
   if (e != cudaSuccess) return e;
   return slim_launch_accum(ctx, p, scores, 1, st);
 }

@@ -20,7 +20,9 @@ struct SlimDecodeParams {
   int d, H, d_k, half;           // half = d_k / 2
   int batch, t_cap;
   int rope;                      // 0 / 1
-  int dtype;                     // slim_dtype
+  int dtype;                     // slim_dtype of q and W_KV (f32 or bf16)
+  int kdtype;                    // slim_dtype of the cache elements (f32, bf16 or fp8 codes)
+  const signed char* k_exp;      // fp8 cache: [batch][t_cap][H] exponents (stored key = code * 2^exponent), else NULL
   int workers;                   // context-split workers (W)
   int cl;                        // tensor-core path: CTAs per worker (1 or 2)
   int min_tiles;                 // a worker gets at least this many tiles if it gets any
@@ -48,7 +50,8 @@ struct SlimDecodeParams {
 };
 
 struct slim_ctx {
-  int d, H, d_k, dtype;
+  int d, H, d_k, dtype;          // dtype: q and W_KV (f32 or bf16)
+  int kdtype;                    // cache elements: dtype, or SLIM_FP8
   double rope_theta;
   int device;
   int num_sms;
@@ -80,6 +83,7 @@ struct slim_ctx {
 struct slim_cache {
   slim_ctx* ctx;
   void* k;
+  signed char* k_exp;            // fp8 cache: exponents behind the codes, else NULL
   int batch, t_cap;              // paged: t_cap = max_pages * page_rows
   const int32_t* block_table;    // paged: device [batch][max_pages]; NULL for a contiguous cache
   int page_rows, max_pages, num_pages;

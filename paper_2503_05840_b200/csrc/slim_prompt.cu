@@ -180,7 +180,7 @@ cudaError_t slim_launch_values(const slim_ctx* ctx, const void* K, int n, float*
   SlimDecodeParams cp;
   memset(&cp, 0, sizeof(cp));
   if (cache) {
-    if (!tc || ((uintptr_t)cache->k & 15)) {         // no fused store on this path: the append kernel first
+    if (!tc || ctx->kdtype == SLIM_FP8 || ((uintptr_t)cache->k & 15)) {   // no fused store on this path (an 8-bit cache quantises): the append kernel first
       cudaError_t e = slim_launch_append(ctx, cache, K, positions, n_new, 0, st);
       if (e != cudaSuccess) return e;
     } else {

@@ -8,6 +8,8 @@
 //          W_KV[h][j][0..d_k): a partial sum over its j-slice, written to
 //          o_part[js][b][h*d_k + c].
 //   tail2: o[b][:] = sum_js o_part[js][b][:]   (fixed order => deterministic)
+#include <cuda_fp8.h>
+
 #include "slim_internal.h"
 #include "slim_sched.cuh"
 
@@ -170,6 +172,46 @@ __global__ void slim_append_kernel(KT* __restrict__ cache, const KT* __restrict_
   }
 }
 
+// 8-bit cache: quantise the new bf16 rows.  Per (row, head): exponent e = the smallest integer with
+// max|k| * 2^-e <= 448 (the E4M3 range), code = E4M3(k * 2^-e) rounded to nearest even; the scaling by
+// a power of two is exact, so the codes depend on the input bits only.  One warp per head.
+__global__ void __launch_bounds__(256)
+slim_append_fp8_kernel(unsigned char* __restrict__ codes, signed char* __restrict__ exps, const __nv_bfloat16* __restrict__ k_new,
+                       const int32_t* __restrict__ positions, int d, int H, int d_k, int t_cap, int n_new, int* status,
+                       int pos_is_length) {
+  slim_pdl_trigger();
+  slim_pdl_wait();
+  const int b = blockIdx.x, r = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int pos = positions[b];
+  if (pos_is_length) {
+    if (pos <= 0) return;
+    pos -= 1;
+  }
+  if (pos < 0 || pos > t_cap - n_new) {
+    if (threadIdx.x == 0) atomicMax(status, (int)SLIM_ERR_CAPACITY);
+    return;
+  }
+  const __nv_bfloat16* src = k_new + ((size_t)b * n_new + r) * d;
+  const size_t row = (size_t)b * t_cap + pos + r;
+  for (int h = warp; h < H; h += blockDim.x >> 5) {
+    float amax = 0.f;
+    for (int c = lane; c < d_k; c += 32) amax = fmaxf(amax, fabsf(__bfloat162float(src[h * d_k + c])));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    int e = 0;
+    if (amax > 0.f && amax <= 3.0e38f) {
+      int x;
+      const float m = frexpf(amax, &x);                 // amax = m 2^x, 0.5 <= m < 1; 448 = 0.875 * 2^9
+      e = m <= 0.875f ? x - 9 : x - 8;
+      e = max(-126, min(127, e));
+    }
+    const float inv = __int_as_float((127 - e) << 23);  // 2^-e (e >= -126 keeps it finite: 2^126 at most)
+    for (int c = lane; c < d_k; c += 32)
+      codes[row * d + h * d_k + c] = (unsigned char)__nv_cvt_float_to_fp8(__bfloat162float(src[h * d_k + c]) * inv, __NV_SATFINITE, __NV_E4M3);
+    if (lane == 0) exps[row * H + h] = (signed char)e;
+  }
+}
+
 }  // namespace
 
 size_t slim_tail_opart_floats(int d, int batch) {
@@ -214,6 +256,10 @@ cudaError_t slim_launch_tail(const slim_ctx* ctx, const SlimDecodeParams& p, cud
 cudaError_t slim_launch_append(const slim_ctx* ctx, const slim_cache* c, const void* k_new,
                                const int32_t* positions, int n_new, int pos_is_length, cudaStream_t st) {
   dim3 grid(c->batch, n_new);
+  if (ctx->kdtype == SLIM_FP8)
+    return slim_launch_pdl(slim_append_fp8_kernel, grid, dim3(256), 0, st, (unsigned char*)c->k, c->k_exp,
+                           (const __nv_bfloat16*)k_new, positions, ctx->d, ctx->H, ctx->d_k, c->t_cap, n_new, ctx->status,
+                           pos_is_length);
   if (ctx->dtype == SLIM_BF16)
     return slim_launch_pdl(slim_append_kernel<__nv_bfloat16>, grid, dim3(256), 0, st, (__nv_bfloat16*)c->k,
                            (const __nv_bfloat16*)k_new, positions, ctx->d, c->t_cap, n_new, ctx->status, c->block_table,

@@ -17,10 +17,14 @@ class SlimLayer:
         self.device = torch.device(device)
         self.d, self.H, self.d_k, self.batch, self.t_cap = d, H, d_k, batch, t_cap
         self.dtype = dtype
-        self.tdtype = torch.bfloat16 if dtype == "bf16" else torch.float32
+        # type of q, of new key rows and of W_KV; an "fp8" layer keeps only its cache in 8 bits
+        self.tdtype = torch.float32 if dtype == "f32" else torch.bfloat16
         with torch.cuda.device(self.device):
-            self.ctx = B.slim_create(d, H, d_k, rope_theta, B.SLIM_BF16 if dtype == "bf16" else B.SLIM_F32)
-            self.k = torch.zeros((batch, t_cap, d), dtype=self.tdtype, device=self.device)
+            self.ctx = B.slim_create(d, H, d_k, rope_theta, {"f32": B.SLIM_F32, "bf16": B.SLIM_BF16, "fp8": B.SLIM_FP8}[dtype])
+            if dtype == "fp8":     # codes [batch][t_cap][d], then the exponents: filled through append_k only
+                self.k = torch.zeros(B.slim_cache_bytes(self.ctx, batch, t_cap), dtype=torch.uint8, device=self.device)
+            else:
+                self.k = torch.zeros((batch, t_cap, d), dtype=self.tdtype, device=self.device)
             self.cache = B.slim_cache_create(self.ctx, self.k, batch, t_cap)
             need = B.slim_workspace_bytes(self.ctx, batch, t_cap)
             if workspace is None:      # layers that run one after another on a stream may share one

@@ -178,8 +178,11 @@ def kcache_values(d: int, layers: int, tokens: int) -> int:
 def kcache_bytes_per_step(cfg: SlimConfig, lengths: np.ndarray) -> int:
     """Algorithmic K bytes one decode step reads: layers * sum(lengths) * d *
     sizeof(dtype)  (the 'n d reads' of Table 2, per layer and sequence)."""
+    rows = int(cfg.layers) * int(np.sum(lengths, dtype=np.int64))
+    if cfg.dtype == "fp8":                       # one byte per value plus one exponent byte per (row, head)
+        return rows * (cfg.d + cfg.H)
     size = 2 if cfg.dtype == "bf16" else 4
-    return int(cfg.layers) * int(np.sum(lengths, dtype=np.int64)) * cfg.d * size
+    return rows * cfg.d * size
 
 
 # ---------------------------------------------------------------- device-side drawing (full-size configs)

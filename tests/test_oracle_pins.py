@@ -554,3 +554,49 @@ def test_prompt_values_from_keys_are_the_vanilla_values():
     assert np.allclose(V, X @ W_V, rtol=1e-9, atol=1e-11)
     K = np.array([[1.0, 2.0], [0.0, -1.0]]); W = np.array([[3.0, 1.0], [2.0, 0.5]])
     assert np.array_equal(so.oracle_prompt_values(K, W), np.array([[7.0, 2.0], [-2.0, -0.5]]))
+
+
+# ---- 8-bit K-cache: the E4M3 format and the per-(row, head) power-of-two exponent -----------------
+def test_e4m3_table_and_rounding_against_the_published_format():
+    tab = so.e4m3_decode_table()
+    # values fixed by the OCP FP8 definition: largest finite 448 = 0x7e, 1.0 = 0x38, smallest normal
+    # 2^-6 = 0x08, smallest subnormal 2^-9 = 0x01, 0x7f and 0xff are NaN, negative half mirrors
+    assert tab[0x7E] == 448.0 and tab[0x38] == 1.0 and tab[0x08] == 2.0 ** -6 and tab[0x01] == 2.0 ** -9
+    assert tab[0x00] == 0.0 and np.isnan(tab[0x7F]) and np.isnan(tab[0xFF]) and tab[0xB8] == -1.0
+    assert tab[0x3C] == 1.5 and tab[0x40] == 2.0 and tab[0x47] == 3.75
+    assert np.all(np.diff(tab[:0x7F]) > 0)                       # codes are ordered like their values
+    enc = so.e4m3_encode
+    assert list(enc(np.array([448.0, 1.0, 1.5, -1.0, 0.0, 1e9, -1e9]))) == [0x7E, 0x38, 0x3C, 0xB8, 0x00, 0x7E, 0xFE]
+    # every finite code survives decode -> encode; midpoints go to the even code (hand: 1.0625 is halfway
+    # between 1.0 = 0x38 and 1.125 = 0x39 -> 0x38; 1.1875 halfway between 0x39 and 0x3a -> 0x3a)
+    finite = [c for c in range(256) if not np.isnan(tab[c]) and c != 0x80]
+    assert all(int(enc(np.array([tab[c]]))[0]) == c for c in finite)
+    assert list(enc(np.array([1.0625, 1.1875, 1.06, 1.07, 2.0 ** -10, 1.5 * 2.0 ** -9]))) == [0x38, 0x3A, 0x38, 0x39, 0x00, 0x02]
+    # relative error of a normal value is at most half a mantissa step, 2^-4
+    x = np.random.default_rng(0).uniform(2.0 ** -6, 448.0, size=2000)
+    assert np.max(np.abs(tab[enc(x)] - x) / x) <= 2.0 ** -4
+
+
+def test_fp8_key_quantisation_exponent_and_exactness():
+    # exponent = smallest e with max|k| 2^-e <= 448: 448 -> 0, 449 -> 1, 224 -> -1, 1 -> -8 (448/2^9 < 1 <= 448/2^8)
+    K = np.zeros((5, 4))
+    K[0] = [448.0, 1.0, 0.0, 0.0]; K[1] = [449.0, 0.0, 0.0, 0.0]; K[2] = [224.0, -3.0, 0.0, 0.0]
+    K[3] = [1.0, 0.5, 0.0, 0.0]
+    codes, exps, deq = so.quantize_keys_e4m3(K, 2)
+    assert list(exps[:, 0]) == [0, 1, -1, -8, 0] and list(exps[:, 1]) == [0, 0, 0, 0, 0]
+    assert deq[0, 0] == 448.0 and deq[1, 0] == 448.0 and deq[2, 0] == 224.0 and deq[3, 0] == 1.0 and deq[3, 1] == 0.5
+    # values with at most 4 significant bits inside a head slice are stored exactly; others to 2^-4
+    g = np.random.default_rng(1)
+    K2 = synth.round_to_bf16(g.standard_normal((50, 64)) * g.uniform(0.01, 30.0, size=(50, 1))).astype(np.float64)
+    c2, e2, d2 = so.quantize_keys_e4m3(K2, 4)
+    amax = np.max(np.abs(K2.reshape(50, 4, 16)), axis=2)
+    assert np.all(amax * np.exp2(-e2.astype(np.float64)) <= 448.0) and np.all(amax * np.exp2(-(e2 - 1.0)) > 448.0)
+    err = np.abs(d2 - K2).reshape(50, 4, 16)
+    assert np.all(err <= amax[:, :, None] * 2.0 ** -4)           # half a step of the largest binade at worst
+    # the attention over the stored keys is ordinary slim attention on the dequantised rows
+    W = g.standard_normal((64, 64)) / 8; q = g.standard_normal(64)
+    assert np.array_equal(so.oracle_slim_fp8(q, K2, W, 4, 1.0e4), so.oracle_slim(q, d2, W, 4, 1.0e4))
+    # and, for keys of ordinary size, close to the unquantised result (keys perturbed by <= 2^-4 of their slice maximum)
+    K3 = synth.round_to_bf16(g.standard_normal((50, 64))).astype(np.float64)
+    ref = so.oracle_slim(q, K3, W, 4, 1.0e4)
+    assert so.err_rms_norm(so.oracle_slim_fp8(q, K3, W, 4, 1.0e4), ref) < 0.2
