@@ -236,6 +236,35 @@ size_t      slim_xcache_workspace_bytes(const slim_ctx* ctx, int batch, int t_ca
 slim_status slim_xcache_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,
                                float* o, void* workspace, void* stream);
 
+/* One context split over several GPUs (the complexity section's remark that the scheme works with
+ * flash-style splitting; Eq. 2 and Eq. 7 Option 2 evaluated slice by slice).  Every rank caches a
+ * slice of the rows of each sequence, starting at a multiple of 16 rows, and calls
+ * slim_decode_partial on it; the ranks exchange the results (an all-gather of H (d + 1) floats per
+ * sequence -- the caller's job, e.g. with NCCL) and slim_combine_project joins them.
+ *   slim_reserve_positions  grows the RoPE tables to cover absolute positions < max_position
+ *                           (a slice's cache only covers its own t_cap rows).  Synchronous; call
+ *                           it at set-up.  Positions outside the tables are clamped and reported as
+ *                           SLIM_ERR_CAPACITY by the device status.
+ *   slim_decode_partial     q, cache, lengths as for slim_decode, lengths[b] = rows of the slice;
+ *                           first_tile  device int32 [batch]: absolute row of the slice's row 0, / 16
+ *                           q_pos       device int32 [batch]: absolute position of the query
+ *                           lse_out     device float [batch][H]: log2 of the slice's softmax
+ *                                       denominator (arguments in log2 units); -inf for an empty slice
+ *                           u_out       device float [batch][H][d]: the slice's weighted sum of keys
+ *                                       divided by that denominator
+ *                           bf16 and f32 caches (not SLIM_FP8)
+ *   slim_combine_project    lse_all [ranks][batch][H], u_all [ranks][batch][H][d] (device, rank
+ *                           order free), total_lengths device int32 [batch] (0 gives a zero row):
+ *                           u = sum_r w_r u_r with w_r = 2^(lse_r - max) / sum_r' 2^(lse_r' - max),
+ *                           then the per-head projection with W_KV; o device float [batch][d];
+ *                           workspace >= slim_workspace_bytes(ctx, batch, 16); ranks <= 64.      */
+slim_status slim_reserve_positions(slim_ctx* ctx, int max_position);
+slim_status slim_decode_partial(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,
+                                const int32_t* first_tile, const int32_t* q_pos, float* lse_out, float* u_out,
+                                void* workspace, void* stream);
+slim_status slim_combine_project(slim_ctx* ctx, const float* lse_all, const float* u_all, int ranks,
+                                 const int32_t* total_lengths, int batch, float* o, void* workspace, void* stream);
+
 /* Synchronises `stream`, returns the sticky device status (SLIM_OK,
  * SLIM_ERR_CAPACITY or SLIM_ERR_TIMEOUT) and clears it.                        */
 slim_status slim_device_status(slim_ctx* ctx, void* stream);

@@ -339,6 +339,51 @@ def oracle_slim_fp8(q: np.ndarray, K: np.ndarray, W_KV: np.ndarray, H: int, rope
     return oracle_slim(q, quantize_keys_e4m3(K, H)[2], W_KV, H, rope_theta)
 
 
+# --------------------------------------------------------------------------
+# One context split into slices (several GPUs): per-slice partial results and their join
+# --------------------------------------------------------------------------
+def oracle_slim_partial(q: np.ndarray, K_slice: np.ndarray, first_pos: int, q_pos: int, H: int, rope_theta: float = 0.0):
+    """Rows K_slice [n, d] sit at absolute positions first_pos .. first_pos + n - 1, the query at q_pos.
+    Per head: z_t = RoPE_{q_pos}(q_i) . RoPE_t(k_{t,i}) / sqrt(d_k) (natural-log units),
+    lse = log2 sum_t e^{z_t}  (reported in log2 units, as the library does), u = sum_t e^{z_t} K[t, :] / sum_t e^{z_t}.
+    An empty slice gives lse = -inf and u = 0.  Returns (lse [H], u [H, d])."""
+    q = np.asarray(q, dtype=F64)
+    K_slice = np.asarray(K_slice, dtype=F64)
+    n, d = K_slice.shape
+    d_k = d // H
+    lse = np.full(H, -np.inf)
+    u = np.zeros((H, d), dtype=F64)
+    if n == 0:
+        return lse, u
+    pos = first_pos + np.arange(n)
+    for i in range(H):
+        sl = slice(i * d_k, (i + 1) * d_k)
+        z = rope_encode(K_slice[:, sl], pos, rope_theta) @ rope_encode(q[sl], q_pos, rope_theta) / math.sqrt(d_k)
+        zmax = np.max(z)
+        e = np.exp(z - zmax)
+        lse[i] = (zmax + math.log(np.sum(e))) / math.log(2.0)
+        u[i] = (e @ K_slice) / np.sum(e)
+    return lse, u
+
+
+def oracle_combine_partials(lse_all: np.ndarray, u_all: np.ndarray, W_KV: np.ndarray) -> np.ndarray:
+    """Join of R slices: lse_all [R, H] (log2 units), u_all [R, H, d].  Per head w_r = 2^lse_r / sum_r' 2^lse_r',
+    u = sum_r w_r u_r, head_i = u W_KV,i (Eq. 7 Option 2).  All slices empty gives zeros."""
+    lse_all = np.asarray(lse_all, dtype=F64)
+    u_all = np.asarray(u_all, dtype=F64)
+    W_KV = np.asarray(W_KV, dtype=F64)
+    R, H, d = u_all.shape
+    d_k = d // H
+    out = np.zeros(d, dtype=F64)
+    for i in range(H):
+        if not np.any(np.isfinite(lse_all[:, i])):
+            continue
+        w = np.exp2(lse_all[:, i] - np.max(lse_all[:, i]))
+        w = w / np.sum(w)
+        out[i * d_k:(i + 1) * d_k] = (w @ u_all[:, i, :]) @ W_KV[:, i * d_k:(i + 1) * d_k]
+    return out
+
+
 def oracle_slim_batch(q: np.ndarray, K: np.ndarray, lengths, W_KV: np.ndarray, H: int,
                       rope_theta: float = 0.0) -> np.ndarray:
     """Ragged batch: q [B, d], K [B, T_cap, d], lengths[b] rows valid.

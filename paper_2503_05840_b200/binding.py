@@ -42,6 +42,9 @@ SIGNATURES = {
     "slim_xcache_set_weights": (c_int, [c_void_p, c_void_p, c_void_p, c_int]),
     "slim_xcache_workspace_bytes": (c_size_t, [c_void_p, c_int, c_int]),
     "slim_xcache_decode": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "slim_reserve_positions": (c_int, [c_void_p, c_int]),
+    "slim_decode_partial": (c_int, [c_void_p] * 10),
+    "slim_combine_project": (c_int, [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
     "slim_device_status": (c_int, [c_void_p, c_void_p]),
     "slim_selftest_bounded_wait": (c_int, [c_void_p, c_void_p]),
     "slim_profile_enable": (c_int, [c_void_p, c_int]),
@@ -221,6 +224,20 @@ def slim_xcache_workspace_bytes(ctx: int, batch: int, t_cap: int) -> int:
 def slim_xcache_decode(ctx: int, q, cache: int, lengths, o, workspace, stream: int = 0) -> None:
     _check(lib().slim_xcache_decode(c_void_p(ctx), _ptr(q), c_void_p(cache), _ptr(lengths), _ptr(o), _ptr(workspace),
                                     c_void_p(stream)), "slim_xcache_decode")
+
+
+def slim_reserve_positions(ctx: int, max_position: int) -> None:
+    _check(lib().slim_reserve_positions(c_void_p(ctx), int(max_position)), "slim_reserve_positions")
+
+
+def slim_decode_partial(ctx: int, q, cache: int, lengths, first_tile, q_pos, lse_out, u_out, workspace, stream: int = 0) -> None:
+    _check(lib().slim_decode_partial(c_void_p(ctx), _ptr(q), c_void_p(cache), _ptr(lengths), _ptr(first_tile), _ptr(q_pos),
+                                     _ptr(lse_out), _ptr(u_out), _ptr(workspace), c_void_p(stream)), "slim_decode_partial")
+
+
+def slim_combine_project(ctx: int, lse_all, u_all, ranks: int, total_lengths, batch: int, o, workspace, stream: int = 0) -> None:
+    _check(lib().slim_combine_project(c_void_p(ctx), _ptr(lse_all), _ptr(u_all), ranks, _ptr(total_lengths), batch, _ptr(o),
+                                      _ptr(workspace), c_void_p(stream)), "slim_combine_project")
 
 
 def slim_device_status(ctx: int, stream: int = 0) -> int:

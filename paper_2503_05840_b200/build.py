@@ -9,8 +9,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libslim.so")
-SOURCES = ["slim_api.cu", "slim_generic.cu", "slim_tail.cu", "slim_wkv.cu", "slim_tc.cu", "slim_proj.cu", "slim_xscores.cu", "slim_prompt.cu"]
-HEADERS = ["slim_internal.h", "slim_sched.cuh", "slim_ptx.cuh"]
+SOURCES = ["slim_api.cu", "slim_generic.cu", "slim_tail.cu", "slim_wkv.cu", "slim_tc.cu", "slim_proj.cu", "slim_xscores.cu", "slim_prompt.cu", "slim_split.cu"]
+HEADERS = ["slim_internal.h", "slim_sched.cuh", "slim_ptx.cuh", "slim_combine.cuh"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC"]
 

@@ -420,10 +420,18 @@ slim_status slim_append_k(slim_ctx* ctx, slim_cache* cache, const void* k_new, c
 }
 
 namespace {
+// What a context-split rank asks for instead of the projected output: the slice's (lse, u) per (sequence, head).
+struct PartialOut {
+  const int32_t* first_tile;     // device [batch]: absolute tile of the cache's first row
+  const int32_t* q_pos;          // device [batch]: absolute position of the query
+  float* lse;                    // device [batch][H]
+  float* u;                      // device [batch][H][d]
+};
+
 // k_new != NULL: the generate-phase step (newest key rows written at lengths[b] - 1 first)
 slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths, float* o,
-                        void* workspace, void* stream, bool xcache, const void* k_new = nullptr) {
-  if (!ctx || !q || !cache || !lengths || !o || !workspace || cache->ctx != ctx) return SLIM_ERR_INVALID_ARG;
+                        void* workspace, void* stream, bool xcache, const void* k_new = nullptr, const PartialOut* part = nullptr) {
+  if (!ctx || !q || !cache || !lengths || (!o && !part) || !workspace || cache->ctx != ctx) return SLIM_ERR_INVALID_ARG;
   if (((uintptr_t)workspace & 255) || ((uintptr_t)q & 15) || ((uintptr_t)o & 15)) return SLIM_ERR_INVALID_ARG;
   if (!ctx->has_weights) return SLIM_ERR_NO_WEIGHTS;
   int path = path_in_use(ctx);
@@ -469,7 +477,10 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   // with a flagged unit is recomputed by the combine kernel (no append kernel, no redo kernel)
   const bool tc_kcache = !xcache && path == SLIM_PATH_TC && !ctx->opt_legacy_flow;
   p.k_new = tc_kcache ? k_new : nullptr;
-  p.redo_in_combine = (tc_kcache && ctx->proj_ok) ? 1 : 0;
+  p.redo_in_combine = (tc_kcache && ctx->proj_ok && !part) ? 1 : 0;
+  p.pos_tiles = part ? part->first_tile : nullptr;
+  p.q_pos = part ? part->q_pos : nullptr;
+  p.rope_tiles = ctx->rope_base_tiles;
   cudaStream_t st = (cudaStream_t)stream;
   int launches = 0;
   if (k_new && !p.k_new) {                           // no fused update on this path: the append kernel first
@@ -508,7 +519,10 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
     launches += 2;                                   // scores, accumulation
   }
   if (ctx->prof_on) cudaEventRecord(ctx->prof_ev[1], st);
-  if (e == cudaSuccess) {
+  if (e == cudaSuccess && part) {                    // a rank of a split context: (lse, u) of its slice, no projection
+    e = slim_launch_partial_out(ctx, p, part->lse, part->u, st);
+    ++launches;
+  } else if (e == cudaSuccess) {
     if (ctx->proj_ok) {
       float* o_part = reinterpret_cast<float*>(ws + L.o_part);
       e = slim_launch_proj(ctx, p, reinterpret_cast<unsigned char*>(ws + L.u_tiled), o_part, st);
@@ -534,6 +548,54 @@ slim_status slim_decode_step(slim_ctx* ctx, const void* q, const void* k_new, sl
                              float* o, void* workspace, void* stream) {
   if (!k_new || ((uintptr_t)k_new & 15)) return SLIM_ERR_INVALID_ARG;
   return decode_impl(ctx, q, cache, lengths, o, workspace, stream, false, k_new);
+}
+
+slim_status slim_reserve_positions(slim_ctx* ctx, int max_position) {
+  if (!ctx || max_position <= 0) return SLIM_ERR_INVALID_ARG;
+  return grow_rope_base(ctx, max_position);
+}
+
+slim_status slim_decode_partial(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,
+                                const int32_t* first_tile, const int32_t* q_pos, float* lse_out, float* u_out,
+                                void* workspace, void* stream) {
+  if (!first_tile || !q_pos || !lse_out || !u_out) return SLIM_ERR_INVALID_ARG;
+  if (ctx && ctx->kdtype == SLIM_FP8) return SLIM_ERR_UNSUPPORTED;
+  const PartialOut part = {first_tile, q_pos, lse_out, u_out};
+  return decode_impl(ctx, q, cache, lengths, nullptr, workspace, stream, false, nullptr, &part);
+}
+
+slim_status slim_combine_project(slim_ctx* ctx, const float* lse_all, const float* u_all, int ranks, const int32_t* total_lengths,
+                                 int batch, float* o, void* workspace, void* stream) {
+  if (!ctx || !lse_all || !u_all || !total_lengths || !o || !workspace) return SLIM_ERR_INVALID_ARG;
+  if (ranks <= 0 || ranks > 64 || batch <= 0 || batch > SLIM_MAX_BATCH) return SLIM_ERR_INVALID_ARG;
+  if (((uintptr_t)workspace & 255) || ((uintptr_t)o & 15)) return SLIM_ERR_INVALID_ARG;
+  if (!ctx->has_weights) return SLIM_ERR_NO_WEIGHTS;
+  // the joined result is laid down as one finished unit per sequence (worker 0 owns every tile of the
+  // schedule below), and the ordinary combine + projection tail completes the step
+  const WsLayout L = ws_layout(ctx, batch, SLIM_TT);
+  char* ws = static_cast<char*>(workspace);
+  SlimDecodeParams p;
+  std::memset(&p, 0, sizeof(p));
+  p.d = ctx->d; p.H = ctx->H; p.d_k = ctx->d_k; p.half = ctx->d_k / 2;
+  p.batch = batch; p.t_cap = 0x3fffffff;
+  p.dtype = ctx->dtype; p.kdtype = ctx->kdtype;
+  p.workers = 1; p.cl = 0; p.min_tiles = 1; p.unit_cost = 0;
+  p.lengths = total_lengths; p.wkv = ctx->wkv;
+  p.part_u = reinterpret_cast<float*>(ws + L.part_u);
+  p.part_m = reinterpret_cast<float*>(ws + L.part_m);
+  p.part_l = reinterpret_cast<float*>(ws + L.part_l);
+  p.unit_flags = reinterpret_cast<int*>(ws + L.flags);
+  p.u = reinterpret_cast<float*>(ws + L.o_part);
+  p.o = o; p.status = ctx->status; p.any_flag = ctx->any_flag;
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = slim_launch_rank_combine(ctx, p, lse_all, u_all, ranks, st);
+  if (e == cudaSuccess) {
+    if (ctx->proj_ok) e = slim_launch_proj(ctx, p, reinterpret_cast<unsigned char*>(ws + L.u_tiled), p.u, st);
+    else e = slim_launch_tail(ctx, p, st);
+  }
+  ctx->launches_last = 3;
+  if (e != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
+  return SLIM_OK;
 }
 
 slim_status slim_xcache_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,

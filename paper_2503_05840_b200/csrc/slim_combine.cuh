@@ -22,8 +22,9 @@ __device__ __forceinline__ uint32_t u_offset(int n, int k) {
 //   w_i = 2^(m_i - M) / sum_j 2^(m_j - M) l_j,   M = max_j (m_j + log2 l_j),
 // so that u = sum_i w_i U_i.  The partials may have been written by other SMs of the same grid:
 // they are read from L2.
-__device__ __forceinline__ void weights_warp(const float* part_m, const float* part_l, int unit0, int wn, int H, int h,
-                                             float* s_w, int lane) {
+// Returns M + log2(sum_j 2^(m_j - M) l_j): the log2 of the sum of 2^argument over the sequence's rows.
+__device__ __forceinline__ float weights_warp(const float* part_m, const float* part_l, int unit0, int wn, int H, int h,
+                                              float* s_w, int lane) {
   float M = -INFINITY;
   for (int i = lane; i < wn; i += 32) {
     const size_t ui = (size_t)(unit0 + i) * H + h;
@@ -43,6 +44,7 @@ __device__ __forceinline__ void weights_warp(const float* part_m, const float* p
   const float inv = 1.f / L;
   __syncwarp();
   for (int i = lane; i < wn; i += 32) s_w[i] *= inv;
+  return M + log2f(L);
 }
 
 // u[b][h][j0 .. j0+8) as hi = bf16(u), lo = bf16(u - hi) into the operand tiles
@@ -75,7 +77,7 @@ __device__ __forceinline__ void fma8(float (&acc)[8], float wg, const float4& a,
 // rotated after the read, written as the query rotated against the key).  Slow by design: it only
 // runs for a sequence one of whose units was flagged.  Called by all threads of the CTA (bf16 cache).
 // s_x: d_k + 2 SLIM_TT + 4 floats of shared memory.
-__device__ __noinline__ void exact_groups(const SlimDecodeParams& p, unsigned char* u_tiled, int hp, int b, int h, int jg0,
+static __device__ __noinline__ void exact_groups(const SlimDecodeParams& p, unsigned char* u_tiled, int hp, int b, int h, int jg0,
                                           int ngroups, float* s_x) {
   const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
   const int d = p.d, dk = p.d_k, half = p.half;
@@ -88,7 +90,7 @@ __device__ __noinline__ void exact_groups(const SlimDecodeParams& p, unsigned ch
   const __nv_bfloat16* __restrict__ Q = reinterpret_cast<const __nv_bfloat16*>(p.q) + (size_t)b * d;
   __syncthreads();
   {
-    const int m = len - 1, mt = m / SLIM_TT, mi = m % SLIM_TT;
+    const int m = slim_query_pos(p, b, len), mt = m / SLIM_TT, mi = m % SLIM_TT;
     for (int jj = tid; jj < dk; jj += nthr) {
       float v;
       if (p.rope) {
@@ -121,7 +123,7 @@ __device__ __noinline__ void exact_groups(const SlimDecodeParams& p, unsigned ch
           const float k1 = __bfloat162float(kr[j]), k2 = __bfloat162float(kr[j + half]);
           const float q1 = s_q[j], q2 = s_q[j + half];
           if (p.rope) {
-            const float2 cb = p.rope_base[(size_t)(t0 / SLIM_TT) * half + j], co = p.rope_off[t * half + j];
+            const float2 cb = p.rope_base[(size_t)(t0 / SLIM_TT + slim_tile_offset(p, b)) * half + j], co = p.rope_off[t * half + j];
             const float c = cb.x * co.x - cb.y * co.y, sn = cb.y * co.x + cb.x * co.y;
             a += c * (q1 * k1 + q2 * k2) + sn * (q1 * k2 - q2 * k1);
           } else {

@@ -85,7 +85,7 @@ slim_exact_kernel(SlimDecodeParams p, int only_flagged) {
     // ---- a2: rotate and scale the query of this sequence --------------------
     __syncthreads();
     {
-      const int m = len - 1, mt = m / SLIM_TT, mi = m % SLIM_TT;
+      const int m = slim_query_pos(p, b, len), mt = m / SLIM_TT, mi = m % SLIM_TT;
       for (int e = tid; e < d; e += GEN_THREADS) {
         const int h = e / dk, jj = e - h * dk;
         float v;
@@ -124,7 +124,7 @@ slim_exact_kernel(SlimDecodeParams p, int only_flagged) {
             const float k1 = ld_k(kr + j), k2 = ld_k(kr + j + half);
             const float q1 = qh[j], q2 = qh[j + half];
             if (p.rope) {
-              const float2 cb = p.rope_base[(size_t)tile * half + j], co = p.rope_off[t * half + j];
+              const float2 cb = p.rope_base[(size_t)(tile + slim_tile_offset(p, b)) * half + j], co = p.rope_off[t * half + j];
               const float c = cb.x * co.x - cb.y * co.y, s = cb.y * co.x + cb.x * co.y;
               a += c * (q1 * k1 + q2 * k2) + s * (q1 * k2 - q2 * k1);
             } else {
@@ -270,7 +270,7 @@ slim_scores_kernel(SlimDecodeParams p, float* __restrict__ scores) {
     __syncthreads();
     if (b != cur_b) {                       // a2: rotate + scale the query of sequence b
       cur_b = b;
-      const int m = len - 1, mt = m / SLIM_TT, mi = m % SLIM_TT;
+      const int m = slim_query_pos(p, b, len), mt = m / SLIM_TT, mi = m % SLIM_TT;
       for (int e = tid; e < d; e += GEN_THREADS) {
         const int h = e / dk, jj = e - h * dk;
         float v;
@@ -299,7 +299,7 @@ slim_scores_kernel(SlimDecodeParams p, float* __restrict__ scores) {
         const float* q2 = q1 + half;
         float a = 0.f;
         if (p.rope) {
-          const float2* cbp = p.rope_base + (size_t)tile * half + j0;
+          const float2* cbp = p.rope_base + (size_t)(tile + slim_tile_offset(p, b)) * half + j0;
           const float2* cop = p.rope_off + t * half + j0;
 #pragma unroll
           for (int x = 0; x < VEC; ++x) {

@@ -45,6 +45,11 @@ struct SlimDecodeParams {
   const float* ext_scores;       // X-cache scheme: precomputed softmax arguments [batch][H][t_cap] (else NULL)
   const int32_t* block_table;    // paged cache: [batch][max_pages] page ids (NULL = contiguous [batch][t_cap][d])
   int page_rows, max_pages, num_pages;
+  // a cache that holds a slice of a longer context (context split over several GPUs): its rows start at absolute
+  // position SLIM_TT * pos_tiles[b] and the query sits at absolute position q_pos[b] (both NULL otherwise)
+  const int32_t* pos_tiles;
+  const int32_t* q_pos;
+  int rope_tiles;                // entries of rope_base (positions < SLIM_TT * rope_tiles are covered)
   const void* k_new;             // tensor-core path: [batch][d] newest key rows, written at row lengths[b]-1 before the read (or NULL)
   int redo_in_combine;           // 1: the combine kernel recomputes the sequences that have a flagged unit (no redo kernel runs)
 };
@@ -169,6 +174,11 @@ size_t slim_xscores_qt_bytes(int d, int batch);
 cudaError_t slim_xscores_make_tmap(const slim_ctx* ctx, slim_cache* c);
 cudaError_t slim_launch_xscores_tc(const slim_ctx* ctx, const slim_cache* c, const SlimDecodeParams& p, const float* W_K,
                                    unsigned char* qt_tiled, float* scores, cudaStream_t st);
+
+// context split over several GPUs (slim_split.cu)
+cudaError_t slim_launch_partial_out(const slim_ctx* ctx, const SlimDecodeParams& p, float* lse_out, float* u_out, cudaStream_t st);
+cudaError_t slim_launch_rank_combine(const slim_ctx* ctx, const SlimDecodeParams& p, const float* lse_all, const float* u_all,
+                                     int ranks, cudaStream_t st);
 
 // prompt phase: V = K W_KV for n rows (slim_prompt.cu)
 cudaError_t slim_launch_values(const slim_ctx* ctx, const void* K, int n, float* V, cudaStream_t st,

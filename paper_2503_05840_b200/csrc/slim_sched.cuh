@@ -113,3 +113,22 @@ __device__ __forceinline__ long long slim_cache_row(const SlimDecodeParams& p, i
   }
   return (long long)b * p.t_cap + t0;
 }
+
+// A cache may hold a slice of a longer context (context split over several GPUs): then its row t sits at
+// absolute position SLIM_TT * pos_tiles[b] + t and the query at q_pos[b].  Otherwise row t is position t and
+// the query sits at the newest row.
+// Positions beyond the RoPE table (slim_reserve_positions) are clamped into it and reported as SLIM_ERR_CAPACITY.
+__device__ __forceinline__ int slim_query_pos(const SlimDecodeParams& p, int b, int len) {
+  if (!p.q_pos) return len - 1;
+  int q = p.q_pos[b];
+  const int top = p.rope_tiles * SLIM_TT - 1;
+  if (q < 0 || q > top) { atomicMax(p.status, (int)SLIM_ERR_CAPACITY); q = q < 0 ? 0 : top; }
+  return q;
+}
+__device__ __forceinline__ int slim_tile_offset(const SlimDecodeParams& p, int b) {
+  if (!p.pos_tiles) return 0;
+  int off = p.pos_tiles[b];
+  const int top = p.rope_tiles - 1 - (p.t_cap + SLIM_TT - 1) / SLIM_TT;      // the slice's last tile must stay inside the table
+  if (off < 0 || off > top) { atomicMax(p.status, (int)SLIM_ERR_CAPACITY); off = off < 0 || top < 0 ? 0 : top; }
+  return off;
+}

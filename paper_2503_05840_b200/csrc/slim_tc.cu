@@ -230,6 +230,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
         const int tile0 = gg - s_prefix[b], ntile = seg_end - gg;
         const int unit = w + b;
         const int len = min(max(p.lengths[b], 0), p.t_cap);
+        const int toff = ROPE ? slim_tile_offset(p, b) : 0;       // absolute tile of the cache's first row
         // ---- a2: this thread's slice of the query at its own position, scaled ----
         float qh1[8], qh2[8];
 #pragma unroll
@@ -240,7 +241,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           unpack8(__ldg(reinterpret_cast<const uint4*>(Q)), a);
           unpack8(__ldg(reinterpret_cast<const uint4*>(Q + PAIRS)), c);
           if (ROPE) {
-            const int m = len - 1, mt = m / SLIM_TT, mi = m % SLIM_TT;
+            const int m = slim_query_pos(p, b, len), mt = m / SLIM_TT, mi = m % SLIM_TT;
 #pragma unroll
             for (int x = 0; x < 8; ++x) {
               const float2 cb = p.rope_base[(size_t)mt * PAIRS + 8 * jl + x], co = p.rope_off[mi * PAIRS + 8 * jl + x];
@@ -272,7 +273,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
               // exact Q at this thread's first row of the tile (position t0 + rp)
 #pragma unroll
               for (int x = 0; x < 4; ++x) {
-                const float4 cb = __ldg(reinterpret_cast<const float4*>(p.rope_base + (size_t)tile * PAIRS + 8 * jl + 2 * x));
+                const float4 cb = __ldg(reinterpret_cast<const float4*>(p.rope_base + (size_t)(tile + toff) * PAIRS + 8 * jl + 2 * x));
                 const float4 co = __ldg(reinterpret_cast<const float4*>(p.rope_off + rp * PAIRS + 8 * jl + 2 * x));
                 const float c0 = cb.x * co.x - cb.y * co.y, s0 = cb.y * co.x + cb.x * co.y;
                 const float c1 = cb.z * co.z - cb.w * co.w, s1 = cb.w * co.z + cb.z * co.w;
@@ -365,7 +366,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
               lsum = 0.f;
             }
             float x = sv - mref;
-            if (valid && x > TC_XMAX) { p.unit_flags[2 * unit + (int)rank] = 1; if (EXT) *p.any_flag = 1; x = TC_XMAX; }
+            if (valid && x > TC_XMAX) { p.unit_flags[2 * unit + (int)rank] = 1; if (EXT || !p.redo_in_combine) *p.any_flag = 1; x = TC_XMAX; }
             const float pf = valid ? ex2_approx(x) : 0.f;
             const __nv_bfloat16 pb = __float2bfloat16_rn(pf);
             if ((jl % DUP) == 0) lsum += __bfloat162float(pb);

@@ -93,3 +93,54 @@ def test_spawn_replicas_starts_one_process_per_rank(tmp_path):
         line = json.load(f)
     assert line["n_gpus"] == 2 and line["ms_per_step"] == 6.0 and line["scaling"] == "weak"
     assert np.isclose(line["value"], 16 * 2 / 6e-3)
+
+
+def _split_rank(rank, world, out_dir):
+    """One rank of a split context on CPU: its slice's partial comes from the oracle (the CUDA kernels
+    need a GPU), the exchange and the index logic are the package's own."""
+    sys.path.insert(0, ROOT)
+    import json
+    import torch
+    import torch.distributed as dist
+    from oracle import slim_oracle as so
+    from paper_2503_05840_b200 import context_split as cs
+    from paper_2503_05840_b200 import synth
+    dist.init_process_group("gloo")
+    cfg = synth.SlimConfig("split", 32, 2, 16, 3, 100, 1, 1.0e4, "f32")
+    lengths = np.array([100, 37, 0], dtype=np.int32)
+    L = synth.make_layer(cfg, 2468, lengths=lengths)                  # same seed on every rank: the same context
+    W_KV = so.oracle_wkv(L.W_K, L.W_V)
+    first, count = cs.shard_batch(lengths, world, rank)
+    lse = np.empty((cfg.batch, cfg.H)); u = np.empty((cfg.batch, cfg.H, cfg.d))
+    for b in range(cfg.batch):
+        a = first[b] * cs.TILE
+        lse[b], u[b] = so.oracle_slim_partial(L.q[b], L.K[b, a:a + count[b]], a, int(lengths[b]) - 1, cfg.H, cfg.rope_theta)
+    lse_all, u_all = cs.gather_partials(torch.from_numpy(lse), torch.from_numpy(u), dist)
+    assert tuple(lse_all.shape) == (world, cfg.batch, cfg.H) and tuple(u_all.shape) == (world, cfg.batch, cfg.H, cfg.d)
+    worst = 0.0
+    for b in range(cfg.batch):
+        out = so.oracle_combine_partials(lse_all[:, b].numpy(), u_all[:, b].numpy(), W_KV)
+        ref = so.oracle_slim_batch(L.q, L.K, lengths, W_KV, cfg.H, cfg.rope_theta)[b]
+        worst = max(worst, float(np.max(np.abs(out - ref))))
+    dist.barrier()
+    with open(os.path.join(out_dir, f"rank{rank}.json"), "w") as f:
+        json.dump({"worst": worst, "count": count, "first": first}, f)
+    dist.destroy_process_group()
+
+
+def test_context_split_two_ranks_exchange_and_join(tmp_path):
+    import json
+    sys.path.insert(0, ROOT)
+    from paper_2503_05840_b200 import context_split as cs
+    from paper_2503_05840_b200 import replicas
+    # slices are whole tiles, cover the context once, and the ragged tail goes to the last non-empty slice
+    for n in (0, 1, 15, 16, 17, 100, 131072):
+        for world in (1, 2, 3, 8):
+            cuts = [cs.shard_rows(n, world, r) for r in range(world)]
+            assert cuts[0][0] == 0 and cuts[-1][1] == n
+            assert all(a[1] == b[0] for a, b in zip(cuts[:-1], cuts[1:]))
+            assert all(a % cs.TILE == 0 for a, _ in cuts if a < n)
+    replicas.spawn_replicas(_split_rank, 2, (str(tmp_path),))
+    res = [json.load(open(tmp_path / f"rank{r}.json")) for r in range(2)]
+    assert all(r["worst"] < 1e-12 for r in res)                       # every rank holds the whole-context result
+    assert [a + b for a, b in zip(res[0]["count"], res[1]["count"])] == [100, 37, 0]

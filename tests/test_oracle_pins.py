@@ -600,3 +600,30 @@ def test_fp8_key_quantisation_exponent_and_exactness():
     K3 = synth.round_to_bf16(g.standard_normal((50, 64))).astype(np.float64)
     ref = so.oracle_slim(q, K3, W, 4, 1.0e4)
     assert so.err_rms_norm(so.oracle_slim_fp8(q, K3, W, 4, 1.0e4), ref) < 0.2
+
+
+# ---- one context split into slices ---------------------------------------------------------------
+def test_partials_of_any_split_join_to_the_whole_context():
+    T, d, H = 77, 16, 2
+    X, W_Q, W_K, W_V = _rand_case(50, T, d, H)
+    K, q, W_KV = X @ W_K, X[-1] @ W_Q, so.oracle_wkv(W_K, W_V)
+    for theta in (0.0, 1.0e4):
+        whole = so.oracle_vanilla(X, W_Q, W_K, W_V, H, theta)
+        for cuts in ([0, T], [0, 16, 48, T], [0, 32, 32, 64, T], [0, 1, T]):      # incl. an empty slice and a one-row slice
+            parts = [so.oracle_slim_partial(q, K[a:b], a, T - 1, H, theta) for a, b in zip(cuts[:-1], cuts[1:])]
+            out = so.oracle_combine_partials(np.stack([p[0] for p in parts]), np.stack([p[1] for p in parts]), W_KV)
+            assert np.max(np.abs(out - whole)) <= 1e-10 * np.max(np.abs(whole))
+
+
+def test_partial_hand_case_single_row_and_two_equal_rows():
+    # one head of width 2, no RoPE.  One row k: lse = (q.k / sqrt 2) / ln 2, u = k.  Two identical rows: lse grows by exactly 1.
+    q = np.array([2.0, 0.0]); k = np.array([[math.sqrt(2.0) * math.log(2.0) * 1.5, 7.0]])
+    lse, u = so.oracle_slim_partial(q, k, 0, 0, 1, 0.0)
+    assert abs(lse[0] - 3.0) < 1e-12 and np.array_equal(u[0], k[0])          # q.k / sqrt 2 = 3 ln 2
+    lse2, u2 = so.oracle_slim_partial(q, np.vstack([k, k]), 0, 1, 1, 0.0)
+    assert abs(lse2[0] - 4.0) < 1e-12 and np.allclose(u2[0], k[0])
+    lse0, u0 = so.oracle_slim_partial(q, np.zeros((0, 2)), 0, 0, 1, 0.0)
+    assert lse0[0] == -np.inf and np.all(u0 == 0)
+    # join by hand: slices with lse 3 and 4 weigh 1/3 and 2/3
+    out = so.oracle_combine_partials(np.array([[3.0], [4.0]]), np.array([[[3.0, 0.0]], [[0.0, 3.0]]]), np.eye(2))
+    assert np.allclose(out, [1.0, 2.0])
