@@ -49,6 +49,7 @@ struct SlimDecodeParams {
   // position SLIM_TT * pos_tiles[b] and the query sits at absolute position q_pos[b] (both NULL otherwise)
   const int32_t* pos_tiles;
   const int32_t* q_pos;
+  int k_evict_first;             // tensor-core path: key tiles are loaded with the L2 evict-first hint
   int rope_tiles;                // entries of rope_base (positions < SLIM_TT * rope_tiles are covered)
   const void* k_new;             // tensor-core path: [batch][d] newest key rows, written at row lengths[b]-1 before the read (or NULL)
   int redo_in_combine;           // 1: the combine kernel recomputes the sequences that have a flagged unit (no redo kernel runs)
@@ -81,6 +82,7 @@ struct slim_ctx {
   int opt_tc_rt;                 // SLIM_TC_RT: rows per thread and tile (0 = default)
   int opt_unit_cost;             // SLIM_TC_UNIT_COST: boundary cost of the schedule in tiles (-1 = default)
   int opt_xscores_cuda;          // SLIM_XSCORES_CUDA: dense X-cache scores on CUDA cores
+  int opt_k_evict;               // SLIM_TC_K_EVICT (0/1): L2 evict-first hint on the key loads (default on)
   int opt_legacy_flow;           // SLIM_TC_LEGACY: append and exact redo as kernels of their own (for side-by-side timing)
   alignas(64) unsigned char wmap[128];   // CUtensorMap over W_KV for the projection kernel
 };

@@ -497,6 +497,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
         int it = 0, st = 0;
         uint32_t kph = 0;
         bool ok = true;
+        const uint64_t l2pol = l2_policy_evict_first();
         {
           // Clear this CTA's redo flags of the worker's units.  A score warp can only raise one after
           // it has seen a k_full phase, which takes this thread's arming arrival (a release) below:
@@ -518,8 +519,12 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
                  mbar_wait<false>(bar_p_empty + 8 * (PAIR ? st >> 1 : st), kph ^ 1, s_abort, p.status);
             if (!ok) break;
             mbar_arrive_expect_tx(bar_k_full + 8 * st, (uint32_t)g.stage_bytes);
-            tma_load_3d(k_stage0 + (uint32_t)st * g.stage_bytes, &tmap, bar_k_full + 8 * st, 0,
-                        (int)slim_cache_row(p, b, (tile0 + kt) * SLIM_TT), (int)rank * g.nc64);
+            if (p.k_evict_first)
+              tma_load_3d_hint(k_stage0 + (uint32_t)st * g.stage_bytes, &tmap, bar_k_full + 8 * st, 0,
+                               (int)slim_cache_row(p, b, (tile0 + kt) * SLIM_TT), (int)rank * g.nc64, l2pol);
+            else
+              tma_load_3d(k_stage0 + (uint32_t)st * g.stage_bytes, &tmap, bar_k_full + 8 * st, 0,
+                          (int)slim_cache_row(p, b, (tile0 + kt) * SLIM_TT), (int)rank * g.nc64);
           }
           gg = seg_end;
         }
