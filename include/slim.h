@@ -41,7 +41,7 @@ extern "C" {
 typedef enum {
   SLIM_OK = 0,
   SLIM_ERR_INVALID_ARG = 1,  /* NULL pointer, non-positive size, bad enum          */
-  SLIM_ERR_UNSUPPORTED = 2,  /* d != H*d_k, d_k not a multiple of 16, H > 64, ...   */
+  SLIM_ERR_UNSUPPORTED = 2,  /* d != H*d_k, odd d_k, H > 64, ...                       */
   SLIM_ERR_SINGULAR = 3,     /* W_K has a (numerically) zero pivot                  */
   SLIM_ERR_CAPACITY = 4,     /* append beyond t_cap / length beyond t_cap (device)  */
   SLIM_ERR_OOM = 5,          /* a library-owned allocation failed                   */
@@ -77,7 +77,8 @@ typedef struct slim_cache slim_cache; /* view of caller-owned key storage [B][t_
 
 /* One layer of shape (d, H, d_k); rope_theta = 0 disables RoPE; dtype is the
  * type of the K-cache and of q.  Requires d == H*d_k (Eq. 6 needs a square
- * W_K), H <= 64, d_k a multiple of 16 and <= 256.  Uses the current CUDA device. */
+ * W_K), H <= 64, d_k even and <= 256 (the tensor-core kernels take d_k = 64, 96, 128; other
+ * widths, e.g. d_k = 100, run on the CUDA-core kernels).  Uses the current CUDA device. */
 slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta, int dtype);
 void        slim_destroy(slim_ctx* ctx);
 

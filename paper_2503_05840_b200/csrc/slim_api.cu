@@ -151,7 +151,7 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
   const int kdtype = dtype;
   if (dtype == SLIM_FP8) dtype = SLIM_BF16;            // 8-bit cache; queries, new rows and W_KV are bf16
   if ((long long)H * d_k != d) return SLIM_ERR_UNSUPPORTED;       // Eq. 6 needs a square W_K
-  if (H > SLIM_MAX_H || d_k > 256 || (d_k % 16) != 0 || d > 16384) return SLIM_ERR_UNSUPPORTED;
+  if (H > SLIM_MAX_H || d_k > 256 || (d_k % 2) != 0 || d > 16384) return SLIM_ERR_UNSUPPORTED;      // rotation pairs need an even width
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return SLIM_ERR_CUDA;
   cudaDeviceProp prop;

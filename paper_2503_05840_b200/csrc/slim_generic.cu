@@ -287,6 +287,33 @@ slim_scores_kernel(SlimDecodeParams p, float* __restrict__ scores) {
       }
       __syncthreads();
     }
+    if (half % VEC != 0) {
+      // head widths whose half is not a multiple of the vector width (e.g. d_k = 100): element loads,
+      // one warp per row, the lanes share the pairs of a head
+      for (int t = wid; t < SLIM_TT; t += GEN_THREADS / 32) {
+        if (t0 + t >= len) continue;
+        const long long row = slim_cache_row(p, b, t0) + t;
+        const KT* kr = Kc + (size_t)row * d;
+        for (int h = 0; h < H; ++h) {
+          const float* q1 = s_q + h * dk;
+          float a = 0.f;
+          for (int j = lane; j < half; j += 32) {
+            const float k1 = ld_k(kr + h * dk + j), k2 = ld_k(kr + h * dk + j + half);
+            if (p.rope) {
+              const float2 cb = __ldg(p.rope_base + (size_t)(tile + slim_tile_offset(p, b)) * half + j), co = __ldg(p.rope_off + t * half + j);
+              const float c = cb.x * co.x - cb.y * co.y, s = cb.y * co.x + cb.x * co.y;
+              a += c * (q1[j] * k1 + q1[j + half] * k2) + s * (q1[j] * k2 - q1[j + half] * k1);
+            } else {
+              a += q1[j] * k1 + q1[j + half] * k2;
+            }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+          if (lane == 0) scores[((size_t)b * H + h) * p.t_cap + t0 + t] = a * k_scale(p, row, h);
+        }
+      }
+      continue;
+    }
     for (int t = wid; t < SLIM_TT; t += GEN_THREADS / 32) {
       if (t0 + t >= len) continue;
       const KT* kr = Kc + (size_t)(slim_cache_row(p, b, t0) + t) * d;

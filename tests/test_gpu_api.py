@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-@pytest.mark.parametrize("d,H", [(32, 2), (96, 3), (384, 6), (960, 10), (1280, 20)])
+@pytest.mark.parametrize("d,H", [(32, 2), (96, 3), (384, 6), (1000, 10), (1280, 20)])
 def test_set_weights_matches_oracle_and_closed_form(d, H):
     W_Q, W_K, W_V, Qo, s = synth.make_weights(d, 77 + d)
     layer = SlimLayer(d, H, d // H, 0.0, "f32", 1, 16, DEV)

@@ -76,6 +76,9 @@ SMALL_SHAPES = [
     (1280, 20, 64, 0.0, "bf16"),
     (768, 8, 96, 1.0e4, "bf16"),
     (1024, 8, 128, 1.0e6, "bf16"),
+    (200, 2, 100, 1.0e4, "f32"),        # head widths outside the vector paths (d_k = 100, as in a d = 3200 / 32-head model)
+    (400, 4, 100, 0.0, "bf16"),
+    (168, 4, 42, 1.0e4, "f32"),
 ]
 
 
