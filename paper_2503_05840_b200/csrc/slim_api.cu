@@ -24,7 +24,7 @@ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 inline size_t esize(int dtype) { return dtype == SLIM_BF16 ? 2 : 4; }
 
 struct WsLayout {
-  size_t part_u, part_m, part_l, flags, o_part, scores, u_tiled, total;
+  size_t part_u, part_m, part_l, flags, o_part, scores, u_tiled, u32, su, total;
   int units;
 };
 
@@ -39,6 +39,8 @@ WsLayout ws_layout(const slim_ctx* ctx, int batch, int t_cap) {
   L.o_part = off; off = align256(off + sizeof(float) * slim_tail_opart_floats(ctx->d, batch));
   L.scores = off; off = align256(off + sizeof(float) * (size_t)batch * ctx->H * t_cap);   // generic path only
   L.u_tiled = off; off = align256(off + (ctx->proj_ok ? slim_proj_u_bytes(ctx->d, ctx->H, batch) : 0));   // tensor-core tail only
+  L.u32 = off; off = align256(off + (ctx->proj_ok ? sizeof(float) * (size_t)batch * ctx->H * ctx->d : 0));
+  L.su = off; off = align256(off + (ctx->proj_ok ? sizeof(float) * (size_t)((batch + 15) / 16) * 16 * ctx->H : 0));
   L.total = off;
   return L;
 }
@@ -171,6 +173,7 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
     c->opt_unit_cost = ((e = getenv("SLIM_TC_UNIT_COST")) && atoi(e) >= 0 && atoi(e) <= 64) ? atoi(e) : -1;
     c->opt_xscores_cuda = getenv("SLIM_XSCORES_CUDA") ? 1 : 0;
     c->opt_legacy_flow = getenv("SLIM_TC_LEGACY") ? 1 : 0;
+    c->opt_proj_ns = (e = getenv("SLIM_PROJ_NS")) ? atoi(e) : 0;
     c->opt_k_evict = (e = getenv("SLIM_TC_K_EVICT")) ? atoi(e) : 1;      // measured side by side: ~1 % per step
   }
   if (cudaMalloc(&c->status, sizeof(int)) != cudaSuccess) { delete c; return SLIM_ERR_OOM; }
@@ -178,6 +181,12 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
   if (cudaMalloc(&c->any_flag, sizeof(int)) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
   cudaMemset(c->any_flag, 0, sizeof(int));
   if (cudaMalloc(&c->wkv, esize(dtype) * (size_t)d * d + 256) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
+  if (dtype == SLIM_BF16) {
+    if (cudaMalloc(&c->wkv_h, 2 * (size_t)d * d + 256) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
+    cudaMemset(c->wkv_h, 0, 2 * (size_t)d * d + 256);
+    if (cudaMalloc(&c->wkv_hscale, sizeof(float) * SLIM_MAX_H) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
+    cudaMemset(c->wkv_hscale, 0, sizeof(float) * SLIM_MAX_H);
+  }
   if (rope_theta != 0.0) {
     const int half = d_k / 2;
     std::vector<float2> off((size_t)SLIM_TT * half);
@@ -213,6 +222,8 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
 void slim_destroy(slim_ctx* ctx) {
   if (!ctx) return;
   cudaFree(ctx->wkv);
+  cudaFree(ctx->wkv_h);
+  cudaFree(ctx->wkv_hscale);
   cudaFree(ctx->rope_off);
   cudaFree(ctx->rope_base);
   cudaFree(ctx->status);
@@ -253,7 +264,7 @@ slim_status slim_set_weights(slim_ctx* ctx, const void* W_K, const void* W_V, in
     if (cudaMemcpy(wkv_out, B, sizeof(double) * nn, cudaMemcpyDeviceToHost) != cudaSuccess) st = SLIM_ERR_CUDA;
   }
   if (st == SLIM_OK) {
-    if (slim_wkv_store(B, ctx->d, ctx->H, ctx->d_k, ctx->dtype, ctx->wkv) != cudaSuccess ||
+    if (slim_wkv_store(B, ctx->d, ctx->H, ctx->d_k, ctx->dtype, ctx->wkv, ctx->wkv_h, ctx->wkv_hscale) != cudaSuccess ||
         cudaDeviceSynchronize() != cudaSuccess)
       st = SLIM_ERR_CUDA;
     else
@@ -294,7 +305,7 @@ slim_status slim_set_weights_nonsquare(slim_ctx* ctx, const void* W_K, const voi
   }
   if (st == SLIM_OK && wkv_out && cudaMemcpy(wkv_out, X, sizeof(double) * ee, cudaMemcpyDeviceToHost) != cudaSuccess) st = SLIM_ERR_CUDA;
   if (st == SLIM_OK) {
-    if (slim_wkv_store(X, ctx->d, ctx->H, ctx->d_k, ctx->dtype, ctx->wkv) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess)
+    if (slim_wkv_store(X, ctx->d, ctx->H, ctx->d_k, ctx->dtype, ctx->wkv, ctx->wkv_h, ctx->wkv_hscale) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess)
       st = SLIM_ERR_CUDA;
     else
       ctx->has_weights = 1;
@@ -327,7 +338,7 @@ slim_status slim_set_wkv(slim_ctx* ctx, const void* W_KV, int host_dtype) {
   double* X = nullptr;
   slim_status st = upload_f64(W_KV, host_dtype, (size_t)ctx->d * ctx->d, &X);
   if (st != SLIM_OK) return st;
-  if (slim_wkv_store(X, ctx->d, ctx->H, ctx->d_k, ctx->dtype, ctx->wkv) != cudaSuccess ||
+  if (slim_wkv_store(X, ctx->d, ctx->H, ctx->d_k, ctx->dtype, ctx->wkv, ctx->wkv_h, ctx->wkv_hscale) != cudaSuccess ||
       cudaDeviceSynchronize() != cudaSuccess)
     st = SLIM_ERR_CUDA;
   else
@@ -527,8 +538,9 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   } else if (e == cudaSuccess) {
     if (ctx->proj_ok) {
       float* o_part = reinterpret_cast<float*>(ws + L.o_part);
-      e = slim_launch_proj(ctx, p, reinterpret_cast<unsigned char*>(ws + L.u_tiled), o_part, st);
-      launches += 2;                                 // combine, projection
+      e = slim_launch_proj(ctx, p, reinterpret_cast<unsigned char*>(ws + L.u_tiled), reinterpret_cast<float*>(ws + L.u32),
+                           reinterpret_cast<float*>(ws + L.su), st);
+      launches += 2 + slim_proj_needs_convert(ctx, p.batch);      // combine (, operand conversion), projection
     } else {
       e = slim_launch_tail(ctx, p, st);
       launches += 2;                                 // combine + projection slices, slice sum
@@ -592,7 +604,8 @@ slim_status slim_combine_project(slim_ctx* ctx, const float* lse_all, const floa
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e = slim_launch_rank_combine(ctx, p, lse_all, u_all, ranks, st);
   if (e == cudaSuccess) {
-    if (ctx->proj_ok) e = slim_launch_proj(ctx, p, reinterpret_cast<unsigned char*>(ws + L.u_tiled), p.u, st);
+    if (ctx->proj_ok) e = slim_launch_proj(ctx, p, reinterpret_cast<unsigned char*>(ws + L.u_tiled), reinterpret_cast<float*>(ws + L.u32),
+                                           reinterpret_cast<float*>(ws + L.su), st);
     else e = slim_launch_tail(ctx, p, st);
   }
   ctx->launches_last = 3;

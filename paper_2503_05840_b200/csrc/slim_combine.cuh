@@ -1,7 +1,15 @@
 // Pieces of the log-sum-exp combine kernels (slim_proj.cu): the weights of a sequence's units, the
-// store of eight combined values as a bf16 (hi, lo) pair in the operand layout of the projection
+// store of combined values as a scaled float16 (hi, lo) pair in the operand layout of the projection
 // MMA, and the exact recomputation of one head of a sequence whose tensor-core partials cannot be
 // used (a softmax argument ran far above a unit's reference exponent).
+//
+// Operand format.  The projection multiplies float16 operands (11-bit mantissas; bf16 weights alone
+// cost about 1e-2 of the output RMS).  float16 has a narrow exponent range, so every row u[b][h][:]
+// is divided by 2^e, e = exponent of the row's largest magnitude (row values end up in (-1, 1)), and
+// stored as hi = f16(v), lo = f16(v - hi); 2^e goes to su[b][h] and is multiplied back in the
+// projection's epilogue.  Entries far below the row maximum lose relative precision, but their
+// absolute error stays below 2^-24 of the row maximum.
+#include <cuda_fp16.h>
 #pragma once
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -47,22 +55,75 @@ __device__ __forceinline__ float weights_warp(const float* part_m, const float* 
   return M + log2f(L);
 }
 
-// u[b][h][j0 .. j0+8) as hi = bf16(u), lo = bf16(u - hi) into the operand tiles
-__device__ __forceinline__ void store_u8(unsigned char* u_tiled, int d, int H, int hp, int b, int h, int j0, const float (&acc)[8]) {
+// u[b][h][j0 .. j0+8) * inv as hi = f16(v), lo = f16(v - hi) into the operand tiles
+__device__ __forceinline__ void store_u8_h(unsigned char* u_tiled, int d, int H, int hp, int b, int h, int j0, const float (&acc)[8],
+                                           float inv) {
   uint32_t hi[4], lo[4];
 #pragma unroll
   for (int x = 0; x < 4; ++x) {
-    const __nv_bfloat16 h0 = __float2bfloat16_rn(acc[2 * x]), h1 = __float2bfloat16_rn(acc[2 * x + 1]);
-    const __nv_bfloat16 l0 = __float2bfloat16_rn(acc[2 * x] - __bfloat162float(h0));
-    const __nv_bfloat16 l1 = __float2bfloat16_rn(acc[2 * x + 1] - __bfloat162float(h1));
-    hi[x] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-    lo[x] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+    const float v0 = acc[2 * x] * inv, v1 = acc[2 * x + 1] * inv;
+    const __half h0 = __float2half_rn(v0), h1 = __float2half_rn(v1);
+    const __half l0 = __float2half_rn(v0 - __half2float(h0)), l1 = __float2half_rn(v1 - __half2float(h1));
+    hi[x] = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
+    lo[x] = (uint32_t)__half_as_ushort(l0) | ((uint32_t)__half_as_ushort(l1) << 16);
   }
   const int bg = b / PJ_BG, n = b % PJ_BG;
   const size_t tile_bytes = (size_t)1024 * hp;
   unsigned char* t = u_tiled + ((size_t)(bg * (H / hp) + h / hp) * (d / 16) + j0 / 16) * tile_bytes + (size_t)(h % hp) * 1024;
   *reinterpret_cast<uint4*>(t + u_offset(n, j0 & 15)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
   *reinterpret_cast<uint4*>(t + u_offset(PJ_BG + n, j0 & 15)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+}
+// the same eight values as plain floats into the row scratch u32[b][h][:]
+__device__ __forceinline__ void store_u8_f32(float* u32, int d, int H, int b, int h, int j0, const float (&acc)[8]) {
+  float4* t = reinterpret_cast<float4*>(u32 + ((size_t)b * H + h) * d + j0);
+  t[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+  t[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+}
+// largest |v| over the CTA (all threads call it; s_red: 33 floats of shared memory)
+__device__ __forceinline__ float block_absmax(float v, float* s_red) {
+  v = fabsf(v);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float w = threadIdx.x < (blockDim.x >> 5) ? s_red[threadIdx.x] : 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) w = fmaxf(w, __shfl_xor_sync(0xffffffffu, w, o));
+    if (threadIdx.x == 0) s_red[32] = w;
+  }
+  __syncthreads();
+  return s_red[32];
+}
+// 2^-e and 2^e for a row whose largest magnitude is mx: mx 2^-e in [0.5, 1); (1, 1) for a zero or non-finite row
+__device__ __forceinline__ void row_scale(float mx, float& inv, float& scale) {
+  inv = 1.f; scale = 1.f;
+  if (mx > 0.f && mx <= 3.0e38f) {
+    int x;
+    frexpf(mx, &x);
+    x = max(-120, min(120, x));
+    inv = exp2f((float)-x); scale = exp2f((float)x);
+  }
+}
+// The CTA turns the finished float row u32[b][h][:] into operand tiles and records its scale.
+__device__ __forceinline__ void convert_row(const float* u32, unsigned char* u_tiled, float* su, int d, int H, int hp, int b, int h,
+                                            float* s_red) {
+  const float* row = u32 + ((size_t)b * H + h) * d;
+  float mx = 0.f;
+  for (int j = threadIdx.x * 4; j < d; j += blockDim.x * 4) {
+    const float4 v = *reinterpret_cast<const float4*>(row + j);
+    mx = fmaxf(fmaxf(mx, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
+  }
+  mx = block_absmax(mx, s_red);
+  float inv, scale;
+  row_scale(mx, inv, scale);
+  for (int j0 = threadIdx.x * 8; j0 < d; j0 += blockDim.x * 8) {
+    const float4 a = *reinterpret_cast<const float4*>(row + j0), c = *reinterpret_cast<const float4*>(row + j0 + 4);
+    const float acc[8] = {a.x, a.y, a.z, a.w, c.x, c.y, c.z, c.w};
+    store_u8_h(u_tiled, d, H, hp, b, h, j0, acc, inv);
+  }
+  if (threadIdx.x == 0) su[(size_t)b * H + h] = scale;
 }
 
 // acc[0..8) += wg * (eight floats at U)
@@ -77,7 +138,8 @@ __device__ __forceinline__ void fma8(float (&acc)[8], float wg, const float4& a,
 // rotated after the read, written as the query rotated against the key).  Slow by design: it only
 // runs for a sequence one of whose units was flagged.  Called by all threads of the CTA (bf16 cache).
 // s_x: d_k + 2 SLIM_TT + 4 floats of shared memory.
-static __device__ __noinline__ void exact_groups(const SlimDecodeParams& p, unsigned char* u_tiled, int hp, int b, int h, int jg0,
+// The result goes to the float row scratch u32[b][h][:].
+static __device__ __noinline__ void exact_groups(const SlimDecodeParams& p, float* u32, int b, int h, int jg0,
                                           int ngroups, float* s_x) {
   const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
   const int d = p.d, dk = p.d_k, half = p.half;
@@ -172,7 +234,7 @@ static __device__ __noinline__ void exact_groups(const SlimDecodeParams& p, unsi
     const float inv = 1.f / s_sc[2];
 #pragma unroll
     for (int x = 0; x < 8; ++x) acc[x] *= inv;
-    store_u8(u_tiled, d, p.H, hp, b, h, j0, acc);
+    store_u8_f32(u32, d, p.H, b, h, j0, acc);
   }
   __syncthreads();
 }

@@ -64,6 +64,9 @@ struct slim_ctx {
   int path_req;                  // slim_path requested
   int has_weights;
   void* wkv;                     // device [H][d][d_k] ctx dtype
+  void* wkv_h;                   // bf16 contexts: device [H][d][d_k] float16, W_KV,h * 2^a_h (head maximum in [2^14, 2^15)): the
+                                 // operand of the tensor-core projection (11-bit mantissa instead of bf16's 8)
+  float* wkv_hscale;             // device [H]: 2^-a_h
   float2* rope_off;              // device [TT][half]
   float2* rope_base;             // device table, grown by slim_cache_create
   int rope_base_tiles;
@@ -83,8 +86,10 @@ struct slim_ctx {
   int opt_unit_cost;             // SLIM_TC_UNIT_COST: boundary cost of the schedule in tiles (-1 = default)
   int opt_xscores_cuda;          // SLIM_XSCORES_CUDA: dense X-cache scores on CUDA cores
   int opt_k_evict;               // SLIM_TC_K_EVICT (0/1): L2 evict-first hint on the key loads (default on)
+  int opt_proj_ns;               // SLIM_PROJ_NS: stages of the projection kernel (0 = default)
   int opt_legacy_flow;           // SLIM_TC_LEGACY: append and exact redo as kernels of their own (for side-by-side timing)
   alignas(64) unsigned char wmap[128];   // CUtensorMap over W_KV for the projection kernel
+  alignas(64) unsigned char wmap_h[128];    // the same over wkv_h
 };
 
 struct slim_cache {
@@ -125,7 +130,7 @@ cudaError_t slim_wkv_solve_rhs(double* A, double* B, int n, int m, int* info_hos
 cudaError_t slim_dgemm(const double* A, const double* B, double* C, int M, int N, int K, int ta, int tb);
 cudaError_t slim_absdiff_max(const double* A, const double* B, size_t n, double* res_host);
 cudaError_t slim_wkv_residual(const double* Wk, const double* X, const double* Wv, int n, double* res_host);
-cudaError_t slim_wkv_store(const double* X, int d, int H, int d_k, int dtype, void* dst);
+cudaError_t slim_wkv_store(const double* X, int d, int H, int d_k, int dtype, void* dst, void* dst_h, float* hscale);
 
 // tensor-core path (slim_tc.cu)
 int  slim_tc_shape_ok(int d, int H, int d_k, int dtype, int rope, int cl);
@@ -141,9 +146,11 @@ cudaError_t slim_tmap_encode_3d(void* out_map, void* base, const unsigned long l
 // tensor-core combine + projection (slim_proj.cu)
 int    slim_proj_shape_ok(int d, int H, int d_k, int dtype);
 int    slim_proj_jsplit(int d);
+int    slim_proj_needs_convert(const slim_ctx* ctx, int batch);      // 1: the combine writes float rows and a conversion kernel follows
 size_t slim_proj_u_bytes(int d, int H, int batch);
 cudaError_t slim_proj_make_wmap(slim_ctx* ctx);
-cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, unsigned char* u_tiled, float* o_part,
+// u32: [batch][H][d] float scratch, su: [16 ceil(batch / 16)][H] float scales of the operand rows
+cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, unsigned char* u_tiled, float* u32, float* su,
                              cudaStream_t st);
 cudaError_t slim_launch_sum_slices(const float* o_part, float* o, int n, int nsplit, cudaStream_t st);
 

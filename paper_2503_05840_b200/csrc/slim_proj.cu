@@ -2,15 +2,16 @@
 //
 //   slim_combine_kernel   log-sum-exp combine of the context-split partials:
 //                         u[b][h][:] = sum_s w_s U_s[h][:] / sum_s w_s l_s over the
-//                         units s of sequence b.  u is written as a bf16 pair
-//                         (hi = bf16(u), lo = bf16(u - hi)) directly in the
-//                         shared-memory operand layout of the projection MMA, so
-//                         the projection kernel fetches it with plain bulk copies.
+//                         units s of sequence b.  u is written as a scaled float16
+//                         pair (row divided by 2^e, hi = f16(v), lo = f16(v - hi);
+//                         see slim_combine.cuh) directly in the shared-memory
+//                         operand layout of the projection MMA, so the projection
+//                         kernel fetches it with plain bulk copies.
 //   slim_proj_tc_kernel   the per-head projection o_h = u_h W_KV,h of Eq. 7
 //                         (Option 2) for 16 sequences at a time:
 //                         O^T[128 x N] += W_tile^T[128 x 16] u^T[16 x N] with one
 //                         tcgen05.mma per 16 rows of W_KV,h; A = the TMA-staged
-//                         weights used MN-major, B = the u tiles, D in tensor
+//                         float16 weights (scaled per head) used MN-major, B = the u tiles, D in tensor
 //                         memory.  N = 32 per head (16 sequences x {hi, lo}); for
 //                         d_k = 64 two heads share an instruction (M = 2 x 64,
 //                         N = 2 x 32) and the off-diagonal quadrants are ignored; for
@@ -36,7 +37,8 @@ using slim_comb::PJ_BG;
 
 constexpr int PJ_ROWS = 64;                    // rows of W_KV,h per stage (4 MMA k-steps)
 constexpr int PJ_W_BYTES = PJ_ROWS * 128 * 2;  // two 64-column atoms x 64 rows x 128 B
-constexpr int PJ_NS = 4;                       // stages
+constexpr int PJ_NS = 4;                       // stages (at most; a CTA uses g.ns of them)
+constexpr int COMBINE_SMEM_ROW = 8192;         // widest row u[b][h][:] the combine kernel collects in shared memory
 
 struct ProjGeom {
   int hp;        // heads per MMA: 1 (d_k = 96, 128) or 2 (d_k = 64)
@@ -45,6 +47,7 @@ struct ProjGeom {
   int nst;       // stages per CTA = d / 64 / jsplit
   int nbg;       // 16-sequence groups
   int u_bytes;   // bytes of u per stage = 4 k-steps x hp x 1 KB
+  int ns;        // stages in use: as many as keep two CTAs on an SM
 };
 
 // weights [workers], info [4], prefix [batch + 1]; behind them, 16-byte aligned, the scratch of the exact path
@@ -71,7 +74,8 @@ __device__ __forceinline__ void combine_prologue(const SlimDecodeParams& p, cons
 
 // (launch bounds: the register budget of the hot loop; the exact path, a call, may spill under it)
 __global__ void __launch_bounds__(256, 4)
-slim_combine_kernel(const __grid_constant__ SlimDecodeParams p, unsigned char* __restrict__ u_tiled, const int hp) {
+slim_combine_kernel(const __grid_constant__ SlimDecodeParams p, unsigned char* __restrict__ u_tiled, float* __restrict__ u32,
+                    float* __restrict__ su, const int hp) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* s_w = reinterpret_cast<float*>(smem_raw);                 // [workers]
   int* s_info = reinterpret_cast<int*>(s_w + p.workers);           // wlo, wn, flagged
@@ -87,19 +91,31 @@ slim_combine_kernel(const __grid_constant__ SlimDecodeParams p, unsigned char* _
   if (tid < 32) combine_prologue(p, sc, s_prefix, b, h, s_w, s_info, lane);
   __syncthreads();
   const int wlo = s_info[0], wn = s_info[1];
-  if (s_info[2]) {                               // a flagged unit: this (head, sequence) is recomputed exactly
-    float* s_x = reinterpret_cast<float*>(smem_raw + exact_scratch_offset(p));
-    for (int jg0 = 0; jg0 < d / 8; jg0 += blockDim.x)
-      slim_comb::exact_groups(p, u_tiled, hp, b, h, jg0, min((int)blockDim.x, d / 8 - jg0), s_x);
+  float* s_x = reinterpret_cast<float*>(smem_raw + exact_scratch_offset(p));     // d_k + 36 floats (>= the 33 of a reduction)
+  const int ngroups = d / 8;
+  if (b >= p.batch) {                            // padding sequence of a 16-sequence group: zero operand columns
+    const float zero[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int jg = tid; jg < ngroups; jg += blockDim.x) slim_comb::store_u8_h(u_tiled, d, H, hp, b, h, jg * 8, zero, 1.f);
     return;
   }
-  for (int jg = tid; jg < d / 8; jg += blockDim.x) {
+  if (s_info[2]) {                               // a flagged unit: this (head, sequence) is recomputed exactly
+    for (int jg0 = 0; jg0 < ngroups; jg0 += blockDim.x)
+      slim_comb::exact_groups(p, u32, b, h, jg0, min((int)blockDim.x, ngroups - jg0), s_x);
+    slim_comb::convert_row(u32, u_tiled, su, d, H, hp, b, h, s_x);
+    return;
+  }
+  // The row is first collected as floats -- in shared memory when it fits (d <= 8192), else in the global
+  // scratch -- so that its scale is known before anything is stored as float16.
+  const size_t ustride = (size_t)H * d;
+  const bool in_smem = d <= COMBINE_SMEM_ROW;
+  float* s_row = s_x + p.d_k + 2 * SLIM_TT + 4 + 36;
+  float mx = 0.f;
+  for (int jg = tid; jg < ngroups; jg += blockDim.x) {
     const int j0 = jg * 8;
     float acc[8];
 #pragma unroll
     for (int x = 0; x < 8; ++x) acc[x] = 0.f;
     const float* Ub = p.part_u + ((size_t)(wlo + b) * H + h) * d + j0;        // unit i lives H*d floats further
-    const size_t ustride = (size_t)H * d;
     int i = 0;
     for (; i + 4 <= wn; i += 4) {                // four units' loads in flight
       float4 a[4], c[4];
@@ -109,28 +125,44 @@ slim_combine_kernel(const __grid_constant__ SlimDecodeParams p, unsigned char* _
         a[k] = __ldcs(U); c[k] = __ldcs(U + 1);
       }
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const float wg = s_w[i + k];
-        acc[0] = fmaf(wg, a[k].x, acc[0]); acc[1] = fmaf(wg, a[k].y, acc[1]); acc[2] = fmaf(wg, a[k].z, acc[2]); acc[3] = fmaf(wg, a[k].w, acc[3]);
-        acc[4] = fmaf(wg, c[k].x, acc[4]); acc[5] = fmaf(wg, c[k].y, acc[5]); acc[6] = fmaf(wg, c[k].z, acc[6]); acc[7] = fmaf(wg, c[k].w, acc[7]);
-      }
+      for (int k = 0; k < 4; ++k) slim_comb::fma8(acc, s_w[i + k], a[k], c[k]);
     }
     for (; i < wn; ++i) {
-      const float wg = s_w[i];
       const float4* U = reinterpret_cast<const float4*>(Ub + (size_t)i * ustride);
-      const float4 a = __ldcs(U), c = __ldcs(U + 1);
-      acc[0] = fmaf(wg, a.x, acc[0]); acc[1] = fmaf(wg, a.y, acc[1]); acc[2] = fmaf(wg, a.z, acc[2]); acc[3] = fmaf(wg, a.w, acc[3]);
-      acc[4] = fmaf(wg, c.x, acc[4]); acc[5] = fmaf(wg, c.y, acc[5]); acc[6] = fmaf(wg, c.z, acc[6]); acc[7] = fmaf(wg, c.w, acc[7]);
+      slim_comb::fma8(acc, s_w[i], __ldcs(U), __ldcs(U + 1));
     }
-    slim_comb::store_u8(u_tiled, d, H, hp, b, h, j0, acc);
+    if (in_smem) {
+#pragma unroll
+      for (int x = 0; x < 8; ++x) mx = fmaxf(mx, fabsf(acc[x]));
+      float4* t = reinterpret_cast<float4*>(s_row + j0);
+      t[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+      t[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+    } else {
+      slim_comb::store_u8_f32(u32, d, H, b, h, j0, acc);
+    }
   }
+  if (!in_smem) {                                // wide rows: through the float scratch
+    __syncthreads();
+    slim_comb::convert_row(u32, u_tiled, su, d, H, hp, b, h, s_x);
+    return;
+  }
+  mx = slim_comb::block_absmax(mx, s_x);         // (its barriers also order the row stores before the reads below)
+  float inv, scale;
+  slim_comb::row_scale(mx, inv, scale);
+  for (int jg = tid; jg < ngroups; jg += blockDim.x) {       // each thread converts what it wrote itself
+    const float4 a = *reinterpret_cast<const float4*>(s_row + jg * 8), c = *reinterpret_cast<const float4*>(s_row + jg * 8 + 4);
+    const float acc[8] = {a.x, a.y, a.z, a.w, c.x, c.y, c.z, c.w};
+    slim_comb::store_u8_h(u_tiled, d, H, hp, b, h, jg * 8, acc, inv);
+  }
+  if (tid == 0) su[(size_t)b * H + h] = scale;
 }
 
 // The same for small batches, where a sequence has many units and few (head, sequence) pairs exist:
 // grid.z CTAs share the d / 8 column groups of a pair, a CTA takes G of them per pass and spreads the
-// units over UL = 256 / G thread rows, whose sums meet in shared memory.
+// units over UL = 256 / G thread rows, whose sums meet in shared memory.  No CTA sees a whole row here,
+// so the rows are left as floats in u32 and slim_convert_kernel turns them into operand tiles.
 __global__ void __launch_bounds__(256, 4)
-slim_combine_split_kernel(const __grid_constant__ SlimDecodeParams p, unsigned char* __restrict__ u_tiled, const int hp, const int G) {
+slim_combine_split_kernel(const __grid_constant__ SlimDecodeParams p, float* __restrict__ u32, const int G) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* s_w = reinterpret_cast<float*>(smem_raw);                 // [workers]
   int* s_info = reinterpret_cast<int*>(s_w + p.workers);           // wlo, wn, flagged
@@ -150,7 +182,7 @@ slim_combine_split_kernel(const __grid_constant__ SlimDecodeParams p, unsigned c
   const int wlo = s_info[0], wn = s_info[1];
   if (s_info[2]) {                               // a flagged unit: this CTA's column groups are recomputed exactly
     for (int jg0 = blockIdx.z * G; jg0 < d / 8; jg0 += gridDim.z * G)
-      slim_comb::exact_groups(p, u_tiled, hp, b, h, jg0, min(G, d / 8 - jg0), s_red);
+      slim_comb::exact_groups(p, u32, b, h, jg0, min(G, d / 8 - jg0), s_red);
     return;
   }
   const int UL = 256 / G, gi = tid % G, ul = tid / G;
@@ -202,12 +234,23 @@ slim_combine_split_kernel(const __grid_constant__ SlimDecodeParams p, unsigned c
       }
     }
     if (ul != 0 || !live) continue;
-    slim_comb::store_u8(u_tiled, d, H, hp, b, h, j0, acc);
+    slim_comb::store_u8_f32(u32, d, H, b, h, j0, acc);
   }
 }
 
+// operand tiles and row scales from the float rows (one CTA per (head, sequence))
+__global__ void __launch_bounds__(256)
+slim_convert_kernel(const float* __restrict__ u32, unsigned char* __restrict__ u_tiled, float* __restrict__ su, const int d,
+                    const int H, const int hp) {
+  __shared__ float s_red[33];
+  slim_pdl_trigger();
+  slim_pdl_wait();
+  slim_comb::convert_row(u32, u_tiled, su, d, H, hp, blockIdx.y, blockIdx.x, s_red);
+}
+
 __global__ void __launch_bounds__(128)
-slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned char* __restrict__ u_tiled,
+slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const float* __restrict__ hscale, const float* __restrict__ su,
+                    const unsigned char* __restrict__ u_tiled,
                     float* __restrict__ o, const ProjGeom g, const int d, const int d_k, const int batch,
                     int* status, const int32_t* __restrict__ lengths) {
   extern __shared__ unsigned char smem_raw[];
@@ -215,7 +258,8 @@ slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned cha
   const uint32_t base = (raw_u32 + 1023u) & ~1023u;
   unsigned char* sm = smem_raw + (base - raw_u32);
   const uint32_t stage_bytes = (uint32_t)(PJ_W_BYTES + g.u_bytes);
-  const uint32_t bars = base + PJ_NS * stage_bytes;
+  const int NS = g.ns;
+  const uint32_t bars = base + (uint32_t)NS * stage_bytes;
   const uint32_t bar_full = bars, bar_empty = bars + 8 * PJ_NS, bar_done = bars + 16 * PJ_NS;
   unsigned char* misc = sm + (bar_done + 8 - base);
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc);
@@ -226,7 +270,8 @@ slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned cha
   const uint32_t tmem_cols = (uint32_t)(32 * g.hp);
 
   if (tid == 0) {
-    for (int i = 0; i < PJ_NS; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
+    prefetch_tensormap(&wmap);
+    for (int i = 0; i < NS; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
     mbar_init(bar_done, 1);
     *s_abort = 0;
     fence_mbar_init();
@@ -241,13 +286,16 @@ slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned cha
   // The weights do not depend on the kernels before this one: the producer starts the W_KV tiles
   // of the first stages before the dependency wait, so they stream in while the combine kernel
   // still runs; the u tiles of those stages follow after the wait (same barrier, one byte count).
-  const int npre = g.nst < PJ_NS ? g.nst : PJ_NS;
+  const int npre = g.nst < NS ? g.nst : NS;
+  // the weight tile of stage s (rows row0 + s * PJ_ROWS ..) into the stage at dst
+  auto load_w = [&](uint32_t dst, uint32_t bar, int s) {
+    if (g.hp == 1) tma_load_3d(dst, &wmap, bar, 0, hg * d + row0 + s * PJ_ROWS, 0);
+    else           tma_load_3d(dst, &wmap, bar, 0, row0 + s * PJ_ROWS, 2 * hg);
+  };
   if (warp == 0 && lane == 0) {
     for (int s = 0; s < npre; ++s) {
-      const uint32_t dst = base + (uint32_t)s * stage_bytes;
       mbar_arrive_expect_tx(bar_full + 8 * s, stage_bytes);
-      if (g.hp == 1) tma_load_3d(dst, &wmap, bar_full + 8 * s, 0, hg * d + row0 + s * PJ_ROWS, 0);
-      else           tma_load_3d(dst, &wmap, bar_full + 8 * s, 0, row0 + s * PJ_ROWS, 2 * hg);
+      load_w(base + (uint32_t)s * stage_bytes, bar_full + 8 * s, s);
     }
   }
   slim_pdl_wait();                                             // u tiles come from the combine kernel
@@ -260,31 +308,30 @@ slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned cha
     for (; s < npre; ++s)
       bulk_load(base + (uint32_t)s * stage_bytes + PJ_W_BYTES, usrc + (size_t)s * g.u_bytes, (uint32_t)g.u_bytes, bar_full + 8 * s);
     for (; s < g.nst; ++s) {
-      const int st = s % PJ_NS;
-      ok = mbar_wait<false>(bar_empty + 8 * st, ((s / PJ_NS) & 1) ^ 1, s_abort, status);
+      const int st = s % NS;
+      ok = mbar_wait<false>(bar_empty + 8 * st, ((s / NS) & 1) ^ 1, s_abort, status);
       if (!ok) break;
       const uint32_t dst = base + (uint32_t)st * stage_bytes;
       mbar_arrive_expect_tx(bar_full + 8 * st, stage_bytes);
-      if (g.hp == 1) tma_load_3d(dst, &wmap, bar_full + 8 * st, 0, hg * d + row0 + s * PJ_ROWS, 0);
-      else           tma_load_3d(dst, &wmap, bar_full + 8 * st, 0, row0 + s * PJ_ROWS, 2 * hg);
+      load_w(dst, bar_full + 8 * st, s);
       bulk_load(dst + PJ_W_BYTES, usrc + (size_t)s * g.u_bytes, (uint32_t)g.u_bytes, bar_full + 8 * st);
     }
     if (!ok) {
       // gave up: let the copies that were issued land before the CTA goes away
-      const int issued = s < PJ_NS ? s : PJ_NS;
+      const int issued = s < NS ? s : NS;
       for (int k = 0; k < issued; ++k) {
-        const int j = s - 1 - k, st = j % PJ_NS;
+        const int j = s - 1 - k, st = j % NS;
         const unsigned long long t0 = globaltimer();
-        while (!mbar_try_wait(bar_full + 8 * st, (j / PJ_NS) & 1) && globaltimer() - t0 < SLIM_WAIT_NS) {}
+        while (!mbar_try_wait(bar_full + 8 * st, (j / NS) & 1) && globaltimer() - t0 < SLIM_WAIT_NS) {}
       }
     }
   } else if (warp == 1 && lane == 0) {
     // =========================== MMA issuer ===========================
-    const uint32_t idesc = umma_idesc((uint32_t)(32 * g.hp));
+    const uint32_t idesc = umma_idesc_f16((uint32_t)(32 * g.hp));      // both operands float16
     bool ok = true;
     for (int s = 0; s < g.nst && ok; ++s) {
-      const int st = s % PJ_NS;
-      ok = mbar_wait<false>(bar_full + 8 * st, (s / PJ_NS) & 1, s_abort, status);
+      const int st = s % NS;
+      ok = mbar_wait<false>(bar_full + 8 * st, (s / NS) & 1, s_abort, status);
       if (!ok) break;
       tc_fence_after();
       const uint32_t wbase = base + (uint32_t)st * stage_bytes, ubase = wbase + PJ_W_BYTES;
@@ -305,6 +352,17 @@ slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned cha
   const int upper = g.hp == 2 ? (warp >> 1) : 0;              // d_k = 64: lanes 64..127 hold the second head
   const int head = hg * g.hp + upper;
   const int c = g.hp == 2 ? (m & 63) : m;
+  // the scales taken out of the operands, fetched while the MMAs run: 2^e of the rows u[b][head][:] and 2^-a of
+  // the head's weights
+  float sc[PJ_BG];
+  {
+    const float hs = hscale[head];
+#pragma unroll
+    for (int n = 0; n < PJ_BG; ++n) {
+      const int b = bg * PJ_BG + n;
+      sc[n] = b < batch ? __ldg(su + (size_t)b * (g.hg * g.hp) + head) * hs : 0.f;
+    }
+  }
   {
     bool ok = mbar_wait<false>(bar_done, 0, s_abort, status);
     ok = __all_sync(0xffffffffu, ok);
@@ -315,9 +373,10 @@ slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned cha
       tc_fence_after();
       tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(32 * upper), r);
     }
+    // (hi + lo) columns of a sequence, times the scales
     float* tile = reinterpret_cast<float*>(sm);
 #pragma unroll
-    for (int n = 0; n < PJ_BG; ++n) tile[n * 128 + m] = __uint_as_float(r[n]) + __uint_as_float(r[PJ_BG + n]);
+    for (int n = 0; n < PJ_BG; ++n) tile[n * 128 + m] = (__uint_as_float(r[n]) + __uint_as_float(r[PJ_BG + n])) * sc[n];
   }
   cluster_sync_all();
   {
@@ -339,7 +398,7 @@ slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const unsigned cha
   }
 }
 
-ProjGeom make_proj_geom(int d, int H, int d_k, int batch) {
+ProjGeom make_proj_geom(int d, int H, int d_k, int batch, int ns_opt = 0) {
   ProjGeom g;
   g.hp = d_k == 64 ? 2 : 1;
   g.hg = H / g.hp;
@@ -351,10 +410,12 @@ ProjGeom make_proj_geom(int d, int H, int d_k, int batch) {
   g.nst = stages / js;
   g.nbg = (batch + PJ_BG - 1) / PJ_BG;
   g.u_bytes = (PJ_ROWS / 16) * 1024 * g.hp;
+  g.ns = PJ_NS;
+  if (ns_opt >= 2 && ns_opt <= PJ_NS) g.ns = ns_opt;          // sweeps
   return g;
 }
 
-size_t proj_smem_bytes(const ProjGeom& g) { return 1024 + (size_t)PJ_NS * (PJ_W_BYTES + g.u_bytes) + 16 * PJ_NS + 8 + 16 + 64; }
+size_t proj_smem_bytes(const ProjGeom& g) { return 1024 + (size_t)g.ns * (PJ_W_BYTES + g.u_bytes) + 16 * PJ_NS + 8 + 16 + 64; }
 
 }  // namespace
 
@@ -384,38 +445,57 @@ cudaError_t slim_proj_make_wmap(slim_ctx* ctx) {
     dims[0] = 64; dims[1] = d; dims[2] = H;
     strides[0] = 128; strides[1] = (unsigned long long)d * 128;
   }
+  // (the float16 copy is described as a 16-bit type of the same size: the copy engine only moves bits)
   cudaError_t e = slim_tmap_encode_3d(ctx->wmap, ctx->wkv, dims, strides, box);
+  if (e == cudaSuccess) e = slim_tmap_encode_3d(ctx->wmap_h, ctx->wkv_h, dims, strides, box);
   if (e != cudaSuccess) return e;
-  const ProjGeom g = make_proj_geom(d, H, d_k, 1);
+  const ProjGeom g = make_proj_geom(d, H, d_k, 1, PJ_NS);      // the largest stage count a sweep may ask for
   return cudaFuncSetAttribute((const void*)slim_proj_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)proj_smem_bytes(g));
 }
 
-cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, unsigned char* u_tiled, float* o_part,
+// Small batches (fewer than two (head, sequence) pairs per SM): the combine is split over column slices
+// (grid.z) so that ~2 CTAs per SM exist; returns the slice count (1 = the one-CTA-per-row kernel).
+static int combine_slices(const slim_ctx* ctx, int H, int batch, int d) {
+  const int ngroups = d / 8;
+  int nslice = 1;
+  while (nslice < 16 && (long long)H * batch * nslice < 2 * ctx->num_sms && ngroups / (2 * nslice) >= 32) nslice <<= 1;
+  return nslice;
+}
+
+int slim_proj_needs_convert(const slim_ctx* ctx, int batch) { return combine_slices(ctx, ctx->H, batch, ctx->d) > 1 ? 1 : 0; }
+
+cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, unsigned char* u_tiled, float* u32, float* su,
                              cudaStream_t st) {
-  const ProjGeom g = make_proj_geom(p.d, p.H, p.d_k, p.batch);
+  const ProjGeom g = make_proj_geom(p.d, p.H, p.d_k, p.batch, ctx->opt_proj_ns);
   {
-    // Small batches: no CTAs for the padding sequences of a 16-sequence group (their columns of the
-    // projection's B operand stay unwritten and only feed outputs that are never stored), and slices
-    // of the columns across grid.z so that ~2 CTAs per SM exist.
+    // No CTAs for the padding sequences of a 16-sequence group in the split variant (their columns of the
+    // projection's B operand stay unwritten and only feed outputs that are never stored).
     const int ngroups = p.d / 8;
-    int nslice = 1;
-    while (nslice < 16 && (long long)p.H * p.batch * nslice < 2 * ctx->num_sms && ngroups / (2 * nslice) >= 32) nslice <<= 1;
+    const int nslice = combine_slices(ctx, p.H, p.batch, p.d);
     cudaError_t e;
     if (nslice > 1) {
       int G = 256;
       while (G > 32 && G / 2 * nslice >= ngroups) G >>= 1;
       const size_t smem = sizeof(float) * p.workers + sizeof(int) * (4 + p.batch + 1) + 16 + sizeof(float) * 7 * 256;
-      e = slim_launch_pdl(slim_combine_split_kernel, dim3(p.H, p.batch, nslice), dim3(256), smem, st, p, u_tiled, g.hp, G);
+      e = slim_launch_pdl(slim_combine_split_kernel, dim3(p.H, p.batch, nslice), dim3(256), smem, st, p, u32, G);
+      if (e == cudaSuccess)
+        e = slim_launch_pdl(slim_convert_kernel, dim3(p.H, p.batch), dim3(256), 0, st, (const float*)u32, u_tiled, su, p.d, p.H, g.hp);
     } else {
       dim3 grid(p.H, g.nbg * PJ_BG);
-      const size_t smem = sizeof(float) * p.workers + sizeof(int) * (4 + p.batch + 1) + 16 + sizeof(float) * (p.d_k + 2 * SLIM_TT + 4);
-      e = slim_launch_pdl(slim_combine_kernel, grid, dim3(256), smem, st, p, u_tiled, g.hp);
+      // weights, info, prefix | exact path / reduction scratch | the float row
+      const size_t smem = sizeof(float) * p.workers + sizeof(int) * (4 + p.batch + 1) + 16 + sizeof(float) * (p.d_k + 2 * SLIM_TT + 4 + 36) +
+                          sizeof(float) * (p.d <= COMBINE_SMEM_ROW ? p.d : 0) + 16;
+      if (smem > 48 * 1024) {
+        e = cudaFuncSetAttribute((const void*)slim_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+      }
+      e = slim_launch_pdl(slim_combine_kernel, grid, dim3(256), smem, st, p, u_tiled, u32, su, g.hp);
     }
     if (e != cudaSuccess) return e;
   }
   CUtensorMap map;
-  memcpy(&map, ctx->wmap, sizeof(map));
+  memcpy(&map, ctx->wmap_h, sizeof(map));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(g.hg, g.jsplit, g.nbg);
   cfg.blockDim = dim3(128);
@@ -427,6 +507,6 @@ cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, uns
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, slim_proj_tc_kernel, map, (const unsigned char*)u_tiled, p.o, g, p.d, p.d_k, p.batch, p.status,
-                            p.lengths);
+  return cudaLaunchKernelEx(&cfg, slim_proj_tc_kernel, map, (const float*)ctx->wkv_hscale, (const float*)su, (const unsigned char*)u_tiled,
+                            p.o, g, p.d, p.d_k, p.batch, p.status, p.lengths);
 }

@@ -161,6 +161,11 @@ __host__ __device__ constexpr uint32_t umma_idesc(uint32_t n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
+// The same for float16 operands (A and B of one instruction always share their type).
+__host__ __device__ constexpr uint32_t umma_idesc_f16(uint32_t n) {
+  return (1u << 4) | (1u << 15) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
 // K-major operand, 128-byte swizzle, as TMA delivers a [rows][64 elements] tile: 8-row groups
 // 1024 B apart; the 16-element k-step is selected by the start address (+32 B per step).
 __device__ __forceinline__ uint64_t desc_kmajor_sw128(uint32_t addr) {

@@ -5,6 +5,8 @@
 // side may have any number of columns m (M is n x (n + m)): the non-square case
 // (section "Support for non-square weight matrices", Option 1) solves
 // (W_K W_K^T) Y = W_V with n = d_model and m = e.
+#include <cuda_fp16.h>
+
 #include "slim_internal.h"
 
 namespace {
@@ -293,14 +295,49 @@ __global__ void __launch_bounds__(256) residual_kernel(const double* __restrict_
 }
 
 template <typename WT>
-__global__ void store_wkv_kernel(const double* __restrict__ X, WT* __restrict__ dst, int d, int H, int dk) {
+__global__ void store_wkv_kernel(const double* __restrict__ X, WT* __restrict__ dst, __half* __restrict__ dst_h,
+                                 const float* __restrict__ hscale, int d, int H, int dk) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= (size_t)d * d) return;
   const int c = (int)(i % dk);
   const size_t rest = i / dk;
   const int j = (int)(rest % d), h = (int)(rest / d);
   const double v = X[(size_t)j * d + h * dk + c];
-  if constexpr (sizeof(WT) == 2) dst[i] = __double2bfloat16(v); else dst[i] = (float)v;
+  if constexpr (sizeof(WT) == 2) {
+    dst[i] = __double2bfloat16(v);
+    if (dst_h) dst_h[i] = __double2half(v / (double)hscale[h]);      // power-of-two scale: exact
+  } else {
+    dst[i] = (float)v;
+  }
+}
+
+// hscale[h] = 2^-a with max |W_KV,h| * 2^a in [2^14, 2^15) (1 for an all-zero head): one CTA per head
+__global__ void head_scale_kernel(const double* __restrict__ X, float* __restrict__ hscale, int d, int dk) {
+  __shared__ double s_max[256];
+  const int h = blockIdx.x;
+  double m = 0.0;
+  for (size_t i = threadIdx.x; i < (size_t)d * dk; i += blockDim.x) {
+    const double v = fabs(X[(i / dk) * d + (size_t)h * dk + i % dk]);
+    m = v > m ? v : m;
+  }
+  s_max[threadIdx.x] = m;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) s_max[threadIdx.x] = fmax(s_max[threadIdx.x], s_max[threadIdx.x + o]);
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    float sc = 1.f;
+    const double mx = s_max[0];
+    if (mx > 0.0 && mx < 1e300) {
+      int x;
+      frexp(mx, &x);                                   // mx = m 2^x, 0.5 <= m < 1  =>  mx 2^(15 - x) in [2^14, 2^15)
+      int a = 15 - x;
+      a = a < -100 ? -100 : (a > 100 ? 100 : a);
+      sc = exp2f((float)-a);
+    }
+    hscale[h] = sc;
+  }
 }
 
 #define CK(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) { cudaFree(M); cudaFree(piv); cudaFree(scal); return e_; } } while (0)
@@ -364,12 +401,14 @@ cudaError_t slim_wkv_residual(const double* Wk, const double* X, const double* W
   return e;
 }
 
-cudaError_t slim_wkv_store(const double* X, int d, int H, int d_k, int dtype, void* dst) {
+cudaError_t slim_wkv_store(const double* X, int d, int H, int d_k, int dtype, void* dst, void* dst_h, float* hscale) {
   const size_t nn = (size_t)d * d;
-  if (dtype == SLIM_BF16)
-    store_wkv_kernel<__nv_bfloat16><<<(unsigned)((nn + 255) / 256), 256>>>(X, (__nv_bfloat16*)dst, d, H, d_k);
-  else
-    store_wkv_kernel<float><<<(unsigned)((nn + 255) / 256), 256>>>(X, (float*)dst, d, H, d_k);
+  if (dtype == SLIM_BF16) {
+    if (dst_h) head_scale_kernel<<<H, 256>>>(X, hscale, d, d_k);
+    store_wkv_kernel<__nv_bfloat16><<<(unsigned)((nn + 255) / 256), 256>>>(X, (__nv_bfloat16*)dst, (__half*)dst_h, hscale, d, H, d_k);
+  } else {
+    store_wkv_kernel<float><<<(unsigned)((nn + 255) / 256), 256>>>(X, (float*)dst, nullptr, nullptr, d, H, d_k);
+  }
   return cudaGetLastError();
 }
 
