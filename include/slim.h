@@ -223,15 +223,25 @@ slim_status slim_decode_static_ws(slim_ctx* ctx, const void* q, const slim_cache
  * inputs X (or the encoder output E, which all decoder layers may share: wrap the same
  * storage with slim_cache_create for every layer's ctx) instead of keys.  Per head
  *   A_i = ((x_n W_Q,i + b) W_K,i^T) X^T,   head_i = [softmax(A_i / sqrt(d_k)) X] W_V,i.
- * No RoPE (the ctx must have rope_theta = 0); square projections (d = H*d_k) only.
- *   slim_xcache_set_weights   W_K, W_V host row-major [d][d]; W_K is kept in float32 for the
+ * No RoPE (the ctx must have rope_theta = 0).  Projections need not be square here: with
+ * slim_xcache_create the model width d (cache rows, the inner index of W_K and W_V) and the
+ * projection width e = H*d_k (queries, outputs) are independent, W_K, W_V in R^{d x e}
+ * (section "Support for non-square weight matrices", Option 2: e > d as in T5-style models, or
+ * e < d).  A context from slim_create (d = e) works as well.
+ *   slim_xcache_create        d_model = width of a cache row; H <= 64, even d_k <= 256,
+ *                             d_model, H*d_k <= 16384; SLIM_F32 or SLIM_BF16.  Such a context
+ *                             serves the slim_xcache_* calls and slim_cache_create only (the K-cache
+ *                             calls return SLIM_ERR_UNSUPPORTED unless d_model = H*d_k)
+ *   slim_xcache_set_weights   W_K, W_V host row-major [d][e]; W_K is kept in float32 for the
  *                             per-token query transform, W_V replaces W_KV in the projection
- *   slim_xcache_decode        as slim_decode: q = x_n W_Q (+ bias) [batch][d], `cache` holds
- *                             X rows; workspace >= slim_xcache_workspace_bytes
+ *   slim_xcache_decode        as slim_decode: q = x_n W_Q (+ bias) [batch][e], `cache` holds
+ *                             X rows [batch][t_cap][d], o is [batch][e];
+ *                             workspace >= slim_xcache_workspace_bytes
  * bf16 caches with d % 64 == 0 and H <= 32 run on the tensor cores (dense scores: cache rows
  * as a K-major TMA operand against bf16 hi/lo query tiles; weighted sum and projection: the
  * kernels of slim_decode); other shapes use the CUDA-core kernels.  The cache is read twice
  * per layer (scores, then the weighted sum).                                            */
+slim_status slim_xcache_create(slim_ctx** out, int d_model, int H, int d_k, int dtype);
 slim_status slim_xcache_set_weights(slim_ctx* ctx, const void* W_K, const void* W_V, int host_dtype);
 size_t      slim_xcache_workspace_bytes(const slim_ctx* ctx, int batch, int t_cap);
 slim_status slim_xcache_decode(slim_ctx* ctx, const void* q, const slim_cache* cache, const int32_t* lengths,

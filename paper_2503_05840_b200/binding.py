@@ -39,6 +39,7 @@ SIGNATURES = {
     "slim_decode_step": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
     "slim_static_workspace_max": (c_size_t, []),
     "slim_decode_static_ws": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "slim_xcache_create": (c_int, [POINTER(c_void_p), c_int, c_int, c_int, c_int]),
     "slim_xcache_set_weights": (c_int, [c_void_p, c_void_p, c_void_p, c_int]),
     "slim_xcache_workspace_bytes": (c_size_t, [c_void_p, c_int, c_int]),
     "slim_xcache_decode": (c_int, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -209,6 +210,13 @@ def slim_decode_static_ws(ctx: int, q, cache: int, lengths, o, stream: int = 0) 
     """slim_decode with the library's built-in scratch: for callers that must not allocate."""
     _check(lib().slim_decode_static_ws(c_void_p(ctx), _ptr(q), c_void_p(cache), _ptr(lengths), _ptr(o),
                                        c_void_p(stream)), "slim_decode_static_ws")
+
+
+def slim_xcache_create(d_model: int, H: int, d_k: int, dtype: int) -> int:
+    """X-cache context whose cache rows are d_model wide while queries and outputs are H*d_k wide."""
+    h = c_void_p()
+    _check(lib().slim_xcache_create(byref(h), d_model, H, d_k, dtype), "slim_xcache_create")
+    return h.value
 
 
 def slim_xcache_set_weights(ctx: int, W_K, W_V) -> None:

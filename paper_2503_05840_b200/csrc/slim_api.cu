@@ -9,7 +9,7 @@
 
 #include "slim_internal.h"
 
-size_t slim_tail_opart_floats(int d, int batch);
+size_t slim_tail_opart_floats(int d, int e, int batch);
 
 // Built-in scratch for slim_decode_static_ws: device memory that exists from the moment
 // the library is loaded on a GPU until the process exits, so that entry point never has
@@ -36,7 +36,7 @@ WsLayout ws_layout(const slim_ctx* ctx, int batch, int t_cap) {
   L.part_m = off; off = align256(off + sizeof(float) * (size_t)L.units * ctx->H);
   L.part_l = off; off = align256(off + sizeof(float) * (size_t)L.units * ctx->H);
   L.flags = off;  off = align256(off + sizeof(int) * 2 * (size_t)L.units);
-  L.o_part = off; off = align256(off + sizeof(float) * slim_tail_opart_floats(ctx->d, batch));
+  L.o_part = off; off = align256(off + sizeof(float) * slim_tail_opart_floats(ctx->d, ctx->e, batch));
   L.scores = off; off = align256(off + sizeof(float) * (size_t)batch * ctx->H * t_cap);   // generic path only
   L.u_tiled = off; off = align256(off + (ctx->proj_ok ? slim_proj_u_bytes(ctx->d, ctx->H, batch) : 0));   // tensor-core tail only
   L.u32 = off; off = align256(off + (ctx->proj_ok ? sizeof(float) * (size_t)batch * ctx->H * ctx->d : 0));
@@ -145,15 +145,32 @@ const char* slim_strerror(int status) {
   }
 }
 
+namespace {
+// d: width of a cache row.  For the K-cache scheme d == H * d_k (square projections); an X-cache
+// context may have d != e = H * d_k (xcache_only).
+slim_status create_impl(slim_ctx** out, int d, int H, int d_k, double rope_theta, int dtype, bool xcache_only);
+}
+
 slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta, int dtype) {
+  return create_impl(out, d, H, d_k, rope_theta, dtype, false);
+}
+
+slim_status slim_xcache_create(slim_ctx** out, int d_model, int H, int d_k, int dtype) {
+  return create_impl(out, d_model, H, d_k, 0.0, dtype, true);
+}
+
+namespace {
+slim_status create_impl(slim_ctx** out, int d, int H, int d_k, double rope_theta, int dtype, bool xcache_only) {
   if (!out) return SLIM_ERR_INVALID_ARG;
   *out = nullptr;
   if (d <= 0 || H <= 0 || d_k <= 0 || !(rope_theta >= 0.0) || (dtype != SLIM_F32 && dtype != SLIM_BF16 && dtype != SLIM_FP8))
     return SLIM_ERR_INVALID_ARG;
   const int kdtype = dtype;
   if (dtype == SLIM_FP8) dtype = SLIM_BF16;            // 8-bit cache; queries, new rows and W_KV are bf16
-  if ((long long)H * d_k != d) return SLIM_ERR_UNSUPPORTED;       // Eq. 6 needs a square W_K
-  if (H > SLIM_MAX_H || d_k > 256 || (d_k % 2) != 0 || d > 16384) return SLIM_ERR_UNSUPPORTED;      // rotation pairs need an even width
+  if ((long long)H * d_k != d && !xcache_only) return SLIM_ERR_UNSUPPORTED;       // Eq. 6 needs a square W_K
+  if (xcache_only && dtype == SLIM_FP8) return SLIM_ERR_UNSUPPORTED;
+  if (H > SLIM_MAX_H || d_k > 256 || (d_k % 2) != 0 || d > 16384 || (long long)H * d_k > 16384) return SLIM_ERR_UNSUPPORTED;      // rotation pairs need an even width
+  const int e = H * d_k;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return SLIM_ERR_CUDA;
   cudaDeviceProp prop;
@@ -161,7 +178,7 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
   slim_ctx* c = new (std::nothrow) slim_ctx();
   if (!c) return SLIM_ERR_OOM;
   std::memset(c, 0, sizeof(*c));
-  c->d = d; c->H = H; c->d_k = d_k; c->dtype = dtype; c->kdtype = kdtype; c->rope_theta = rope_theta;
+  c->d = d; c->e = e; c->H = H; c->d_k = d_k; c->dtype = dtype; c->kdtype = kdtype; c->rope_theta = rope_theta;
   c->device = dev; c->num_sms = prop.multiProcessorCount;
   c->path_req = SLIM_PATH_AUTO;
   {
@@ -180,10 +197,10 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
   cudaMemset(c->status, 0, sizeof(int));
   if (cudaMalloc(&c->any_flag, sizeof(int)) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
   cudaMemset(c->any_flag, 0, sizeof(int));
-  if (cudaMalloc(&c->wkv, esize(dtype) * (size_t)d * d + 256) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
+  if (cudaMalloc(&c->wkv, esize(dtype) * (size_t)d * e + 256) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
   if (dtype == SLIM_BF16) {
-    if (cudaMalloc(&c->wkv_h, 2 * (size_t)d * d + 256) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
-    cudaMemset(c->wkv_h, 0, 2 * (size_t)d * d + 256);
+    if (cudaMalloc(&c->wkv_h, 2 * (size_t)d * e + 256) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
+    cudaMemset(c->wkv_h, 0, 2 * (size_t)d * e + 256);
     if (cudaMalloc(&c->wkv_hscale, sizeof(float) * SLIM_MAX_H) != cudaSuccess) { slim_destroy(c); return SLIM_ERR_OOM; }
     cudaMemset(c->wkv_hscale, 0, sizeof(float) * SLIM_MAX_H);
   }
@@ -201,7 +218,7 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
       return SLIM_ERR_CUDA;
     }
   }
-  cudaMemset(c->wkv, 0, esize(dtype) * (size_t)d * d + 256);
+  cudaMemset(c->wkv, 0, esize(dtype) * (size_t)d * e + 256);
   c->proj_ok = prop.major == 10 ? slim_proj_shape_ok(d, H, d_k, dtype) : 0;
   if (c->proj_ok && slim_proj_make_wmap(c) != cudaSuccess) { cudaGetLastError(); c->proj_ok = 0; }
   {
@@ -218,6 +235,7 @@ slim_status slim_create(slim_ctx** out, int d, int H, int d_k, double rope_theta
   *out = c;
   return SLIM_OK;
 }
+}  // namespace
 
 void slim_destroy(slim_ctx* ctx) {
   if (!ctx) return;
@@ -238,6 +256,7 @@ slim_status slim_set_weights(slim_ctx* ctx, const void* W_K, const void* W_V, in
                              double* wkv_out, double* residual_out) {
   if (!ctx || !W_K || !W_V || (host_dtype != SLIM_HOST_F32 && host_dtype != SLIM_HOST_F64))
     return SLIM_ERR_INVALID_ARG;
+  if (ctx->e != ctx->d) return SLIM_ERR_UNSUPPORTED;              // an X-cache context with non-square projections
   const int n = ctx->d;
   const size_t nn = (size_t)n * n;
   double *A = nullptr, *B = nullptr, *A0 = nullptr, *B0 = nullptr;
@@ -278,6 +297,7 @@ slim_status slim_set_weights(slim_ctx* ctx, const void* W_K, const void* W_V, in
 slim_status slim_set_weights_nonsquare(slim_ctx* ctx, const void* W_K, const void* W_V, int d_model, int host_dtype,
                                        double* wkv_out, double* residual_out) {
   if (!ctx || !W_K || !W_V || (host_dtype != SLIM_HOST_F32 && host_dtype != SLIM_HOST_F64)) return SLIM_ERR_INVALID_ARG;
+  if (ctx->e != ctx->d) return SLIM_ERR_UNSUPPORTED;
   const int e = ctx->d;                                  // width of K and V: e = H d_k
   if (d_model <= 0 || d_model > e) return SLIM_ERR_INVALID_ARG;
   const size_t de = (size_t)d_model * e, ee = (size_t)e * e, dd = (size_t)d_model * d_model;
@@ -319,7 +339,7 @@ slim_status slim_xcache_set_weights(slim_ctx* ctx, const void* W_K, const void* 
   if (!ctx || !W_K || !W_V || (host_dtype != SLIM_HOST_F32 && host_dtype != SLIM_HOST_F64)) return SLIM_ERR_INVALID_ARG;
   if (ctx->rope_theta != 0.0) return SLIM_ERR_UNSUPPORTED;          // the scheme has no place for RoPE
   if (ctx->kdtype == SLIM_FP8) return SLIM_ERR_UNSUPPORTED;
-  const size_t nn = (size_t)ctx->d * ctx->d;
+  const size_t nn = (size_t)ctx->d * ctx->e;              // W_K, W_V: [d][e]
   std::vector<float> wk(nn);
   if (host_dtype == SLIM_HOST_F64) { const double* s = static_cast<const double*>(W_K); for (size_t i = 0; i < nn; ++i) wk[i] = (float)s[i]; }
   else std::memcpy(wk.data(), W_K, sizeof(float) * nn);
@@ -336,7 +356,7 @@ size_t slim_xcache_workspace_bytes(const slim_ctx* ctx, int batch, int t_cap) {
 slim_status slim_set_wkv(slim_ctx* ctx, const void* W_KV, int host_dtype) {
   if (!ctx || !W_KV || (host_dtype != SLIM_HOST_F32 && host_dtype != SLIM_HOST_F64)) return SLIM_ERR_INVALID_ARG;
   double* X = nullptr;
-  slim_status st = upload_f64(W_KV, host_dtype, (size_t)ctx->d * ctx->d, &X);
+  slim_status st = upload_f64(W_KV, host_dtype, (size_t)ctx->d * ctx->e, &X);
   if (st != SLIM_OK) return st;
   if (slim_wkv_store(X, ctx->d, ctx->H, ctx->d_k, ctx->dtype, ctx->wkv, ctx->wkv_h, ctx->wkv_hscale) != cudaSuccess ||
       cudaDeviceSynchronize() != cudaSuccess)
@@ -448,6 +468,7 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   if (!ctx->has_weights) return SLIM_ERR_NO_WEIGHTS;
   int path = path_in_use(ctx);
   if (xcache && !ctx->xc_wk) return SLIM_ERR_NO_WEIGHTS;
+  if (!xcache && ctx->e != ctx->d) return SLIM_ERR_UNSUPPORTED;   // the K-cache scheme needs square projections
   if (xcache && cache->block_table) return SLIM_ERR_UNSUPPORTED;
   if (path < 0) return SLIM_ERR_UNSUPPORTED;
   // CTAs per worker: the pair when the kernel computes the scores, the lone CTA with external scores
@@ -464,7 +485,7 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   const WsLayout L = ws_layout(ctx, cache->batch, cache->t_cap);
   char* ws = static_cast<char*>(workspace);
   SlimDecodeParams p;
-  p.d = ctx->d; p.H = ctx->H; p.d_k = ctx->d_k; p.half = ctx->d_k / 2;
+  p.d = ctx->d; p.e = ctx->e; p.H = ctx->H; p.d_k = ctx->d_k; p.half = ctx->d_k / 2;
   p.batch = cache->batch; p.t_cap = cache->t_cap;
   p.rope = ctx->rope_theta != 0.0; p.dtype = ctx->dtype; p.kdtype = ctx->kdtype; p.k_exp = cache->k_exp;
   p.workers = path == SLIM_PATH_TC ? ctx->tc_workers[cl - 1] : ctx->gen_workers;
@@ -590,7 +611,7 @@ slim_status slim_combine_project(slim_ctx* ctx, const float* lse_all, const floa
   char* ws = static_cast<char*>(workspace);
   SlimDecodeParams p;
   std::memset(&p, 0, sizeof(p));
-  p.d = ctx->d; p.H = ctx->H; p.d_k = ctx->d_k; p.half = ctx->d_k / 2;
+  p.d = ctx->d; p.e = ctx->e; p.H = ctx->H; p.d_k = ctx->d_k; p.half = ctx->d_k / 2;
   p.batch = batch; p.t_cap = 0x3fffffff;
   p.dtype = ctx->dtype; p.kdtype = ctx->kdtype;
   p.workers = 1; p.cl = 0; p.min_tiles = 1; p.unit_cost = 0;
@@ -620,6 +641,7 @@ slim_status slim_xcache_decode(slim_ctx* ctx, const void* q, const slim_cache* c
 
 slim_status slim_values_from_keys(slim_ctx* ctx, const void* K, int n, float* V, void* stream) {
   if (!ctx || !K || !V || n <= 0) return SLIM_ERR_INVALID_ARG;
+  if (ctx->e != ctx->d) return SLIM_ERR_UNSUPPORTED;
   if (!ctx->has_weights) return SLIM_ERR_NO_WEIGHTS;
   if (slim_launch_values(ctx, K, n, V, (cudaStream_t)stream) != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
   return SLIM_OK;
@@ -630,7 +652,7 @@ slim_status slim_prefill(slim_ctx* ctx, slim_cache* cache, const void* k_new, co
   if (!ctx || !cache || !k_new || !positions || !V || cache->ctx != ctx) return SLIM_ERR_INVALID_ARG;
   if (n_new <= 0 || n_new > 65535) return SLIM_ERR_INVALID_ARG;
   if (n_new > cache->t_cap) return SLIM_ERR_CAPACITY;
-  if ((long long)cache->batch * n_new > 0x7fffffffLL) return SLIM_ERR_UNSUPPORTED;
+  if ((long long)cache->batch * n_new > 0x7fffffffLL || ctx->e != ctx->d) return SLIM_ERR_UNSUPPORTED;
   if (!ctx->has_weights) return SLIM_ERR_NO_WEIGHTS;
   if (slim_launch_values(ctx, k_new, cache->batch * n_new, V, (cudaStream_t)stream, cache, positions, n_new) != cudaSuccess) {
     cudaGetLastError();

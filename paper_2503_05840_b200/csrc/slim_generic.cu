@@ -460,11 +460,11 @@ slim_xq_kernel(SlimDecodeParams p, const float* __restrict__ W_K, float* __restr
   float* s_q = reinterpret_cast<float*>(smem_raw);                   // [d_k]
   const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int d = p.d, dk = p.d_k;
-  const KT* Q = reinterpret_cast<const KT*>(p.q) + (size_t)b * d + h * dk;
+  const KT* Q = reinterpret_cast<const KT*>(p.q) + (size_t)b * p.e + h * dk;
   for (int c = tid; c < dk; c += GEN_THREADS) s_q[c] = ld_k(Q + c) * p.qscale;
   __syncthreads();
   for (int j = wid; j < d; j += GEN_THREADS / 32) {
-    const float* w = W_K + (size_t)j * d + h * dk;
+    const float* w = W_K + (size_t)j * p.e + h * dk;
     float a = 0.f;
     for (int c = lane; c < dk; c += 32) a = fmaf(s_q[c], __ldg(w + c), a);
 #pragma unroll

@@ -17,7 +17,8 @@
 
 // Parameters every decode kernel receives (passed by value).
 struct SlimDecodeParams {
-  int d, H, d_k, half;           // half = d_k / 2
+  int d, H, d_k, half;           // d: width of a cache row (and of u); half = d_k / 2
+  int e;                         // width of q and o: H * d_k (= d except for a non-square X-cache)
   int batch, t_cap;
   int rope;                      // 0 / 1
   int dtype;                     // slim_dtype of q and W_KV (f32 or bf16)
@@ -56,7 +57,8 @@ struct SlimDecodeParams {
 };
 
 struct slim_ctx {
-  int d, H, d_k, dtype;          // dtype: q and W_KV (f32 or bf16)
+  int d, H, d_k, dtype;          // d: width of a cache row; dtype: q and W_KV (f32 or bf16)
+  int e;                         // width of q and o: H * d_k; differs from d only for an X-cache context with non-square projections
   int kdtype;                    // cache elements: dtype, or SLIM_FP8
   double rope_theta;
   int device;
@@ -130,6 +132,7 @@ cudaError_t slim_wkv_solve_rhs(double* A, double* B, int n, int m, int* info_hos
 cudaError_t slim_dgemm(const double* A, const double* B, double* C, int M, int N, int K, int ta, int tb);
 cudaError_t slim_absdiff_max(const double* A, const double* B, size_t n, double* res_host);
 cudaError_t slim_wkv_residual(const double* Wk, const double* X, const double* Wv, int n, double* res_host);
+// X: [d][H * d_k] row-major (d rows: the contraction index of the projection)
 cudaError_t slim_wkv_store(const double* X, int d, int H, int d_k, int dtype, void* dst, void* dst_h, float* hscale);
 
 // tensor-core path (slim_tc.cu)

@@ -252,7 +252,7 @@ __global__ void __launch_bounds__(128)
 slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const float* __restrict__ hscale, const float* __restrict__ su,
                     const unsigned char* __restrict__ u_tiled,
                     float* __restrict__ o, const ProjGeom g, const int d, const int d_k, const int batch,
-                    int* status, const int32_t* __restrict__ lengths) {
+                    int* status, const int32_t* __restrict__ lengths, const int e) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_u32 = smem_u32(smem_raw);
   const uint32_t base = (raw_u32 + 1023u) & ~1023u;
@@ -386,7 +386,7 @@ slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const float* __res
       float a = 0.f;
       for (int sl = 0; sl < g.jsplit; ++sl) a += ld_cluster_f32(mapa(base + (uint32_t)(n * 128 + m) * 4u, (uint32_t)sl));
       // an empty sequence has no partials: its operand columns hold whatever an earlier call left
-      if (b < batch && c < d_k) o[(size_t)b * d + head * d_k + c] = lengths[b] > 0 ? a : 0.f;
+      if (b < batch && c < d_k) o[(size_t)b * e + head * d_k + c] = lengths[b] > 0 ? a : 0.f;
     }
   }
   cluster_sync_all();                                          // nobody leaves while its tile may still be read
@@ -508,5 +508,5 @@ cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, uns
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, slim_proj_tc_kernel, map, (const float*)ctx->wkv_hscale, (const float*)su, (const unsigned char*)u_tiled,
-                            p.o, g, p.d, p.d_k, p.batch, p.status, p.lengths);
+                            p.o, g, p.d, p.d_k, p.batch, p.status, p.lengths, p.e);
 }

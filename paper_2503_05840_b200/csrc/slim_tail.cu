@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(256) slim_tail1_kernel(SlimDecodeParams p, int
 #pragma unroll
       for (int i = 0; i < BPT; ++i) {
         const int bi = bg * BPT + i;
-        if (bi < nb) o_part[((size_t)js * p.batch + b0 + bi) * d + h * dk + c] = acc[i];
+        if (bi < nb) o_part[((size_t)js * p.batch + b0 + bi) * p.e + h * dk + c] = acc[i];
       }
     }
   }
@@ -214,9 +214,9 @@ slim_append_fp8_kernel(unsigned char* __restrict__ codes, signed char* __restric
 
 }  // namespace
 
-size_t slim_tail_opart_floats(int d, int batch) {
+size_t slim_tail_opart_floats(int d, int e, int batch) {
   const int slices = (d + JR - 1) / JR;
-  return (size_t)(slices > 8 ? slices : 8) * batch * d;      // the tensor-core projection writes up to 8 slices
+  return (size_t)(slices > 8 ? slices : 8) * batch * e;
 }
 
 cudaError_t slim_launch_sum_slices(const float* o_part, float* o, int n, int nsplit, cudaStream_t st) {
@@ -248,7 +248,7 @@ cudaError_t slim_launch_tail(const slim_ctx* ctx, const SlimDecodeParams& p, cud
   }
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  const int n = p.batch * p.d;
+  const int n = p.batch * p.e;
   slim_tail2_kernel<<<(n + 255) / 256, 256, 0, st>>>(o_part, p.o, n, nsplit);
   return cudaGetLastError();
 }

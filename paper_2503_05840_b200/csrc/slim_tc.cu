@@ -235,7 +235,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
         float qh1[8], qh2[8];
 #pragma unroll
         for (int x = 0; x < 8; ++x) { qh1[x] = 0.f; qh2[x] = 0.f; }
-        if (active) {
+        if (active && !EXT) {         // (with external scores the query is not needed here, and its rows are H d_k wide, not d)
           const __nv_bfloat16* Q = reinterpret_cast<const __nv_bfloat16*>(p.q) + (size_t)b * p.d + my_n * DK + 8 * jl;
           float a[8], c[8];
           unpack8(__ldg(reinterpret_cast<const uint4*>(Q)), a);

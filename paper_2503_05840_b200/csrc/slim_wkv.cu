@@ -298,11 +298,11 @@ template <typename WT>
 __global__ void store_wkv_kernel(const double* __restrict__ X, WT* __restrict__ dst, __half* __restrict__ dst_h,
                                  const float* __restrict__ hscale, int d, int H, int dk) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= (size_t)d * d) return;
+  if (i >= (size_t)d * H * dk) return;
   const int c = (int)(i % dk);
   const size_t rest = i / dk;
   const int j = (int)(rest % d), h = (int)(rest / d);
-  const double v = X[(size_t)j * d + h * dk + c];
+  const double v = X[(size_t)j * H * dk + h * dk + c];
   if constexpr (sizeof(WT) == 2) {
     dst[i] = __double2bfloat16(v);
     if (dst_h) dst_h[i] = __double2half(v / (double)hscale[h]);      // power-of-two scale: exact
@@ -312,12 +312,12 @@ __global__ void store_wkv_kernel(const double* __restrict__ X, WT* __restrict__ 
 }
 
 // hscale[h] = 2^-a with max |W_KV,h| * 2^a in [2^14, 2^15) (1 for an all-zero head): one CTA per head
-__global__ void head_scale_kernel(const double* __restrict__ X, float* __restrict__ hscale, int d, int dk) {
+__global__ void head_scale_kernel(const double* __restrict__ X, float* __restrict__ hscale, int d, int dk, int e) {
   __shared__ double s_max[256];
   const int h = blockIdx.x;
   double m = 0.0;
   for (size_t i = threadIdx.x; i < (size_t)d * dk; i += blockDim.x) {
-    const double v = fabs(X[(i / dk) * d + (size_t)h * dk + i % dk]);
+    const double v = fabs(X[(i / dk) * e + (size_t)h * dk + i % dk]);
     m = v > m ? v : m;
   }
   s_max[threadIdx.x] = m;
@@ -402,9 +402,9 @@ cudaError_t slim_wkv_residual(const double* Wk, const double* X, const double* W
 }
 
 cudaError_t slim_wkv_store(const double* X, int d, int H, int d_k, int dtype, void* dst, void* dst_h, float* hscale) {
-  const size_t nn = (size_t)d * d;
+  const size_t nn = (size_t)d * H * d_k;
   if (dtype == SLIM_BF16) {
-    if (dst_h) head_scale_kernel<<<H, 256>>>(X, hscale, d, d_k);
+    if (dst_h) head_scale_kernel<<<H, 256>>>(X, hscale, d, d_k, H * d_k);
     store_wkv_kernel<__nv_bfloat16><<<(unsigned)((nn + 255) / 256), 256>>>(X, (__nv_bfloat16*)dst, (__half*)dst_h, hscale, d, H, d_k);
   } else {
     store_wkv_kernel<float><<<(unsigned)((nn + 255) / 256), 256>>>(X, (float*)dst, nullptr, nullptr, d, H, d_k);

@@ -36,7 +36,7 @@ slim_xq_tiled_kernel(SlimDecodeParams p, const float* __restrict__ W_K, unsigned
   const int h = blockIdx.x, j0 = blockIdx.y * XQ_J, tid = threadIdx.x;
   for (int e = tid; e < XQ_J * dk; e += 256) {
     const int j = e / dk, c = e % dk;
-    s_w[j * (dk + 1) + c] = (j0 + j < d) ? __ldg(W_K + (size_t)(j0 + j) * d + h * dk + c) : 0.f;
+    s_w[j * (dk + 1) + c] = (j0 + j < d) ? __ldg(W_K + (size_t)(j0 + j) * p.e + h * dk + c) : 0.f;
   }
   const int j = tid & (XQ_J - 1), bq = tid >> 6;                     // a thread: row j, sequences 4 bq .. 4 bq + 3 of a pass
   for (int b0 = 0; b0 < p.batch; b0 += XQ_B) {
@@ -44,7 +44,7 @@ slim_xq_tiled_kernel(SlimDecodeParams p, const float* __restrict__ W_K, unsigned
     for (int e = tid; e < XQ_B * dk; e += 256) {                     // s_q[c][bb]: four sequences of one c in 16 bytes
       const int bb = e / dk, c = e % dk;
       s_q[c * XQ_B + bb] = (b0 + bb < p.batch)
-                               ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.q)[(size_t)(b0 + bb) * d + h * dk + c]) * p.qscale : 0.f;
+                               ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.q)[(size_t)(b0 + bb) * p.e + h * dk + c]) * p.qscale : 0.f;
     }
     __syncthreads();
     if (j0 + j >= d) continue;

@@ -145,3 +145,61 @@ def test_xcache_batch_above_sixteen_small_ragged():
     lengths = g.integers(1, 120, size=40).astype(np.int32)
     lengths[[3, 17, 33]] = [0, 1, 119]
     _xcache_device_case(256, 4, 64, 40, 119, lengths, list(range(40)), 3004)
+
+
+@pytest.mark.parametrize("d,H,d_k,dtype", [(512, 8, 128, "bf16"),      # e = 1024 > d, tensor-core kernels (a T5-style widening)
+                                           (512, 2, 128, "bf16"),      # e = 256 < d
+                                           (1280, 10, 64, "bf16"),     # e = 640, two heads per projection MMA
+                                           (192, 4, 64, "f32"),        # CUDA-core kernels, e = 256
+                                           (320, 6, 100, "f32")])      # a head width outside the vector paths, e = 600
+def test_xcache_nonsquare_projections_match_oracle(d, H, d_k, dtype):
+    """Non-square projections (section "Support for non-square weight matrices", Option 2): the cache
+    holds d-wide inputs, W_K and W_V are d x e with e = H d_k != d, queries and outputs are e wide."""
+    e = H * d_k
+    g = np.random.default_rng(d + e)
+    lengths = np.array([700, 333, 0, 17, 1, 129], dtype=np.int32)
+    batch, t_cap = len(lengths), 700
+    X = np.zeros((batch, t_cap, d), dtype=np.float32)
+    for b in range(batch):
+        X[b, :lengths[b]] = synth.round_to_dtype(g.standard_normal((int(lengths[b]), d)), dtype)
+    if e > d:
+        W_Q, W_K, W_V, _, _ = synth.make_weights_nonsquare(d, e, 500 + d)
+    else:
+        W_Q, W_K, W_V = (g.standard_normal((d, e)) / np.sqrt(d) for _ in range(3))
+    bias = g.standard_normal(e) * 0.1
+    q = np.zeros((batch, e), dtype=np.float32)
+    for b in range(batch):
+        if lengths[b]:
+            q[b] = synth.round_to_dtype(X[b, lengths[b] - 1].astype(np.float64) @ W_Q + bias, dtype)
+    with torch.cuda.device(DEV):
+        storage = to_device_keys(X, dtype, DEV)
+        storage[1, lengths[1]:] = float("nan")
+        ctx = B.slim_xcache_create(d, H, d_k, B.SLIM_BF16 if dtype == "bf16" else B.SLIM_F32)
+        cache = None
+        try:
+            cache = B.slim_cache_create(ctx, storage, batch, t_cap)
+            ws = torch.empty(B.slim_xcache_workspace_bytes(ctx, batch, t_cap), dtype=torch.uint8, device=DEV)
+            o = torch.full((batch, e), float("nan"), dtype=torch.float32, device=DEV)
+            st = torch.cuda.current_stream().cuda_stream
+            B.slim_xcache_set_weights(ctx, W_K, W_V)
+            B.slim_xcache_decode(ctx, to_device_keys(q, dtype, DEV), cache, torch.from_numpy(lengths).to(DEV), o, ws, st)
+            assert B.slim_device_status(ctx, st) == B.SLIM_OK
+            got = o.cpu().numpy().astype(np.float64)
+            assert np.all(np.isfinite(got))
+            for b in range(batch):
+                n = int(lengths[b])
+                if n == 0:
+                    assert np.all(got[b] == 0)
+                    continue
+                ref = so.oracle_xcache(q[b], X[b, :n], W_K, W_V, H)
+                err = _err(got[b], ref, dtype)
+                assert err <= TOL[dtype], f"seq {b}: {err:.3e}"
+            # the K-cache calls have no meaning on such a context (W_K is not square)
+            if e != d:
+                with pytest.raises(B.SlimError) as ei:
+                    B.slim_decode(ctx, to_device_keys(q, dtype, DEV), cache, torch.from_numpy(lengths).to(DEV), o, ws, st)
+                assert ei.value.status == B.SLIM_ERR_UNSUPPORTED
+        finally:
+            if cache:
+                B.slim_cache_destroy(cache)
+            B.slim_destroy(ctx)
