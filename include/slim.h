@@ -295,6 +295,13 @@ slim_status slim_selftest_bounded_wait(slim_ctx* ctx, void* stream);
 slim_status slim_profile_enable(slim_ctx* ctx, int enable);
 slim_status slim_profile_read(slim_ctx* ctx, float* main_ms, float* tail_ms);
 
+/* Per-tile timing of the tensor-core decode kernel, for builds of the library compiled with
+ * -DSLIM_TC_TRACE (python -m paper_2503_05840_b200.trace builds one and prints the statistics; the
+ * default build returns SLIM_ERR_UNSUPPORTED).  device_buffer: device int64 [CTAs][192][8], zeroed by
+ * the caller; while set, every slim_decode of this ctx records, for the first 192 tiles of each CTA,
+ * the SM clock at eight points of the producer, score-warp and MMA loops.  NULL switches it off.  */
+slim_status slim_set_trace(slim_ctx* ctx, void* device_buffer);
+
 slim_status slim_set_path(slim_ctx* ctx, int path);
 long long   slim_query(const slim_ctx* ctx, int key);
 const char* slim_strerror(int status);

@@ -50,6 +50,7 @@ SIGNATURES = {
     "slim_selftest_bounded_wait": (c_int, [c_void_p, c_void_p]),
     "slim_profile_enable": (c_int, [c_void_p, c_int]),
     "slim_profile_read": (c_int, [c_void_p, POINTER(ctypes.c_float), POINTER(ctypes.c_float)]),
+    "slim_set_trace": (c_int, [c_void_p, c_void_p]),
     "slim_set_path": (c_int, [c_void_p, c_int]),
     "slim_query": (c_longlong, [c_void_p, c_int]),
     "slim_strerror": (c_char_p, [c_int]),
@@ -65,13 +66,15 @@ class SlimError(RuntimeError):
 
 
 def lib() -> ctypes.CDLL:
-    """Load libslim.so (once).  Raises if it has not been built."""
+    """Load libslim.so (once).  Raises if it has not been built.  SLIM_LIBRARY names another build of the
+    library (the instrumented one of trace.py)."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2503_05840_b200.build` "
+        path = os.environ.get("SLIM_LIBRARY", LIB_PATH)
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: run `python -m paper_2503_05840_b200.build` "
                                "(there is no CPU fallback)")
-        L = ctypes.CDLL(LIB_PATH)
+        L = ctypes.CDLL(path)
         for name, (res, args) in SIGNATURES.items():
             fn = getattr(L, name)
             fn.restype = res
@@ -265,6 +268,10 @@ def slim_profile_read(ctx: int):
     a, b = ctypes.c_float(0), ctypes.c_float(0)
     _check(lib().slim_profile_read(c_void_p(ctx), byref(a), byref(b)), "slim_profile_read")
     return a.value, b.value
+
+
+def slim_set_trace(ctx: int, device_buffer) -> None:
+    _check(lib().slim_set_trace(c_void_p(ctx), _ptr(device_buffer)), "slim_set_trace")
 
 
 def slim_set_path(ctx: int, path: int) -> None:

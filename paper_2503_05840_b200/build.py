@@ -31,17 +31,27 @@ def needs_build() -> bool:
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+TRACE_LIB = os.path.join(HERE, "libslim_trace.so")
+
+
+def build(force: bool = False, verbose: bool = False, trace: bool = False) -> str:
+    """trace=True builds libslim_trace.so, the library with the per-tile instrumentation of the
+    tensor-core decode kernel compiled in (-DSLIM_TC_TRACE)."""
+    if trace:
+        return _build(TRACE_LIB, os.path.join(HERE, "_build", "trace"), ["-DSLIM_TC_TRACE"], verbose)
     if not force and not needs_build():
         return LIB
+    return _build(LIB, os.path.join(HERE, "_build"), [], verbose)
+
+
+def _build(lib_path: str, bdir: str, extra: list, verbose: bool) -> str:
     nvcc = _nvcc()
-    bdir = os.path.join(HERE, "_build")
     os.makedirs(bdir, exist_ok=True)
     objs = []
     procs = []
     for s in SOURCES:
         o = os.path.join(bdir, s.replace(".cu", ".o"))
-        cmd = [nvcc] + FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
+        cmd = [nvcc] + FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + \
               ["-c", os.path.join(CSRC, s), "-o", o]
         procs.append((s, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(o)
@@ -51,12 +61,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
             sys.stderr.write(out)
         if p.returncode:
             raise RuntimeError(f"nvcc failed on {s}")
-    cmd = [nvcc, "-shared", "-o", LIB] + objs + ["-lcudart"]
+    cmd = [nvcc, "-shared", "-o", lib_path] + objs + ["-lcudart"]
     r = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
     if r.returncode:
         sys.stderr.write(r.stdout)
         raise RuntimeError("link failed")
-    return LIB
+    return lib_path
 
 
 if __name__ == "__main__":

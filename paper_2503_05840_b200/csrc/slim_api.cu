@@ -515,6 +515,7 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   p.q_pos = part ? part->q_pos : nullptr;
   p.rope_tiles = ctx->rope_base_tiles;
   p.k_evict_first = ctx->opt_k_evict;
+  p.trace = ctx->trace;
   cudaStream_t st = (cudaStream_t)stream;
   int launches = 0;
   if (k_new && !p.k_new) {                           // no fused update on this path: the append kernel first
@@ -719,6 +720,17 @@ slim_status slim_profile_read(slim_ctx* ctx, float* main_ms, float* tail_ms) {
       cudaEventElapsedTime(tail_ms, ctx->prof_ev[1], ctx->prof_ev[2]) != cudaSuccess)
     return SLIM_ERR_CUDA;
   return SLIM_OK;
+}
+
+slim_status slim_set_trace(slim_ctx* ctx, void* device_buffer) {
+  if (!ctx) return SLIM_ERR_INVALID_ARG;
+#ifdef SLIM_TC_TRACE
+  ctx->trace = static_cast<long long*>(device_buffer);
+  return SLIM_OK;
+#else
+  (void)device_buffer;
+  return SLIM_ERR_UNSUPPORTED;                    // this build of the library carries no instrumentation
+#endif
 }
 
 slim_status slim_set_path(slim_ctx* ctx, int path) {

@@ -14,6 +14,7 @@
 #define SLIM_TT 16
 #define SLIM_MAX_H 64
 #define SLIM_MAX_BATCH 2048
+#define SLIM_TRACE_TILES 192      // tiles per CTA that a trace build records
 
 // Parameters every decode kernel receives (passed by value).
 struct SlimDecodeParams {
@@ -52,6 +53,7 @@ struct SlimDecodeParams {
   const int32_t* q_pos;
   int k_evict_first;             // tensor-core path: key tiles are loaded with the L2 evict-first hint
   int rope_tiles;                // entries of rope_base (positions < SLIM_TT * rope_tiles are covered)
+  long long* trace;              // builds with SLIM_TC_TRACE only: [CTAs][SLIM_TRACE_TILES][8] SM clocks (else NULL, unused)
   const void* k_new;             // tensor-core path: [batch][d] newest key rows, written at row lengths[b]-1 before the read (or NULL)
   int redo_in_combine;           // 1: the combine kernel recomputes the sequences that have a flagged unit (no redo kernel runs)
 };
@@ -88,6 +90,7 @@ struct slim_ctx {
   int opt_unit_cost;             // SLIM_TC_UNIT_COST: boundary cost of the schedule in tiles (-1 = default)
   int opt_xscores_cuda;          // SLIM_XSCORES_CUDA: dense X-cache scores on CUDA cores
   int opt_k_evict;               // SLIM_TC_K_EVICT (0/1): L2 evict-first hint on the key loads (default on)
+  long long* trace;              // device buffer set by slim_set_trace (trace builds)
   int opt_proj_ns;               // SLIM_PROJ_NS: stages of the projection kernel (0 = default)
   int opt_legacy_flow;           // SLIM_TC_LEGACY: append and exact redo as kernels of their own (for side-by-side timing)
   alignas(64) unsigned char wmap[128];   // CUtensorMap over W_KV for the projection kernel

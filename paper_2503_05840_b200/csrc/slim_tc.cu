@@ -68,6 +68,22 @@
 namespace {
 using namespace slim_ptx;
 
+// Compile-time instrumentation, off by default (-DSLIM_TC_TRACE, see build.py and trace.py): for the first
+// SLIM_TRACE_TILES tiles of every CTA one thread of each role stores the SM clock at fixed points of its
+// per-tile loop.  Slots: 0 producer at the top of its loop, 1 producer when the stage is free (load issued),
+// 2 score warp 0 when the keys have landed, 3 when its probabilities are computed, 4 when the P stage is
+// free, 5 when it has shipped and released, 6 MMA thread when the tile's probabilities are complete,
+// 7 when its MMAs and the commit are issued.
+#ifdef SLIM_TC_TRACE
+#define TC_TRACE(slot, tile_no)                                                                              \
+  do {                                                                                                       \
+    if (p.trace && (tile_no) < SLIM_TRACE_TILES)                                                             \
+      p.trace[((size_t)blockIdx.x * SLIM_TRACE_TILES + (tile_no)) * 8 + (slot)] = clock64();                 \
+  } while (0)
+#else
+#define TC_TRACE(slot, tile_no) do {} while (0)
+#endif
+
 constexpr int TC_P_BYTES = 1024;         // [32 heads][16 rows] bf16
 constexpr int TC_MAX_NS = 8;             // K stages
 constexpr int TC_MAX_SW = 16;            // score warps
@@ -284,6 +300,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             // a wait that ran out is acted on after the vote below (until then the lanes only
             // touch their own registers and this CTA's shared memory)
             ok = mbar_wait<false>(bar_k_full + 8 * st, kph, s_abort, p.status);
+            if (warp == 0 && lane == 0) TC_TRACE(2, it_own);
             // rows at or beyond the sequence end must not reach the tensor core (0 x NaN)
             if (t0 + SLIM_TT > len) {
               const int nz = len - t0;
@@ -370,10 +387,12 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             const float pf = valid ? ex2_approx(x) : 0.f;
             const __nv_bfloat16 pb = __float2bfloat16_rn(pf);
             if ((jl % DUP) == 0) lsum += __bfloat162float(pb);
+            if (warp == 0 && lane == 0) TC_TRACE(3, it_own);
             // the P stage is free once the MMAs of tile it - ns are done in both CTAs
             ok = mbar_wait<false>(bar_p_empty + 8 * (PAIR ? st >> 1 : st), kph ^ 1, s_abort, p.status) && ok;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
+            if (warp == 0 && lane == 0) TC_TRACE(4, it_own);
             {
               // stage this warp's probabilities in the K-major order of the P tile, then ship
               // them in 16-byte pieces (8 rows of one head) to both CTAs
@@ -397,6 +416,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             if (lane == 0) {
               mbar_arrive_expect_tx(bar_p_full + 8 * st, p_bytes_w);
               mbar_arrive(bar_k_empty + 8 * st);
+              if (warp == 0) TC_TRACE(5, it_own);
             }
             if (ROPE && active && SETS == 2) {
               // the other set's tile: RT row steps of RP rows keep the stepped rotation in step
@@ -515,9 +535,11 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           const int tile0 = gg - s_prefix[b], ntile = seg_end - gg;
           for (int kt = 0; kt < ntile; ++kt, ++it, st = (st + 1 == g.ns ? 0 : st + 1), kph ^= (st == 0)) {
             // free once the score warps have read the keys and the tensor core has consumed them
+            TC_TRACE(0, it);
             ok = mbar_wait<false>(bar_k_empty + 8 * st, kph ^ 1, s_abort, p.status) &&
                  mbar_wait<false>(bar_p_empty + 8 * (PAIR ? st >> 1 : st), kph ^ 1, s_abort, p.status);
             if (!ok) break;
+            TC_TRACE(1, it);
             mbar_arrive_expect_tx(bar_k_full + 8 * st, (uint32_t)g.stage_bytes);
             if (p.k_evict_first)
               tma_load_3d_hint(k_stage0 + (uint32_t)st * g.stage_bytes, &tmap, bar_k_full + 8 * st, 0,
@@ -564,6 +586,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             if (ok && two) ok = mbar_wait<true>(bar_p_full + 8 * (st + 1), kph, s_abort, p.status);
             if (ok && kt == 0 && uc > 0) ok = mbar_wait<false>(bar_u_empty, (uc - 1) & 1, s_abort, p.status);
             if (!ok) break;
+            TC_TRACE(6, it);
             fence_proxy_async_smem();        // P pieces and zero-filled key rows -> tensor-core reads
             tc_fence_after();
             // One instruction per 128-column chunk.  The tensor core takes one of these every ~65
@@ -587,6 +610,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             } else if (last & 1) {               // the odd stage closes the pair (the even one is older)
               if (CL == 2) umma_commit_pair(bar_p_empty + 8 * (last >> 1)); else umma_commit(bar_p_empty + 8 * (last >> 1));
             }
+            TC_TRACE(7, it);
             const int adv = two ? 2 : 1;
             kt += adv; it += adv; st += adv;
             if (st >= g.ns) { st -= g.ns; kph ^= 1u; }
