@@ -148,6 +148,160 @@ slim_values_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
   }
 }
 
+// The same product on a CTA pair (cluster of two along the prompt rows): one tcgen05.mma.cta_group::2 with
+// M = 256 covers the 128 rows of each CTA; each CTA stages its own key rows and only HALF of the W_KV tile
+// (64 of the 128 columns: its half of B's N), so the weight bytes fetched per flop are halved.  The even CTA
+// issues the MMAs.  Both CTAs' loads of a stage count their bytes on the EVEN CTA's barrier (pair form of the
+// TMA load), so the issuer waits on one barrier and no thread relays anything; one multicast commit frees
+// the stage in both CTAs.
+constexpr int PV2_B_BYTES = PV_J * 64 * 2;          // one 64-column atom x 64 rows x 128 B = 8 KB
+#ifndef PV2_NS_X
+#define PV2_NS_X 4
+#endif
+constexpr int PV2_NS = PV2_NS_X;
+constexpr uint32_t PV2_STAGE = PV_A_BYTES + PV2_B_BYTES;
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128)
+slim_values_tc2_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap wmap1, float* __restrict__ V,
+                       const int n, const int d, const int d_k, const int hp, int* status, const SlimDecodeParams cp) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw_u32 = smem_u32(smem_raw);
+  const uint32_t base = (raw_u32 + 1023u) & ~1023u;
+  unsigned char* sm = smem_raw + (base - raw_u32);
+  const uint32_t bars = base + PV2_NS * PV2_STAGE;
+  // full: (even CTA's copy only) both CTAs' loads of a stage have landed; empty: the pair's MMAs on the stage
+  // are done (commit from the even CTA, to both); done: the accumulator is complete
+  const uint32_t bar_full = bars, bar_empty = bars + 8 * PV2_NS, bar_done = bars + 16 * PV2_NS;
+  unsigned char* misc = sm + (bar_done + 8 - base);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 4);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // One-dimensional grid, a pair = two neighbouring CTAs (the pair of a cta_group::2 instruction is the two CTAs
+  // whose cluster rank differs in the last bit, along x).  Pairs are numbered with the head groups fastest: the
+  // pairs in flight share a few key tiles and all of W_KV (L2-resident).
+  const uint32_t rank = cluster_ctarank();
+  const int ngroups_h = (d / d_k) / hp;
+  const int pair = blockIdx.x >> 1, hg = pair % ngroups_h;
+  const int t0 = (2 * (pair / ngroups_h) + (int)rank) * PV_ROWS;
+  const int nst = d / PV_J;
+
+  if (tid == 0) {
+    prefetch_tensormap(&kmap);
+    prefetch_tensormap(&wmap1);
+    for (int i = 0; i < PV2_NS; ++i) {
+      mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1);
+    }
+    mbar_init(bar_done, 1);
+    *s_abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) tmem_alloc2(smem_u32(s_tmem), 128);       // the same warp of both CTAs
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                      // the peer's barriers exist before anything is sent to them
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  slim_pdl_wait();
+
+  if (warp == 0 && lane == 0) {
+    // ---- producer: this CTA's 128 key rows and its half (atom `rank`) of the W_KV tile; the bytes of both
+    // CTAs are expected (by the even CTA's producer) and counted on the even CTA's barrier ----
+    int s = 0;
+    bool ok = true;
+    for (; s < nst; ++s) {
+      const int st = s % PV2_NS;
+      ok = mbar_wait<false>(bar_empty + 8 * st, ((s / PV2_NS) & 1) ^ 1, s_abort, status);
+      if (!ok) break;
+      const uint32_t dst = base + (uint32_t)st * PV2_STAGE;
+      const uint32_t full0 = mapa(bar_full + 8 * st, 0);
+      if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * st, 2 * PV2_STAGE);
+      tma_load_3d_pair(dst, &kmap, full0, s * PV_J, t0, 0);
+      if (hp == 1) tma_load_3d_pair(dst + PV_A_BYTES, &wmap1, full0, 0, hg * d + s * PV_J, (int)rank);
+      else         tma_load_3d_pair(dst + PV_A_BYTES, &wmap1, full0, 0, s * PV_J, 2 * hg + (int)rank);
+    }
+    if (!ok) {
+      // Gave up (a wait ran out two seconds after the last progress): whatever was issued has landed long
+      // since; the even CTA still waits, bounded, on the barriers that count both CTAs' bytes, the odd CTA
+      // lets a fixed time pass.  Neither leaves before the final cluster barrier.
+      if (rank == 0) {
+        const int issued = s < PV2_NS ? s : PV2_NS;
+        for (int k = 0; k < issued; ++k) {
+          const int j = s - 1 - k, st = j % PV2_NS;
+          const unsigned long long tt = globaltimer();
+          while (!mbar_try_wait(bar_full + 8 * st, (j / PV2_NS) & 1) && globaltimer() - tt < SLIM_WAIT_NS) {}
+        }
+      } else {
+        const unsigned long long tt = globaltimer();
+        while (globaltimer() - tt < 200000ull) {}
+      }
+    }
+  } else if (warp >= 2 && hg == 0 && cp.k != nullptr) {
+    // bulk append (as in the single-CTA kernel)
+    const int n_new = cp.workers, t64 = tid - 64;
+    const uint4* src = reinterpret_cast<const uint4*>(cp.q);
+    uint4* dst = reinterpret_cast<uint4*>(const_cast<void*>(cp.k));
+    const int vec_per_row = d / 8;
+    for (int r = t0; r < min(t0 + PV_ROWS, n); ++r) {
+      const int b = r / n_new, i = r - b * n_new;
+      const int pos = cp.lengths[b];
+      if (pos < 0 || pos > cp.t_cap - n_new) { if (t64 == 0) atomicMax(status, (int)SLIM_ERR_CAPACITY); continue; }
+      const long long row = slim_cache_row(cp, b, pos + i);
+      for (int e = t64; e < vec_per_row; e += 64) dst[(size_t)row * vec_per_row + e] = __ldg(src + (size_t)r * vec_per_row + e);
+    }
+  }
+  if (warp == 1 && lane == 0 && rank == 0) {
+    // ---- MMA issuer of the pair ----
+    bool ok = true;
+    int st = 0;
+    uint32_t ph = 0;
+    const uint64_t ad0 = desc_kmajor_sw128(base), bd0 = desc_a(base + PV_A_BYTES, PV_J * 128);
+    const uint32_t a_lo0 = (uint32_t)ad0, a_hi = (uint32_t)(ad0 >> 32), b_lo0 = (uint32_t)bd0, b_hi = (uint32_t)(bd0 >> 32);
+    constexpr uint32_t idesc = umma_idesc_mn(256, 128, 0, 1);          // A K-major, B MN-major
+    for (int s = 0; s < nst && ok; ++s, st = (st + 1 == PV2_NS ? 0 : st + 1), ph ^= (st == 0)) {
+      ok = mbar_wait<true>(bar_full + 8 * st, ph, s_abort, status);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t a_lo = a_lo0 + (uint32_t)st * (PV2_STAGE >> 4), b_lo = b_lo0 + (uint32_t)st * (PV2_STAGE >> 4);
+#pragma unroll
+      for (int kk = 0; kk < PV_J / 16; ++kk)
+        umma2_bf16_words(tmem_base, a_lo + (uint32_t)kk * (32u >> 4), a_hi, b_lo + (uint32_t)kk * (2048u >> 4), b_hi, idesc,
+                         (s | kk) ? 1u : 0u);
+      umma2_commit_pair(bar_empty + 8 * st);
+      if (s == nst - 1) umma2_commit_pair(bar_done);
+    }
+  }
+  __syncwarp();
+  {
+    bool ok = mbar_wait<false>(bar_done, 0, s_abort, status);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after();
+      const int row = t0 + warp * 32 + lane;                   // accumulator row = prompt row (this CTA's 128 TMEM lanes)
+      const int ncols = hp == 2 ? 128 : d_k;
+      float* out = V + (size_t)row * d + (size_t)hg * hp * d_k;
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, r);
+        if (row < n) {
+#pragma unroll
+          for (int c = 0; c < 32; c += 4)
+            if (c0 + c < ncols)
+              *reinterpret_cast<float4*>(out + c0 + c) = make_float4(__uint_as_float(r[c]), __uint_as_float(r[c + 1]),
+                                                                    __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
+        }
+      }
+    }
+  }
+  // nobody leaves (or frees the pair's tensor memory) while the other CTA may still be reached
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc2(tmem_base, 128);
+  }
+}
+
 // CUDA-core version: V[t][h d_k + c] = sum_j K[t][j] W[h][j][c]; 16 x 16 output tile per CTA.
 template <typename KT>
 __global__ void __launch_bounds__(256)
@@ -169,6 +323,7 @@ slim_values_kernel(const KT* __restrict__ K, const KT* __restrict__ W, float* __
 }
 
 constexpr size_t PV_SMEM = 1024 + (size_t)PV_NS * (PV_A_BYTES + PV_B_BYTES) + 16 * PV_NS + 8 + 16 + 64;
+constexpr size_t PV2_SMEM = 1024 + (size_t)PV2_NS * PV2_STAGE + 16 * PV2_NS + 8 + 16 + 64;
 
 }  // namespace
 
@@ -204,8 +359,28 @@ cudaError_t slim_launch_values(const slim_ctx* ctx, const void* K, int n, float*
     const unsigned int box[3] = {PV_J, PV_ROWS, 1};
     cudaError_t e = slim_tmap_encode_3d(&kmap, const_cast<void*>(K), dims, strides, box);
     if (e != cudaSuccess) return e;
-    memcpy(&wmap, ctx->wmap, sizeof(wmap));
     const int hp = d_k == 64 ? 2 : 1;
+    if (ctx->opt_prompt_pair && n > PV_ROWS) {           // CTA pairs over the prompt rows (grid.y even)
+      static bool attr2_set[64] = {};
+      if (ctx->device < 0 || ctx->device >= 64 || !attr2_set[ctx->device]) {
+        e = cudaFuncSetAttribute((const void*)slim_values_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PV2_SMEM);
+        if (e != cudaSuccess) return e;
+        if (ctx->device >= 0 && ctx->device < 64) attr2_set[ctx->device] = true;
+      }
+      memcpy(&wmap, ctx->wmap1, sizeof(wmap));
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(2 * (H / hp) * ((n + 2 * PV_ROWS - 1) / (2 * PV_ROWS)));
+      cfg.blockDim = dim3(128);
+      cfg.dynamicSmemBytes = PV2_SMEM;
+      cfg.stream = st;
+      cudaLaunchAttribute attr[1];                   // (the cluster shape (2, 1, 1) is a compile-time property of the kernel)
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr; cfg.numAttrs = 1;
+      e = cudaLaunchKernelEx(&cfg, slim_values_tc2_kernel, kmap, wmap, V, n, d, d_k, hp, ctx->status, cp);
+      return e;
+    }
+    memcpy(&wmap, ctx->wmap, sizeof(wmap));
     return slim_launch_pdl(slim_values_tc_kernel, dim3(H / hp, (n + PV_ROWS - 1) / PV_ROWS), dim3(128), PV_SMEM, st, kmap, wmap, V, n,
                            d, d_k, hp, ctx->status, cp);
   }

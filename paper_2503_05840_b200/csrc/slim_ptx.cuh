@@ -120,6 +120,36 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {   // arrives on
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                ::"r"(bar), "h"((unsigned short)3) : "memory");
 }
+// ---- CTA-pair forms (cta_group::2): one MMA instruction, issued by the even CTA of a cluster of two, drives the
+// tensor cores of both; each CTA supplies its own 128 rows of A and its half of B's N columns from its own shared
+// memory (same offsets in both CTAs), and receives its 128 rows of D in its own tensor memory.
+__device__ __forceinline__ void tmem_alloc2(uint32_t dst_smem, uint32_t cols) {      // by the same warp of BOTH CTAs
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma2_bf16_words(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                 uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\tmov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma2_commit_pair(uint32_t bar) {   // arrives on the barrier at this offset in both CTAs
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+// TMA load of a CTA pair: the destination is this CTA's shared memory, the bytes are counted on an mbarrier
+// that may live in either CTA of the pair (cluster_bar: an address from mapa), so the pair's MMA issuer
+// waits on one barrier for both CTAs' halves of a stage.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t cluster_bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(cluster_bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
 // 32 consecutive accumulator columns of this warp's 32 TMEM lanes; the registers are valid
 // after tmem_ld_wait().
 __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
@@ -164,6 +194,11 @@ __host__ __device__ constexpr uint32_t umma_idesc(uint32_t n) {
 // The same for float16 operands (A and B of one instruction always share their type).
 __host__ __device__ constexpr uint32_t umma_idesc_f16(uint32_t n) {
   return (1u << 4) | (1u << 15) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// General form: bf16 x bf16 -> f32, M = m (128, or 256 for a CTA pair), N = n, explicit operand majors.
+__host__ __device__ constexpr uint32_t umma_idesc_mn(uint32_t m, uint32_t n, uint32_t a_mn, uint32_t b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn << 15) | (b_mn << 16) | ((n >> 3) << 17) | ((m >> 4) << 24);
 }
 
 // K-major operand, 128-byte swizzle, as TMA delivers a [rows][64 elements] tile: 8-row groups
