@@ -154,16 +154,23 @@ slim_values_tc_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
 // issues the MMAs.  Both CTAs' loads of a stage count their bytes on the EVEN CTA's barrier (pair form of the
 // TMA load), so the issuer waits on one barrier and no thread relays anything; one multicast commit frees
 // the stage in both CTAs.
-constexpr int PV2_B_BYTES = PV_J * 64 * 2;          // one 64-column atom x 64 rows x 128 B = 8 KB
-#ifndef PV2_NS_X
-#define PV2_NS_X 4
-#endif
-constexpr int PV2_NS = PV2_NS_X;
-constexpr uint32_t PV2_STAGE = PV_A_BYTES + PV2_B_BYTES;
+// NB = 64-column atoms of W_KV per CTA: NB = 1 is the 256 x 128 pair tile (four 24 KB stages), NB = 2 the
+// 256 x 256 one (three 32 KB stages, 256 accumulator columns): per flop it fetches two thirds of the bytes.
+// Either way two CTAs (of different pairs) share an SM, one's epilogue under the other's MMAs.
+template <int NB> struct Pv2 {
+  static constexpr int B_BYTES = PV_J * 64 * 2 * NB;        // NB atoms x 64 rows x 128 B
+  static constexpr int NS = NB == 1 ? 4 : 3;
+  static constexpr uint32_t STAGE = PV_A_BYTES + B_BYTES;
+  static constexpr int NCOL = 128 * NB;                     // accumulator columns = N of the pair's MMA
+  static constexpr size_t SMEM = 1024 + (size_t)NS * STAGE + 16 * NS + 8 + 16 + 64;
+};
 
+template <int NB>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128)
-slim_values_tc2_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap wmap1, float* __restrict__ V,
+slim_values_tc2_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap wmapb, float* __restrict__ V,
                        const int n, const int d, const int d_k, const int hp, int* status, const SlimDecodeParams cp) {
+  constexpr int PV2_NS = Pv2<NB>::NS, NCOL = Pv2<NB>::NCOL;
+  constexpr uint32_t PV2_STAGE = Pv2<NB>::STAGE;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_u32 = smem_u32(smem_raw);
   const uint32_t base = (raw_u32 + 1023u) & ~1023u;
@@ -180,14 +187,14 @@ slim_values_tc2_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_co
   // whose cluster rank differs in the last bit, along x).  Pairs are numbered with the head groups fastest: the
   // pairs in flight share a few key tiles and all of W_KV (L2-resident).
   const uint32_t rank = cluster_ctarank();
-  const int ngroups_h = (d / d_k) / hp;
+  const int ngroups_h = (d / d_k) / hp / NB;               // column groups of the output (NB = 2: hp d_k = 128)
   const int pair = blockIdx.x >> 1, hg = pair % ngroups_h;
   const int t0 = (2 * (pair / ngroups_h) + (int)rank) * PV_ROWS;
   const int nst = d / PV_J;
 
   if (tid == 0) {
     prefetch_tensormap(&kmap);
-    prefetch_tensormap(&wmap1);
+    prefetch_tensormap(&wmapb);
     for (int i = 0; i < PV2_NS; ++i) {
       mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1);
     }
@@ -195,7 +202,7 @@ slim_values_tc2_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_co
     *s_abort = 0;
     fence_mbar_init();
   }
-  if (warp == 1) tmem_alloc2(smem_u32(s_tmem), 128);       // the same warp of both CTAs
+  if (warp == 1) tmem_alloc2(smem_u32(s_tmem), NCOL);      // the same warp of both CTAs
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();                                      // the peer's barriers exist before anything is sent to them
@@ -216,8 +223,15 @@ slim_values_tc2_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_co
       const uint32_t full0 = mapa(bar_full + 8 * st, 0);
       if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * st, 2 * PV2_STAGE);
       tma_load_3d_pair(dst, &kmap, full0, s * PV_J, t0, 0);
-      if (hp == 1) tma_load_3d_pair(dst + PV_A_BYTES, &wmap1, full0, 0, hg * d + s * PV_J, (int)rank);
-      else         tma_load_3d_pair(dst + PV_A_BYTES, &wmap1, full0, 0, s * PV_J, 2 * hg + (int)rank);
+      // this CTA's half of the tile's columns: atom `rank` of the group (NB = 1, map with one-atom boxes), or
+      // the two atoms of head (hp = 1) / head pair (hp = 2) number 2 hg + rank (NB = 2, two-atom boxes)
+      if (NB == 1) {
+        if (hp == 1) tma_load_3d_pair(dst + PV_A_BYTES, &wmapb, full0, 0, hg * d + s * PV_J, (int)rank);
+        else         tma_load_3d_pair(dst + PV_A_BYTES, &wmapb, full0, 0, s * PV_J, 2 * hg + (int)rank);
+      } else {
+        if (hp == 1) tma_load_3d_pair(dst + PV_A_BYTES, &wmapb, full0, 0, (2 * hg + (int)rank) * d + s * PV_J, 0);
+        else         tma_load_3d_pair(dst + PV_A_BYTES, &wmapb, full0, 0, s * PV_J, 2 * (2 * hg + (int)rank));
+      }
     }
     if (!ok) {
       // Gave up (a wait ran out two seconds after the last progress): whatever was issued has landed long
@@ -256,7 +270,7 @@ slim_values_tc2_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_co
     uint32_t ph = 0;
     const uint64_t ad0 = desc_kmajor_sw128(base), bd0 = desc_a(base + PV_A_BYTES, PV_J * 128);
     const uint32_t a_lo0 = (uint32_t)ad0, a_hi = (uint32_t)(ad0 >> 32), b_lo0 = (uint32_t)bd0, b_hi = (uint32_t)(bd0 >> 32);
-    constexpr uint32_t idesc = umma_idesc_mn(256, 128, 0, 1);          // A K-major, B MN-major
+    constexpr uint32_t idesc = umma_idesc_mn(256, NCOL, 0, 1);         // A K-major, B MN-major
     for (int s = 0; s < nst && ok; ++s, st = (st + 1 == PV2_NS ? 0 : st + 1), ph ^= (st == 0)) {
       ok = mbar_wait<true>(bar_full + 8 * st, ph, s_abort, status);
       if (!ok) break;
@@ -277,9 +291,9 @@ slim_values_tc2_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_co
     if (ok) {
       tc_fence_after();
       const int row = t0 + warp * 32 + lane;                   // accumulator row = prompt row (this CTA's 128 TMEM lanes)
-      const int ncols = hp == 2 ? 128 : d_k;
-      float* out = V + (size_t)row * d + (size_t)hg * hp * d_k;
-      for (int c0 = 0; c0 < 128; c0 += 32) {
+      const int ncols = NB == 2 ? NCOL : (hp == 2 ? 128 : d_k);
+      float* out = V + (size_t)row * d + (NB == 2 ? (size_t)hg * NCOL : (size_t)hg * hp * d_k);
+      for (int c0 = 0; c0 < NCOL; c0 += 32) {
         uint32_t r[32];
         tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, r);
         if (row < n) {
@@ -298,7 +312,7 @@ slim_values_tc2_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_co
   cluster_sync_all();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc2(tmem_base, 128);
+    tmem_dealloc2(tmem_base, NCOL);
   }
 }
 
@@ -323,7 +337,30 @@ slim_values_kernel(const KT* __restrict__ K, const KT* __restrict__ W, float* __
 }
 
 constexpr size_t PV_SMEM = 1024 + (size_t)PV_NS * (PV_A_BYTES + PV_B_BYTES) + 16 * PV_NS + 8 + 16 + 64;
-constexpr size_t PV2_SMEM = 1024 + (size_t)PV2_NS * PV2_STAGE + 16 * PV2_NS + 8 + 16 + 64;
+
+// Launch of the pair kernel (its cluster shape (2, 1, 1) is a compile-time property) behind the previous
+// kernel's programmatic completion.  Function attributes are kept per device: opt in once on each.
+template <int NB>
+cudaError_t launch_pair(int device, dim3 grid, cudaStream_t st, const CUtensorMap& kmap, const CUtensorMap& wmap, float* V, int n,
+                        int d, int d_k, int hp, int* status, const SlimDecodeParams& cp) {
+  static bool attr_set[64] = {};
+  if (device < 0 || device >= 64 || !attr_set[device]) {
+    cudaError_t e = cudaFuncSetAttribute((const void*)slim_values_tc2_kernel<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)Pv2<NB>::SMEM);
+    if (e != cudaSuccess) return e;
+    if (device >= 0 && device < 64) attr_set[device] = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(128);
+  cfg.dynamicSmemBytes = Pv2<NB>::SMEM;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, slim_values_tc2_kernel<NB>, kmap, wmap, V, n, d, d_k, hp, status, cp);
+}
 
 }  // namespace
 
@@ -360,25 +397,14 @@ cudaError_t slim_launch_values(const slim_ctx* ctx, const void* K, int n, float*
     cudaError_t e = slim_tmap_encode_3d(&kmap, const_cast<void*>(K), dims, strides, box);
     if (e != cudaSuccess) return e;
     const int hp = d_k == 64 ? 2 : 1;
-    if (ctx->opt_prompt_pair && n > PV_ROWS) {           // CTA pairs over the prompt rows (grid.y even)
-      static bool attr2_set[64] = {};
-      if (ctx->device < 0 || ctx->device >= 64 || !attr2_set[ctx->device]) {
-        e = cudaFuncSetAttribute((const void*)slim_values_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PV2_SMEM);
-        if (e != cudaSuccess) return e;
-        if (ctx->device >= 0 && ctx->device < 64) attr2_set[ctx->device] = true;
-      }
-      memcpy(&wmap, ctx->wmap1, sizeof(wmap));
-      cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3(2 * (H / hp) * ((n + 2 * PV_ROWS - 1) / (2 * PV_ROWS)));
-      cfg.blockDim = dim3(128);
-      cfg.dynamicSmemBytes = PV2_SMEM;
-      cfg.stream = st;
-      cudaLaunchAttribute attr[1];                   // (the cluster shape (2, 1, 1) is a compile-time property of the kernel)
-      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-      attr[0].val.programmaticStreamSerializationAllowed = 1;
-      cfg.attrs = attr; cfg.numAttrs = 1;
-      e = cudaLaunchKernelEx(&cfg, slim_values_tc2_kernel, kmap, wmap, V, n, d, d_k, hp, ctx->status, cp);
-      return e;
+    if (ctx->opt_prompt_pair && n > PV_ROWS) {           // CTA pairs over the prompt rows
+      // 256-column pair tiles where a tile is two whole 128-column groups (d_k = 128 or 64) and the groups pair up
+      const bool wide = ctx->opt_prompt_pair >= 2 && hp * d_k == 128 && (H / hp) % 2 == 0;
+      memcpy(&wmap, wide ? ctx->wmap : ctx->wmap1, sizeof(wmap));
+      const int groups = wide ? H / hp / 2 : H / hp;
+      const dim3 grid(2 * groups * ((n + 2 * PV_ROWS - 1) / (2 * PV_ROWS)));
+      return wide ? launch_pair<2>(ctx->device, grid, st, kmap, wmap, V, n, d, d_k, hp, ctx->status, cp)
+                  : launch_pair<1>(ctx->device, grid, st, kmap, wmap, V, n, d, d_k, hp, ctx->status, cp);
     }
     memcpy(&wmap, ctx->wmap, sizeof(wmap));
     return slim_launch_pdl(slim_values_tc_kernel, dim3(H / hp, (n + PV_ROWS - 1) / PV_ROWS), dim3(128), PV_SMEM, st, kmap, wmap, V, n,

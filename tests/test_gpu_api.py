@@ -327,7 +327,8 @@ def test_nonsquare_weights_right_inverse_matches_oracle_and_decodes():
         layer.close()
 
 
-@pytest.mark.parametrize("d,H,d_k,dtype", [(512, 4, 128, "bf16"), (1280, 20, 64, "bf16"), (384, 4, 96, "bf16"), (256, 4, 64, "f32"), (192, 2, 96, "bf16")])
+@pytest.mark.parametrize("d,H,d_k,dtype", [(512, 4, 128, "bf16"), (1280, 20, 64, "bf16"), (384, 4, 96, "bf16"), (256, 4, 64, "f32"), (192, 2, 96, "bf16"),
+                                          (384, 6, 64, "bf16"), (384, 3, 128, "bf16")])
 def test_prompt_phase_values_from_keys(d, H, d_k, dtype):
     # Fig. 3(a): V = K W_KV for a whole prompt; equals X W_V up to the rounding of the stored keys
     n = 300
