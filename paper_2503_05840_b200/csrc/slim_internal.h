@@ -91,12 +91,11 @@ struct slim_ctx {
   int opt_xscores_cuda;          // SLIM_XSCORES_CUDA: dense X-cache scores on CUDA cores
   int opt_k_evict;               // SLIM_TC_K_EVICT (0/1): L2 evict-first hint on the key loads (default on)
   long long* trace;              // device buffer set by slim_set_trace (trace builds)
-  int opt_prompt_pair;           // SLIM_PROMPT_PAIR: the prompt GEMM on CTA pairs (0 off, 1 256 x 128 tiles, 2 = default: 256 x 256 where the shape allows)
+  int opt_prompt_pair;           // SLIM_PROMPT_PAIR=0: the prompt GEMM never runs on CTA pairs (for comparisons)
   int opt_proj_ns;               // SLIM_PROJ_NS: stages of the projection kernel (0 = default)
   int opt_legacy_flow;           // SLIM_TC_LEGACY: append and exact redo as kernels of their own (for side-by-side timing)
   alignas(64) unsigned char wmap[128];   // CUtensorMap over W_KV for the projection kernel
   alignas(64) unsigned char wmap_h[128];    // the same over wkv_h
-  alignas(64) unsigned char wmap1[128];     // over W_KV (cache dtype) with a one-half box, for the prompt kernel's CTA pair
 };
 
 struct slim_cache {

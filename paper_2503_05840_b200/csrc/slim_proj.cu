@@ -448,10 +448,6 @@ cudaError_t slim_proj_make_wmap(slim_ctx* ctx) {
   // (the float16 copy is described as a 16-bit type of the same size: the copy engine only moves bits)
   cudaError_t e = slim_tmap_encode_3d(ctx->wmap, ctx->wkv, dims, strides, box);
   if (e == cudaSuccess) e = slim_tmap_encode_3d(ctx->wmap_h, ctx->wkv_h, dims, strides, box);
-  if (e == cudaSuccess) {                      // one 64-column half of a tile: what a CTA of the prompt kernel's pair stages
-    unsigned int box1[3] = {64, PJ_ROWS, 1};
-    e = slim_tmap_encode_3d(ctx->wmap1, ctx->wkv, dims, strides, box1);
-  }
   if (e != cudaSuccess) return e;
   const ProjGeom g = make_proj_geom(d, H, d_k, 1, PJ_NS);      // the largest stage count a sweep may ask for
   return cudaFuncSetAttribute((const void*)slim_proj_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

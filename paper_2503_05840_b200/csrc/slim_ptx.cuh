@@ -141,6 +141,11 @@ __device__ __forceinline__ void umma2_commit_pair(uint32_t bar) {   // arrives o
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                ::"r"(bar), "h"((unsigned short)3) : "memory");
 }
+// arrival on a barrier of any CTA of the cluster (address from mapa); orders this thread's earlier reads and
+// writes before it at cluster scope
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
 // TMA load of a CTA pair: the destination is this CTA's shared memory, the bytes are counted on an mbarrier
 // that may live in either CTA of the pair (cluster_bar: an address from mapa), so the pair's MMA issuer
 // waits on one barrier for both CTAs' halves of a stage.
