@@ -301,7 +301,7 @@ def run_prompt(args):
     cfg = synth.CONFIGS[args.config]
     dev = "cuda:0"
     torch.cuda.set_device(0)
-    n = min(cfg.batch * cfg.context, 262144)
+    n = min((args.batch or cfg.batch) * cfg.context, 262144)
     ctx = B.slim_create(cfg.d, cfg.H, cfg.d_k, 0.0, B.SLIM_BF16 if cfg.dtype == "bf16" else B.SLIM_F32)
     B.slim_set_wkv(ctx, np.random.default_rng(0).standard_normal((cfg.d, cfg.d)) / np.sqrt(cfg.d))
     tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
