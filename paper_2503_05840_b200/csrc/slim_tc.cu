@@ -73,7 +73,9 @@ using namespace slim_ptx;
 // per-tile loop.  Slots: 0 producer at the top of its loop, 1 producer when the stage is free (load issued),
 // 2 score warp 0 when the keys have landed, 3 when its probabilities are computed, 4 when the P stage is
 // free, 5 when it has shipped and released, 6 MMA thread when the tile's probabilities are complete,
-// 7 when its MMAs and the commit are issued.
+// 7 when its MMAs and the commit are issued.  The last tile index (SLIM_TRACE_TILES - 1, beyond any worker's
+// tile count at the traced shapes) holds whole-kernel marks of thread 0: slot 0 kernel entry, 1 set-up done,
+// 2 / 3 begin / end of the drain of its last unit's accumulator, 4 kernel exit.
 #ifdef SLIM_TC_TRACE
 #define TC_TRACE(slot, tile_no)                                                                              \
   do {                                                                                                       \
@@ -83,6 +85,7 @@ using namespace slim_ptx;
 #else
 #define TC_TRACE(slot, tile_no) do {} while (0)
 #endif
+#define TC_TRACE_MARK(slot) do { if (threadIdx.x == 0) TC_TRACE(slot, SLIM_TRACE_TILES - 1); } while (0)
 
 constexpr int TC_P_BYTES = 1024;         // [32 heads][16 rows] bf16
 constexpr int TC_MAX_NS = 8;             // K stages
@@ -158,6 +161,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   const uint32_t rank = cluster_ctarank();
   const int w = blockIdx.x / CL;                  // worker = cluster index
   const int producer_warp = g.nswl, mma_warp = g.nswl + 1;
+  TC_TRACE_MARK(0);
 
   // ---- set-up -------------------------------------------------------------------
   const int nepi = (g.nswl / 4) * 4;              // warps that drain the accumulator at a unit's end
@@ -194,6 +198,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
   const int g_begin = in_range ? slim_worker_start(sc, w) : 0;
   const int g_end = in_range ? slim_worker_start(sc, w + 1) : 0;
   const bool have_work = g_end > g_begin;
+  TC_TRACE_MARK(1);
 
   if (have_work) {
     if (warp < g.nswl) {
@@ -465,6 +470,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           ok = mbar_wait<false>(bar_u_full, uc & 1, s_abort, p.status);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
+          TC_TRACE_MARK(2);
           tc_fence_after();
           const int q = warp & 3, cstep = nepi >> 2;
           const uint32_t tlane = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -490,6 +496,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_u_empty);
+          TC_TRACE_MARK(3);
         }
         gg = seg_end;
         it_base += ntile;
@@ -636,6 +643,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)g.tmem_cols);
   }
+  TC_TRACE_MARK(4);
 }
 
 // ------------------------------------------------------------------ host side
