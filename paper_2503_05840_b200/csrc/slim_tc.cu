@@ -85,6 +85,10 @@ using namespace slim_ptx;
 #else
 #define TC_TRACE(slot, tile_no) do {} while (0)
 #endif
+// the score warp whose per-tile points are recorded (-DSLIM_TC_TRACE_WARP=n to look at another one)
+#ifndef SLIM_TC_TRACE_WARP
+#define SLIM_TC_TRACE_WARP 0
+#endif
 #define TC_TRACE_MARK(slot) do { if (threadIdx.x == 0) TC_TRACE(slot, SLIM_TRACE_TILES - 1); } while (0)
 
 constexpr int TC_P_BYTES = 1024;         // [32 heads][16 rows] bf16
@@ -305,7 +309,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             // a wait that ran out is acted on after the vote below (until then the lanes only
             // touch their own registers and this CTA's shared memory)
             ok = mbar_wait<false>(bar_k_full + 8 * st, kph, s_abort, p.status);
-            if (warp == 0 && lane == 0) TC_TRACE(2, it_own);
+            if (warp == SLIM_TC_TRACE_WARP && lane == 0) TC_TRACE(2, it_own);
             // rows at or beyond the sequence end must not reach the tensor core (0 x NaN)
             if (t0 + SLIM_TT > len) {
               const int nz = len - t0;
@@ -392,12 +396,12 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             const float pf = valid ? ex2_approx(x) : 0.f;
             const __nv_bfloat16 pb = __float2bfloat16_rn(pf);
             if ((jl % DUP) == 0) lsum += __bfloat162float(pb);
-            if (warp == 0 && lane == 0) TC_TRACE(3, it_own);
+            if (warp == SLIM_TC_TRACE_WARP && lane == 0) TC_TRACE(3, it_own);
             // the P stage is free once the MMAs of tile it - ns are done in both CTAs
             ok = mbar_wait<false>(bar_p_empty + 8 * (PAIR ? st >> 1 : st), kph ^ 1, s_abort, p.status) && ok;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            if (warp == 0 && lane == 0) TC_TRACE(4, it_own);
+            if (warp == SLIM_TC_TRACE_WARP && lane == 0) TC_TRACE(4, it_own);
             {
               // stage this warp's probabilities in the K-major order of the P tile, then ship
               // them in 16-byte pieces (8 rows of one head) to both CTAs
@@ -421,7 +425,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
             if (lane == 0) {
               mbar_arrive_expect_tx(bar_p_full + 8 * st, p_bytes_w);
               mbar_arrive(bar_k_empty + 8 * st);
-              if (warp == 0) TC_TRACE(5, it_own);
+              if (warp == SLIM_TC_TRACE_WARP) TC_TRACE(5, it_own);
             }
             if (ROPE && active && SETS == 2) {
               // the other set's tile: RT row steps of RP rows keep the stepped rotation in step

@@ -32,10 +32,11 @@ def main(argv=None) -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--steps", type=int, default=4)
+    ap.add_argument("--library", default="", help="an instrumented library built by hand (e.g. with -DSLIM_TC_TRACE_WARP=7)")
     args = ap.parse_args(argv)
 
     from . import build as _build
-    os.environ["SLIM_LIBRARY"] = _build.build(trace=True)
+    os.environ["SLIM_LIBRARY"] = args.library or _build.build(trace=True)
     import torch
     from . import binding as B
     from . import synth
