@@ -234,11 +234,18 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
       const uint32_t p_bytes_w = (uint32_t)(CL * 32 * nvalid);
       // e^{i RP theta}: one step of this thread's rows
       f32x2 stc[4], sts[4], stn[4];
+      // Three-term form of the same step, Q(n+1) = 2 cos(RP theta) Q(n) - Q(n-1), used for a tile's rows from
+      // the third on: one packed FMA per register instead of two packed operations.  The subtraction is
+      // folded into the signs: Z(n) = sg(n) Q(n) with sg = + + - - + + ..., Z(n+1) = a(n) Z(n) + Z(n-1),
+      // a(n) = -/+ 2 cos alternating; a row's sum takes sg(n) back, and sg(RT) = + (RT a multiple of 4).
+      constexpr bool CHEB = ROPE && RT % 4 == 0;
+      f32x2 tcp[4], tcn[4];
       if (ROPE && active) {
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
           const float2 a = p.rope_off[RP * PAIRS + 8 * jl + 2 * x], b = p.rope_off[RP * PAIRS + 8 * jl + 2 * x + 1];
           stc[x] = pack2(a.x, b.x); sts[x] = pack2(a.y, b.y); stn[x] = pack2(-a.y, -b.y);
+          if (CHEB) { tcp[x] = pack2(2.f * a.x, 2.f * b.x); tcn[x] = pack2(-2.f * a.x, -2.f * b.x); }
         }
       }
 
@@ -328,6 +335,7 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
 #pragma unroll
             for (int i = 0; i < RT; ++i) v[i] = 0.f;
             if (active) {
+              f32x2 Pa[4], Pb[4];                        // Z(n-1) of the three-term step
 #pragma unroll
               for (int i = 0; i < RT; ++i) {
                 const int row = row_of(i);
@@ -340,13 +348,24 @@ slim_tc_kernel(const __grid_constant__ CUtensorMap tmap, const SlimDecodeParams 
                 acc0 = fma2(unpack2(ka.y), Qa[1], acc0); acc1 = fma2(unpack2(kb.y), Qb[1], acc1);
                 acc0 = fma2(unpack2(ka.z), Qa[2], acc0); acc1 = fma2(unpack2(kb.z), Qb[2], acc1);
                 acc0 = fma2(unpack2(ka.w), Qa[3], acc0); acc1 = fma2(unpack2(kb.w), Qb[3], acc1);
-                v[i] = sum2(add2(acc0, acc1));
+                v[i] = (CHEB && (i & 2)) ? -sum2(add2(acc0, acc1)) : sum2(add2(acc0, acc1));
                 if (ROPE) {
+                  if (!CHEB || i == 0) {
 #pragma unroll
-                  for (int x = 0; x < 4; ++x) {
-                    const f32x2 na = fma2(Qb[x], stn[x], mul2(Qa[x], stc[x]));
-                    Qb[x] = fma2(Qa[x], sts[x], mul2(Qb[x], stc[x]));
-                    Qa[x] = na;
+                    for (int x = 0; x < 4; ++x) {
+                      if (CHEB) { Pa[x] = Qa[x]; Pb[x] = Qb[x]; }
+                      const f32x2 na = fma2(Qb[x], stn[x], mul2(Qa[x], stc[x]));
+                      Qb[x] = fma2(Qa[x], sts[x], mul2(Qb[x], stc[x]));
+                      Qa[x] = na;
+                    }
+                  } else {
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {
+                      const f32x2 tw = (i & 1) ? tcn[x] : tcp[x];
+                      const f32x2 na = fma2(tw, Qa[x], Pa[x]), nb = fma2(tw, Qb[x], Pb[x]);
+                      Pa[x] = Qa[x]; Pb[x] = Qb[x];
+                      Qa[x] = na; Qb[x] = nb;
+                    }
                   }
                 }
               }
