@@ -11,7 +11,7 @@ leaving them out changes a head's output by at most eps times the largest value 
                 feeds whole tiles to the tensor core could leave out)
 `sharp` multiplies the query (1 = the workload's recipe; larger = more peaked softmax).
 
-    python -m oracle.sparsity_survey            # prints the table quoted in the design doc
+    python -m oracle.sparsity_survey            # prints one line per workload shape and query sharpness
 """
 from __future__ import annotations
 
