@@ -46,7 +46,7 @@ def parse():
     ap.add_argument("--variant", default="kcache", choices=["kcache", "xcache", "prompt", "fp8"],
                     help="xcache: the X/E-cache scheme, one cache shared by all layers (configs without RoPE); "
                          "prompt: the prompt-phase V = K W_KV of the config's shape; "
-                         "fp8: the K-cache path with an 8-bit cache (CUDA-core kernels)")
+                         "fp8: the K-cache path with an 8-bit cache")
     ap.add_argument("--paged", type=int, default=0, help="K-cache in a shuffled pool of pages of this many rows (0 = contiguous)")
     return ap.parse_args()
 
@@ -661,7 +661,7 @@ def main():
             "metric": "decode_attention_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
-            "dtype": {"bf16": "bf16", "f32": "f32", "fp8": "f32 arithmetic on an e4m3 cache (bf16 queries and W_KV)"}[cfg.dtype],
+            "dtype": {"bf16": "bf16", "f32": "f32", "fp8": "e4m3 cache decoded exactly to bf16, then the bf16 path (bf16 queries and W_KV)"}[cfg.dtype],
             "data": "synthetic",
             "config": {"workload": f"config{args.config}:{cfg.name}" + (" (8-bit K-cache)" if fp8 else ""), "layers": layers_n, "batch_per_gpu": cfg.batch,
                        "global_batch": tokens, "context": cfg.context, "sum_lengths": int(lengths.sum()),
@@ -676,7 +676,10 @@ def main():
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": ncu_traffic(args.config) if not fp8 else None, "peak_kind": peak_kind,
                          "kernel": "main decode kernel (per layer launch)" if not fp8 else
-                                   "score + accumulation kernels (CUDA cores; the 8-bit keys are read twice per layer)",
+                                   ("decode of the 8-bit rows into the bf16 scratch + main decode kernel on the scratch "
+                                    "(1 + 2 + 2 bytes of DRAM traffic per key element)"
+                                    if layers[0].query(B.SLIM_Q_PATH_IN_USE) == 2 else
+                                    "score + accumulation kernels (CUDA cores; the 8-bit keys are read twice per layer)"),
                          "main_ms": main_ms, "tail_ms": tail_ms, "bytes_per_launch": k_bytes_layer,
                          "timing": "CUDA events recorded by the library inside a sustained loop of the same step "
                                    "(last step, mean over layers); that loop ran at %.4f ms per step" % ms_prof},

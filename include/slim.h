@@ -115,8 +115,11 @@ slim_status slim_set_wkv(slim_ctx* ctx, const void* W_KV, int host_dtype);
  * [batch][t_cap][H]: the stored key is code * 2^exponent, the exponent being the smallest one
  * for which the head slice of the row fits the E4M3 range (|value| <= 448), codes rounded to
  * nearest even.  Such a cache is filled only through slim_append_k / slim_decode_step /
- * slim_prefill (which quantise bf16 rows); it is contiguous (no paged variant), has no X-cache
- * mode, and is read by the CUDA-core kernels.                                            */
+ * slim_prefill (which quantise bf16 rows); it is contiguous (no paged variant) and has no X-cache
+ * mode.  Where the shape fits the tensor-core kernels, slim_decode first decodes the live rows
+ * exactly into a bf16 copy inside the workspace (slim_workspace_bytes then includes
+ * 2 * batch * t_cap * d bytes for it) and runs the bf16 kernels on the copy; otherwise, and with
+ * SLIM_PATH_GENERIC, the CUDA-core kernels read the codes directly.                       */
 size_t slim_cache_bytes(const slim_ctx* ctx, int batch, int t_cap);
 size_t slim_workspace_bytes(const slim_ctx* ctx, int batch, int t_cap);
 

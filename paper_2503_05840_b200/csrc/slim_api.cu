@@ -24,7 +24,7 @@ inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 inline size_t esize(int dtype) { return dtype == SLIM_BF16 ? 2 : 4; }
 
 struct WsLayout {
-  size_t part_u, part_m, part_l, flags, o_part, scores, u_tiled, u32, su, total;
+  size_t part_u, part_m, part_l, flags, o_part, scores, u_tiled, u32, su, kscratch, total;
   int units;
 };
 
@@ -41,6 +41,8 @@ WsLayout ws_layout(const slim_ctx* ctx, int batch, int t_cap) {
   L.u_tiled = off; off = align256(off + (ctx->proj_ok ? slim_proj_u_bytes(ctx->d, ctx->H, batch) : 0));   // tensor-core tail only
   L.u32 = off; off = align256(off + (ctx->proj_ok ? sizeof(float) * (size_t)batch * ctx->H * ctx->d : 0));
   L.su = off; off = align256(off + (ctx->proj_ok ? sizeof(float) * (size_t)((batch + 15) / 16) * 16 * ctx->H : 0));
+  // 8-bit cache on the tensor-core path: one layer's keys as bf16 (the cache itself stays in 8 bits)
+  L.kscratch = off; off = align256(off + ((ctx->kdtype == SLIM_FP8 && ctx->tc_ok) ? 2 * (size_t)batch * t_cap * ctx->d : 0));
   L.total = off;
   return L;
 }
@@ -228,7 +230,7 @@ slim_status create_impl(slim_ctx** out, int d, int H, int d_k, double rope_theta
   }
   c->tc_ok = 0;
   for (int cl = 1; cl <= 2; ++cl) {
-    c->tc_workers[cl - 1] = (prop.major == 10 && kdtype != SLIM_FP8 && slim_tc_shape_ok(d, H, d_k, dtype, rope_theta != 0.0, cl)) ? slim_tc_workers(c, cl) : 0;
+    c->tc_workers[cl - 1] = (prop.major == 10 && slim_tc_shape_ok(d, H, d_k, dtype, rope_theta != 0.0, cl)) ? slim_tc_workers(c, cl) : 0;
     if (c->tc_workers[cl - 1] < 0) c->tc_workers[cl - 1] = 0;
     if (c->tc_workers[cl - 1] > 0) c->tc_ok = 1;
   }
@@ -397,7 +399,7 @@ slim_status slim_cache_create(slim_ctx* ctx, slim_cache** out, void* k_storage, 
   c->total_rows = (long long)batch * t_cap;
   for (int cl = 1; cl <= 2; ++cl) {
     c->has_tmap[cl - 1] = 0;
-    if (ctx->tc_workers[cl - 1] > 0) {
+    if (ctx->tc_workers[cl - 1] > 0 && ctx->kdtype != SLIM_FP8) {       // (an 8-bit cache is read through a bf16 scratch)
       if (slim_tc_make_tmap(ctx, c, cl) == cudaSuccess) c->has_tmap[cl - 1] = 1;
       else cudaGetLastError();
     }
@@ -474,10 +476,11 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   if (path < 0) return SLIM_ERR_UNSUPPORTED;
   // CTAs per worker: the pair when the kernel computes the scores, the lone CTA with external scores
   int cl = 0;
+  const bool fp8_tc = path == SLIM_PATH_TC && ctx->kdtype == SLIM_FP8;      // decoded into a bf16 scratch first
   if (path == SLIM_PATH_TC) {
     const int pref = xcache ? 1 : 2, other = 3 - pref;
-    if (ctx->tc_workers[pref - 1] > 0 && cache->has_tmap[pref - 1]) cl = pref;
-    else if (ctx->tc_workers[other - 1] > 0 && cache->has_tmap[other - 1]) cl = other;
+    if (ctx->tc_workers[pref - 1] > 0 && (fp8_tc || cache->has_tmap[pref - 1])) cl = pref;
+    else if (ctx->tc_workers[other - 1] > 0 && (fp8_tc || cache->has_tmap[other - 1])) cl = other;
   }
   if (path == SLIM_PATH_TC && cl == 0) {
     if (ctx->path_req == SLIM_PATH_TC) return SLIM_ERR_UNSUPPORTED;
@@ -510,7 +513,7 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   // K-cache path on the tensor cores: the decode kernel writes the newest key rows itself, and a sequence
   // with a flagged unit is recomputed by the combine kernel (no append kernel, no redo kernel)
   const bool tc_kcache = !xcache && path == SLIM_PATH_TC && !ctx->opt_legacy_flow;
-  p.k_new = tc_kcache ? k_new : nullptr;
+  p.k_new = (tc_kcache && !fp8_tc) ? k_new : nullptr;        // (new rows of an 8-bit cache go through the quantising append)
   p.redo_in_combine = (tc_kcache && ctx->proj_ok && !part) ? 1 : 0;
   p.pos_tiles = part ? part->first_tile : nullptr;
   p.q_pos = part ? part->q_pos : nullptr;
@@ -525,6 +528,24 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
   }
   if (ctx->prof_on) cudaEventRecord(ctx->prof_ev[0], st);
   cudaError_t e;
+  slim_cache view;                                   // what the tensor-core kernel reads when the cache is 8-bit
+  const slim_cache* tc_cache = cache;
+  if (fp8_tc) {
+    // 8-bit cache on the tensor cores: decode the live rows into the bf16 scratch of the workspace and run the
+    // bf16 kernels on that (contiguous) copy; codes x 2^exponent are exact in bf16, so the result is the one
+    // the CUDA-core kernels get from the codes, up to the rounding of P
+    void* scratch = ws + L.kscratch;
+    if (slim_launch_dequant(ctx, cache, lengths, scratch, st) != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
+    ++launches;
+    view = *cache;
+    view.k = scratch; view.k_exp = nullptr; view.block_table = nullptr;
+    view.total_rows = (long long)cache->batch * cache->t_cap;
+    view.has_tmap[0] = view.has_tmap[1] = 0;
+    if (slim_tc_make_tmap(ctx, &view, cl) != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
+    view.has_tmap[cl - 1] = 1;
+    tc_cache = &view;
+    p.k = scratch; p.kdtype = SLIM_BF16; p.k_exp = nullptr;
+  }
   float* scores = reinterpret_cast<float*>(ws + L.scores);
   if (xcache) {
     // dense scores first; then P.X on the tensor cores where the shape allows it (an argument that
@@ -547,7 +568,7 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
       }
     }
   } else if (path == SLIM_PATH_TC) {
-    e = slim_launch_tc(ctx, cache, p, st);
+    e = slim_launch_tc(ctx, tc_cache, p, st);
     ++launches;
     if (e == cudaSuccess && !p.redo_in_combine) { e = slim_launch_exact_flagged(ctx, p, st); ++launches; }
   } else {

@@ -125,6 +125,9 @@ cudaError_t slim_launch_accum(const slim_ctx* ctx, const SlimDecodeParams& p, co
 cudaError_t slim_launch_exact_flagged(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st);
 cudaError_t slim_launch_tail(const slim_ctx* ctx, const SlimDecodeParams& p, cudaStream_t st);
 // pos_is_length = 1: positions[b] holds the length AFTER the append (row positions[b]-1 is written; 0 writes nothing)
+// 8-bit cache on the tensor-core path: rows [0, lengths[b]) of every sequence are decoded (code * 2^exponent,
+// exact in bf16) into `scratch`, a contiguous bf16 cache [batch][t_cap][d] that the bf16 kernels then read
+cudaError_t slim_launch_dequant(const slim_ctx* ctx, const slim_cache* c, const int32_t* lengths, void* scratch, cudaStream_t st);
 cudaError_t slim_launch_append(const slim_ctx* ctx, const slim_cache* c, const void* k_new,
                                const int32_t* positions, int n_new, int pos_is_length, cudaStream_t st);
 // fp64 solve W_K X = W_V on the device; A and B are device row-major [n][n]

@@ -212,7 +212,50 @@ slim_append_fp8_kernel(unsigned char* __restrict__ codes, signed char* __restric
   }
 }
 
+// 8-bit cache -> bf16 rows for the tensor-core kernels: stored key = code * 2^exponent, one exponent per (row,
+// head).  An E4M3 code has four significant bits, so the product is exact in bf16 (as long as the sum of the two
+// exponents stays in bf16's range, which the quantiser's clamp of the exponent together with the code's own range
+// leaves a wide margin for).  A thread decodes 16 codes of one head (d_k is a multiple of 16); a CTA takes
+// DQ_ROWS rows of one sequence; rows at or beyond lengths[b] are left as they are (the decode kernel masks them).
+constexpr int DQ_ROWS = 8;
+__global__ void __launch_bounds__(256)
+slim_dequant_kernel(const unsigned char* __restrict__ codes, const signed char* __restrict__ exps, __nv_bfloat16* __restrict__ out,
+                    const int32_t* __restrict__ lengths, int d, int H, int d_k, int t_cap) {
+  slim_pdl_trigger();
+  slim_pdl_wait();
+  const int b = blockIdx.y, t0 = blockIdx.x * DQ_ROWS;
+  const int len = min(max(lengths[b], 0), t_cap);
+  if (t0 >= len) return;
+  const int vec_per_row = d / 16;
+  const int n = min(DQ_ROWS, len - t0) * vec_per_row;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const int r = i / vec_per_row, v = i - r * vec_per_row;
+    const size_t row = (size_t)b * t_cap + t0 + r;
+    const uint4 c = __ldcs(reinterpret_cast<const uint4*>(codes + row * d) + v);
+    const float scale = __int_as_float(((int)__ldg(exps + row * H + (v * 16) / d_k) + 127) << 23);
+    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+    uint32_t o[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const uint32_t pair = (w[k >> 1] >> (16 * (k & 1))) & 0xffffu;                  // two codes
+      const __half2_raw h2 = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)pair, __NV_E4M3);
+      const float2 f = __half22float2(__half2(h2));
+      const __nv_bfloat162 bb = __floats2bfloat162_rn(f.x * scale, f.y * scale);
+      o[k] = *reinterpret_cast<const uint32_t*>(&bb);
+    }
+    uint4* dst = reinterpret_cast<uint4*>(out + row * d) + 2 * v;
+    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+  }
+}
+
 }  // namespace
+
+cudaError_t slim_launch_dequant(const slim_ctx* ctx, const slim_cache* c, const int32_t* lengths, void* scratch, cudaStream_t st) {
+  return slim_launch_pdl(slim_dequant_kernel, dim3((c->t_cap + DQ_ROWS - 1) / DQ_ROWS, c->batch), dim3(256), 0, st,
+                         (const unsigned char*)c->k, (const signed char*)c->k_exp, (__nv_bfloat16*)scratch, lengths, ctx->d, ctx->H,
+                         ctx->d_k, c->t_cap);
+}
 
 size_t slim_tail_opart_floats(int d, int e, int batch) {
   const int slices = (d + JR - 1) / JR;

@@ -49,7 +49,12 @@ def test_fp8_cache_codes_bitwise_and_decode_matches_oracle(d, H, d_k, theta):
                 k_new[b] = Kd[b, lengths[b] - 1]
         got = layer.decode_step(q, k_new, ld).cpu().numpy().astype(np.float64)
         assert layer.device_status() == B.SLIM_OK
-        assert layer.query(B.SLIM_Q_PATH_IN_USE) == B.SLIM_PATH_GENERIC
+        # shapes the tensor-core kernels take are decoded into a bf16 scratch and run there; the others stay on CUDA cores
+        probe = B.slim_create(d, H, d_k, theta, B.SLIM_BF16)       # what a bf16 cache of this shape would run on
+        B.slim_set_wkv(probe, np.eye(d))
+        tc_shape = B.slim_query(probe, B.SLIM_Q_PATH_IN_USE) == B.SLIM_PATH_TC
+        B.slim_destroy(probe)
+        assert layer.query(B.SLIM_Q_PATH_IN_USE) == (B.SLIM_PATH_TC if tc_shape else B.SLIM_PATH_GENERIC)
         codes, exps = _stored(layer, batch, t_cap, d, H)
         for b in range(batch):
             n = int(lengths[b])
@@ -65,12 +70,25 @@ def test_fp8_cache_codes_bitwise_and_decode_matches_oracle(d, H, d_k, theta):
         # plain decode over the stored keys gives the same bits as the step call did
         again = layer.decode(q, ld).cpu().numpy().astype(np.float64)
         assert np.array_equal(again, got)
+        if tc_shape:
+            # the CUDA-core kernels read the same codes directly: same tolerance against the oracle
+            layer.set_path(B.SLIM_PATH_GENERIC)
+            gen = layer.decode(q, ld).cpu().numpy().astype(np.float64)
+            assert layer.device_status() == B.SLIM_OK
+            for b in range(batch):
+                n = int(lengths[b])
+                if n == 0:
+                    assert np.all(gen[b] == 0)
+                    continue
+                _, _, deq = so.quantize_keys_e4m3(K[b, :n], H)
+                e = so.err_rms_norm(gen[b], so.oracle_slim(L.q[b], deq, W_KV, H, theta))
+                assert e <= 2e-2, f"CUDA-core path, sequence {b}: {e:.3e}"
     finally:
         layer.close()
 
 
 def test_fp8_cache_refuses_what_it_does_not_support():
-    ctx = B.slim_create(256, 4, 64, 0.0, B.SLIM_FP8)
+    ctx = B.slim_create(256, 16, 16, 0.0, B.SLIM_FP8)          # (d_k = 16: no tensor-core kernel for this shape)
     try:
         with pytest.raises(B.SlimError) as ei:
             B.slim_xcache_set_weights(ctx, np.eye(256), np.eye(256))
