@@ -193,6 +193,7 @@ slim_status create_impl(slim_ctx** out, int d, int H, int d_k, double rope_theta
     c->opt_xscores_cuda = getenv("SLIM_XSCORES_CUDA") ? 1 : 0;
     c->opt_legacy_flow = getenv("SLIM_TC_LEGACY") ? 1 : 0;
     c->opt_proj_ns = (e = getenv("SLIM_PROJ_NS")) ? atoi(e) : 0;
+    c->opt_tail_fused = (e = getenv("SLIM_TAIL_FUSED")) ? atoi(e) : 1;
     c->opt_prompt_pair = ((e = getenv("SLIM_PROMPT_PAIR")) && atoi(e) == 0) ? 0 : 1;
     c->opt_k_evict = (e = getenv("SLIM_TC_K_EVICT")) ? atoi(e) : 1;      // measured side by side: ~1 % per step
   }
@@ -583,7 +584,7 @@ slim_status decode_impl(slim_ctx* ctx, const void* q, const slim_cache* cache, c
     if (ctx->proj_ok) {
       e = slim_launch_proj(ctx, p, reinterpret_cast<unsigned char*>(ws + L.u_tiled), reinterpret_cast<float*>(ws + L.u32),
                            reinterpret_cast<float*>(ws + L.su), st);
-      launches += 2 + slim_proj_needs_convert(ctx, p.batch);      // combine (, operand conversion), projection
+      launches += slim_proj_launch_count(ctx, p);                 // combine (, operand conversion), projection -- or the fused kernel
     } else {
       e = slim_launch_tail(ctx, p, st);
       launches += 2;                                 // combine + projection slices, slice sum

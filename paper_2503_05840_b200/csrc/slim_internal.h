@@ -91,6 +91,7 @@ struct slim_ctx {
   int opt_xscores_cuda;          // SLIM_XSCORES_CUDA: dense X-cache scores on CUDA cores
   int opt_k_evict;               // SLIM_TC_K_EVICT (0/1): L2 evict-first hint on the key loads (default on)
   long long* trace;              // device buffer set by slim_set_trace (trace builds)
+  int opt_tail_fused;            // SLIM_TAIL_FUSED: combine + projection in one kernel: 0 never, 1 where it pays (default), 2 wherever possible
   int opt_prompt_pair;           // SLIM_PROMPT_PAIR=0: the prompt GEMM never runs on CTA pairs (for comparisons)
   int opt_proj_ns;               // SLIM_PROJ_NS: stages of the projection kernel (0 = default)
   int opt_legacy_flow;           // SLIM_TC_LEGACY: append and exact redo as kernels of their own (for side-by-side timing)
@@ -157,6 +158,7 @@ cudaError_t slim_tmap_encode_3d(void* out_map, void* base, const unsigned long l
 int    slim_proj_shape_ok(int d, int H, int d_k, int dtype);
 int    slim_proj_jsplit(int d);
 int    slim_proj_needs_convert(const slim_ctx* ctx, int batch);      // 1: the combine writes float rows and a conversion kernel follows
+int    slim_proj_launch_count(const slim_ctx* ctx, const SlimDecodeParams& p);   // kernels slim_launch_proj enqueues
 size_t slim_proj_u_bytes(int d, int H, int batch);
 cudaError_t slim_proj_make_wmap(slim_ctx* ctx);
 // u32: [batch][H][d] float scratch, su: [16 ceil(batch / 16)][H] float scales of the operand rows

@@ -398,6 +398,291 @@ slim_proj_tc_kernel(const __grid_constant__ CUtensorMap wmap, const float* __res
   }
 }
 
+// Combine and projection in one kernel.  The CTA of (head group, row slice js of W_KV,h, 16-sequence group)
+// needs exactly the columns [row0, row0 + ncols) of u[b][h][:] for its 16 sequences, and no other CTA needs
+// them: it forms them itself from the context-split partials (the weights, the sums, the scaled float16
+// (hi, lo) pair written straight into the operand layout in shared memory) while the first stages of its
+// weight tiles, requested before the dependency wait, stream in.  The scale is per (sequence, head, slice) --
+// each slice's result is multiplied back before the slices are summed -- so nothing has to know a whole row.
+// Against the two kernels this saves a launch boundary, the trip of u through global memory, and the combine
+// kernel's own prologue.  A sequence with a flagged unit is recomputed exactly for the CTA's columns first.
+// PF_MAXR rounds of 256 (item, column group) pairs per CTA keep the combined values in registers between the
+// pass that finds the scales and the pass that stores the operands.
+constexpr int PF_THREADS = 256;
+constexpr int PF_MAXR = 8;                 // (the kernel is instantiated for 4 and 8 rounds)
+
+struct FusedSmem {              // offsets (bytes) behind the barriers; all 16-byte aligned
+  uint32_t prefix, info, amax, x, w, total;
+};
+__host__ __device__ inline FusedSmem fused_smem(const ProjGeom& g, int batch, int workers, int d_k) {
+  const uint32_t items = (uint32_t)(PJ_BG * g.hp);
+  FusedSmem f;
+  uint32_t off = 0;
+  f.prefix = off; off += (uint32_t)((sizeof(int) * (batch + 1) + 15) & ~15u);
+  f.info = off;   off += 16u * items;
+  f.amax = off;   off += (uint32_t)((4u * items + 15) & ~15u);
+  f.x = off;      off += (uint32_t)((sizeof(float) * (d_k + 2 * SLIM_TT + 4 + 36) + 15) & ~15u);
+  f.w = off;      off += (uint32_t)((sizeof(float) * items * workers + 15) & ~15u);
+  f.total = off;
+  return f;
+}
+
+template <int MAXR>
+__global__ void __launch_bounds__(PF_THREADS, 2)
+slim_tail_fused_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_constant__ SlimDecodeParams p,
+                       const float* __restrict__ hscale, float* __restrict__ u32, const ProjGeom g) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw_u32 = smem_u32(smem_raw);
+  const uint32_t base = (raw_u32 + 1023u) & ~1023u;
+  unsigned char* sm = smem_raw + (base - raw_u32);
+  const int NS = g.ns;
+  const uint32_t u_region = base + (uint32_t)NS * PJ_W_BYTES;              // all nst stages of u operand tiles
+  const uint32_t bars = u_region + (uint32_t)(g.nst * g.u_bytes);
+  const uint32_t bar_full = bars, bar_empty = bars + 8 * PJ_NS, bar_done = bars + 16 * PJ_NS;
+  unsigned char* misc = sm + (bar_done + 8 - base);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(misc);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(misc + 4);
+  const FusedSmem fs = fused_smem(g, p.batch, p.workers, p.d_k);
+  unsigned char* area = misc + 24;                            // (16-byte aligned: the barriers end 8 bytes short of it)
+  int* s_prefix = reinterpret_cast<int*>(area + fs.prefix);
+  int* s_info = reinterpret_cast<int*>(area + fs.info);                    // per item: first worker, unit count, flagged
+  int* s_amax = reinterpret_cast<int*>(area + fs.amax);                    // per item: bits of the largest magnitude
+  float* s_x = reinterpret_cast<float*>(area + fs.x);
+  float* s_w = reinterpret_cast<float*>(area + fs.w);                      // per item: [workers] weights
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int hg = blockIdx.x, js = blockIdx.y, bg = blockIdx.z;
+  const int d = p.d, H = p.H, hp = g.hp;
+  const uint32_t tmem_cols = (uint32_t)(32 * hp);
+  const int items = PJ_BG * hp;                               // (sequence, head of the group) pairs of this CTA
+
+  if (tid == 0) {
+    prefetch_tensormap(&wmap);
+    for (int i = 0; i < NS; ++i) { mbar_init(bar_full + 8 * i, 1); mbar_init(bar_empty + 8 * i, 1); }
+    mbar_init(bar_done, 1);
+    *s_abort = 0;
+    fence_mbar_init();
+  }
+  if (tid < items) s_amax[tid] = 0;
+  if (warp == 1) tmem_alloc(smem_u32(s_tmem), tmem_cols);
+  slim_pdl_trigger();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  const int row0 = js * g.nst * PJ_ROWS;                      // first row of W_KV,h = first column of u of this CTA
+  const int ncols = g.nst * PJ_ROWS;
+  const int npre = g.nst < NS ? g.nst : NS;
+  auto load_w = [&](uint32_t dst, uint32_t bar, int s) {
+    if (hp == 1) tma_load_3d(dst, &wmap, bar, 0, hg * d + row0 + s * PJ_ROWS, 0);
+    else         tma_load_3d(dst, &wmap, bar, 0, row0 + s * PJ_ROWS, 2 * hg);
+  };
+  // the weights do not depend on the kernels before this one: the first stages are requested now
+  if (warp == 0 && lane == 0) {
+    for (int s = 0; s < npre; ++s) {
+      mbar_arrive_expect_tx(bar_full + 8 * s, PJ_W_BYTES);
+      load_w(base + (uint32_t)s * PJ_W_BYTES, bar_full + 8 * s, s);
+    }
+  }
+  slim_pdl_wait();                                             // the partials come from the decode kernel
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && tid == 0) *p.any_flag = 0;
+
+  // ---- combine: units and weights of the CTA's (sequence, head) items ----
+  const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
+  {
+    // All items at once: LPI = 256 / items lanes (16 or 8, a power of two within a warp) share an item and take its
+    // units i = sub, sub + LPI, ...:  w_i = 2^(m_i - M) / sum_j 2^(m_j - M) l_j,  M = max_j (m_j + log2 l_j).
+    const int LPI = PF_THREADS / items, item = tid / LPI, sub = tid % LPI;
+    const int b = bg * PJ_BG + item / hp, h = hg * hp + item % hp;
+    float* sw = s_w + (size_t)item * p.workers;
+    int wlo = 0, wn = 0, flagged = 0;
+    if (b < p.batch && s_prefix[b + 1] > s_prefix[b]) {
+      wlo = slim_worker_of_tile(sc, s_prefix[b]);
+      wn = slim_worker_of_tile(sc, s_prefix[b + 1] - 1) - wlo + 1;
+      if (p.redo_in_combine)
+        for (int i = sub; i < 2 * wn; i += LPI) flagged |= p.unit_flags[2 * (wlo + b) + i];
+    }
+    float M = -INFINITY, m0 = 0.f, l0 = 0.f;                  // (m, l) of this lane's first unit stay in registers
+    for (int i = sub; i < wn; i += LPI) {
+      const size_t ui = (size_t)(wlo + b + i) * H + h;
+      const float mi = __ldcg(p.part_m + ui), li = __ldcg(p.part_l + ui);
+      if (i == sub) { m0 = mi; l0 = li; }
+      M = fmaxf(M, mi + log2f(li));
+    }
+    for (int o = LPI >> 1; o > 0; o >>= 1) {
+      M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+      flagged |= __shfl_xor_sync(0xffffffffu, flagged, o);
+    }
+    float L = 0.f;
+    for (int i = sub; i < wn; i += LPI) {
+      const size_t ui = (size_t)(wlo + b + i) * H + h;
+      const float mi = i == sub ? m0 : __ldcg(p.part_m + ui), li = i == sub ? l0 : __ldcg(p.part_l + ui);
+      const float wg = exp2f(mi - M);
+      sw[i] = wg;
+      L += wg * li;
+    }
+    for (int o = LPI >> 1; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+    const float inv = 1.f / L;
+    __syncwarp();
+    for (int i = sub; i < wn; i += LPI) sw[i] *= inv;
+    if (sub == 0) { s_info[4 * item] = wlo; s_info[4 * item + 1] = wn; s_info[4 * item + 2] = flagged != 0; }
+  }
+  __syncthreads();
+  // a sequence with a flagged unit: its columns are recomputed exactly into the float scratch first (rare)
+  for (int item = 0; item < items; ++item)
+    if (s_info[4 * item + 2]) slim_comb::exact_groups(p, u32, bg * PJ_BG + item / hp, hg * hp + item % hp, row0 / 8, ncols / 8, s_x);
+  __syncthreads();
+  const int gpi = ncols / 8;                                  // column groups per item
+  const int total = items * gpi, rounds = (total + PF_THREADS - 1) / PF_THREADS;
+  const size_t ustride = (size_t)H * d;
+  constexpr int UB = MAXR <= 4 ? 8 : 4;                       // units whose loads are in flight together
+  float acc[MAXR][8];
+#pragma unroll
+  for (int r = 0; r < MAXR; ++r) {
+#pragma unroll
+    for (int x = 0; x < 8; ++x) acc[r][x] = 0.f;
+    const int idx = r * PF_THREADS + tid;
+    if (r < rounds && idx < total) {
+      const int item = idx / gpi, jg = idx - item * gpi;
+      const int b = bg * PJ_BG + item / hp, h = hg * hp + item % hp, j0 = row0 + jg * 8;
+      const int wlo = s_info[4 * item], wn = s_info[4 * item + 1];
+      if (b < p.batch) {
+        if (s_info[4 * item + 2]) {
+          const float4* U = reinterpret_cast<const float4*>(u32 + ((size_t)b * H + h) * d + j0);
+          const float4 a = U[0], c = U[1];
+          acc[r][0] = a.x; acc[r][1] = a.y; acc[r][2] = a.z; acc[r][3] = a.w; acc[r][4] = c.x; acc[r][5] = c.y; acc[r][6] = c.z; acc[r][7] = c.w;
+        } else {
+          const float* sw = s_w + (size_t)item * p.workers;
+          const float* Ub = p.part_u + ((size_t)(wlo + b) * H + h) * d + j0;        // unit i lives H*d floats further
+          for (int i = 0; i < wn; i += UB) {         // UB units' loads in flight (a short last batch repeats its last unit with weight 0)
+            float4 a[UB], c[UB];
+#pragma unroll
+            for (int k = 0; k < UB; ++k) {
+              const float4* U = reinterpret_cast<const float4*>(Ub + (size_t)min(i + k, wn - 1) * ustride);
+              a[k] = __ldcs(U); c[k] = __ldcs(U + 1);
+            }
+#pragma unroll
+            for (int k = 0; k < UB; ++k) slim_comb::fma8(acc[r], i + k < wn ? sw[i + k] : 0.f, a[k], c[k]);
+          }
+        }
+        float mx = 0.f;
+#pragma unroll
+        for (int x = 0; x < 8; ++x) mx = fmaxf(mx, fabsf(acc[r][x]));
+        if (!(mx <= 3.0e38f)) mx = 3.4e38f;          // a NaN or an infinity: the row keeps scale 1 (row_scale)
+        atomicMax(s_amax + item, __float_as_int(mx));
+      }
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < MAXR; ++r) {
+    const int idx = r * PF_THREADS + tid;
+    if (r < rounds && idx < total) {
+      const int item = idx / gpi, jg = idx - item * gpi;
+      float inv, scale;
+      slim_comb::row_scale(__int_as_float(s_amax[item]), inv, scale);
+      uint32_t hi[4], lo[4];
+#pragma unroll
+      for (int x = 0; x < 4; ++x) {
+        const float v0 = acc[r][2 * x] * inv, v1 = acc[r][2 * x + 1] * inv;
+        const __half h0 = __float2half_rn(v0), h1 = __float2half_rn(v1);
+        const __half l0 = __float2half_rn(v0 - __half2float(h0)), l1 = __float2half_rn(v1 - __half2float(h1));
+        hi[x] = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
+        lo[x] = (uint32_t)__half_as_ushort(l0) | ((uint32_t)__half_as_ushort(l1) << 16);
+      }
+      const int n = item / hp, jl = jg * 8;                   // column within the CTA's slice
+      const uint32_t t = u_region + (uint32_t)(jl / 16) * (uint32_t)(1024 * hp) + (uint32_t)(item % hp) * 1024u;
+      sts128(t + slim_comb::u_offset(n, jl & 15), make_uint4(hi[0], hi[1], hi[2], hi[3]));
+      sts128(t + slim_comb::u_offset(PJ_BG + n, jl & 15), make_uint4(lo[0], lo[1], lo[2], lo[3]));
+    }
+  }
+  fence_proxy_async_smem();                                    // operand tiles: generic-proxy stores -> tensor-core reads
+  __syncthreads();
+
+  if (warp == 0 && lane == 0) {
+    // =========================== producer: the remaining weight stages ===========================
+    int s = npre;
+    bool ok = true;
+    for (; s < g.nst; ++s) {
+      const int st = s % NS;
+      ok = mbar_wait<false>(bar_empty + 8 * st, ((s / NS) & 1) ^ 1, s_abort, p.status);
+      if (!ok) break;
+      mbar_arrive_expect_tx(bar_full + 8 * st, PJ_W_BYTES);
+      load_w(base + (uint32_t)st * PJ_W_BYTES, bar_full + 8 * st, s);
+    }
+    if (!ok) {
+      // gave up: let the copies that were issued land before the CTA goes away
+      const int issued = s < NS ? s : NS;
+      for (int k = 0; k < issued; ++k) {
+        const int j = s - 1 - k, st = j % NS;
+        const unsigned long long t0 = globaltimer();
+        while (!mbar_try_wait(bar_full + 8 * st, (j / NS) & 1) && globaltimer() - t0 < SLIM_WAIT_NS) {}
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // =========================== MMA issuer ===========================
+    const uint32_t idesc = umma_idesc_f16((uint32_t)(32 * hp));        // both operands float16
+    bool ok = true;
+    for (int s = 0; s < g.nst && ok; ++s) {
+      const int st = s % NS;
+      ok = mbar_wait<false>(bar_full + 8 * st, (s / NS) & 1, s_abort, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t wbase = base + (uint32_t)st * PJ_W_BYTES, ubase = u_region + (uint32_t)(s * g.u_bytes);
+#pragma unroll
+      for (int kk = 0; kk < PJ_ROWS / 16; ++kk)
+        umma_bf16(tmem_base, desc_a(wbase + (uint32_t)kk * 2048u, PJ_ROWS * 128), desc_b(ubase + (uint32_t)(kk * 1024 * hp)),
+                  idesc, (s | kk) ? 1u : 0u);
+      umma_commit(bar_empty + 8 * st);
+      if (s == g.nst - 1) umma_commit(bar_done);
+    }
+  }
+  __syncwarp();
+  // =========================== epilogue (warps 0-3 hold the 128 accumulator rows) ===========================
+  const int m = (warp & 3) * 32 + lane;                       // accumulator row = TMEM lane
+  const int upper = hp == 2 ? ((warp & 3) >> 1) : 0;          // d_k = 64: lanes 64..127 hold the second head
+  const int head = hg * hp + upper;
+  const int c = hp == 2 ? (m & 63) : m;
+  if (warp < 4) {
+    bool ok = mbar_wait<false>(bar_done, 0, s_abort, p.status);
+    ok = __all_sync(0xffffffffu, ok);
+    uint32_t r[32];
+#pragma unroll
+    for (int n = 0; n < 32; ++n) r[n] = 0u;
+    if (ok) {
+      tc_fence_after();
+      tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(32 * upper), r);
+    }
+    // (hi + lo) columns of a sequence, times the scales taken out of the operands: 2^e of the item's slice and
+    // 2^-a of the head's weights
+    const float hs = hscale[head];
+    float* tile = reinterpret_cast<float*>(sm);
+#pragma unroll
+    for (int n = 0; n < PJ_BG; ++n) {
+      float inv, scale;
+      slim_comb::row_scale(__int_as_float(s_amax[n * hp + upper]), inv, scale);
+      tile[n * 128 + m] = (__uint_as_float(r[n]) + __uint_as_float(r[PJ_BG + n])) * (scale * hs);
+    }
+  }
+  cluster_sync_all();
+  if (warp < 4) {
+    const int n_lo = (js * PJ_BG) / g.jsplit, n_hi = ((js + 1) * PJ_BG) / g.jsplit;
+    for (int n = n_lo; n < n_hi; ++n) {
+      const int b = bg * PJ_BG + n;
+      float a = 0.f;
+      for (int sl = 0; sl < g.jsplit; ++sl) a += ld_cluster_f32(mapa(base + (uint32_t)(n * 128 + m) * 4u, (uint32_t)sl));
+      if (b < p.batch && c < p.d_k) p.o[(size_t)b * p.e + head * p.d_k + c] = p.lengths[b] > 0 ? a : 0.f;
+    }
+  }
+  cluster_sync_all();                                          // nobody leaves while its tile may still be read
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, tmem_cols);
+  }
+}
+
 ProjGeom make_proj_geom(int d, int H, int d_k, int batch, int ns_opt = 0) {
   ProjGeom g;
   g.hp = d_k == 64 ? 2 : 1;
@@ -416,6 +701,9 @@ ProjGeom make_proj_geom(int d, int H, int d_k, int batch, int ns_opt = 0) {
 }
 
 size_t proj_smem_bytes(const ProjGeom& g) { return 1024 + (size_t)g.ns * (PJ_W_BYTES + g.u_bytes) + 16 * PJ_NS + 8 + 16 + 64; }
+size_t fused_smem_bytes(const ProjGeom& g, int batch, int workers, int d_k) {
+  return 1024 + (size_t)g.ns * PJ_W_BYTES + (size_t)g.nst * g.u_bytes + 16 * PJ_NS + 8 + 24 + fused_smem(g, batch, workers, d_k).total + 64;
+}
 
 }  // namespace
 
@@ -465,9 +753,55 @@ static int combine_slices(const slim_ctx* ctx, int H, int batch, int d) {
 
 int slim_proj_needs_convert(const slim_ctx* ctx, int batch) { return combine_slices(ctx, ctx->H, batch, ctx->d) > 1 ? 1 : 0; }
 
+// Combine and projection in one kernel?  (see slim_tail_fused_kernel)  Measured: where the tail is a chain of
+// latencies over little data (many short sequences: 64 x 1500 rows at d = 1280: step 2.53 -> 2.40 ms) the fused
+// kernel wins; where a CTA has a lot of partials to pull out of L2 (16 long sequences at d = 4096: 184 KB per
+// CTA) the separate combine kernel with four times the threads per SM is faster (step 10.47 against 10.70 ms).
+// The partial bytes per CTA are estimated from the unit count a sequence has on average.
+static bool tail_fused(const slim_ctx* ctx, const SlimDecodeParams& p, const ProjGeom& g) {
+  if (!ctx->opt_tail_fused || combine_slices(ctx, p.H, p.batch, p.d) != 1 || g.hp * (g.nst * PJ_ROWS) > 128 * PF_MAXR ||
+      fused_smem_bytes(g, p.batch, p.workers, p.d_k) > (size_t)227 * 1024)
+    return false;
+  if (ctx->opt_tail_fused >= 2) return true;                  // forced (sweeps)
+  const double units_per_seq = (double)(p.workers + p.batch) / p.batch;
+  return 4.0 * PJ_BG * g.hp * (g.nst * PJ_ROWS) * units_per_seq <= 128.0 * 1024;
+}
+int slim_proj_launch_count(const slim_ctx* ctx, const SlimDecodeParams& p) {
+  const ProjGeom g = make_proj_geom(p.d, p.H, p.d_k, p.batch, ctx->opt_proj_ns);
+  return tail_fused(ctx, p, g) ? 1 : 2 + slim_proj_needs_convert(ctx, p.batch);
+}
+
 cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, unsigned char* u_tiled, float* u32, float* su,
                              cudaStream_t st) {
   const ProjGeom g = make_proj_geom(p.d, p.H, p.d_k, p.batch, ctx->opt_proj_ns);
+  // One kernel for combine and projection where every (head, sequence) row has a CTA of its own anyway (no
+  // column-split combine) and a CTA's share of the combined values fits its registers.
+  if (tail_fused(ctx, p, g)) {
+    const size_t smem = fused_smem_bytes(g, p.batch, p.workers, p.d_k);
+    const bool r4 = g.hp * (g.nst * PJ_ROWS) <= 128 * 4;      // rounds of 256 (item, column group) pairs per CTA
+    void (*kern)(const CUtensorMap, const SlimDecodeParams, const float*, float*, const ProjGeom) =
+        r4 ? slim_tail_fused_kernel<4> : slim_tail_fused_kernel<8>;
+    static size_t attr_set[64][2] = {};              // function attributes are kept per device
+    if (ctx->device < 0 || ctx->device >= 64 || attr_set[ctx->device][r4] < smem) {
+      cudaError_t e = cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      if (ctx->device >= 0 && ctx->device < 64) attr_set[ctx->device][r4] = smem;
+    }
+    CUtensorMap map;
+    memcpy(&map, ctx->wmap_h, sizeof(map));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(g.hg, g.jsplit, g.nbg);
+    cfg.blockDim = dim3(PF_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;            // the row slices of one output tile
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = g.jsplit; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, kern, map, p, (const float*)ctx->wkv_hscale, u32, g);
+  }
   {
     // No CTAs for the padding sequences of a 16-sequence group in the split variant (their columns of the
     // projection's B operand stay unwritten and only feed outputs that are never stored).
