@@ -22,6 +22,9 @@
 //                         each adds, in slice order, a share of the output rows
 //                         through distributed shared memory (bitwise repeatable).
 //
+//   slim_tail_fused_kernel  both of the above in one kernel: the projection CTA forms its own columns of u
+//                         from the partials (used where a CTA has few partial bytes to pull; see tail_fused).
+//
 // Every mbarrier wait is bounded in time; a wait that runs out sets the device
 // status to SLIM_ERR_TIMEOUT and the CTA drains and exits.
 #include <cstring>
