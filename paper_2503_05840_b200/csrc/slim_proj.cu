@@ -760,14 +760,16 @@ int slim_proj_needs_convert(const slim_ctx* ctx, int batch) { return combine_sli
 // latencies over little data (many short sequences: 64 x 1500 rows at d = 1280: step 2.53 -> 2.40 ms) the fused
 // kernel wins; where a CTA has a lot of partials to pull out of L2 (16 long sequences at d = 4096: 184 KB per
 // CTA) the separate combine kernel with four times the threads per SM is faster (step 10.47 against 10.70 ms).
-// The partial bytes per CTA are estimated from the unit count a sequence has on average.
+// In between (the same 64 sequences with lone-CTA workers, 148 of them: 108 KB) the separate kernels still win
+// (X-cache scheme: 5.21 against 5.69 ms).  The partial bytes per CTA are estimated from the unit count a
+// sequence has on average.
 static bool tail_fused(const slim_ctx* ctx, const SlimDecodeParams& p, const ProjGeom& g) {
   if (!ctx->opt_tail_fused || combine_slices(ctx, p.H, p.batch, p.d) != 1 || g.hp * (g.nst * PJ_ROWS) > 128 * PF_MAXR ||
       fused_smem_bytes(g, p.batch, p.workers, p.d_k) > (size_t)227 * 1024)
     return false;
   if (ctx->opt_tail_fused >= 2) return true;                  // forced (sweeps)
   const double units_per_seq = (double)(p.workers + p.batch) / p.batch;
-  return 4.0 * PJ_BG * g.hp * (g.nst * PJ_ROWS) * units_per_seq <= 128.0 * 1024;
+  return 4.0 * PJ_BG * g.hp * (g.nst * PJ_ROWS) * units_per_seq <= 80.0 * 1024;
 }
 int slim_proj_launch_count(const slim_ctx* ctx, const SlimDecodeParams& p) {
   const ProjGeom g = make_proj_geom(p.d, p.H, p.d_k, p.batch, ctx->opt_proj_ns);
