@@ -25,7 +25,7 @@ __device__ __forceinline__ uint32_t qt_offset(int n, int k) {     // K-major 8x8
 // q~[b][h][j] = qscale sum_c q[b][h d_k + c] W_K[j][h d_k + c], written as bf16 hi / lo rows h and 32 + h
 // of the [64 x 16] tile of k-step j / 16.  CTA = (head, 64 rows j of W_K): the weight tile is read once
 // and used for every sequence of the batch.
-constexpr int XQ_J = 64, XQ_B = 16;
+constexpr int XQ_J = 64, XQ_B = 64;             // rows of W_K per CTA; sequences per pass (one pass up to batch 64)
 __global__ void __launch_bounds__(256)
 slim_xq_tiled_kernel(SlimDecodeParams p, const float* __restrict__ W_K, unsigned char* __restrict__ qt_tiled) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -38,27 +38,34 @@ slim_xq_tiled_kernel(SlimDecodeParams p, const float* __restrict__ W_K, unsigned
     const int j = e / dk, c = e % dk;
     s_w[j * (dk + 1) + c] = (j0 + j < d) ? __ldg(W_K + (size_t)(j0 + j) * p.e + h * dk + c) : 0.f;
   }
-  const int j = tid & (XQ_J - 1), bq = tid >> 6;                     // a thread: row j, sequences 4 bq .. 4 bq + 3 of a pass
+  constexpr int XQ_S = XQ_B / 4;                                     // sequences per thread and pass
+  const int j = tid & (XQ_J - 1), bq = tid >> 6;                     // a thread: row j, sequences XQ_S bq .. XQ_S bq + XQ_S - 1 of a pass
   for (int b0 = 0; b0 < p.batch; b0 += XQ_B) {
     __syncthreads();
-    for (int e = tid; e < XQ_B * dk; e += 256) {                     // s_q[c][bb]: four sequences of one c in 16 bytes
+    for (int e = tid; e < XQ_B * dk; e += 256) {                     // s_q[c][bb]: the sequences of one c side by side
       const int bb = e / dk, c = e % dk;
       s_q[c * XQ_B + bb] = (b0 + bb < p.batch)
                                ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.q)[(size_t)(b0 + bb) * p.e + h * dk + c]) * p.qscale : 0.f;
     }
     __syncthreads();
-    if (j0 + j >= d) continue;
+    if (j0 + j >= d || b0 + XQ_S * bq >= p.batch) continue;
     const float* w = s_w + j * (dk + 1);
-    float a[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 8
+    float a[XQ_S];
+#pragma unroll
+    for (int x = 0; x < XQ_S; ++x) a[x] = 0.f;
+#pragma unroll 4
     for (int c = 0; c < dk; ++c) {
       const float wc = w[c];
-      const float4 qv = *reinterpret_cast<const float4*>(s_q + c * XQ_B + 4 * bq);
-      a[0] = fmaf(qv.x, wc, a[0]); a[1] = fmaf(qv.y, wc, a[1]); a[2] = fmaf(qv.z, wc, a[2]); a[3] = fmaf(qv.w, wc, a[3]);
+#pragma unroll
+      for (int x4 = 0; x4 < XQ_S / 4; ++x4) {
+        const float4 qv = *reinterpret_cast<const float4*>(s_q + c * XQ_B + XQ_S * bq + 4 * x4);
+        a[4 * x4] = fmaf(qv.x, wc, a[4 * x4]); a[4 * x4 + 1] = fmaf(qv.y, wc, a[4 * x4 + 1]);
+        a[4 * x4 + 2] = fmaf(qv.z, wc, a[4 * x4 + 2]); a[4 * x4 + 3] = fmaf(qv.w, wc, a[4 * x4 + 3]);
+      }
     }
 #pragma unroll
-    for (int x = 0; x < 4; ++x) {
-      const int b = b0 + 4 * bq + x;
+    for (int x = 0; x < XQ_S; ++x) {
+      const int b = b0 + XQ_S * bq + x;
       if (b >= p.batch) continue;
       const __nv_bfloat16 hi = __float2bfloat16_rn(a[x]), lo = __float2bfloat16_rn(a[x] - __bfloat162float(hi));
       unsigned char* t = qt_tiled + ((size_t)b * (d / 16) + (j0 + j) / 16) * 2048;
@@ -187,7 +194,17 @@ cudaError_t slim_xscores_make_tmap(const slim_ctx* ctx, slim_cache* c) {
 
 cudaError_t slim_launch_xscores_tc(const slim_ctx* ctx, const slim_cache* c, const SlimDecodeParams& p, const float* W_K,
                                    unsigned char* qt_tiled, float* scores, cudaStream_t st) {
-  slim_xq_tiled_kernel<<<dim3(p.H, (p.d + XQ_J - 1) / XQ_J), 256, sizeof(float) * (XQ_J * (p.d_k + 1) + XQ_B * p.d_k), st>>>(p, W_K, qt_tiled);
+  const size_t xq_smem = sizeof(float) * (XQ_J * (p.d_k + 1) + XQ_B * p.d_k);
+  if (xq_smem > 48 * 1024) {                         // function attributes are kept per device: opt in once on each
+    static bool attr_set[64] = {};
+    if (ctx->device < 0 || ctx->device >= 64 || !attr_set[ctx->device]) {
+      cudaError_t ea = cudaFuncSetAttribute((const void*)slim_xq_tiled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+      if (ea != cudaSuccess) return ea;
+      if (ctx->device >= 0 && ctx->device < 64) attr_set[ctx->device] = true;
+    }
+  }
+  // (a plain launch: letting this kernel start under the one before it was measured slower, 5.16 -> 5.44 ms per step)
+  slim_xq_tiled_kernel<<<dim3(p.H, (p.d + XQ_J - 1) / XQ_J), 256, xq_smem, st>>>(p, W_K, qt_tiled);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   CUtensorMap map;
