@@ -242,3 +242,39 @@ def test_random_ragged_batches(seed):
     cfg = synth.SlimConfig("ragged", d, H, d_k, batch, t_cap, 1, theta, "bf16")
     L = synth.make_layer(cfg, 9000 + seed, lengths=lengths)
     _run_host_case(cfg, L)
+
+
+@pytest.mark.parametrize("d,H,d_k,theta", [(1024, 8, 128, 1.0e6), (1280, 20, 64, 0.0), (768, 8, 96, 1.0e4)])
+@pytest.mark.parametrize("fused", [0, 2])
+def test_tail_as_one_kernel_and_as_two(d, H, d_k, theta, fused, monkeypatch):
+    """The split combine and the projection (Eq. 7, Option 2) run either as two kernels or fused into one; which
+    one a shape gets by default is a matter of speed.  Both are forced here (the switch is read when the context
+    is created) on a ragged batch of 40 sequences with an empty one, against the oracle, and the launch count
+    tells that the intended kernels ran."""
+    monkeypatch.setenv("SLIM_TAIL_FUSED", str(fused))
+    g = np.random.default_rng(7)
+    lengths = g.integers(1, 400, size=40).astype(np.int32)
+    lengths[5] = 0
+    cfg = synth.SlimConfig("tail", d, H, d_k, len(lengths), 400, 1, theta, "bf16")
+    L = synth.make_layer(cfg, 4321 + d, lengths=lengths)
+    layer = SlimLayer(cfg.d, cfg.H, cfg.d_k, cfg.rope_theta, cfg.dtype, cfg.batch, cfg.context, DEV)
+    try:
+        try:
+            layer.set_path(B.SLIM_PATH_TC)
+        except B.SlimError:
+            pytest.skip("no tensor-core kernels for this shape on this device")
+        layer.k.copy_(to_device_keys(L.K, cfg.dtype, DEV))
+        layer.set_weights(L.W_K, L.W_V)
+        q = to_device_keys(L.q, cfg.dtype, DEV)
+        ld = torch.from_numpy(L.lengths).to(DEV)
+        got = layer.decode(q, ld).cpu().numpy().astype(np.float64)
+        assert layer.device_status() == B.SLIM_OK
+        assert layer.query(B.SLIM_Q_LAUNCHES_PER_DECODE) == (2 if fused else 3)
+        ref = so.oracle_slim_batch(L.q, L.K, L.lengths, so.oracle_wkv(L.W_K, L.W_V), cfg.H, cfg.rope_theta)
+        for b in range(cfg.batch):
+            if L.lengths[b] == 0:
+                assert np.all(got[b] == 0)
+            else:
+                assert _err(got[b], ref[b], "bf16") <= TOL["bf16"], f"sequence {b}"
+    finally:
+        layer.close()
