@@ -433,7 +433,9 @@ __host__ __device__ inline FusedSmem fused_smem(const ProjGeom& g, int batch, in
 template <int MAXR>
 __global__ void __launch_bounds__(PF_THREADS, 2)
 slim_tail_fused_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_constant__ SlimDecodeParams p,
-                       const float* __restrict__ hscale, float* __restrict__ u32, const ProjGeom g) {
+                       const float* __restrict__ hscale, float* __restrict__ u32, const ProjGeom g, const int from_u32) {
+  // from_u32: the rows u[b][h][:] are already combined (float rows in u32, written by the column-split combine of
+  // small batches); the CTA only turns its columns into operand tiles, which saves the conversion kernel.
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw_u32 = smem_u32(smem_raw);
   const uint32_t base = (raw_u32 + 1023u) & ~1023u;
@@ -488,9 +490,10 @@ slim_tail_fused_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_co
     }
   }
   slim_pdl_wait();                                             // the partials come from the decode kernel
-  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && tid == 0) *p.any_flag = 0;
+  if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && tid == 0 && !from_u32) *p.any_flag = 0;
 
   // ---- combine: units and weights of the CTA's (sequence, head) items ----
+  if (!from_u32) {
   const SlimSched sc = slim_sched_build(p.lengths, p.batch, p.t_cap, p.workers, p.min_tiles, s_prefix, p.status, p.unit_cost);
   {
     // All items at once: LPI = 256 / items lanes (16 or 8, a power of two within a warp) share an item and take its
@@ -534,6 +537,9 @@ slim_tail_fused_kernel(const __grid_constant__ CUtensorMap wmap, const __grid_co
   // a sequence with a flagged unit: its columns are recomputed exactly into the float scratch first (rare)
   for (int item = 0; item < items; ++item)
     if (s_info[4 * item + 2]) slim_comb::exact_groups(p, u32, bg * PJ_BG + item / hp, hg * hp + item % hp, row0 / 8, ncols / 8, s_x);
+  } else if (tid < items) {
+    s_info[4 * tid] = 0; s_info[4 * tid + 1] = 0; s_info[4 * tid + 2] = 1;         // every row comes from the float scratch
+  }
   __syncthreads();
   const int gpi = ncols / 8;                                  // column groups per item
   const int total = items * gpi, rounds = (total + PF_THREADS - 1) / PF_THREADS;
@@ -763,17 +769,54 @@ int slim_proj_needs_convert(const slim_ctx* ctx, int batch) { return combine_sli
 // In between (the same 64 sequences with lone-CTA workers, 148 of them: 108 KB) the separate kernels still win
 // (X-cache scheme: 5.21 against 5.69 ms).  The partial bytes per CTA are estimated from the unit count a
 // sequence has on average.
+static bool fused_possible(const slim_ctx* ctx, const SlimDecodeParams& p, const ProjGeom& g) {
+  return ctx->opt_tail_fused && g.hp * (g.nst * PJ_ROWS) <= 128 * PF_MAXR &&
+         fused_smem_bytes(g, p.batch, p.workers, p.d_k) <= (size_t)227 * 1024;
+}
 static bool tail_fused(const slim_ctx* ctx, const SlimDecodeParams& p, const ProjGeom& g) {
-  if (!ctx->opt_tail_fused || combine_slices(ctx, p.H, p.batch, p.d) != 1 || g.hp * (g.nst * PJ_ROWS) > 128 * PF_MAXR ||
-      fused_smem_bytes(g, p.batch, p.workers, p.d_k) > (size_t)227 * 1024)
-    return false;
+  if (!fused_possible(ctx, p, g) || combine_slices(ctx, p.H, p.batch, p.d) != 1) return false;
   if (ctx->opt_tail_fused >= 2) return true;                  // forced (sweeps)
   const double units_per_seq = (double)(p.workers + p.batch) / p.batch;
   return 4.0 * PJ_BG * g.hp * (g.nst * PJ_ROWS) * units_per_seq <= 80.0 * 1024;
 }
+// Small batches (column-split combine into float rows): the fused kernel takes the rows from there and makes
+// the operand tiles itself, so no conversion kernel runs.
+static bool convert_fused(const slim_ctx* ctx, const SlimDecodeParams& p, const ProjGeom& g) {
+  return fused_possible(ctx, p, g) && combine_slices(ctx, p.H, p.batch, p.d) > 1;
+}
 int slim_proj_launch_count(const slim_ctx* ctx, const SlimDecodeParams& p) {
   const ProjGeom g = make_proj_geom(p.d, p.H, p.d_k, p.batch, ctx->opt_proj_ns);
-  return tail_fused(ctx, p, g) ? 1 : 2 + slim_proj_needs_convert(ctx, p.batch);
+  if (tail_fused(ctx, p, g)) return 1;
+  if (convert_fused(ctx, p, g)) return 2;
+  return 2 + slim_proj_needs_convert(ctx, p.batch);
+}
+
+static cudaError_t launch_fused(const slim_ctx* ctx, const SlimDecodeParams& p, const ProjGeom& g, float* u32, int from_u32,
+                                cudaStream_t st) {
+  const size_t smem = fused_smem_bytes(g, p.batch, p.workers, p.d_k);
+  const bool r4 = g.hp * (g.nst * PJ_ROWS) <= 128 * 4;      // rounds of 256 (item, column group) pairs per CTA
+  void (*kern)(const CUtensorMap, const SlimDecodeParams, const float*, float*, const ProjGeom, const int) =
+      r4 ? slim_tail_fused_kernel<4> : slim_tail_fused_kernel<8>;
+  static size_t attr_set[64][2] = {};              // function attributes are kept per device
+  if (ctx->device < 0 || ctx->device >= 64 || attr_set[ctx->device][r4] < smem) {
+    cudaError_t e = cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    if (ctx->device >= 0 && ctx->device < 64) attr_set[ctx->device][r4] = smem;
+  }
+  CUtensorMap map;
+  memcpy(&map, ctx->wmap_h, sizeof(map));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(g.hg, g.jsplit, g.nbg);
+  cfg.blockDim = dim3(PF_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;            // the row slices of one output tile
+  attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = g.jsplit; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, kern, map, p, (const float*)ctx->wkv_hscale, u32, g, from_u32);
 }
 
 cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, unsigned char* u_tiled, float* u32, float* su,
@@ -781,32 +824,7 @@ cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, uns
   const ProjGeom g = make_proj_geom(p.d, p.H, p.d_k, p.batch, ctx->opt_proj_ns);
   // One kernel for combine and projection where every (head, sequence) row has a CTA of its own anyway (no
   // column-split combine) and a CTA's share of the combined values fits its registers.
-  if (tail_fused(ctx, p, g)) {
-    const size_t smem = fused_smem_bytes(g, p.batch, p.workers, p.d_k);
-    const bool r4 = g.hp * (g.nst * PJ_ROWS) <= 128 * 4;      // rounds of 256 (item, column group) pairs per CTA
-    void (*kern)(const CUtensorMap, const SlimDecodeParams, const float*, float*, const ProjGeom) =
-        r4 ? slim_tail_fused_kernel<4> : slim_tail_fused_kernel<8>;
-    static size_t attr_set[64][2] = {};              // function attributes are kept per device
-    if (ctx->device < 0 || ctx->device >= 64 || attr_set[ctx->device][r4] < smem) {
-      cudaError_t e = cudaFuncSetAttribute((const void*)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e != cudaSuccess) return e;
-      if (ctx->device >= 0 && ctx->device < 64) attr_set[ctx->device][r4] = smem;
-    }
-    CUtensorMap map;
-    memcpy(&map, ctx->wmap_h, sizeof(map));
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(g.hg, g.jsplit, g.nbg);
-    cfg.blockDim = dim3(PF_THREADS);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;            // the row slices of one output tile
-    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = g.jsplit; attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, kern, map, p, (const float*)ctx->wkv_hscale, u32, g);
-  }
+  if (tail_fused(ctx, p, g)) return launch_fused(ctx, p, g, u32, 0, st);
   {
     // No CTAs for the padding sequences of a 16-sequence group in the split variant (their columns of the
     // projection's B operand stay unwritten and only feed outputs that are never stored).
@@ -818,6 +836,7 @@ cudaError_t slim_launch_proj(const slim_ctx* ctx, const SlimDecodeParams& p, uns
       while (G > 32 && G / 2 * nslice >= ngroups) G >>= 1;
       const size_t smem = sizeof(float) * p.workers + sizeof(int) * (4 + p.batch + 1) + 16 + sizeof(float) * 7 * 256;
       e = slim_launch_pdl(slim_combine_split_kernel, dim3(p.H, p.batch, nslice), dim3(256), smem, st, p, u32, G);
+      if (e == cudaSuccess && convert_fused(ctx, p, g)) return launch_fused(ctx, p, g, u32, 1, st);
       if (e == cudaSuccess)
         e = slim_launch_pdl(slim_convert_kernel, dim3(p.H, p.batch), dim3(256), 0, st, (const float*)u32, u_tiled, su, p.d, p.H, g.hp);
     } else {

@@ -423,14 +423,14 @@ def test_decode_step_capacity_and_launch_count():
         assert layer.device_status() == B.SLIM_ERR_CAPACITY          # sequence 0: beyond t_cap, nothing written
         assert torch.equal(layer.k[0], keep[0])
         assert torch.all(layer.k[1, 63] == 9.0) and torch.equal(layer.k[1, :63], keep[1, :63])
-        # tensor-core path: decode kernel, combine (for so small a batch: split combine + operand conversion),
-        # projection; the update needs no kernel of its own
+        # tensor-core path: decode kernel, column-split combine (so small a batch), projection (which makes its own
+        # operand tiles from the combined rows); the update needs no kernel of its own
         assert layer.query(B.SLIM_Q_PATH_IN_USE) == B.SLIM_PATH_TC
-        assert layer.query(B.SLIM_Q_LAUNCHES_PER_DECODE) == 4
+        assert layer.query(B.SLIM_Q_LAUNCHES_PER_DECODE) == 3
         layer.set_path(B.SLIM_PATH_GENERIC)
         layer.decode_step(q, k_new, torch.tensor([3, 64], dtype=torch.int32, device=DEV))
         assert layer.device_status() == B.SLIM_OK
-        assert layer.query(B.SLIM_Q_LAUNCHES_PER_DECODE) == 6         # append, scores, accumulation, combine, conversion, projection
+        assert layer.query(B.SLIM_Q_LAUNCHES_PER_DECODE) == 5         # append, scores, accumulation, column-split combine, projection
     finally:
         layer.close()
 
