@@ -652,7 +652,7 @@ slim_status slim_combine_project(slim_ctx* ctx, const float* lse_all, const floa
                                            reinterpret_cast<float*>(ws + L.su), st);
     else e = slim_launch_tail(ctx, p, st);
   }
-  ctx->launches_last = 3;
+  ctx->launches_last = 1 + (ctx->proj_ok ? slim_proj_launch_count(ctx, p) : 2);      // join, then the tail's kernels
   if (e != cudaSuccess) { cudaGetLastError(); return SLIM_ERR_CUDA; }
   return SLIM_OK;
 }
