@@ -278,3 +278,30 @@ def test_tail_as_one_kernel_and_as_two(d, H, d_k, theta, fused, monkeypatch):
                 assert _err(got[b], ref[b], "bf16") <= TOL["bf16"], f"sequence {b}"
     finally:
         layer.close()
+
+
+@pytest.mark.parametrize("fused", [0, 1])
+def test_small_batch_tail_with_and_without_the_conversion_kernel(fused, monkeypatch):
+    """Few sequences: the combine is split over column slices and leaves float rows; the operand tiles are then made
+    either by a conversion kernel (switch off) or by the projection kernel itself (default).  Both against the oracle."""
+    monkeypatch.setenv("SLIM_TAIL_FUSED", str(fused))
+    lengths = np.array([300, 257, 16], dtype=np.int32)
+    cfg = synth.SlimConfig("tail-small", 1024, 8, 128, len(lengths), 300, 1, 1.0e4, "bf16")
+    L = synth.make_layer(cfg, 99, lengths=lengths)
+    layer = SlimLayer(cfg.d, cfg.H, cfg.d_k, cfg.rope_theta, cfg.dtype, cfg.batch, cfg.context, DEV)
+    try:
+        try:
+            layer.set_path(B.SLIM_PATH_TC)
+        except B.SlimError:
+            pytest.skip("no tensor-core kernels for this shape on this device")
+        layer.k.copy_(to_device_keys(L.K, cfg.dtype, DEV))
+        layer.set_weights(L.W_K, L.W_V)
+        q = to_device_keys(L.q, cfg.dtype, DEV)
+        got = layer.decode(q, torch.from_numpy(L.lengths).to(DEV)).cpu().numpy().astype(np.float64)
+        assert layer.device_status() == B.SLIM_OK
+        assert layer.query(B.SLIM_Q_LAUNCHES_PER_DECODE) == (3 if fused else 4)
+        ref = so.oracle_slim_batch(L.q, L.K, L.lengths, so.oracle_wkv(L.W_K, L.W_V), cfg.H, cfg.rope_theta)
+        for b in range(cfg.batch):
+            assert _err(got[b], ref[b], "bf16") <= TOL["bf16"], f"sequence {b}"
+    finally:
+        layer.close()
